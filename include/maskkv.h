@@ -1,0 +1,165 @@
+/* maskkv.h - C ABI of the MaskKV compress-and-attend path for NVIDIA B200 (sm_100a).
+ *
+ * The path, per transformer layer of a diffusion LLM (paper: "Mask Tokens as Prophet", Section
+ * "The MaskKV Framework"):
+ *
+ *   maskkv_score    Stage 1, Eq. 6-7: the mask-token queries vote on the prompt keys through softmax
+ *                   attention; also the two attention-mass sums of Eq. 14.
+ *   maskkv_budget   Stage 2, Eq. 14-15: per-head budgets from the prompt preference, plus the exclusive
+ *                   prefix sum that lays out the ragged cache.  (maskkv_layer_budgets: Eq. 9-13, host.)
+ *   maskkv_select   Eq. 16: per head, keep the top-k prompt tokens.
+ *   maskkv_compact  gather the kept K/V rows into the ragged per-head cache.
+ *   maskkv_attend   a later denoising step: attention over [compacted prompt segment ; live keys]
+ *                   (appendix, proof step 3: out_m = sum_j softmax(q_m k_j / sqrt(d_k)) V_j).
+ *
+ * Conventions that hold for every function:
+ *   - Return value: 0 (MASKKV_OK) or a negative MASKKV_E_* code.  Nothing throws, aborts or prints.
+ *   - Pointers named *_dev are DEVICE pointers owned by the caller; the library neither frees nor keeps
+ *     them past the call.  Pointers named *_host (and the *_cu arrays of the descriptor) are HOST
+ *     pointers that only need to stay valid until the call returns.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default stream) and the
+ *     call returns without synchronising.  The only synchronising call is maskkv_check_status.
+ *   - Device pointers must be 16-byte aligned (MASKKV_E_ALIGN otherwise); head_dim is contiguous.
+ *   - Arguments are validated before anything is launched.  A failed validation launches nothing.
+ *   - Outputs are fully written for every valid (request, head) segment and untouched elsewhere.
+ *     The same inputs give bit-identical outputs on every call (no order-dependent float atomics).
+ *   - No call allocates device memory; scratch comes from the caller's workspace
+ *     (maskkv_workspace_bytes).  maskkv_create allocates one 256-byte status block.
+ *   - Requests are independent.  A batch of layers can be run in one call by treating
+ *     (layer, request) as the request axis.
+ *
+ * Tensor layouts (T = MASKKV_F32 or MASKKV_BF16, chosen by desc.dtype for every Q/K/V/O tensor):
+ *   q_mask, q_live, out    T   [sum_M][H   ][d]   token stride q_token_stride, head stride q_head_stride
+ *   k_prompt, v_prompt     T   [sum_N][H_kv][d]   token stride kv_token_stride, head stride kv_head_stride
+ *   k_mask, k_live, v_live T   [sum_M][H_kv][d]   same kv strides
+ *   scores                 f32 [H_kv][sum_N]      I_j of Eq. 7, one contiguous segment per (head, request)
+ *   mass_p, mass_m         f32 [R][H_kv]          S_{m->p}, S_{m->m} of Eq. 14
+ *   budgets                i32 [R][H_kv]          k_{l,h} of Eq. 15
+ *   offsets                i32 [R*H_kv + 1]       exclusive prefix sum of budgets; segment s = r*H_kv + h
+ *   kept_idx               i32 [capacity]         request-local prompt indices, ascending within a segment
+ *   kc, vc                 T   [capacity][d]      compacted cache; rows of segment s are contiguous
+ *   lse                    f32 [H][sum_M]         log of the softmax denominator (optional)
+ * sum_N = prompt_cu[R], sum_M = live_cu[R].  Strides are in elements.
+ */
+#ifndef MASKKV_H_
+#define MASKKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  MASKKV_OK = 0,
+  MASKKV_E_INVALID = -1,      /* null pointer, negative size, inconsistent descriptor */
+  MASKKV_E_UNSUPPORTED = -2,  /* dtype / head_dim / device the library has no kernel for */
+  MASKKV_E_ALIGN = -3,        /* a device pointer or stride breaks the 16-byte rule */
+  MASKKV_E_WORKSPACE = -4,    /* workspace missing or smaller than maskkv_workspace_bytes */
+  MASKKV_E_CAPACITY = -5,     /* capacity too small for what the host can bound */
+  MASKKV_E_CUDA = -6,         /* a CUDA runtime or driver call failed */
+  MASKKV_E_TIMEOUT = -7       /* reported by maskkv_check_status: a bounded device wait expired */
+};
+
+enum { MASKKV_F32 = 0, MASKKV_BF16 = 1 };
+
+/* Bits of the device status word returned by maskkv_check_status. */
+enum {
+  MASKKV_FLAG_TIMEOUT = 1u,   /* a bounded mbarrier wait gave up; that launch's outputs are invalid */
+  MASKKV_FLAG_CAPACITY = 2u,  /* maskkv_budget clipped budgets to fit `capacity` */
+  MASKKV_FLAG_BOUNDS = 4u     /* an index read from device memory was out of range and was skipped */
+};
+
+typedef struct maskkv_ctx maskkv_ctx;
+
+/* Opens the library on CUDA device `device` (which must be compute capability 10.x, else
+ * MASKKV_E_UNSUPPORTED).  Allocates the status block and resolves the tensor-map encoder.
+ * The context may be used from one host thread at a time. */
+int maskkv_create(maskkv_ctx** out, int device);
+int maskkv_destroy(maskkv_ctx* ctx);
+
+/* Static, human-readable name of a return code. */
+const char* maskkv_status_string(int code);
+
+/* Waits for `stream`, then returns the device status flags accumulated since the last call in
+ * *flags_out (may be NULL) and clears them.  Returns MASKKV_E_TIMEOUT if the TIMEOUT flag was set,
+ * MASKKV_E_CUDA if the stream reported an error, else MASKKV_OK. */
+int maskkv_check_status(maskkv_ctx* ctx, void* stream, uint32_t* flags_out);
+
+typedef struct {
+  int32_t dtype;              /* MASKKV_F32 | MASKKV_BF16 */
+  int32_t n_q_heads;          /* H */
+  int32_t n_kv_heads;         /* H_kv, divides H */
+  int32_t head_dim;           /* d: 64 or 128 */
+  int32_t n_requests;         /* R >= 1 */
+  float softmax_scale;        /* <= 0 selects 1/sqrt(head_dim) (Eq. 6) */
+  const int32_t* prompt_cu;   /* HOST [R+1] cumulative prompt lengths, prompt_cu[0] = 0 */
+  const int32_t* live_cu;     /* HOST [R+1] cumulative mask/live lengths */
+  const int32_t* prompt_cu_dev; /* DEVICE copies of the two arrays */
+  const int32_t* live_cu_dev;
+  int64_t q_token_stride, q_head_stride;     /* elements; 0 selects the packed layout */
+  int64_t kv_token_stride, kv_head_stride;
+} maskkv_desc_t;
+
+/* Bytes of scratch that maskkv_score and maskkv_select may need for this descriptor (the larger of
+ * the two).  Never fails; returns 0 for an invalid descriptor. */
+size_t maskkv_workspace_bytes(const maskkv_ctx* ctx, const maskkv_desc_t* desc);
+
+/* Eq. 9-13, host only: splits the total budget k_p (in per-head units, i.e. n_layers x the nominal
+ * per-head budget) over the layers.  importance_host [n_layers] is the offline layer-importance
+ * profile (Eq. 8); is_boundary_host [n_layers] marks the boundary group (NULL = first and last layer).
+ * k_group values stay real until the floor of Eq. 13; floors are floor(x + 1e-6) in double precision.
+ * Writes k_l_out_host [n_layers]. */
+int maskkv_layer_budgets(int64_t k_p, double beta, int32_t n_layers, const double* importance_host,
+                         const uint8_t* is_boundary_host, int32_t* k_l_out_host);
+
+/* Eq. 6-7 and the sums of Eq. 14.  For every request r and KV head h: softmax (fp32) of
+ * scale * q_i . k_j over the request's N_r prompt keys followed by its M_r mask keys, for each of the
+ * H/H_kv query heads that share h; scores[h][prompt_cu[r] + j] = sum over those heads and mask rows i of
+ * w_i * A_ij; mass_p = the same sum over prompt j; mass_m = over mask j.  row_weights_dev (f32 [sum_M],
+ * NULL = all ones) weights each voting row.  The M x N weight matrix is never written to memory. */
+int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_dev,
+                 const void* k_prompt_dev, const void* k_mask_dev, const float* row_weights_dev,
+                 float* scores_dev, float* mass_p_dev, float* mass_m_dev, void* workspace_dev,
+                 size_t workspace_bytes, void* stream);
+
+/* Eq. 14-15, clamp and prefix sum, all on the device (no host synchronisation):
+ *   P = mass_p / (mass_p + mass_m); Phat = P / sum_h P (ascending h);
+ *   x = alpha*k_l + ((1-alpha)*(H_kv*k_l))*Phat; k = floor(x + 1e-6) clamped to [0, N_r]
+ * in IEEE double precision without fused multiply-add, so equal inputs give equal integers on any
+ * conforming implementation.  k_l applies to every request unless k_l_per_request_dev (i32 [R]) is
+ * given.  If the running total would exceed `capacity` (rows available in kept_idx / kc / vc) the
+ * segment that crosses it is clipped, later ones get 0, and MASKKV_FLAG_CAPACITY is raised. */
+int maskkv_budget(maskkv_ctx* ctx, const maskkv_desc_t* desc, int32_t k_l,
+                  const int32_t* k_l_per_request_dev, double alpha, const float* mass_p_dev,
+                  const float* mass_m_dev, int64_t capacity, int32_t* budgets_dev, int32_t* offsets_dev,
+                  void* stream);
+
+/* Eq. 16.  For segment s = (r, h): kept_idx[offsets[s] .. offsets[s+1]) receives the indices of the
+ * budgets[s] largest scores of scores[h][prompt_cu[r] .. prompt_cu[r+1]) under the total order
+ * (score descending, index ascending; NaN below every number), written in ascending index order.
+ * Exact: no tolerance is involved. */
+int maskkv_select(maskkv_ctx* ctx, const maskkv_desc_t* desc, const float* scores_dev,
+                  const int32_t* budgets_dev, const int32_t* offsets_dev, int32_t* kept_idx_dev,
+                  void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* kc[offsets[s] + t] = k_prompt[prompt_cu[r] + kept_idx[offsets[s] + t]][h][:], same for v: a byte copy.
+ * `capacity` is the number of rows kc/vc/kept_idx hold; rows at or beyond it are never touched. */
+int maskkv_compact(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* k_prompt_dev,
+                   const void* v_prompt_dev, const int32_t* kept_idx_dev, const int32_t* offsets_dev,
+                   int64_t capacity, void* kc_dev, void* vc_dev, void* stream);
+
+/* One attention step of the live region.  For request r and query head h (KV head h / (H/H_kv)):
+ * softmax of scale * q_i . k over the rows [offsets[s], offsets[s+1]) of kc followed by the request's
+ * M_r live keys (no mask, own key included); out = weights x [vc rows ; v_live].  bf16: fp32 accumulation
+ * and softmax, weights rounded to bf16 before the second product; f32: fp32 throughout.
+ * lse_dev (f32 [H][sum_M]) may be NULL. */
+int maskkv_attend(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_live_dev,
+                  const void* k_live_dev, const void* v_live_dev, const void* kc_dev, const void* vc_dev,
+                  const int32_t* offsets_dev, void* out_dev, float* lse_dev, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MASKKV_H_ */

@@ -1,0 +1,77 @@
+// Shared declarations of the MaskKV CUDA library (sm_100a): context, resolved problem shape,
+// element loads.  Internal; the public surface is include/maskkv.h.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "maskkv.h"
+
+struct maskkv_ctx {
+  int device;
+  int sm_count;
+  int smem_optin;          // max opt-in dynamic shared memory per block
+  uint32_t* status_dev;    // 256-byte block; word 0 = status flags, word 1 = where a wait gave up
+  void* encode_tiled;      // cuTensorMapEncodeTiled, resolved through the runtime
+};
+
+// The descriptor after validation, passed to kernels by value.
+struct Shape {
+  int dtype, H, Hkv, g, d, R;
+  float scale;
+  long long q_ts, q_hs, kv_ts, kv_hs;     // strides in elements
+  const int32_t* prompt_cu;               // device
+  const int32_t* live_cu;                 // device
+  int sumN, sumM, maxN, maxM;
+};
+
+namespace mkv {
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// Load `n` consecutive elements (n * sizeof(T) a multiple of 16, src 16-byte aligned) into floats.
+template <int n>
+__device__ __forceinline__ void load_row(const float* __restrict__ src, float* dst) {
+#pragma unroll
+  for (int c = 0; c < n; c += 4) {
+    float4 v = *reinterpret_cast<const float4*>(src + c);
+    dst[c] = v.x; dst[c + 1] = v.y; dst[c + 2] = v.z; dst[c + 3] = v.w;
+  }
+}
+template <int n>
+__device__ __forceinline__ void load_row(const __nv_bfloat16* __restrict__ src, float* dst) {
+#pragma unroll
+  for (int c = 0; c < n; c += 8) {
+    uint4 v = *reinterpret_cast<const uint4*>(src + c);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      dst[c + 2 * t] = __uint_as_float(w[t] << 16);
+      dst[c + 2 * t + 1] = __uint_as_float(w[t] & 0xffff0000u);
+    }
+  }
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Request that owns row `row` of a cumulative array cu[0..R].
+__device__ __forceinline__ int find_request(const int32_t* __restrict__ cu, int R, int row) {
+  int lo = 0, hi = R;  // invariant: cu[lo] <= row < cu[hi]
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (cu[mid] <= row) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+}  // namespace mkv

@@ -1,0 +1,54 @@
+// Gather of the kept K/V rows into the ragged per-head cache: a pure byte copy, one warp per kept
+// row, 16 bytes per lane per access (K row on the lower half-warp, V row on the upper one when a row
+// is 256 bytes).  Bound by HBM; the source rows are scattered 256-byte pieces, the destination is
+// contiguous.
+#pragma once
+
+#include "common.cuh"
+
+namespace mkv {
+
+constexpr int kCompactThreads = 256;
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+// row_bytes = d * sizeof(T); strides in bytes.  grid-stride over the rows in use (offsets[S], read on the device).
+__global__ void __launch_bounds__(kCompactThreads)
+compact_kernel(Shape sh, int row_bytes, long long ts_bytes, long long hs_bytes, const unsigned char* __restrict__ kp,
+               const unsigned char* __restrict__ vp, const int32_t* __restrict__ kept_idx,
+               const int32_t* __restrict__ offsets, long long capacity, unsigned char* __restrict__ kc,
+               unsigned char* __restrict__ vc, uint32_t* __restrict__ status) {
+  const int S = sh.R * sh.Hkv;
+  long long total = offsets[S];
+  if (total > capacity) total = capacity;
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = kCompactThreads / 32;
+  const int vec_per_row = row_bytes / 16;               // 16-byte pieces per row (8, 16 or 32)
+  const int pieces = 2 * vec_per_row;                   // K row then V row
+  for (long long t = (long long)blockIdx.x * warps_per_block + (threadIdx.x >> 5); t < total;
+       t += (long long)gridDim.x * warps_per_block) {
+    const int s = find_request(offsets, S, (int)t);     // segment that owns output row t
+    const int r = s / sh.Hkv, hk = s % sh.Hkv;
+    const int p0 = sh.prompt_cu[r], N = sh.prompt_cu[r + 1] - p0;
+    const int j = kept_idx[t];
+    if (j < 0 || j >= N) {                              // never dereference a bad index
+      if (lane == 0) atomicOr(status, (uint32_t)MASKKV_FLAG_BOUNDS);
+      continue;
+    }
+    const long long src = (long long)(p0 + j) * ts_bytes + (long long)hk * hs_bytes;
+    const long long dst = t * row_bytes;
+    for (int e = lane; e < pieces; e += 32) {
+      const bool is_v = e >= vec_per_row;
+      const int off = (is_v ? e - vec_per_row : e) * 16;
+      const uint4 v = ld_stream(reinterpret_cast<const uint4*>((is_v ? vp : kp) + src + off));
+      *reinterpret_cast<uint4*>((is_v ? vc : kc) + dst + off) = v;
+    }
+  }
+}
+
+}  // namespace mkv

@@ -1,0 +1,331 @@
+// C ABI of the MaskKV library: argument validation, workspace carving and kernel launches.
+// Every entry point validates first and launches nothing on failure (see include/maskkv.h).
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "attend_simt.cuh"
+#include "budget.cuh"
+#include "common.cuh"
+#include "compact.cuh"
+#include "score_simt.cuh"
+#include "select.cuh"
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() { if (switched) cudaSetDevice(prev); }
+};
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int elem_size(int dtype) { return dtype == MASKKV_F32 ? 4 : 2; }
+
+// Validates the descriptor and resolves defaults.  Returns MASKKV_OK or an error code.
+int resolve(const maskkv_desc_t* d, Shape* sh) {
+  if (d == nullptr) return MASKKV_E_INVALID;
+  if (d->dtype != MASKKV_F32 && d->dtype != MASKKV_BF16) return MASKKV_E_UNSUPPORTED;
+  if (d->head_dim != 64 && d->head_dim != 128) return MASKKV_E_UNSUPPORTED;
+  if (d->n_q_heads <= 0 || d->n_kv_heads <= 0 || d->n_q_heads % d->n_kv_heads != 0) return MASKKV_E_INVALID;
+  if (d->n_requests <= 0) return MASKKV_E_INVALID;
+  if (d->prompt_cu == nullptr || d->live_cu == nullptr || d->prompt_cu_dev == nullptr || d->live_cu_dev == nullptr)
+    return MASKKV_E_INVALID;
+  if (d->prompt_cu[0] != 0 || d->live_cu[0] != 0) return MASKKV_E_INVALID;
+  sh->dtype = d->dtype;
+  sh->H = d->n_q_heads;
+  sh->Hkv = d->n_kv_heads;
+  sh->g = sh->H / sh->Hkv;
+  sh->d = d->head_dim;
+  sh->R = d->n_requests;
+  sh->scale = d->softmax_scale > 0.f ? d->softmax_scale : (float)(1.0 / sqrt((double)d->head_dim));
+  sh->maxN = sh->maxM = 0;
+  for (int r = 0; r < sh->R; ++r) {
+    const long long n = (long long)d->prompt_cu[r + 1] - d->prompt_cu[r];
+    const long long m = (long long)d->live_cu[r + 1] - d->live_cu[r];
+    if (n < 0 || m < 0) return MASKKV_E_INVALID;
+    if (n > sh->maxN) sh->maxN = (int)n;
+    if (m > sh->maxM) sh->maxM = (int)m;
+  }
+  sh->sumN = d->prompt_cu[sh->R];
+  sh->sumM = d->live_cu[sh->R];
+  sh->q_hs = d->q_head_stride > 0 ? d->q_head_stride : sh->d;
+  sh->q_ts = d->q_token_stride > 0 ? d->q_token_stride : (long long)sh->H * sh->q_hs;
+  sh->kv_hs = d->kv_head_stride > 0 ? d->kv_head_stride : sh->d;
+  sh->kv_ts = d->kv_token_stride > 0 ? d->kv_token_stride : (long long)sh->Hkv * sh->kv_hs;
+  const long long es = elem_size(sh->dtype);
+  if ((sh->q_hs * es) % 16 || (sh->q_ts * es) % 16 || (sh->kv_hs * es) % 16 || (sh->kv_ts * es) % 16) return MASKKV_E_ALIGN;
+  if (sh->q_hs < sh->d || sh->kv_hs < sh->d) return MASKKV_E_INVALID;
+  if ((reinterpret_cast<uintptr_t>(d->prompt_cu_dev) & 3u) || (reinterpret_cast<uintptr_t>(d->live_cu_dev) & 3u)) return MASKKV_E_ALIGN;
+  sh->prompt_cu = d->prompt_cu_dev;
+  sh->live_cu = d->live_cu_dev;
+  return MASKKV_OK;
+}
+
+struct ScoreWorkspace {
+  size_t lse_off, part_off, mass_off, total;
+  int C, Tmax;
+};
+
+ScoreWorkspace score_workspace(const Shape& sh) {
+  ScoreWorkspace w;
+  const long long keys = (long long)sh.maxN + sh.maxM;
+  w.C = (int)((keys + mkv::kStatsChunk - 1) / mkv::kStatsChunk);
+  if (w.C < 1) w.C = 1;
+  w.Tmax = (int)((keys + mkv::kSimtThreads - 1) / mkv::kSimtThreads);
+  if (w.Tmax < 1) w.Tmax = 1;
+  size_t off = 0;
+  w.lse_off = off;  off = align_up(off + sizeof(float) * (size_t)sh.H * sh.sumM, 256);
+  w.part_off = off; off = align_up(off + sizeof(float2) * (size_t)sh.H * sh.sumM * w.C, 256);
+  w.mass_off = off; off = align_up(off + sizeof(float2) * (size_t)sh.R * sh.Hkv * w.Tmax, 256);
+  w.total = off;
+  return w;
+}
+
+inline int launch_status() { return cudaGetLastError() == cudaSuccess ? MASKKV_OK : MASKKV_E_CUDA; }
+
+template <typename T, int D>
+int launch_score_simt(const Shape& sh, const ScoreWorkspace& w, const void* q, const void* kp, const void* km,
+                      const float* rw, float* scores, float* mass_p, float* mass_m, unsigned char* ws, cudaStream_t st) {
+  float* lse = reinterpret_cast<float*>(ws + w.lse_off);
+  float2* part = reinterpret_cast<float2*>(ws + w.part_off);
+  float2* mass_part = reinterpret_cast<float2*>(ws + w.mass_off);
+  const int S = sh.R * sh.Hkv;
+  if (sh.sumM > 0) {
+    const int q_tiles = (sh.maxM + mkv::kSimtThreads - 1) / mkv::kSimtThreads;
+    dim3 g1(w.C, sh.H, sh.R * q_tiles);
+    mkv::score_stats_simt<T, D><<<g1, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, part, w.C);
+    const long long rows = (long long)sh.H * sh.sumM;
+    mkv::score_merge_stats<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(sh, part, w.C, lse);
+  }
+  dim3 g2(w.Tmax, sh.Hkv, sh.R);
+  mkv::score_colsum_simt<T, D><<<g2, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, lse, rw,
+                                                                  scores, mass_part, w.Tmax);
+  mkv::score_mass_reduce<<<(S + 3) / 4, 128, 0, st>>>(S, mass_part, w.Tmax, mass_p, mass_m);
+  return launch_status();
+}
+
+template <typename T, int D>
+int launch_attend_simt(const Shape& sh, const void* q, const void* kl, const void* vl, const void* kc, const void* vc,
+                       const int32_t* offsets, void* out, float* lse, cudaStream_t st) {
+  if (sh.maxM == 0) return MASKKV_OK;
+  dim3 grid((sh.maxM + mkv::kAttendWarps - 1) / mkv::kAttendWarps, sh.H, sh.R);
+  mkv::attend_simt<T, D><<<grid, mkv::kAttendWarps * 32, 0, st>>>(sh, (const T*)q, (const T*)kl, (const T*)vl, (const T*)kc,
+                                                                   (const T*)vc, offsets, (T*)out, lse);
+  return launch_status();
+}
+
+}  // namespace
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+const char* maskkv_status_string(int code) {
+  switch (code) {
+    case MASKKV_OK: return "ok";
+    case MASKKV_E_INVALID: return "invalid argument";
+    case MASKKV_E_UNSUPPORTED: return "unsupported dtype, head_dim or device";
+    case MASKKV_E_ALIGN: return "pointer or stride not 16-byte aligned";
+    case MASKKV_E_WORKSPACE: return "workspace missing or too small";
+    case MASKKV_E_CAPACITY: return "capacity too small";
+    case MASKKV_E_CUDA: return "CUDA call failed";
+    case MASKKV_E_TIMEOUT: return "a bounded device wait expired";
+    default: return "unknown status";
+  }
+}
+
+int maskkv_create(maskkv_ctx** out, int device) {
+  if (out == nullptr) return MASKKV_E_INVALID;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return MASKKV_E_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MASKKV_E_CUDA;
+  if (prop.major != 10) return MASKKV_E_UNSUPPORTED;
+  DeviceGuard guard(device);
+  maskkv_ctx* ctx = static_cast<maskkv_ctx*>(calloc(1, sizeof(maskkv_ctx)));
+  if (ctx == nullptr) return MASKKV_E_INVALID;
+  ctx->device = device;
+  ctx->sm_count = prop.multiProcessorCount;
+  ctx->smem_optin = (int)prop.sharedMemPerBlockOptin;
+  if (cudaMalloc(&ctx->status_dev, 256) != cudaSuccess || cudaMemset(ctx->status_dev, 0, 256) != cudaSuccess) {
+    free(ctx);
+    return MASKKV_E_CUDA;
+  }
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->encode_tiled, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    ctx->encode_tiled = nullptr;
+  cudaFuncSetAttribute(mkv::select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - 2048);
+  if (cudaGetLastError() != cudaSuccess) { cudaFree(ctx->status_dev); free(ctx); return MASKKV_E_CUDA; }
+  *out = ctx;
+  return MASKKV_OK;
+}
+
+int maskkv_destroy(maskkv_ctx* ctx) {
+  if (ctx == nullptr) return MASKKV_E_INVALID;
+  DeviceGuard guard(ctx->device);
+  cudaFree(ctx->status_dev);
+  free(ctx);
+  return MASKKV_OK;
+}
+
+int maskkv_check_status(maskkv_ctx* ctx, void* stream, uint32_t* flags_out) {
+  if (ctx == nullptr) return MASKKV_E_INVALID;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t flags = 0;
+  if (cudaMemcpyAsync(&flags, ctx->status_dev, sizeof(flags), cudaMemcpyDeviceToHost, st) != cudaSuccess) return MASKKV_E_CUDA;
+  if (cudaMemsetAsync(ctx->status_dev, 0, 8, st) != cudaSuccess) return MASKKV_E_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return MASKKV_E_CUDA;
+  if (flags_out) *flags_out = flags;
+  return (flags & MASKKV_FLAG_TIMEOUT) ? MASKKV_E_TIMEOUT : MASKKV_OK;
+}
+
+size_t maskkv_workspace_bytes(const maskkv_ctx* ctx, const maskkv_desc_t* desc) {
+  (void)ctx;
+  Shape sh;
+  if (resolve(desc, &sh) != MASKKV_OK) return 0;
+  return score_workspace(sh).total;
+}
+
+int maskkv_layer_budgets(int64_t k_p, double beta, int32_t n_layers, const double* importance_host,
+                         const uint8_t* is_boundary_host, int32_t* k_l_out_host) {
+  if (n_layers <= 0 || importance_host == nullptr || k_l_out_host == nullptr || k_p < 0) return MASKKV_E_INVALID;
+  if (!(beta >= 0.0 && beta <= 1.0)) return MASKKV_E_INVALID;
+  // volatile keeps every intermediate a rounded double (no contraction, no extended precision)
+  volatile double base_real = beta * (double)k_p;
+  base_real = base_real / (double)n_layers;
+  const long long k_base = (long long)floor(base_real + 1e-6);                  // Eq. 9
+  const long long k_imp = k_p - (long long)n_layers * k_base;                   // Eq. 10
+  volatile double i_b = 0.0, i_m = 0.0;
+  int n_b = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    const bool bnd = is_boundary_host ? is_boundary_host[l] != 0 : (l == 0 || l == n_layers - 1);
+    if (bnd) { i_b = i_b + importance_host[l]; ++n_b; } else { i_m = i_m + importance_host[l]; }
+  }
+  const int n_m = n_layers - n_b;
+  volatile double denom = i_b + i_m;
+  volatile double group_b = 0.0;
+  if (denom > 0.0) { group_b = (double)k_imp * i_b; group_b = group_b / denom; } // Eq. 11
+  volatile double group_m = (double)k_imp - group_b;                            // Eq. 12
+  for (int l = 0; l < n_layers; ++l) {                                          // Eq. 13
+    const bool bnd = is_boundary_host ? is_boundary_host[l] != 0 : (l == 0 || l == n_layers - 1);
+    volatile double share = bnd ? group_b / (double)(n_b > 0 ? n_b : 1) : group_m / (double)(n_m > 0 ? n_m : 1);
+    k_l_out_host[l] = (int32_t)(k_base + (long long)floor(share + 1e-6));
+  }
+  return MASKKV_OK;
+}
+
+int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_dev, const void* k_prompt_dev,
+                 const void* k_mask_dev, const float* row_weights_dev, float* scores_dev, float* mass_p_dev,
+                 float* mass_m_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
+  if (ctx == nullptr) return MASKKV_E_INVALID;
+  Shape sh;
+  int rc = resolve(desc, &sh);
+  if (rc != MASKKV_OK) return rc;
+  if (scores_dev == nullptr || mass_p_dev == nullptr || mass_m_dev == nullptr) return MASKKV_E_INVALID;
+  if ((sh.sumM > 0 && (q_mask_dev == nullptr || k_mask_dev == nullptr)) || (sh.sumN > 0 && k_prompt_dev == nullptr))
+    return MASKKV_E_INVALID;
+  if (!aligned16(q_mask_dev) || !aligned16(k_prompt_dev) || !aligned16(k_mask_dev) || !aligned16(scores_dev) ||
+      !aligned16(workspace_dev))
+    return MASKKV_E_ALIGN;
+  const ScoreWorkspace w = score_workspace(sh);
+  if (workspace_dev == nullptr || workspace_bytes < w.total) return MASKKV_E_WORKSPACE;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  unsigned char* ws = static_cast<unsigned char*>(workspace_dev);
+#define MKV_SCORE(T, D) launch_score_simt<T, D>(sh, w, q_mask_dev, k_prompt_dev, k_mask_dev, row_weights_dev, scores_dev, \
+                                                mass_p_dev, mass_m_dev, ws, st)
+  if (sh.dtype == MASKKV_F32) return sh.d == 64 ? MKV_SCORE(float, 64) : MKV_SCORE(float, 128);
+  return sh.d == 64 ? MKV_SCORE(__nv_bfloat16, 64) : MKV_SCORE(__nv_bfloat16, 128);
+#undef MKV_SCORE
+}
+
+int maskkv_budget(maskkv_ctx* ctx, const maskkv_desc_t* desc, int32_t k_l, const int32_t* k_l_per_request_dev,
+                  double alpha, const float* mass_p_dev, const float* mass_m_dev, int64_t capacity,
+                  int32_t* budgets_dev, int32_t* offsets_dev, void* stream) {
+  if (ctx == nullptr) return MASKKV_E_INVALID;
+  Shape sh;
+  int rc = resolve(desc, &sh);
+  if (rc != MASKKV_OK) return rc;
+  if (mass_p_dev == nullptr || mass_m_dev == nullptr || budgets_dev == nullptr || offsets_dev == nullptr) return MASKKV_E_INVALID;
+  if (k_l < 0 || capacity < 0 || capacity > 0x7fffffffLL || !(alpha >= 0.0 && alpha <= 1.0)) return MASKKV_E_INVALID;
+  const int S = sh.R * sh.Hkv;
+  if (S > mkv::kBudgetMaxSegments) return MASKKV_E_UNSUPPORTED;
+  DeviceGuard guard(ctx->device);
+  const size_t smem = sizeof(double) * sh.R + sizeof(int) * S;
+  mkv::budget_kernel<<<1, mkv::kBudgetThreads, smem, static_cast<cudaStream_t>(stream)>>>(
+      sh, k_l, k_l_per_request_dev, alpha, 1.0 - alpha, mass_p_dev, mass_m_dev, (long long)capacity, budgets_dev,
+      offsets_dev, ctx->status_dev);
+  return launch_status();
+}
+
+int maskkv_select(maskkv_ctx* ctx, const maskkv_desc_t* desc, const float* scores_dev, const int32_t* budgets_dev,
+                  const int32_t* offsets_dev, int32_t* kept_idx_dev, void* workspace_dev, size_t workspace_bytes,
+                  void* stream) {
+  (void)workspace_dev; (void)workspace_bytes;
+  if (ctx == nullptr) return MASKKV_E_INVALID;
+  Shape sh;
+  int rc = resolve(desc, &sh);
+  if (rc != MASKKV_OK) return rc;
+  if (scores_dev == nullptr || budgets_dev == nullptr || offsets_dev == nullptr || kept_idx_dev == nullptr) return MASKKV_E_INVALID;
+  DeviceGuard guard(ctx->device);
+  const int max_cache = (ctx->smem_optin - 2048) / 4;
+  const int cache = sh.maxN <= max_cache ? sh.maxN : 0;   // segments that do not fit are read through L2
+  mkv::select_kernel<<<sh.R * sh.Hkv, mkv::kSelectThreads, (size_t)cache * 4, static_cast<cudaStream_t>(stream)>>>(
+      sh, scores_dev, budgets_dev, offsets_dev, kept_idx_dev, cache, ctx->status_dev);
+  return launch_status();
+}
+
+int maskkv_compact(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* k_prompt_dev, const void* v_prompt_dev,
+                   const int32_t* kept_idx_dev, const int32_t* offsets_dev, int64_t capacity, void* kc_dev, void* vc_dev,
+                   void* stream) {
+  if (ctx == nullptr) return MASKKV_E_INVALID;
+  Shape sh;
+  int rc = resolve(desc, &sh);
+  if (rc != MASKKV_OK) return rc;
+  if (kept_idx_dev == nullptr || offsets_dev == nullptr || capacity < 0) return MASKKV_E_INVALID;
+  if (capacity == 0 || sh.sumN == 0) return MASKKV_OK;
+  if (k_prompt_dev == nullptr || v_prompt_dev == nullptr || kc_dev == nullptr || vc_dev == nullptr) return MASKKV_E_INVALID;
+  if (!aligned16(k_prompt_dev) || !aligned16(v_prompt_dev) || !aligned16(kc_dev) || !aligned16(vc_dev)) return MASKKV_E_ALIGN;
+  DeviceGuard guard(ctx->device);
+  const int es = elem_size(sh.dtype);
+  const long long warps = capacity;
+  long long blocks = (warps + (mkv::kCompactThreads / 32) - 1) / (mkv::kCompactThreads / 32);
+  const long long max_blocks = (long long)ctx->sm_count * 8;
+  if (blocks > max_blocks) blocks = max_blocks;
+  mkv::compact_kernel<<<(unsigned)blocks, mkv::kCompactThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      sh, sh.d * es, sh.kv_ts * es, sh.kv_hs * es, static_cast<const unsigned char*>(k_prompt_dev),
+      static_cast<const unsigned char*>(v_prompt_dev), kept_idx_dev, offsets_dev, (long long)capacity,
+      static_cast<unsigned char*>(kc_dev), static_cast<unsigned char*>(vc_dev), ctx->status_dev);
+  return launch_status();
+}
+
+int maskkv_attend(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_live_dev, const void* k_live_dev,
+                  const void* v_live_dev, const void* kc_dev, const void* vc_dev, const int32_t* offsets_dev,
+                  void* out_dev, float* lse_dev, void* stream) {
+  if (ctx == nullptr) return MASKKV_E_INVALID;
+  Shape sh;
+  int rc = resolve(desc, &sh);
+  if (rc != MASKKV_OK) return rc;
+  if (offsets_dev == nullptr) return MASKKV_E_INVALID;
+  if (sh.sumM == 0) return MASKKV_OK;
+  if (q_live_dev == nullptr || k_live_dev == nullptr || v_live_dev == nullptr || out_dev == nullptr) return MASKKV_E_INVALID;
+  if (!aligned16(q_live_dev) || !aligned16(k_live_dev) || !aligned16(v_live_dev) || !aligned16(kc_dev) ||
+      !aligned16(vc_dev) || !aligned16(out_dev))
+    return MASKKV_E_ALIGN;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+#define MKV_ATTEND(T, D) launch_attend_simt<T, D>(sh, q_live_dev, k_live_dev, v_live_dev, kc_dev, vc_dev, offsets_dev, out_dev, lse_dev, st)
+  if (sh.dtype == MASKKV_F32) return sh.d == 64 ? MKV_ATTEND(float, 64) : MKV_ATTEND(float, 128);
+  return sh.d == 64 ? MKV_ATTEND(__nv_bfloat16, 64) : MKV_ATTEND(__nv_bfloat16, 128);
+#undef MKV_ATTEND
+}
+
+#pragma GCC visibility pop
+}  // extern "C"

@@ -1,0 +1,162 @@
+"""GPU edge cases of the C ABI: degenerate segments, clamps, capacity clipping, ties, special values,
+strided inputs and argument validation (a failed validation must launch nothing)."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import maskkv_oracle as O
+from paper_2510_09309_b200 import synth
+from pipeline import ATTEND_ATOL, GpuRun, assert_scores_close, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2510_09309_b200 import binding as B
+    c = B.Context(0)
+    yield c
+    c.close()
+
+
+def _problem(ctx, dtype, H, Hkv, d, lens, M):
+    from paper_2510_09309_b200 import binding as B
+    pcu = np.concatenate([[0], np.cumsum(lens)]).tolist()
+    lcu = [r * M for r in range(len(lens) + 1)]
+    return B.Problem(dtype, H, Hkv, d, pcu, lcu, ctx.device), pcu, lcu
+
+
+def test_select_ties_duplicates_and_special_values(ctx):
+    p, pcu, _ = _problem(ctx, torch.bfloat16, 3, 3, 64, [10, 6, 5, 40000], 4)
+    sc = np.zeros((3, pcu[-1]), np.float32)
+    sc[0, 0:10] = 1.0                                   # all equal -> lowest indices
+    sc[0, 10:16] = [5, 1, 5, 5, 0, 5]                   # duplicates straddling the cut
+    sc[0, 16:21] = [np.nan, 1, -np.inf, 2, np.nan]      # NaN below every number
+    rng = np.random.default_rng(0)
+    sc[0, 21:] = rng.integers(0, 50, 40000) / 7.0       # long segment (beyond the shared-memory cache) with many ties
+    sc[1] = rng.standard_normal(pcu[-1])                # negative values and zeros
+    sc[1, 3] = 0.0; sc[1, 4] = -0.0
+    sc[2] = rng.random(pcu[-1])
+    bud = np.array([[4, 10, 0], [2, 5, 6], [3, 4, 5], [20000, 1, 39999]], np.int32)
+    idx, off = O.select(sc, bud, pcu)
+    kept = torch.full((int(off[-1]) + 8,), -1, dtype=torch.int32, device=ctx.device)
+    ctx.maskkv_select(p, to_dev(sc), to_dev(bud), to_dev(off), kept)
+    torch.cuda.synchronize()
+    assert np.array_equal(kept[:int(off[-1])].cpu().numpy(), idx)
+    assert (kept[int(off[-1]):] == -1).all()
+    assert ctx.maskkv_check_status() == 0
+
+
+def test_budget_clamp_capacity_and_per_request_k(ctx):
+    from paper_2510_09309_b200 import binding as B
+    p, pcu, _ = _problem(ctx, torch.bfloat16, 2, 2, 64, [1000, 40, 1000], 4)
+    mp = np.array([[3, 1], [1, 1], [2, 2]], np.float32); mm = np.array([[1, 3], [1, 1], [2, 2]], np.float32)
+    kl = np.array([100, 50, 10], np.int32)
+    bud = torch.zeros((3, 2), dtype=torch.int32, device=ctx.device); off = torch.zeros(7, dtype=torch.int32, device=ctx.device)
+    for cap in (10 ** 6, 215, 0):
+        ctx.maskkv_budget(p, 0, 0.0, to_dev(mp), to_dev(mm), cap, bud, off, k_l_per_request=to_dev(kl))
+        torch.cuda.synchronize()
+        rb, ro = O.head_budgets(mp, mm, kl, 0.0, [1000, 40, 1000], capacity=cap)
+        assert np.array_equal(bud.cpu().numpy(), rb) and np.array_equal(off.cpu().numpy(), ro)
+        flags = ctx.maskkv_check_status()
+        assert bool(flags & B.MASKKV_FLAG_CAPACITY) == (cap < 290)
+    # golden fixtures through the device kernel
+    from golden_io import head_budget_cases
+    for c in head_budget_cases():
+        Hkv = len(c["expected"])
+        pp, _, _ = _problem(ctx, torch.bfloat16, Hkv, Hkv, 64, [c["n"]], 4)
+        b = torch.zeros((1, Hkv), dtype=torch.int32, device=ctx.device); o = torch.zeros(Hkv + 1, dtype=torch.int32, device=ctx.device)
+        mp32 = np.array([c["mass_p"]], np.float32); mm32 = np.array([c["mass_m"]], np.float32)
+        ctx.maskkv_budget(pp, c["k_l"], c["alpha"], to_dev(mp32), to_dev(mm32), 10 ** 6, b, o)
+        torch.cuda.synchronize()
+        rb, _ = O.head_budgets(mp32, mm32, c["k_l"], c["alpha"], [c["n"]])
+        assert np.array_equal(b.cpu().numpy(), rb)
+
+
+def test_budget_random_bit_exact(ctx):
+    rng = np.random.default_rng(5)
+    for trial in range(20):
+        R, Hkv = int(rng.integers(1, 9)), int(rng.choice([1, 4, 8, 32]))
+        lens = rng.integers(1, 5000, R).tolist()
+        p, _, _ = _problem(ctx, torch.bfloat16, Hkv, Hkv, 128, lens, 8)
+        mp = rng.uniform(0.01, 300, (R, Hkv)).astype(np.float32); mm = rng.uniform(0.01, 300, (R, Hkv)).astype(np.float32)
+        k_l, alpha = int(rng.integers(0, 3000)), float(rng.choice([0.0, 0.1, 0.37, 1.0]))
+        b = torch.zeros((R, Hkv), dtype=torch.int32, device=ctx.device); o = torch.zeros(R * Hkv + 1, dtype=torch.int32, device=ctx.device)
+        ctx.maskkv_budget(p, k_l, alpha, to_dev(mp), to_dev(mm), 2 ** 31 - 1, b, o)
+        torch.cuda.synchronize()
+        rb, ro = O.head_budgets(mp, mm, k_l, alpha, lens)
+        assert np.array_equal(b.cpu().numpy(), rb) and np.array_equal(o.cpu().numpy(), ro)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_empty_and_degenerate_segments(ctx, dtype):
+    """Zero budgets (attend sees only live keys), one-token prompts, a request with one mask row."""
+    wl = synth.scaled(synth.config(2), "degenerate", dtype=dtype, prompt_lens=(1, 257, 31), n_mask=5, n_q_heads=4,
+                      n_kv_heads=2, head_dim=64, mean_budget=0)
+    x = synth.layer_inputs(wl, 0, "cpu"); live = synth.live_inputs(wl, 0, 0, "cpu")
+    xd = {k: to_dev(v) for k, v in x.items() if torch.is_tensor(v)}; ld = {k: to_dev(v) for k, v in live.items()}
+    for k_l in (0, 1, 300):
+        run = GpuRun(ctx, wl, capacity=2000, k_l=k_l)
+        run.score(xd); run.budget(alpha=1.0); run.select(); run.compact(xd); run.attend(ld)
+        torch.cuda.synchronize()
+        sc, mp, mm = O.score(x["q_mask"], x["k_prompt"], x["k_mask"], wl.prompt_cu(), wl.live_cu())
+        assert_scores_close(run.scores.cpu().numpy(), sc)
+        bud, off = O.head_budgets(mp.astype(np.float32), mm.astype(np.float32), k_l, 1.0, wl.prompt_lens)
+        assert np.array_equal(run.budgets.cpu().numpy(), bud)
+        kept = run.kept.cpu().numpy(); offd = run.offsets.cpu().numpy()
+        kc, vc = O.compact(x["k_prompt"], x["v_prompt"], kept, offd, wl.prompt_cu())
+        out, _ = O.attend(live["q_live"], live["k_live"], live["v_live"], kc, vc, offd, wl.live_cu(), wl.n_kv_heads)
+        err = np.abs(run.out.float().cpu().numpy() - out).max()
+        assert err <= ATTEND_ATOL[dtype]
+    assert ctx.maskkv_check_status() == 0
+
+
+def test_strided_inputs(ctx):
+    """Q/K/V taken as views of a fused [tokens, (H + 2 H_kv), d] projection output: non-packed strides."""
+    from paper_2510_09309_b200 import binding as B
+    wl = synth.scaled(synth.config(2), "strided", prompt_lens=(300,), n_mask=64, n_q_heads=4, n_kv_heads=2, mean_budget=32)
+    x = synth.layer_inputs(wl, 0, "cpu")
+    H, Hkv, d, N, M = 4, 2, 128, 300, 64
+    fused_p = torch.zeros(N, H + 2 * Hkv, d, dtype=torch.bfloat16); fused_m = torch.zeros(M, H + 2 * Hkv, d, dtype=torch.bfloat16)
+    fused_p[:, H:H + Hkv] = x["k_prompt"]; fused_m[:, :H] = x["q_mask"]; fused_m[:, H:H + Hkv] = x["k_mask"]
+    fp, fm = to_dev(fused_p), to_dev(fused_m)
+    ts = (H + 2 * Hkv) * d
+    p = B.Problem(torch.bfloat16, H, Hkv, d, [0, N], [0, M], ctx.device, q_strides=(ts, d), kv_strides=(ts, d))
+    scores = torch.zeros((Hkv, N), dtype=torch.float32, device=ctx.device)
+    mp = torch.zeros((1, Hkv), dtype=torch.float32, device=ctx.device); mm = torch.zeros_like(mp)
+    ws = torch.empty(ctx.maskkv_workspace_bytes(p), dtype=torch.uint8, device=ctx.device)
+    ctx.maskkv_score(p, fm, fp[:, H:], fm[:, H:], scores, mp, mm, ws)
+    torch.cuda.synchronize()
+    sc, _, _ = O.score(x["q_mask"], x["k_prompt"], x["k_mask"], [0, N], [0, M])
+    assert_scores_close(scores.cpu().numpy(), sc)
+
+
+def test_validation_launches_nothing(ctx):
+    from paper_2510_09309_b200 import binding as B
+    p, _, _ = _problem(ctx, torch.bfloat16, 4, 2, 128, [64], 8)
+    good = torch.zeros(64 * 2 * 128 + 64, dtype=torch.bfloat16, device=ctx.device)
+    f = torch.zeros(4096, dtype=torch.float32, device=ctx.device)
+    ws = torch.empty(max(ctx.maskkv_workspace_bytes(p), 16), dtype=torch.uint8, device=ctx.device)
+
+    def score_rc(desc, q, k, km, sc, ws_t, ws_bytes):
+        return B.lib.maskkv_score(ctx._h, ctypes.byref(desc), q, k, km, None, sc, f.data_ptr(), f.data_ptr(), ws_t, ws_bytes, None)
+
+    ok = (good.data_ptr(), good.data_ptr(), good.data_ptr(), f.data_ptr(), ws.data_ptr(), ws.numel())
+    assert score_rc(p.desc, ok[0] + 2, *ok[1:]) == B.MASKKV_E_ALIGN
+    assert score_rc(p.desc, None, *ok[1:]) == B.MASKKV_E_INVALID
+    assert score_rc(p.desc, *ok[:4], ws.data_ptr(), 8) == B.MASKKV_E_WORKSPACE
+    assert score_rc(p.desc, *ok[:4], None, 0) == B.MASKKV_E_WORKSPACE
+    for field, val, code in (("head_dim", 96, B.MASKKV_E_UNSUPPORTED), ("dtype", 7, B.MASKKV_E_UNSUPPORTED),
+                             ("n_kv_heads", 3, B.MASKKV_E_INVALID), ("n_requests", 0, B.MASKKV_E_INVALID),
+                             ("kv_token_stride", 100, B.MASKKV_E_ALIGN)):
+        q, _, _ = _problem(ctx, torch.bfloat16, 4, 2, 128, [64], 8)
+        setattr(q.desc, field, val)
+        assert score_rc(q.desc, *ok) == code, field
+    assert B.lib.maskkv_budget(ctx._h, ctypes.byref(p.desc), 10, None, 1.5, f.data_ptr(), f.data_ptr(), 10, f.data_ptr(), f.data_ptr(), None) == B.MASKKV_E_INVALID
+    assert B.lib.maskkv_budget(ctx._h, ctypes.byref(p.desc), -1, None, 0.5, f.data_ptr(), f.data_ptr(), 10, f.data_ptr(), f.data_ptr(), None) == B.MASKKV_E_INVALID
+    assert B.lib.maskkv_select(ctx._h, ctypes.byref(p.desc), None, f.data_ptr(), f.data_ptr(), f.data_ptr(), None, 0, None) == B.MASKKV_E_INVALID
+    assert B.lib.maskkv_attend(None, ctypes.byref(p.desc), *([f.data_ptr()] * 8), None) == B.MASKKV_E_INVALID
+    torch.cuda.synchronize()
+    assert (f == 0).all() and ctx.maskkv_check_status() == 0
