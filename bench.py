@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the MaskKV compress-and-attend path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one transformer layer of the 32k LLaDA-shaped workload (N=32768 prompt keys, M=256 mask
+queries, 32 heads, d=128, bf16, adaptive budgets) through the whole path:
+maskkv_score -> maskkv_budget -> maskkv_select -> maskkv_compact -> maskkv_attend.
+`value` is prompt tokens scored+compacted (and attended once) per second per layer, inputs resident
+in HBM; `e2e` is the same with the layer's inputs in pinned host memory and both copies timed.
+With N > 1 ranks (torchrun) each rank runs its own layers (no data-path collective): weak scaling.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload (rank 0 only).
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch
+
+from paper_2510_09309_b200 import synth
+
+METRIC = "prompt tokens scored+compacted/s per layer at 32k"
+UNIT = "tokens/s"
+RESIDENT_LAYERS = (0, 1, 15, 31)          # layers whose inputs stay resident and are cycled through
+CALLS = ("score", "budget", "select", "compact", "attend")
+
+
+# ----------------------------------------------------------------------------- multi-rank plumbing
+def rank_world():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("LOCAL_RANK", "0"))
+
+
+def shard_layers(n_layers: int, rank: int, world: int):
+    """Layers this rank owns (round-robin): every layer belongs to exactly one rank."""
+    return [l for l in range(n_layers) if l % world == rank]
+
+
+def max_over_ranks(value: float, device=None) -> float:
+    """The slowest rank's time; a no-op without a process group."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(value: float, device=None) -> float:
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.mktemp(prefix="maskkv_clocks_", suffix=".csv")
+        self.proc = None
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        try:
+            for ln in open(self.path):
+                p = [x.strip() for x in ln.split(",")]
+                if len(p) < 9:
+                    continue
+                try:
+                    sm.append(float(p[1])); mx.append(float(p[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ----------------------------------------------------------------------------- our arm
+class LayerBuffers:
+    """Device-side outputs and scratch shared by all layers of the workload (one layer in flight at a time)."""
+
+    def __init__(self, ctx, B, wl, capacity, device):
+        self.p = B.Problem(wl.torch_dtype, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.prompt_cu(), wl.live_cu(), device)
+        R, Hkv, H, d = wl.n_requests, wl.n_kv_heads, wl.n_q_heads, wl.head_dim
+        f32, i32 = torch.float32, torch.int32
+        self.capacity = capacity
+        self.scores = torch.empty((Hkv, self.p.sumN), dtype=f32, device=device)
+        self.mass_p = torch.empty((R, Hkv), dtype=f32, device=device)
+        self.mass_m = torch.empty((R, Hkv), dtype=f32, device=device)
+        self.budgets = torch.empty((R, Hkv), dtype=i32, device=device)
+        self.offsets = torch.zeros(R * Hkv + 1, dtype=i32, device=device)
+        self.kept = torch.empty(capacity, dtype=i32, device=device)
+        self.kc = torch.empty((capacity, d), dtype=wl.torch_dtype, device=device)
+        self.vc = torch.empty((capacity, d), dtype=wl.torch_dtype, device=device)
+        self.out = torch.empty((self.p.sumM, H, d), dtype=wl.torch_dtype, device=device)
+        self.ws = torch.empty(max(ctx.maskkv_workspace_bytes(self.p), 256), dtype=torch.uint8, device=device)
+
+
+def run_layer(ctx, buf, x, live, k_l, alpha, events=None):
+    """The five calls of one layer on the current stream.  `events`: optional list of 6 CUDA events."""
+    p = buf.p
+    if events: events[0].record()
+    ctx.maskkv_score(p, x["q_mask"], x["k_prompt"], x["k_mask"], buf.scores, buf.mass_p, buf.mass_m, buf.ws)
+    if events: events[1].record()
+    ctx.maskkv_budget(p, k_l, alpha, buf.mass_p, buf.mass_m, buf.capacity, buf.budgets, buf.offsets)
+    if events: events[2].record()
+    ctx.maskkv_select(p, buf.scores, buf.budgets, buf.offsets, buf.kept, buf.ws)
+    if events: events[3].record()
+    ctx.maskkv_compact(p, x["k_prompt"], x["v_prompt"], buf.kept, buf.offsets, buf.capacity, buf.kc, buf.vc)
+    if events: events[4].record()
+    ctx.maskkv_attend(p, live["q_live"], live["k_live"], live["v_live"], buf.kc, buf.vc, buf.offsets, buf.out)
+    if events: events[5].record()
+
+
+def algorithmic_work(wl):
+    """Per layer: flops of the one Q K^T product scoring needs, and the bytes each HBM-bound call must move."""
+    N, M, H, d = wl.prompt_lens[0], wl.n_mask, wl.n_q_heads, wl.head_dim
+    return {"score_flops": 2.0 * M * (N + M) * d * H}
+
+
+def bench_ours(args):
+    rank, world, local_rank = rank_world()
+    import torch.distributed as dist
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the MaskKV path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    from paper_2510_09309_b200 import binding as B
+    ctx = B.Context(local_rank)
+
+    wl = synth.config(3)
+    N = wl.prompt_lens[0]
+    k_layers = B.maskkv_layer_budgets(wl.total_budget(), wl.beta, wl.layer_importance())
+    my_layers = shard_layers(wl.n_layers, rank, world)
+    # one rank keeps a boundary/middle mix resident; with several ranks each keeps four of its own layers
+    resident = list(RESIDENT_LAYERS) if world == 1 else (my_layers * 4)[:4]
+    capacity = wl.n_kv_heads * max(k_layers)                      # the host-side bound on rows per layer
+    inputs = [synth.layer_inputs(wl, l, device) for l in resident]
+    lives = [synth.live_inputs(wl, l, 0, device) for l in resident]
+    for x in inputs:
+        x.pop("planted", None); x.pop("v_mask", None)
+    buf = LayerBuffers(ctx, B, wl, capacity, device)
+    torch.cuda.synchronize()
+
+    def step(i, events=None):
+        j = i % len(resident)
+        run_layer(ctx, buf, inputs[j], lives[j], k_layers[resident[j]], wl.alpha, events)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        time.sleep(0.25)
+    per_call = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
+    launches0 = ctx.maskkv_launch_count()
+    barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for i in range(args.steps):
+        step(args.warmup + i, per_call[i])
+    t1.record()
+    barrier()
+    launches = ctx.maskkv_launch_count() - launches0
+    elapsed_ms = max_over_ranks(t0.elapsed_time(t1), device)
+    clocks = sampler.stop() if sampler else {}
+    call_us = {name: 1e3 * statistics.mean(ev[c].elapsed_time(ev[c + 1]) for ev in per_call) for c, name in enumerate(CALLS)}
+    flags = ctx.maskkv_check_status()
+
+    # ---- end to end: the layer's inputs start in pinned host memory, results end in host memory
+    keys_in = ("q_mask", "k_prompt", "v_prompt", "k_mask")
+    keys_live = ("q_live", "k_live", "v_live")
+    host_x = {k: inputs[0][k].cpu().pin_memory() for k in keys_in}
+    host_l = {k: lives[0][k].cpu().pin_memory() for k in keys_live}
+    dev_x = {k: torch.empty_like(inputs[0][k]) for k in keys_in}
+    dev_l = {k: torch.empty_like(lives[0][k]) for k in keys_live}
+    host_out = torch.empty_like(buf.out, device="cpu").pin_memory()
+    host_bud = torch.empty_like(buf.budgets, device="cpu").pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in list(host_x.values()) + list(host_l.values()))
+    d2h = host_out.numel() * host_out.element_size() + host_bud.numel() * host_bud.element_size()
+
+    def e2e_step(i):
+        for k in keys_in:
+            dev_x[k].copy_(host_x[k], non_blocking=True)
+        for k in keys_live:
+            dev_l[k].copy_(host_l[k], non_blocking=True)
+        run_layer(ctx, buf, dev_x, dev_l, k_layers[resident[0]], wl.alpha)
+        host_out.copy_(buf.out, non_blocking=True)
+        host_bud.copy_(buf.budgets, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 20))
+    for i in range(2):
+        e2e_step(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), device)
+
+    if world > 1:
+        dist.destroy_process_group()
+    if rank != 0:
+        return None
+
+    ms_per_step = elapsed_ms / args.steps
+    value = world * N / (ms_per_step * 1e-3)
+    peaks = load_peaks()
+    work = algorithmic_work(wl)
+    score_s = call_us["score"] * 1e-6
+    achieved_tf = work["score_flops"] / score_s / 1e12
+    peak_tf = peaks["bf16_tflops_sustained"]
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "configs[2] llada_stack_32k, one layer per step: N=32768 M=256 H=H_kv=32 d=128, "
+                               "adaptive budgets (k_l 512/238, alpha=0.1)", "layers_resident": len(resident),
+                   "l2": "inputs 545 MB per step > 126 MB L2; resident layers are cycled", "calls": list(CALLS)},
+        "call_us": {k: round(v, 2) for k, v in call_us.items()},
+        "attend_step_us": round(call_us["attend"], 2),
+        "compress_tokens_per_s": N / (1e-6 * (call_us["score"] + call_us["budget"] + call_us["select"] + call_us["compact"])),
+        "e2e": {"value": world * N / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "status_flags": flags,
+        "roofline": {"kernel": "maskkv_score (all its kernels; one Q K^T product counted)", "bound": "tensor",
+                     "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
+                     "peak_source": peaks["source"] + " (sustained bf16)", "traffic": None},
+    }
+    line["cpu_baseline"] = oracle_baseline(wl, budget_s=15.0)
+    return line
+
+
+# ----------------------------------------------------------------------------- peaks and the CPU oracle
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def oracle_sample(wl, n_heads: int, layer: int = 0):
+    """The workload restricted to its first `n_heads` heads (same per-head cost), generated on the CPU."""
+    sub = synth.scaled(wl, wl.name + f"_first{n_heads}heads", n_q_heads=n_heads, n_kv_heads=n_heads, n_layers=wl.n_layers)
+    x = synth.layer_inputs(sub, layer, "cpu")
+    live = synth.live_inputs(sub, layer, 0, "cpu")
+    return sub, x, live
+
+
+def oracle_pass(sub, x, live, k_l):
+    """One pass of the whole path in the CPU oracle (as it stands); returns seconds."""
+    import numpy as np
+    from oracle import maskkv_oracle as O
+    t = time.perf_counter()
+    pcu, lcu = sub.prompt_cu(), sub.live_cu()
+    sc, mp, mm = O.score(x["q_mask"], x["k_prompt"], x["k_mask"], pcu, lcu)
+    bud, off = O.head_budgets(mp.astype(np.float32), mm.astype(np.float32), k_l, sub.alpha, sub.prompt_lens)
+    idx, _ = O.select(sc.astype(np.float32), bud, pcu)
+    kc, vc = O.compact(x["k_prompt"], x["v_prompt"], idx, off, pcu)
+    O.attend(live["q_live"], live["k_live"], live["v_live"], kc, vc, off, lcu, sub.n_kv_heads)
+    return time.perf_counter() - t
+
+
+def oracle_baseline(wl, budget_s: float):
+    """Times the oracle on a bounded sample (a few heads of one layer) and scales to a whole layer."""
+    N, H = wl.prompt_lens[0], wl.n_q_heads
+    sub, x, live = oracle_sample(wl, 1)
+    t1 = oracle_pass(sub, x, live, 238)
+    n_heads = int(max(1, min(H, budget_s / max(t1, 1e-3))))
+    if n_heads > 1:
+        sub, x, live = oracle_sample(wl, n_heads)
+        t = oracle_pass(sub, x, live, 238)
+    else:
+        t = t1
+    return {"value": N / (t * H / n_heads), "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+            "sample": f"{n_heads} of {H} heads of one 32k layer through the whole path (fp64 numpy), {t:.2f} s; "
+                      f"scaled to a full layer by {H}/{n_heads}", "host_cores": os.cpu_count()}
+
+
+def bench_reference(args):
+    rank, world, _ = rank_world()
+    if rank != 0:
+        return None
+    wl = synth.config(3)
+    N, H = wl.prompt_lens[0], wl.n_q_heads
+    n_heads = 1
+    sub, x, live = oracle_sample(wl, n_heads)
+    for _ in range(args.warmup):
+        oracle_pass(sub, x, live, 238)
+    times = [oracle_pass(sub, x, live, 238) for _ in range(args.steps)]
+    t = sum(times) / len(times)
+    value = N / (t * H / n_heads)
+    sample = f"each step = {n_heads} of {H} heads of one 32k layer through the whole path (fp64 numpy oracle); scaled by {H}/{n_heads}"
+    return {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * t * H / n_heads, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "configs[2] llada_stack_32k, one layer per step (sampled)", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 3 if args.steps is None else max(1, args.steps)
+        args.warmup = 1 if args.warmup is None else max(0, args.warmup)
+        line = bench_reference(args)
+    else:
+        args.steps = 40 if args.steps is None else max(1, args.steps)
+        args.warmup = 5 if args.warmup is None else max(3, args.warmup)
+        line = bench_ours(args)
+    if line is not None:
+        print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()

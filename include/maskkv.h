@@ -87,6 +87,10 @@ const char* maskkv_status_string(int code);
  * MASKKV_E_CUDA if the stream reported an error, else MASKKV_OK. */
 int maskkv_check_status(maskkv_ctx* ctx, void* stream, uint32_t* flags_out);
 
+/* Number of kernels this context has launched so far (host counter; for benchmarks and for checking
+ * that a failed validation launched nothing). */
+uint64_t maskkv_launch_count(const maskkv_ctx* ctx);
+
 typedef struct {
   int32_t dtype;              /* MASKKV_F32 | MASKKV_BF16 */
   int32_t n_q_heads;          /* H */

@@ -22,7 +22,8 @@ MASKKV_F32, MASKKV_BF16 = 0, 1
 MASKKV_FLAG_TIMEOUT, MASKKV_FLAG_CAPACITY, MASKKV_FLAG_BOUNDS = 1, 2, 4
 
 EXPORTS = (
-    "maskkv_create", "maskkv_destroy", "maskkv_status_string", "maskkv_check_status", "maskkv_workspace_bytes",
+    "maskkv_create", "maskkv_destroy", "maskkv_status_string", "maskkv_check_status", "maskkv_launch_count",
+    "maskkv_workspace_bytes",
     "maskkv_layer_budgets", "maskkv_score", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend",
 )
 
@@ -57,6 +58,8 @@ def _load() -> C.CDLL:
     lib.maskkv_status_string.argtypes = [C.c_int]
     lib.maskkv_status_string.restype = C.c_char_p
     lib.maskkv_check_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
+    lib.maskkv_launch_count.argtypes = [vp]
+    lib.maskkv_launch_count.restype = C.c_uint64
     lib.maskkv_workspace_bytes.argtypes = [vp, dp]
     lib.maskkv_workspace_bytes.restype = sz
     lib.maskkv_layer_budgets.argtypes = [i64, C.c_double, i32, C.POINTER(C.c_double), C.POINTER(C.c_uint8), C.POINTER(i32)]
@@ -66,7 +69,7 @@ def _load() -> C.CDLL:
     lib.maskkv_compact.argtypes = [vp, dp, vp, vp, vp, vp, i64, vp, vp, vp]
     lib.maskkv_attend.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     for name in EXPORTS:
-        if name not in ("maskkv_status_string", "maskkv_workspace_bytes"):
+        if name not in ("maskkv_status_string", "maskkv_workspace_bytes", "maskkv_launch_count"):
             getattr(lib, name).restype = C.c_int
     return lib
 
@@ -143,6 +146,9 @@ class Context:
             self.close()
         except Exception:
             pass
+
+    def maskkv_launch_count(self) -> int:
+        return int(lib.maskkv_launch_count(self._h))
 
     def maskkv_workspace_bytes(self, p: Problem) -> int:
         return int(lib.maskkv_workspace_bytes(self._h, C.byref(p.desc)))

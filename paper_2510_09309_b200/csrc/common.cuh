@@ -14,6 +14,7 @@ struct maskkv_ctx {
   int smem_optin;          // max opt-in dynamic shared memory per block
   uint32_t* status_dev;    // 256-byte block; word 0 = status flags, word 1 = where a wait gave up
   void* encode_tiled;      // cuTensorMapEncodeTiled, resolved through the runtime
+  unsigned long long launches;  // kernels launched through this context so far
 };
 
 // The descriptor after validation, passed to kernels by value.

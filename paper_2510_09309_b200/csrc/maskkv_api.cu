@@ -86,16 +86,22 @@ ScoreWorkspace score_workspace(const Shape& sh) {
   return w;
 }
 
-inline int launch_status() { return cudaGetLastError() == cudaSuccess ? MASKKV_OK : MASKKV_E_CUDA; }
+// Adds `n` launches to the context's counter and maps the runtime's launch status to a return code.
+inline int launch_status(maskkv_ctx* ctx, int n) {
+  ctx->launches += (unsigned long long)n;
+  return cudaGetLastError() == cudaSuccess ? MASKKV_OK : MASKKV_E_CUDA;
+}
 
 template <typename T, int D>
-int launch_score_simt(const Shape& sh, const ScoreWorkspace& w, const void* q, const void* kp, const void* km,
+int launch_score_simt(maskkv_ctx* ctx, const Shape& sh, const ScoreWorkspace& w, const void* q, const void* kp, const void* km,
                       const float* rw, float* scores, float* mass_p, float* mass_m, unsigned char* ws, cudaStream_t st) {
   float* lse = reinterpret_cast<float*>(ws + w.lse_off);
   float2* part = reinterpret_cast<float2*>(ws + w.part_off);
   float2* mass_part = reinterpret_cast<float2*>(ws + w.mass_off);
   const int S = sh.R * sh.Hkv;
+  int n = 2;
   if (sh.sumM > 0) {
+    n = 4;
     const int q_tiles = (sh.maxM + mkv::kSimtThreads - 1) / mkv::kSimtThreads;
     dim3 g1(w.C, sh.H, sh.R * q_tiles);
     mkv::score_stats_simt<T, D><<<g1, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, part, w.C);
@@ -106,17 +112,17 @@ int launch_score_simt(const Shape& sh, const ScoreWorkspace& w, const void* q, c
   mkv::score_colsum_simt<T, D><<<g2, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, lse, rw,
                                                                   scores, mass_part, w.Tmax);
   mkv::score_mass_reduce<<<(S + 3) / 4, 128, 0, st>>>(S, mass_part, w.Tmax, mass_p, mass_m);
-  return launch_status();
+  return launch_status(ctx, n);
 }
 
 template <typename T, int D>
-int launch_attend_simt(const Shape& sh, const void* q, const void* kl, const void* vl, const void* kc, const void* vc,
+int launch_attend_simt(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kl, const void* vl, const void* kc, const void* vc,
                        const int32_t* offsets, void* out, float* lse, cudaStream_t st) {
   if (sh.maxM == 0) return MASKKV_OK;
   dim3 grid((sh.maxM + mkv::kAttendWarps - 1) / mkv::kAttendWarps, sh.H, sh.R);
   mkv::attend_simt<T, D><<<grid, mkv::kAttendWarps * 32, 0, st>>>(sh, (const T*)q, (const T*)kl, (const T*)vl, (const T*)kc,
                                                                    (const T*)vc, offsets, (T*)out, lse);
-  return launch_status();
+  return launch_status(ctx, 1);
 }
 
 }  // namespace
@@ -186,6 +192,8 @@ int maskkv_check_status(maskkv_ctx* ctx, void* stream, uint32_t* flags_out) {
   return (flags & MASKKV_FLAG_TIMEOUT) ? MASKKV_E_TIMEOUT : MASKKV_OK;
 }
 
+uint64_t maskkv_launch_count(const maskkv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
 size_t maskkv_workspace_bytes(const maskkv_ctx* ctx, const maskkv_desc_t* desc) {
   (void)ctx;
   Shape sh;
@@ -239,7 +247,7 @@ int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_
   DeviceGuard guard(ctx->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   unsigned char* ws = static_cast<unsigned char*>(workspace_dev);
-#define MKV_SCORE(T, D) launch_score_simt<T, D>(sh, w, q_mask_dev, k_prompt_dev, k_mask_dev, row_weights_dev, scores_dev, \
+#define MKV_SCORE(T, D) launch_score_simt<T, D>(ctx, sh, w, q_mask_dev, k_prompt_dev, k_mask_dev, row_weights_dev, scores_dev, \
                                                 mass_p_dev, mass_m_dev, ws, st)
   if (sh.dtype == MASKKV_F32) return sh.d == 64 ? MKV_SCORE(float, 64) : MKV_SCORE(float, 128);
   return sh.d == 64 ? MKV_SCORE(__nv_bfloat16, 64) : MKV_SCORE(__nv_bfloat16, 128);
@@ -262,7 +270,7 @@ int maskkv_budget(maskkv_ctx* ctx, const maskkv_desc_t* desc, int32_t k_l, const
   mkv::budget_kernel<<<1, mkv::kBudgetThreads, smem, static_cast<cudaStream_t>(stream)>>>(
       sh, k_l, k_l_per_request_dev, alpha, 1.0 - alpha, mass_p_dev, mass_m_dev, (long long)capacity, budgets_dev,
       offsets_dev, ctx->status_dev);
-  return launch_status();
+  return launch_status(ctx, 1);
 }
 
 int maskkv_select(maskkv_ctx* ctx, const maskkv_desc_t* desc, const float* scores_dev, const int32_t* budgets_dev,
@@ -279,7 +287,7 @@ int maskkv_select(maskkv_ctx* ctx, const maskkv_desc_t* desc, const float* score
   const int cache = sh.maxN <= max_cache ? sh.maxN : 0;   // segments that do not fit are read through L2
   mkv::select_kernel<<<sh.R * sh.Hkv, mkv::kSelectThreads, (size_t)cache * 4, static_cast<cudaStream_t>(stream)>>>(
       sh, scores_dev, budgets_dev, offsets_dev, kept_idx_dev, cache, ctx->status_dev);
-  return launch_status();
+  return launch_status(ctx, 1);
 }
 
 int maskkv_compact(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* k_prompt_dev, const void* v_prompt_dev,
@@ -303,7 +311,7 @@ int maskkv_compact(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* k_pro
       sh, sh.d * es, sh.kv_ts * es, sh.kv_hs * es, static_cast<const unsigned char*>(k_prompt_dev),
       static_cast<const unsigned char*>(v_prompt_dev), kept_idx_dev, offsets_dev, (long long)capacity,
       static_cast<unsigned char*>(kc_dev), static_cast<unsigned char*>(vc_dev), ctx->status_dev);
-  return launch_status();
+  return launch_status(ctx, 1);
 }
 
 int maskkv_attend(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_live_dev, const void* k_live_dev,
@@ -321,7 +329,7 @@ int maskkv_attend(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_live
     return MASKKV_E_ALIGN;
   DeviceGuard guard(ctx->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-#define MKV_ATTEND(T, D) launch_attend_simt<T, D>(sh, q_live_dev, k_live_dev, v_live_dev, kc_dev, vc_dev, offsets_dev, out_dev, lse_dev, st)
+#define MKV_ATTEND(T, D) launch_attend_simt<T, D>(ctx, sh, q_live_dev, k_live_dev, v_live_dev, kc_dev, vc_dev, offsets_dev, out_dev, lse_dev, st)
   if (sh.dtype == MASKKV_F32) return sh.d == 64 ? MKV_ATTEND(float, 64) : MKV_ATTEND(float, 128);
   return sh.d == 64 ? MKV_ATTEND(__nv_bfloat16, 64) : MKV_ATTEND(__nv_bfloat16, 128);
 #undef MKV_ATTEND
