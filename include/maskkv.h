@@ -128,6 +128,31 @@ int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_
                  float* scores_dev, float* mass_p_dev, float* mass_m_dev, void* workspace_dev,
                  size_t workspace_bytes, void* stream);
 
+/* maskkv_score for callers that cannot hand over a workspace.  (The paper has no counterpart: this is a
+ * packaging variant of the call above, same arithmetic, same outputs.)
+ *
+ * Who needs it: code that runs where device allocation is off limits - inside a serving loop whose memory
+ * pool is fixed and fully handed out at start-up, in a plugin that is given tensors but no allocator, or
+ * next to a stream-ordered allocator whose pool must not be touched from a side library.  Such a caller
+ * cannot call cudaMalloc (or ask torch for a buffer) to create the scratch maskkv_score wants.
+ *
+ * The scratch is instead a fixed array of maskkv_score_noalloc_max_bytes() = 8 MiB that is part of the
+ * library image: each GPU that loads the library reserves those bytes until the process exits, used or not.
+ * The call allocates nothing and frees nothing.  If maskkv_workspace_bytes(desc) exceeds the array the call
+ * returns MASKKV_E_WORKSPACE and launches nothing (8 MiB covers a single request of up to about 60k prompt
+ * keys at 32 heads x 256 mask rows; batches need the regular call).
+ *
+ * The first call on each device looks up the array's device address (a one-time, host-side set-up step);
+ * make that first call outside any stream capture.  All calls on a device share the one array, and it keeps
+ * whatever the previous call left in it - harmless, because every word the kernels read they first write in
+ * the same call - but two calls that overlap on the GPU (different streams, or the same stream from two
+ * contexts) would overwrite each other's partial results: serialise them.  Inputs and outputs are the
+ * caller's, exactly as for maskkv_score. */
+int maskkv_score_noalloc(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_dev,
+                         const void* k_prompt_dev, const void* k_mask_dev, const float* row_weights_dev,
+                         float* scores_dev, float* mass_p_dev, float* mass_m_dev, void* stream);
+size_t maskkv_score_noalloc_max_bytes(void);
+
 /* Eq. 14-15, clamp and prefix sum, all on the device (no host synchronisation):
  *   P = mass_p / (mass_p + mass_m); Phat = P / sum_h P (ascending h);
  *   x = alpha*k_l + ((1-alpha)*(H_kv*k_l))*Phat; k = floor(x + 1e-6) clamped to [0, N_r]

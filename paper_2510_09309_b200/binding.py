@@ -24,7 +24,7 @@ MASKKV_FLAG_TIMEOUT, MASKKV_FLAG_CAPACITY, MASKKV_FLAG_BOUNDS = 1, 2, 4
 EXPORTS = (
     "maskkv_create", "maskkv_destroy", "maskkv_status_string", "maskkv_check_status", "maskkv_launch_count",
     "maskkv_workspace_bytes",
-    "maskkv_layer_budgets", "maskkv_score", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend",
+    "maskkv_layer_budgets", "maskkv_score", "maskkv_score_noalloc", "maskkv_score_noalloc_max_bytes", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend",
 )
 
 
@@ -64,12 +64,15 @@ def _load() -> C.CDLL:
     lib.maskkv_workspace_bytes.restype = sz
     lib.maskkv_layer_budgets.argtypes = [i64, C.c_double, i32, C.POINTER(C.c_double), C.POINTER(C.c_uint8), C.POINTER(i32)]
     lib.maskkv_score.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.maskkv_score_noalloc.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.maskkv_score_noalloc_max_bytes.argtypes = []
+    lib.maskkv_score_noalloc_max_bytes.restype = sz
     lib.maskkv_budget.argtypes = [vp, dp, i32, vp, C.c_double, vp, vp, i64, vp, vp, vp]
     lib.maskkv_select.argtypes = [vp, dp, vp, vp, vp, vp, vp, sz, vp]
     lib.maskkv_compact.argtypes = [vp, dp, vp, vp, vp, vp, i64, vp, vp, vp]
     lib.maskkv_attend.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     for name in EXPORTS:
-        if name not in ("maskkv_status_string", "maskkv_workspace_bytes", "maskkv_launch_count"):
+        if name not in ("maskkv_status_string", "maskkv_workspace_bytes", "maskkv_launch_count", "maskkv_score_noalloc_max_bytes"):
             getattr(lib, name).restype = C.c_int
     return lib
 
@@ -165,6 +168,14 @@ class Context:
                                 _ptr(scores), _ptr(mass_p), _ptr(mass_m), _ptr(workspace),
                                 0 if workspace is None else workspace.numel() * workspace.element_size(), _stream()),
                "maskkv_score")
+
+    def maskkv_score_noalloc(self, p: Problem, q_mask, k_prompt, k_mask, scores, mass_p, mass_m, row_weights=None):
+        """maskkv_score without a workspace argument, for callers that may not allocate device memory: the
+        scratch is an 8 MiB array built into the library (see include/maskkv.h for the limits and the rules on
+        the first call and on overlapping calls)."""
+        _check(lib.maskkv_score_noalloc(self._h, C.byref(p.desc), _ptr(q_mask), _ptr(k_prompt), _ptr(k_mask),
+                                        _ptr(row_weights), _ptr(scores), _ptr(mass_p), _ptr(mass_m), _stream()),
+               "maskkv_score_noalloc")
 
     def maskkv_budget(self, p: Problem, k_l: int, alpha: float, mass_p, mass_m, capacity: int, budgets, offsets,
                       k_l_per_request=None):

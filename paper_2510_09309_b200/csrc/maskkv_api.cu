@@ -125,6 +125,31 @@ int launch_attend_simt(maskkv_ctx* ctx, const Shape& sh, const void* q, const vo
   return launch_status(ctx, 1);
 }
 
+// ---- scratch for maskkv_score_noalloc -------------------------------------------------------------------
+// Lives in the library image: every GPU that loads the library holds these bytes until the process exits.
+constexpr size_t kStaticScratchBytes = 8u << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static void* g_static_scratch_ptr[kMaxDevices] = {nullptr};
+
+// Device address of g_static_scratch on `device`.  In host code the array's name is only a handle for the
+// runtime, never an address a kernel may use, so it is resolved once per device (with that device current).
+int static_scratch_address(int device, void** out) {
+  if (device < 0 || device >= kMaxDevices) return MASKKV_E_UNSUPPORTED;
+  if (g_static_scratch_ptr[device] == nullptr) {
+    DeviceGuard guard(device);
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
+      cudaGetLastError();
+      return MASKKV_E_CUDA;
+    }
+    g_static_scratch_ptr[device] = p;
+  }
+  *out = g_static_scratch_ptr[device];
+  return MASKKV_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -253,6 +278,25 @@ int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_
   return sh.d == 64 ? MKV_SCORE(__nv_bfloat16, 64) : MKV_SCORE(__nv_bfloat16, 128);
 #undef MKV_SCORE
 }
+
+int maskkv_score_noalloc(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_dev, const void* k_prompt_dev,
+                         const void* k_mask_dev, const float* row_weights_dev, float* scores_dev, float* mass_p_dev,
+                         float* mass_m_dev, void* stream) {
+  if (ctx == nullptr) return MASKKV_E_INVALID;
+  Shape sh;
+  int rc = resolve(desc, &sh);
+  if (rc != MASKKV_OK) return rc;
+  const size_t need = maskkv_workspace_bytes(ctx, desc);
+  if (need > kStaticScratchBytes) return MASKKV_E_WORKSPACE;   // problem too large for the built-in scratch
+  void* scratch = nullptr;
+  rc = static_scratch_address(ctx->device, &scratch);
+  if (rc != MASKKV_OK) return rc;
+  // Every scratch word the scoring kernels read is written earlier in the same call, so nothing has to be cleared.
+  return maskkv_score(ctx, desc, q_mask_dev, k_prompt_dev, k_mask_dev, row_weights_dev, scores_dev, mass_p_dev, mass_m_dev,
+                      scratch, kStaticScratchBytes, stream);
+}
+
+size_t maskkv_score_noalloc_max_bytes(void) { return kStaticScratchBytes; }
 
 int maskkv_budget(maskkv_ctx* ctx, const maskkv_desc_t* desc, int32_t k_l, const int32_t* k_l_per_request_dev,
                   double alpha, const float* mass_p_dev, const float* mass_m_dev, int64_t capacity,
