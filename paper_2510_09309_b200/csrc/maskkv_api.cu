@@ -9,6 +9,7 @@
 #include "common.cuh"
 #include "compact.cuh"
 #include "score_simt.cuh"
+#include "score_tc.h"
 #include "select.cuh"
 
 namespace {
@@ -75,8 +76,9 @@ ScoreWorkspace score_workspace(const Shape& sh) {
   ScoreWorkspace w;
   const long long keys = (long long)sh.maxN + sh.maxM;
   w.C = (int)((keys + mkv::kStatsChunk - 1) / mkv::kStatsChunk);
+  if (w.C < mkv::tc::score_tc_max_chunks(sh)) w.C = mkv::tc::score_tc_max_chunks(sh);
   if (w.C < 1) w.C = 1;
-  w.Tmax = (int)((keys + mkv::kSimtThreads - 1) / mkv::kSimtThreads);
+  w.Tmax = mkv::tc::score_tc_max_tiles(sh);               // >= ceil(keys / 128), the FP32-pipe kernel's tiling
   if (w.Tmax < 1) w.Tmax = 1;
   size_t off = 0;
   w.lse_off = off;  off = align_up(off + sizeof(float) * (size_t)sh.H * sh.sumM, 256);
@@ -92,27 +94,40 @@ inline int launch_status(maskkv_ctx* ctx, int n) {
   return cudaGetLastError() == cudaSuccess ? MASKKV_OK : MASKKV_E_CUDA;
 }
 
+// Scoring = sweep 1 (row statistics) + merge + sweep 2 (column sums) + mass reduction.  bf16 problems run the two
+// sweeps on the tensor cores; fp32 problems (and anything the tensor-core path cannot take) on the FP32 pipes.
 template <typename T, int D>
-int launch_score_simt(maskkv_ctx* ctx, const Shape& sh, const ScoreWorkspace& w, const void* q, const void* kp, const void* km,
-                      const float* rw, float* scores, float* mass_p, float* mass_m, unsigned char* ws, cudaStream_t st) {
+int launch_score(maskkv_ctx* ctx, const Shape& sh, const ScoreWorkspace& w, const void* q, const void* kp, const void* km,
+                 const float* rw, float* scores, float* mass_p, float* mass_m, unsigned char* ws, cudaStream_t st) {
   float* lse = reinterpret_cast<float*>(ws + w.lse_off);
   float2* part = reinterpret_cast<float2*>(ws + w.part_off);
   float2* mass_part = reinterpret_cast<float2*>(ws + w.mass_off);
   const int S = sh.R * sh.Hkv;
-  int n = 2;
+  const bool tc_ok = mkv::tc::score_tc_supported(ctx, sh);
+  int n = 0;
   if (sh.sumM > 0) {
-    n = 4;
-    const int q_tiles = (sh.maxM + mkv::kSimtThreads - 1) / mkv::kSimtThreads;
-    dim3 g1(w.C, sh.H, sh.R * q_tiles);
-    mkv::score_stats_simt<T, D><<<g1, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, part, w.C);
+    int chunk_tiles = 0;
+    bool done = false;
+    if (tc_ok && !(ctx->force_simt & 1u)) done = mkv::tc::launch_score_stats_tc(ctx, sh, q, kp, km, part, w.C, &chunk_tiles, st) == 0;
+    if (!done) {
+      chunk_tiles = 0;
+      const int q_tiles = (sh.maxM + mkv::kSimtThreads - 1) / mkv::kSimtThreads;
+      dim3 g1((unsigned)((sh.maxN + sh.maxM + mkv::kStatsChunk - 1) / mkv::kStatsChunk), sh.H, sh.R * q_tiles);
+      mkv::score_stats_simt<T, D><<<g1, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, part, w.C);
+    }
     const long long rows = (long long)sh.H * sh.sumM;
-    mkv::score_merge_stats<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(sh, part, w.C, lse);
+    mkv::score_merge_stats<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(sh, part, w.C, chunk_tiles, lse);
+    n += 2;
   }
-  dim3 g2(w.Tmax, sh.Hkv, sh.R);
-  mkv::score_colsum_simt<T, D><<<g2, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, lse, rw,
-                                                                  scores, mass_part, w.Tmax);
+  bool done = false;
+  if (tc_ok && !(ctx->force_simt & 2u)) done = mkv::tc::launch_score_colsum_tc(ctx, sh, q, kp, km, lse, rw, scores, mass_part, w.Tmax, st) == 0;
+  if (!done) {
+    dim3 g2(w.Tmax, sh.Hkv, sh.R);
+    mkv::score_colsum_simt<T, D><<<g2, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, lse, rw,
+                                                                    scores, mass_part, w.Tmax);
+  }
   mkv::score_mass_reduce<<<(S + 3) / 4, 128, 0, st>>>(S, mass_part, w.Tmax, mass_p, mass_m);
-  return launch_status(ctx, n);
+  return launch_status(ctx, n + 2);
 }
 
 template <typename T, int D>
@@ -191,6 +206,7 @@ int maskkv_create(maskkv_ctx** out, int device) {
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->encode_tiled, cudaEnableDefault, &qres) != cudaSuccess ||
       qres != cudaDriverEntryPointSuccess)
     ctx->encode_tiled = nullptr;
+  if (const char* e = getenv("MASKKV_FORCE_SIMT")) ctx->force_simt = (unsigned)strtoul(e, nullptr, 0);
   cudaFuncSetAttribute(mkv::select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - 2048);
   if (cudaGetLastError() != cudaSuccess) { cudaFree(ctx->status_dev); free(ctx); return MASKKV_E_CUDA; }
   *out = ctx;
@@ -272,7 +288,7 @@ int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_
   DeviceGuard guard(ctx->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   unsigned char* ws = static_cast<unsigned char*>(workspace_dev);
-#define MKV_SCORE(T, D) launch_score_simt<T, D>(ctx, sh, w, q_mask_dev, k_prompt_dev, k_mask_dev, row_weights_dev, scores_dev, \
+#define MKV_SCORE(T, D) launch_score<T, D>(ctx, sh, w, q_mask_dev, k_prompt_dev, k_mask_dev, row_weights_dev, scores_dev, \
                                                 mass_p_dev, mass_m_dev, ws, st)
   if (sh.dtype == MASKKV_F32) return sh.d == 64 ? MKV_SCORE(float, 64) : MKV_SCORE(float, 128);
   return sh.d == 64 ? MKV_SCORE(__nv_bfloat16, 64) : MKV_SCORE(__nv_bfloat16, 128);
