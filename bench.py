@@ -147,7 +147,7 @@ def run_layer(ctx, buf, x, live, k_l, alpha, events=None):
     if events: events[3].record()
     ctx.maskkv_compact(p, x["k_prompt"], x["v_prompt"], buf.kept, buf.offsets, buf.capacity, buf.kc, buf.vc)
     if events: events[4].record()
-    ctx.maskkv_attend(p, live["q_live"], live["k_live"], live["v_live"], buf.kc, buf.vc, buf.offsets, buf.out)
+    ctx.maskkv_attend(p, live["q_live"], live["k_live"], live["v_live"], buf.kc, buf.vc, buf.offsets, buf.capacity, buf.out)
     if events: events[5].record()
 
 

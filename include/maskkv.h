@@ -90,6 +90,8 @@ int maskkv_check_status(maskkv_ctx* ctx, void* stream, uint32_t* flags_out);
 /* Number of kernels this context has launched so far (host counter; for benchmarks and for checking
  * that a failed validation launched nothing). */
 uint64_t maskkv_launch_count(const maskkv_ctx* ctx);
+/* Of those, the launches of tcgen05 (tensor-core) kernels: bf16 scoring sweeps and bf16 attention. */
+uint64_t maskkv_tensor_core_launch_count(const maskkv_ctx* ctx);
 
 typedef struct {
   int32_t dtype;              /* MASKKV_F32 | MASKKV_BF16 */
@@ -183,10 +185,10 @@ int maskkv_compact(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* k_pro
  * softmax of scale * q_i . k over the rows [offsets[s], offsets[s+1]) of kc followed by the request's
  * M_r live keys (no mask, own key included); out = weights x [vc rows ; v_live].  bf16: fp32 accumulation
  * and softmax, weights rounded to bf16 before the second product; f32: fp32 throughout.
- * lse_dev (f32 [H][sum_M]) may be NULL. */
+ * `capacity` is the number of rows kc/vc hold (nothing beyond it is read).  lse_dev (f32 [H][sum_M]) may be NULL. */
 int maskkv_attend(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_live_dev,
                   const void* k_live_dev, const void* v_live_dev, const void* kc_dev, const void* vc_dev,
-                  const int32_t* offsets_dev, void* out_dev, float* lse_dev, void* stream);
+                  const int32_t* offsets_dev, int64_t capacity, void* out_dev, float* lse_dev, void* stream);
 
 #ifdef __cplusplus
 }

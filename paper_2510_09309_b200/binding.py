@@ -23,6 +23,7 @@ MASKKV_FLAG_TIMEOUT, MASKKV_FLAG_CAPACITY, MASKKV_FLAG_BOUNDS = 1, 2, 4
 
 EXPORTS = (
     "maskkv_create", "maskkv_destroy", "maskkv_status_string", "maskkv_check_status", "maskkv_launch_count",
+    "maskkv_tensor_core_launch_count",
     "maskkv_workspace_bytes",
     "maskkv_layer_budgets", "maskkv_score", "maskkv_score_noalloc", "maskkv_score_noalloc_max_bytes", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend",
 )
@@ -60,6 +61,8 @@ def _load() -> C.CDLL:
     lib.maskkv_check_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
     lib.maskkv_launch_count.argtypes = [vp]
     lib.maskkv_launch_count.restype = C.c_uint64
+    lib.maskkv_tensor_core_launch_count.argtypes = [vp]
+    lib.maskkv_tensor_core_launch_count.restype = C.c_uint64
     lib.maskkv_workspace_bytes.argtypes = [vp, dp]
     lib.maskkv_workspace_bytes.restype = sz
     lib.maskkv_layer_budgets.argtypes = [i64, C.c_double, i32, C.POINTER(C.c_double), C.POINTER(C.c_uint8), C.POINTER(i32)]
@@ -70,9 +73,10 @@ def _load() -> C.CDLL:
     lib.maskkv_budget.argtypes = [vp, dp, i32, vp, C.c_double, vp, vp, i64, vp, vp, vp]
     lib.maskkv_select.argtypes = [vp, dp, vp, vp, vp, vp, vp, sz, vp]
     lib.maskkv_compact.argtypes = [vp, dp, vp, vp, vp, vp, i64, vp, vp, vp]
-    lib.maskkv_attend.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.maskkv_attend.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
     for name in EXPORTS:
-        if name not in ("maskkv_status_string", "maskkv_workspace_bytes", "maskkv_launch_count", "maskkv_score_noalloc_max_bytes"):
+        if name not in ("maskkv_status_string", "maskkv_workspace_bytes", "maskkv_launch_count", "maskkv_tensor_core_launch_count",
+                        "maskkv_score_noalloc_max_bytes"):
             getattr(lib, name).restype = C.c_int
     return lib
 
@@ -153,6 +157,9 @@ class Context:
     def maskkv_launch_count(self) -> int:
         return int(lib.maskkv_launch_count(self._h))
 
+    def maskkv_tensor_core_launch_count(self) -> int:
+        return int(lib.maskkv_tensor_core_launch_count(self._h))
+
     def maskkv_workspace_bytes(self, p: Problem) -> int:
         return int(lib.maskkv_workspace_bytes(self._h, C.byref(p.desc)))
 
@@ -191,6 +198,6 @@ class Context:
         _check(lib.maskkv_compact(self._h, C.byref(p.desc), _ptr(k_prompt), _ptr(v_prompt), _ptr(kept_idx), _ptr(offsets),
                                   int(capacity), _ptr(kc), _ptr(vc), _stream()), "maskkv_compact")
 
-    def maskkv_attend(self, p: Problem, q_live, k_live, v_live, kc, vc, offsets, out, lse=None):
+    def maskkv_attend(self, p: Problem, q_live, k_live, v_live, kc, vc, offsets, capacity: int, out, lse=None):
         _check(lib.maskkv_attend(self._h, C.byref(p.desc), _ptr(q_live), _ptr(k_live), _ptr(v_live), _ptr(kc), _ptr(vc),
-                                 _ptr(offsets), _ptr(out), _ptr(lse), _stream()), "maskkv_attend")
+                                 _ptr(offsets), int(capacity), _ptr(out), _ptr(lse), _stream()), "maskkv_attend")

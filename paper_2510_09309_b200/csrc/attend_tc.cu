@@ -1,0 +1,381 @@
+// Attention of a later denoising step over [compacted prompt segment ; live keys] for bf16 inputs on
+// the 5th-generation tensor cores (appendix, proof step 3: out_m = sum_j softmax(q_m k_j / sqrt(d_k)) V_j).
+//
+// One CTA per (128-query tile, query head, request).  Key tiles of 128 rows are walked first over the
+// head's ragged segment of the compacted cache (rows [offsets[s], offsets[s+1]) of kc / vc), then over
+// the request's live rows.  Per tile:
+//     S = Q K^T            tcgen05.mma, operands in shared memory (TMA, 128-byte swizzle), S in tensor memory
+//     P = 2^(S*c - m*c)    one thread per query row: online max / sum in fp32, P rounded to bf16 and
+//                          written back into tensor memory over S
+//     PV = P V             tcgen05.mma with P read from tensor memory and V (row-major, i.e. N-major) from
+//                          shared memory, into a fresh accumulator
+//     O = O*corr + PV      in registers of the row's thread (no rescaling pass over tensor memory)
+// S/P and PV are double-buffered (4 x 128 columns of tensor memory) so the next tile's Q K^T overlaps the
+// softmax.  Columns of a ragged tile's tail are masked to -inf, and the matching V rows are zeroed in
+// shared memory so that stale cache rows can never leak a NaN into the product.
+#include "attend_tc.h"
+
+#include "tc_common.cuh"
+
+namespace mkv {
+namespace tc {
+
+constexpr int kAThreads = 192;         // warp 0: TMA, warp 1: MMA, warps 2-5: softmax (one thread per query row)
+constexpr int kATile = 128;
+constexpr int kAStages = 3;
+constexpr float kALog2e = 1.4426950408889634f;
+
+template <int D>
+struct ASmem {
+  static constexpr int kBoxes = D / 64;
+  static constexpr int kBoxBytes = kATile * 128;
+  static constexpr int kTileBytes = kBoxes * kBoxBytes;
+  static constexpr int kQOff = 0;
+  static constexpr int kKOff = kTileBytes;
+  static constexpr int kVOff = kKOff + kAStages * kTileBytes;
+  static constexpr int kBarOff = kVOff + kAStages * kTileBytes;
+  static constexpr int kNumBars = 1 + 4 * kAStages + 8;
+  static constexpr int kMiscOff = kBarOff + kNumBars * 8;
+  static constexpr int kBytes = kMiscOff + 16;
+  static constexpr int kDynamic = kBytes + 1024;
+};
+
+// Shared-memory descriptor of an N-major (row = k index, 64 contiguous n per 128-byte row) operand with
+// 128-byte swizzle: 8-row groups 1024 bytes apart along k, the next 64 columns `n_stride` bytes away.
+__device__ __forceinline__ uint64_t smem_desc_sw128_nmajor(uint32_t saddr, uint32_t n_stride) {
+  return (uint64_t)((saddr & 0x3ffffu) >> 4) | ((uint64_t)(n_stride >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// bf16 x bf16 -> fp32, A K-major (tensor memory), B N-major.
+__device__ __forceinline__ uint32_t idesc_bf16_f32_bn(uint32_t m, uint32_t n) { return idesc_bf16_f32(m, n) | (1u << 16); }
+
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+      "}\n"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* u) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(u[0]), "r"(u[1]), "r"(u[2]), "r"(u[3]), "r"(u[4]), "r"(u[5]), "r"(u[6]), "r"(u[7]), "r"(u[8]),
+        "r"(u[9]), "r"(u[10]), "r"(u[11]), "r"(u[12]), "r"(u[13]), "r"(u[14]), "r"(u[15]), "r"(u[16]), "r"(u[17]),
+        "r"(u[18]), "r"(u[19]), "r"(u[20]), "r"(u[21]), "r"(u[22]), "r"(u[23]), "r"(u[24]), "r"(u[25]), "r"(u[26]),
+        "r"(u[27]), "r"(u[28]), "r"(u[29]), "r"(u[30]), "r"(u[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+struct ABars {
+  uint64_t* qfull;
+  uint64_t *kfull, *kempty, *vfull, *vempty;   // [kAStages]
+  uint64_t *sfull, *pready, *ofull, *oempty;   // [2]
+};
+__device__ __forceinline__ ABars carve_abars(uint8_t* base, int off) {
+  uint64_t* b = reinterpret_cast<uint64_t*>(base + off);
+  ABars r;
+  r.qfull = b; r.kfull = b + 1; r.kempty = r.kfull + kAStages; r.vfull = r.kempty + kAStages; r.vempty = r.vfull + kAStages;
+  r.sfull = r.vempty + kAStages; r.pready = r.sfull + 2; r.ofull = r.pready + 2; r.oempty = r.ofull + 2;
+  return r;
+}
+
+// Tile j of the key walk: compacted rows first, then live rows.
+struct ATile { bool cache; int row; int valid; };
+__device__ __forceinline__ ATile a_tile(int j, int c0, int nc, int l0, int M) {
+  const int TC = (nc + kATile - 1) / kATile;
+  ATile t;
+  t.cache = j < TC;
+  const int off = (t.cache ? j : j - TC) * kATile;
+  t.row = (t.cache ? c0 : l0) + off;
+  t.valid = min(kATile, (t.cache ? nc : M) - off);
+  return t;
+}
+
+// grid (q tiles, H, R)
+template <int D>
+__global__ void __launch_bounds__(kAThreads, 1)
+attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kl,
+          const __grid_constant__ CUtensorMap map_vl, const __grid_constant__ CUtensorMap map_kc,
+          const __grid_constant__ CUtensorMap map_vc, Shape sh, const int32_t* __restrict__ offsets,
+          __nv_bfloat16* __restrict__ out, float* __restrict__ lse, uint32_t* __restrict__ status) {
+  using S = ASmem<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const ABars bars = carve_abars(base, S::kBarOff);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + S::kMiscOff);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base + S::kMiscOff + 4);
+
+  const int qt = blockIdx.x, h = blockIdx.y, r = blockIdx.z, hk = h / sh.g;
+  const int l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
+  const int q0 = qt * kATile;
+  if (q0 >= M) return;
+  const int seg = r * sh.Hkv + hk;
+  const int c0 = offsets[seg], nc = offsets[seg + 1] - c0;
+  const int nt = (nc + kATile - 1) / kATile + (M + kATile - 1) / kATile;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    mbar_init(bars.qfull, 1);
+    for (int s = 0; s < kAStages; ++s) {
+      mbar_init(bars.kfull + s, 1); mbar_init(bars.kempty + s, 1); mbar_init(bars.vfull + s, 1); mbar_init(bars.vempty + s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bars.sfull + b, 1); mbar_init(bars.pready + b, kATile); mbar_init(bars.ofull + b, 1); mbar_init(bars.oempty + b, kATile);
+    }
+    *abort_flag = 0u;
+    fence_barrier_init();
+  }
+  if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tm_s = tmem_base, tm_o = tmem_base + 256;   // S/P buffers at columns 0 / 128, PV buffers at 256 / 384
+
+  if (warp == 0) {
+    if (lane == 0) {
+      prefetch_tmap(&map_q); prefetch_tmap(&map_kl); prefetch_tmap(&map_vl); prefetch_tmap(&map_kc); prefetch_tmap(&map_vc);
+      mbar_expect_tx(bars.qfull, S::kTileBytes);
+      for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kBoxBytes, &map_q, bars.qfull, b * 64, h, l0 + q0);
+      bool ok = true;
+      int jk = 0, jv = 0;
+      // keys run ahead of values: the Q K^T of tile j+1 is issued before the P V of tile j
+      while (ok && (jk < nt || jv < nt)) {
+        if (jk < nt && jk <= jv + 1) {
+          const int stage = jk % kAStages, use = jk / kAStages;
+          if (!(ok = mbar_wait(bars.kempty + stage, (use & 1) ^ 1, abort_flag, status, 0x301))) break;
+          const ATile t = a_tile(jk, c0, nc, l0, M);
+          mbar_expect_tx(bars.kfull + stage, S::kTileBytes);
+          for (int b = 0; b < S::kBoxes; ++b)
+            tma_load_3d(base + S::kKOff + stage * S::kTileBytes + b * S::kBoxBytes, t.cache ? &map_kc : &map_kl, bars.kfull + stage,
+                        b * 64, t.cache ? 0 : hk, t.row);
+          ++jk;
+        } else {
+          const int stage = jv % kAStages, use = jv / kAStages;
+          if (!(ok = mbar_wait(bars.vempty + stage, (use & 1) ^ 1, abort_flag, status, 0x302))) break;
+          const ATile t = a_tile(jv, c0, nc, l0, M);
+          mbar_expect_tx(bars.vfull + stage, S::kTileBytes);
+          for (int b = 0; b < S::kBoxes; ++b)
+            tma_load_3d(base + S::kVOff + stage * S::kTileBytes + b * S::kBoxBytes, t.cache ? &map_vc : &map_vl, bars.vfull + stage,
+                        b * 64, t.cache ? 0 : hk, t.row);
+          ++jv;
+        }
+      }
+      if (!ok) {   // wait (bounded) for the copies already issued
+        for (int i = max(0, jk - kAStages); i < jk; ++i)
+          for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(bars.kfull + i % kAStages, (i / kAStages) & 1); ++it) __nanosleep(64);
+        for (int i = max(0, jv - kAStages); i < jv; ++i)
+          for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(bars.vfull + i % kAStages, (i / kAStages) & 1); ++it) __nanosleep(64);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc_qk = idesc_bf16_f32(kATile, kATile);
+      const uint32_t idesc_pv = idesc_bf16_f32_bn(kATile, D);
+      const uint32_t q_addr = smem_u32(base + S::kQOff);
+      bool ok = mbar_wait(bars.qfull, 0, abort_flag, status, 0x303);
+      tc_fence_after();
+      auto issue_qk = [&](int j) -> bool {
+        const int stage = j % kAStages, use = j / kAStages;
+        if (!mbar_wait(bars.kfull + stage, use & 1, abort_flag, status, 0x304)) return false;
+        tc_fence_after();
+        const uint32_t k_addr = smem_u32(base + S::kKOff + stage * S::kTileBytes);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint64_t adesc = smem_desc_sw128(q_addr + (kk >> 2) * S::kBoxBytes + (kk & 3) * 32);
+          const uint64_t bdesc = smem_desc_sw128(k_addr + (kk >> 2) * S::kBoxBytes + (kk & 3) * 32);
+          umma_ss(tm_s + (j & 1) * kATile, adesc, bdesc, idesc_qk, kk > 0);
+        }
+        umma_commit(bars.sfull + (j & 1));
+        umma_commit(bars.kempty + stage);
+        return true;
+      };
+      if (ok) ok = issue_qk(0);
+      for (int j = 0; ok && j < nt; ++j) {
+        if (j + 1 < nt && !(ok = issue_qk(j + 1))) break;
+        const int b = j & 1, stage = j % kAStages, use = j / kAStages;
+        if (!(ok = mbar_wait(bars.vfull + stage, use & 1, abort_flag, status, 0x305))) break;
+        if (!(ok = mbar_wait(bars.oempty + b, ((j >> 1) & 1) ^ 1, abort_flag, status, 0x306))) break;
+        if (!(ok = mbar_wait(bars.pready + b, (j >> 1) & 1, abort_flag, status, 0x307))) break;
+        tc_fence_after();
+        const uint32_t v_addr = smem_u32(base + S::kVOff + stage * S::kTileBytes);
+#pragma unroll
+        for (int kk = 0; kk < kATile / 16; ++kk) {
+          const uint64_t bdesc = smem_desc_sw128_nmajor(v_addr + kk * 16 * 128, S::kBoxBytes);
+          umma_ts(tm_o + b * kATile, tm_s + b * kATile + kk * 8, bdesc, idesc_pv, kk > 0);
+        }
+        umma_commit(bars.ofull + b);
+        umma_commit(bars.vempty + stage);
+      }
+    }
+  } else {
+    const int lane_group = warp & 3;
+    const int row = lane_group * 32 + lane;                 // query inside the tile
+    const int tid = (warp - 2) * 32 + lane;                 // 0..127, used for cooperative shared-memory work
+    const uint32_t lane_addr = (uint32_t)(lane_group * 32) << 16;
+    const float cs = sh.scale * kALog2e;
+    float o[D];
+#pragma unroll
+    for (int c = 0; c < D; ++c) o[c] = 0.f;
+    float m = -INFINITY, l = 0.f, corr_prev = 0.f;
+    bool ok = true;
+
+    auto consume_pv = [&](int j, float corr) -> bool {      // O = O*corr + PV(j)
+      const int b = j & 1;
+      if (!mbar_wait(bars.ofull + b, (j >> 1) & 1, abort_flag, status, 0x308)) return false;
+      tc_fence_after();
+#pragma unroll
+      for (int cb = 0; cb < D / 32; ++cb) {
+        float v[32];
+        tmem_ld32(tm_o + lane_addr + b * kATile + cb * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) o[cb * 32 + c] = fmaf(o[cb * 32 + c], corr, v[c]);
+      }
+      tc_fence_before();
+      mbar_arrive(bars.oempty + b);
+      return true;
+    };
+
+    for (int j = 0; ok && j < nt; ++j) {
+      const int b = j & 1;
+      const ATile t = a_tile(j, c0, nc, l0, M);
+      if (t.valid < kATile) {
+        // ragged tail: zero the value rows that do not belong to this tile (every thread clears a slice)
+        const int stage = j % kAStages, use = j / kAStages;
+        if (!(ok = mbar_wait(bars.vfull + stage, use & 1, abort_flag, status, 0x309))) break;
+        uint8_t* v_tile = base + S::kVOff + stage * S::kTileBytes;
+        const int n16 = (kATile - t.valid) * 8;             // 16-byte pieces per box
+        for (int bx = 0; bx < S::kBoxes; ++bx) {
+          uint4* dst = reinterpret_cast<uint4*>(v_tile + bx * S::kBoxBytes + t.valid * 128);
+          for (int e = tid; e < n16; e += kATile) dst[e] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        fence_async_smem();
+      }
+      if (!(ok = mbar_wait(bars.sfull + b, (j >> 1) & 1, abort_flag, status, 0x30a))) break;
+      tc_fence_after();
+      const uint32_t s_addr = tm_s + lane_addr + b * kATile;
+      // pass 1 over the tile: row maximum
+      float tmax = -INFINITY;
+#pragma unroll 1
+      for (int cb = 0; cb < kATile / 32; ++cb) {
+        if (cb * 32 >= t.valid) break;
+        float v[32];
+        tmem_ld32(s_addr + cb * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) if (cb * 32 + c < t.valid) tmax = fmaxf(tmax, v[c]);
+      }
+      const float m_new = fmaxf(m, tmax);
+      const float corr = ex2((m - m_new) * cs);
+      const float neg = -m_new * cs;
+      float rs = 0.f;
+      // pass 2: P = 2^(s*c - m*c), packed to bf16 and written over S (64 packed columns)
+#pragma unroll 1
+      for (int half = 0; half < 2; ++half) {
+        uint32_t packed[32];
+#pragma unroll
+        for (int sub = 0; sub < 2; ++sub) {
+          const int cb = half * 2 + sub;
+          float v[32];
+          if (cb * 32 < t.valid) {
+            tmem_ld32(s_addr + cb * 32, v);
+            tmem_ld_wait();
+          }
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            float p0 = 0.f, p1 = 0.f;
+            if (cb * 32 + c < t.valid) p0 = ex2(fmaf(v[c], cs, neg));
+            if (cb * 32 + c + 1 < t.valid) p1 = ex2(fmaf(v[c + 1], cs, neg));
+            rs += p0 + p1;
+            packed[sub * 16 + c / 2] = pack_bf16(p0, p1);
+          }
+        }
+        // all four chunks of S must be in registers before P overwrites columns 0..63: half 0 writes P columns
+        // 0..31 (keys 0..63) after reading S columns 0..63; half 1 reads S columns 64..127 which P never touches
+        tmem_st32(s_addr + half * 32, packed);
+      }
+      tmem_st_wait();
+      l = l * corr + rs;
+      m = m_new;
+      tc_fence_before();
+      mbar_arrive(bars.pready + b);
+      if (j > 0 && !(ok = consume_pv(j - 1, corr_prev))) break;
+      corr_prev = corr;
+    }
+    if (ok && nt > 0) ok = consume_pv(nt - 1, corr_prev);
+    const int i = q0 + row;
+    if (ok && i < M) {
+      const float inv = 1.f / l;
+      __nv_bfloat16* dst = out + (long long)(l0 + i) * sh.q_ts + (long long)h * sh.q_hs;
+#pragma unroll
+      for (int c = 0; c < D; c += 8) {
+        uint4 w;
+        w.x = pack_bf16(o[c] * inv, o[c + 1] * inv);
+        w.y = pack_bf16(o[c + 2] * inv, o[c + 3] * inv);
+        w.z = pack_bf16(o[c + 4] * inv, o[c + 5] * inv);
+        w.w = pack_bf16(o[c + 6] * inv, o[c + 7] * inv);
+        *reinterpret_cast<uint4*>(dst + c) = w;
+      }
+      if (lse != nullptr) lse[(long long)h * sh.sumM + l0 + i] = m * sh.scale + logf(l);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
+}
+
+namespace {
+template <int D>
+cudaError_t set_attend_attr() {
+  static bool done = false;
+  if (done) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(attend_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, ASmem<D>::kDynamic);
+  done = e == cudaSuccess;
+  return e;
+}
+}  // namespace
+
+bool attend_tc_supported(const maskkv_ctx* ctx, const Shape& sh) {
+  return sh.dtype == MASKKV_BF16 && ctx->encode_tiled != nullptr && sh.sumM > 0 && ctx->smem_optin >= ASmem<128>::kDynamic;
+}
+
+int launch_attend_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kl, const void* vl, const void* kc,
+                     const void* vc, long long cache_rows, const int32_t* offsets, void* out, float* lse, cudaStream_t st) {
+  CUtensorMap mq, mkl, mvl, mkc, mvc;
+  // an empty cache still needs valid maps: point them at the live tensors (no tile of them is ever requested)
+  const void* kc_base = cache_rows > 0 && kc ? kc : kl;
+  const void* vc_base = cache_rows > 0 && vc ? vc : vl;
+  const uint64_t rows = cache_rows > 0 ? (uint64_t)cache_rows : 1;
+  const bool ok = make_tmap_rows(ctx->encode_tiled, &mq, q, sh.d, sh.H, sh.sumM, sh.q_hs * 2, sh.q_ts * 2, kATile) &&
+                  make_tmap_rows(ctx->encode_tiled, &mkl, kl, sh.d, sh.Hkv, sh.sumM, sh.kv_hs * 2, sh.kv_ts * 2, kATile) &&
+                  make_tmap_rows(ctx->encode_tiled, &mvl, vl, sh.d, sh.Hkv, sh.sumM, sh.kv_hs * 2, sh.kv_ts * 2, kATile) &&
+                  make_tmap_rows(ctx->encode_tiled, &mkc, kc_base, sh.d, 1, rows, (uint64_t)sh.d * 2, (uint64_t)sh.d * 2, kATile) &&
+                  make_tmap_rows(ctx->encode_tiled, &mvc, vc_base, sh.d, 1, rows, (uint64_t)sh.d * 2, (uint64_t)sh.d * 2, kATile);
+  if (!ok) return 1;
+  dim3 grid((sh.maxM + kATile - 1) / kATile, sh.H, sh.R);
+  if (sh.d == 128) {
+    if (set_attend_attr<128>() != cudaSuccess) return 1;
+    attend_tc<128><<<grid, kAThreads, ASmem<128>::kDynamic, st>>>(mq, mkl, mvl, mkc, mvc, sh, offsets, (__nv_bfloat16*)out, lse,
+                                                                  ctx->status_dev);
+  } else {
+    if (set_attend_attr<64>() != cudaSuccess) return 1;
+    attend_tc<64><<<grid, kAThreads, ASmem<64>::kDynamic, st>>>(mq, mkl, mvl, mkc, mvc, sh, offsets, (__nv_bfloat16*)out, lse,
+                                                                ctx->status_dev);
+  }
+  return 0;
+}
+
+}  // namespace tc
+}  // namespace mkv

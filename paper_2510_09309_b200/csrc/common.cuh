@@ -15,6 +15,7 @@ struct maskkv_ctx {
   uint32_t* status_dev;    // 256-byte block; word 0 = status flags, word 1 = where a wait gave up
   void* encode_tiled;      // cuTensorMapEncodeTiled, resolved through the runtime
   unsigned long long launches;  // kernels launched through this context so far
+  unsigned long long tc_launches;  // of those, kernels of the tcgen05 (tensor-core) paths
   unsigned force_simt;     // debugging: bit 0 = scoring sweep 1, bit 1 = scoring sweep 2, bit 2 = attention on the FP32 pipes
 };
 

@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include "attend_simt.cuh"
+#include "attend_tc.h"
 #include "budget.cuh"
 #include "common.cuh"
 #include "compact.cuh"
@@ -109,6 +110,7 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const ScoreWorkspace& w, cons
     int chunk_tiles = 0;
     bool done = false;
     if (tc_ok && !(ctx->force_simt & 1u)) done = mkv::tc::launch_score_stats_tc(ctx, sh, q, kp, km, part, w.C, &chunk_tiles, st) == 0;
+    if (done) ++ctx->tc_launches;
     if (!done) {
       chunk_tiles = 0;
       const int q_tiles = (sh.maxM + mkv::kSimtThreads - 1) / mkv::kSimtThreads;
@@ -121,6 +123,7 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const ScoreWorkspace& w, cons
   }
   bool done = false;
   if (tc_ok && !(ctx->force_simt & 2u)) done = mkv::tc::launch_score_colsum_tc(ctx, sh, q, kp, km, lse, rw, scores, mass_part, w.Tmax, st) == 0;
+  if (done) ++ctx->tc_launches;
   if (!done) {
     dim3 g2(w.Tmax, sh.Hkv, sh.R);
     mkv::score_colsum_simt<T, D><<<g2, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, lse, rw,
@@ -234,6 +237,7 @@ int maskkv_check_status(maskkv_ctx* ctx, void* stream, uint32_t* flags_out) {
 }
 
 uint64_t maskkv_launch_count(const maskkv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+uint64_t maskkv_tensor_core_launch_count(const maskkv_ctx* ctx) { return ctx ? ctx->tc_launches : 0; }
 
 size_t maskkv_workspace_bytes(const maskkv_ctx* ctx, const maskkv_desc_t* desc) {
   (void)ctx;
@@ -376,12 +380,12 @@ int maskkv_compact(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* k_pro
 
 int maskkv_attend(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_live_dev, const void* k_live_dev,
                   const void* v_live_dev, const void* kc_dev, const void* vc_dev, const int32_t* offsets_dev,
-                  void* out_dev, float* lse_dev, void* stream) {
+                  int64_t capacity, void* out_dev, float* lse_dev, void* stream) {
   if (ctx == nullptr) return MASKKV_E_INVALID;
   Shape sh;
   int rc = resolve(desc, &sh);
   if (rc != MASKKV_OK) return rc;
-  if (offsets_dev == nullptr) return MASKKV_E_INVALID;
+  if (offsets_dev == nullptr || capacity < 0) return MASKKV_E_INVALID;
   if (sh.sumM == 0) return MASKKV_OK;
   if (q_live_dev == nullptr || k_live_dev == nullptr || v_live_dev == nullptr || out_dev == nullptr) return MASKKV_E_INVALID;
   if (!aligned16(q_live_dev) || !aligned16(k_live_dev) || !aligned16(v_live_dev) || !aligned16(kc_dev) ||
@@ -389,6 +393,12 @@ int maskkv_attend(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_live
     return MASKKV_E_ALIGN;
   DeviceGuard guard(ctx->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (mkv::tc::attend_tc_supported(ctx, sh) && !(ctx->force_simt & 4u) &&
+      mkv::tc::launch_attend_tc(ctx, sh, q_live_dev, k_live_dev, v_live_dev, kc_dev, vc_dev, capacity, offsets_dev, out_dev,
+                                lse_dev, st) == 0) {
+    ++ctx->tc_launches;
+    return launch_status(ctx, 1);
+  }
 #define MKV_ATTEND(T, D) launch_attend_simt<T, D>(ctx, sh, q_live_dev, k_live_dev, v_live_dev, kc_dev, vc_dev, offsets_dev, out_dev, lse_dev, st)
   if (sh.dtype == MASKKV_F32) return sh.d == 64 ? MKV_ATTEND(float, 64) : MKV_ATTEND(float, 128);
   return sh.d == 64 ? MKV_ATTEND(__nv_bfloat16, 64) : MKV_ATTEND(__nv_bfloat16, 128);

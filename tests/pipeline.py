@@ -67,8 +67,8 @@ class GpuRun:
 
     def attend(self, live, kc=None, vc=None, offsets=None):
         self.ctx.maskkv_attend(self.p, live["q_live"], live["k_live"], live["v_live"], self.kc if kc is None else kc,
-                               self.vc if vc is None else vc, self.offsets if offsets is None else offsets, self.out,
-                               self.lse)
+                               self.vc if vc is None else vc, self.offsets if offsets is None else offsets,
+                               (self.kc if kc is None else kc).shape[0], self.out, self.lse)
 
 
 def oracle_layer(wl: synth.Workload, x, live, k_l: int, alpha: float, heads: Optional[Sequence[int]] = None):

@@ -157,6 +157,6 @@ def test_validation_launches_nothing(ctx):
     assert B.lib.maskkv_budget(ctx._h, ctypes.byref(p.desc), 10, None, 1.5, f.data_ptr(), f.data_ptr(), 10, f.data_ptr(), f.data_ptr(), None) == B.MASKKV_E_INVALID
     assert B.lib.maskkv_budget(ctx._h, ctypes.byref(p.desc), -1, None, 0.5, f.data_ptr(), f.data_ptr(), 10, f.data_ptr(), f.data_ptr(), None) == B.MASKKV_E_INVALID
     assert B.lib.maskkv_select(ctx._h, ctypes.byref(p.desc), None, f.data_ptr(), f.data_ptr(), f.data_ptr(), None, 0, None) == B.MASKKV_E_INVALID
-    assert B.lib.maskkv_attend(None, ctypes.byref(p.desc), *([f.data_ptr()] * 8), None) == B.MASKKV_E_INVALID
+    assert B.lib.maskkv_attend(None, ctypes.byref(p.desc), *([f.data_ptr()] * 6), 16, f.data_ptr(), f.data_ptr(), None) == B.MASKKV_E_INVALID
     torch.cuda.synchronize()
     assert (f == 0).all() and ctx.maskkv_check_status() == 0

@@ -167,6 +167,15 @@ def test_chain_on_device(case):
         assert err2 <= ATTEND_ATOL[wl.dtype]
 
 
+def test_bf16_runs_on_the_tensor_core_kernels(case, ctx):
+    """bf16 scoring (two sweeps) and attention must be served by the tcgen05 kernels, fp32 by the FP32 pipes."""
+    run = case["run"]
+    before = ctx.maskkv_tensor_core_launch_count()
+    run.score(case["xd"]); run.attend(case["ld"])
+    torch.cuda.synchronize()
+    assert ctx.maskkv_tensor_core_launch_count() - before == (3 if case["wl"].dtype == "bf16" else 0)
+
+
 def test_full_budget_equals_full_attention(ctx):
     """k >= N for every head: attention over the compacted cache equals attention over the original K/V."""
     wl = synth.scaled(synth.config(2), "full_budget", prompt_lens=(200, 64), n_mask=48, n_q_heads=4, n_kv_heads=2,
