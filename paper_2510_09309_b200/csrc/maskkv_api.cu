@@ -84,7 +84,7 @@ ScoreWorkspace score_workspace(const Shape& sh) {
   size_t off = 0;
   w.lse_off = off;  off = align_up(off + sizeof(float) * (size_t)sh.H * sh.sumM, 256);
   w.part_off = off; off = align_up(off + sizeof(float2) * (size_t)sh.H * sh.sumM * w.C, 256);
-  w.mass_off = off; off = align_up(off + sizeof(float2) * (size_t)sh.R * sh.Hkv * w.Tmax, 256);
+  w.mass_off = off; off = align_up(off + sizeof(float2) * (size_t)sh.R * sh.Hkv * w.Tmax * 4, 256);
   w.total = off;
   return w;
 }
@@ -98,8 +98,9 @@ inline int launch_status(maskkv_ctx* ctx, int n) {
 // Scoring = sweep 1 (row statistics) + merge + sweep 2 (column sums) + mass reduction.  bf16 problems run the two
 // sweeps on the tensor cores; fp32 problems (and anything the tensor-core path cannot take) on the FP32 pipes.
 template <typename T, int D>
-int launch_score(maskkv_ctx* ctx, const Shape& sh, const ScoreWorkspace& w, const void* q, const void* kp, const void* km,
-                 const float* rw, float* scores, float* mass_p, float* mass_m, unsigned char* ws, cudaStream_t st) {
+int launch_score(maskkv_ctx* ctx, const Shape& sh, const ScoreWorkspace& w, bool any_without_voters, const void* q,
+                 const void* kp, const void* km, const float* rw, float* scores, float* mass_p, float* mass_m,
+                 unsigned char* ws, cudaStream_t st) {
   float* lse = reinterpret_cast<float*>(ws + w.lse_off);
   float2* part = reinterpret_cast<float2*>(ws + w.part_off);
   float2* mass_part = reinterpret_cast<float2*>(ws + w.mass_off);
@@ -122,14 +123,16 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const ScoreWorkspace& w, cons
     n += 2;
   }
   bool done = false;
-  if (tc_ok && !(ctx->force_simt & 2u)) done = mkv::tc::launch_score_colsum_tc(ctx, sh, q, kp, km, lse, rw, scores, mass_part, w.Tmax, st) == 0;
-  if (done) ++ctx->tc_launches;
+  if (tc_ok && !(ctx->force_simt & 2u)) {
+    done = mkv::tc::launch_score_colsum_tc(ctx, sh, q, kp, km, lse, rw, scores, mass_part, w.Tmax, any_without_voters, st) == 0;
+    if (done) { ++ctx->tc_launches; n += any_without_voters ? 1 : 0; }
+  }
   if (!done) {
     dim3 g2(w.Tmax, sh.Hkv, sh.R);
     mkv::score_colsum_simt<T, D><<<g2, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, lse, rw,
                                                                     scores, mass_part, w.Tmax);
   }
-  mkv::score_mass_reduce<<<(S + 3) / 4, 128, 0, st>>>(S, mass_part, w.Tmax, mass_p, mass_m);
+  mkv::score_mass_reduce<<<(S + 3) / 4, 128, 0, st>>>(sh, mass_part, w.Tmax, mass_p, mass_m);
   return launch_status(ctx, n + 2);
 }
 
@@ -292,7 +295,9 @@ int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_
   DeviceGuard guard(ctx->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   unsigned char* ws = static_cast<unsigned char*>(workspace_dev);
-#define MKV_SCORE(T, D) launch_score<T, D>(ctx, sh, w, q_mask_dev, k_prompt_dev, k_mask_dev, row_weights_dev, scores_dev, \
+  bool any_without_voters = false;
+  for (int r = 0; r < sh.R; ++r) any_without_voters |= desc->live_cu[r + 1] == desc->live_cu[r];
+#define MKV_SCORE(T, D) launch_score<T, D>(ctx, sh, w, any_without_voters, q_mask_dev, k_prompt_dev, k_mask_dev, row_weights_dev, scores_dev, \
                                                 mass_p_dev, mass_m_dev, ws, st)
   if (sh.dtype == MASKKV_F32) return sh.d == 64 ? MKV_SCORE(float, 64) : MKV_SCORE(float, 128);
   return sh.d == 64 ? MKV_SCORE(__nv_bfloat16, 64) : MKV_SCORE(__nv_bfloat16, 128);

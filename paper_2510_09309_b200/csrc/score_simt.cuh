@@ -87,7 +87,7 @@ score_stats_simt(Shape sh, const T* __restrict__ q, const T* __restrict__ kp, co
 }
 
 // One thread per (h, row): lse[h*sumM + row] = ln sum_j exp(s_j).  chunk_tiles = 0: partials cover kStatsChunk
-// keys each; otherwise they cover chunk_tiles 128-key tiles of the [prompt tiles ; mask tiles] order.
+// keys each; otherwise each chunk of chunk_tiles 128-key tiles of the [prompt tiles ; mask tiles] order has two.
 __global__ void score_merge_stats(Shape sh, const float2* __restrict__ part, int C, int chunk_tiles, float* __restrict__ lse) {
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= (long long)sh.H * sh.sumM) return;
@@ -95,7 +95,7 @@ __global__ void score_merge_stats(Shape sh, const float2* __restrict__ part, int
   const int r = find_request(sh.live_cu, sh.R, row);
   const int N = sh.prompt_cu[r + 1] - sh.prompt_cu[r], M = sh.live_cu[r + 1] - sh.live_cu[r];
   const int tiles = (N + 127) / 128 + (M + 127) / 128;
-  const int chunks = chunk_tiles > 0 ? (tiles + chunk_tiles - 1) / chunk_tiles : (N + M + kStatsChunk - 1) / kStatsChunk;
+  const int chunks = chunk_tiles > 0 ? 2 * ((tiles + chunk_tiles - 1) / chunk_tiles) : (N + M + kStatsChunk - 1) / kStatsChunk;
   const float2* p = part + t * C;
   float m = -INFINITY;
   for (int c = 0; c < chunks; ++c) m = fmaxf(m, p[c].x);
@@ -104,7 +104,8 @@ __global__ void score_merge_stats(Shape sh, const float2* __restrict__ part, int
   lse[t] = m + logf(l);
 }
 
-// grid (key tiles, H_kv, R); block kSimtThreads.  mass_part[(s*T + tile)] = (prompt sum, mask sum), s = r*H_kv + hk.
+// grid (key tiles, H_kv, R); block kSimtThreads.  mass_part[(s*Tmax + tile)*4 + slot] = (prompt sum, mask sum),
+// s = r*H_kv + hk; this kernel puts the tile's total in slot 0 (the tensor-core kernel fills one slot per warp).
 template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads)
 score_colsum_simt(Shape sh, const T* __restrict__ q, const T* __restrict__ kp, const T* __restrict__ km,
@@ -116,11 +117,9 @@ score_colsum_simt(Shape sh, const T* __restrict__ q, const T* __restrict__ kp, c
   const int tile = blockIdx.x, hk = blockIdx.y, r = blockIdx.z;
   const int p0 = sh.prompt_cu[r], N = sh.prompt_cu[r + 1] - p0;
   const int l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
-  float2* mp = mass_part + ((long long)(r * sh.Hkv + hk) * Tmax + tile);
-  if (tile * kSimtThreads >= N + M) {                  // beyond this request's keys (uniform)
-    if (threadIdx.x == 0) *mp = make_float2(0.f, 0.f);
-    return;
-  }
+  float2* mp = mass_part + ((long long)(r * sh.Hkv + hk) * Tmax + tile) * 4;
+  if (threadIdx.x < 4) mp[threadIdx.x] = make_float2(0.f, 0.f);
+  if (tile * kSimtThreads >= N + M) return;            // beyond this request's keys (uniform)
   const int j = tile * kSimtThreads + threadIdx.x;
   const bool valid = j < N + M;
   float kreg[D];
@@ -166,15 +165,18 @@ score_colsum_simt(Shape sh, const T* __restrict__ q, const T* __restrict__ kp, c
   }
 }
 
-// One warp per segment s: fixed-order sum of the tile partials.
-__global__ void score_mass_reduce(int S, const float2* __restrict__ mass_part, int Tmax,
+// One warp per segment s: fixed-order sum of the tile partials (4 slots per tile) of the request's own tiles.
+__global__ void score_mass_reduce(Shape sh, const float2* __restrict__ mass_part, int Tmax,
                                   float* __restrict__ mass_p, float* __restrict__ mass_m) {
   const int s = blockIdx.x * (blockDim.x / 32) + (threadIdx.x >> 5);
-  if (s >= S) return;
+  if (s >= sh.R * sh.Hkv) return;
   const int lane = threadIdx.x & 31;
+  const int r = s / sh.Hkv;
+  const int N = sh.prompt_cu[r + 1] - sh.prompt_cu[r], M = sh.live_cu[r + 1] - sh.live_cu[r];
+  const int entries = ((N + 127) / 128 + (M + 127) / 128) * 4;
   float a = 0.f, b = 0.f;
-  for (int t = lane; t < Tmax; t += 32) {
-    const float2 v = mass_part[(long long)s * Tmax + t];
+  for (int t = lane; t < entries; t += 32) {
+    const float2 v = mass_part[(long long)s * Tmax * 4 + t];
     a += v.x;
     b += v.y;
   }

@@ -6,16 +6,19 @@
 //
 //   sweep 1  score_stats_tc   queries on the TMEM lanes (A = 128-query tile, B = 128-key tile): the thread
 //                             that owns a lane owns a softmax row and keeps its running (max, sum of exp).
-//                             A CTA covers 256 queries (two accumulators) x one chunk of key tiles and
-//                             writes one partial per row; a tiny kernel merges the partials into lse_i.
+//                             A unit covers 256 queries (two accumulators) x one chunk of key tiles and
+//                             yields one partial per row; a tiny kernel merges the partials into lse_i.
 //   sweep 2  score_colsum_tc  keys on the TMEM lanes (A = 128-key tile, B = up to 256 queries): the owning
 //                             thread reads its key's logits against every query, forms
 //                             A_ij = 2^(s_ij*c - lse2_i) and sums over i in a register - the column sum
 //                             needs no cross-thread reduction.
 //
-// Both kernels are warp-specialised: warp 0 issues TMA loads (4-stage ring of key tiles), warp 1 issues
-// the MMAs, warps 2-9 are two epilogue warpgroups working on alternate accumulators so that the tensor
-// pipe and the exponentials overlap.  Tensor memory: 512 columns = 2 x 256 (sweep 2) or 4 x 128 (sweep 1).
+// Both kernels are persistent (one CTA per SM walks a strided list of units, its TMA / MMA / epilogue
+// pipelines running on across unit boundaries) and warp-specialised: warp 0 issues TMA loads (4-stage
+// ring of key tiles), warp 1 issues the MMAs, warps 2-17 are four epilogue warpgroups - two per
+// accumulator, each taking half of its columns - so that every scheduler has four warps of
+// exponentials to interleave while the tensor pipe fills the other accumulator.  Tensor memory: 512 columns
+// = 2 x 256 (sweep 2) or 4 x 128 (sweep 1).  Both sweeps are bound by the exponential (MUFU) rate.
 #include "score_tc.h"
 
 #include "tc_common.cuh"
@@ -23,11 +26,12 @@
 namespace mkv {
 namespace tc {
 
-constexpr int kThreads = 320;          // 10 warps: TMA, MMA, 2 x 4 epilogue
+constexpr int kThreads = 576;          // 18 warps: TMA, MMA, 4 x 4 epilogue
+constexpr int kEpiThreadsPerAcc = 256; // two epilogue warpgroups share one accumulator
 constexpr int kStages = 4;
 constexpr int kTile = 128;             // keys per tile (both sweeps), queries per accumulator (sweep 1)
 constexpr int kQBlock = 256;           // queries resident per CTA
-constexpr int kColsumMaxTiles = 16;    // key tiles per CTA in sweep 2 (bounded by the shared-memory accumulators)
+constexpr int kColsumMaxTiles = 16;    // key tiles per unit in sweep 2 (bounded by the shared-memory accumulators)
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int D>
@@ -40,9 +44,9 @@ struct Smem {
   static constexpr int kQOff = 0;
   static constexpr int kKOff = kQBytes;
   static constexpr int kAccOff = kKOff + kStages * kKBytes;               // float [kColsumMaxTiles][128]
-  static constexpr int kC2Off = kAccOff + kColsumMaxTiles * kTile * 4;     // float [2][256]
-  static constexpr int kRedOff = kC2Off + 2 * kQBlock * 4;                 // float [8]
-  static constexpr int kBarOff = kRedOff + 64;                             // mbarriers
+  static constexpr int kC2Off = kAccOff + kColsumMaxTiles * kTile * 4;     // float [4 warpgroups][2][128]
+  static constexpr int kXchOff = kC2Off + 4 * kQBlock * 4;                 // float [2 accumulators][2][128]
+  static constexpr int kBarOff = kXchOff + 4 * kTile * 4;                  // mbarriers
   static constexpr int kNumBars = 2 * kStages + 2 + 4 + 4;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;                  // tmem base, abort flag
   static constexpr int kBytes = kMiscOff + 16;
@@ -90,39 +94,12 @@ __device__ __forceinline__ KeyTile key_tile(int t, int p0, int N, int l0, int M)
   return k;
 }
 
-// =====================================================================================================
-// sweep 1: per-row (max, sum of exp) over one chunk of key tiles.
-// grid (chunks, H, R * q_pairs); part[(h*sumM + row)*C + chunk] = (max of scaled logits, sum of exp).
-// =====================================================================================================
-template <int D>
-__global__ void __launch_bounds__(kThreads, 1)
-score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kp,
-               const __grid_constant__ CUtensorMap map_km, Shape sh, float2* __restrict__ part, int C, int chunk_tiles,
-               uint32_t* __restrict__ status) {
-  using S = Smem<D>;
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* base = align_1024(smem_raw);
-  const Bars bars = carve_bars(base, S::kBarOff);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + S::kMiscOff);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base + S::kMiscOff + 4);
-
-  const int q_pairs = (sh.maxM + kQBlock - 1) / kQBlock;
-  const int chunk = blockIdx.x, h = blockIdx.y, r = blockIdx.z / q_pairs, qp = blockIdx.z % q_pairs;
-  const int hk = h / sh.g;
-  const int p0 = sh.prompt_cu[r], N = sh.prompt_cu[r + 1] - p0;
-  const int l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
-  const int T = (N + kTile - 1) / kTile + (M + kTile - 1) / kTile;
-  const int q0 = qp * kQBlock;
-  const int t_begin = chunk * chunk_tiles, t_end = min(t_begin + chunk_tiles, T);
-  if (q0 >= M || t_begin >= t_end) return;                 // nothing to do (uniform for the block)
-  const int n_qtiles = (M - q0 > kTile) ? 2 : 1;
-  const int nt = t_end - t_begin;
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+__device__ __forceinline__ void block_setup(const Bars& bars, int n_acc, uint32_t* tmem_slot, volatile uint32_t* abort_flag) {
+  const int warp = threadIdx.x >> 5;
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(bars.full + s, 1); mbar_init(bars.empty + s, 1); }
     mbar_init(bars.qfull, 1); mbar_init(bars.qempty, 1);
-    for (int b = 0; b < 4; ++b) { mbar_init(bars.tfull + b, 1); mbar_init(bars.tempty + b, kTile); }
+    for (int b = 0; b < n_acc; ++b) { mbar_init(bars.tfull + b, 1); mbar_init(bars.tempty + b, kEpiThreadsPerAcc); }
     *abort_flag = 0u;
     fence_barrier_init();
   }
@@ -130,238 +107,304 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+}
+
+__device__ __forceinline__ void block_teardown(uint32_t tmem_base) {
+  tc_fence_before();
+  __syncthreads();
+  if ((threadIdx.x >> 5) == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
+}
+
+// =====================================================================================================
+// sweep 1: per-row (max, sum of exp) over one chunk of key tiles.
+// unit u -> (chunk, h, r, query pair); part[(h*sumM + row)*C + chunk] = (max of scaled logits, sum of exp).
+// =====================================================================================================
+struct StatsUnit { int chunk, h, hk, p0, N, l0, M, q0, t_begin, nt, n_qtiles; bool valid; };
+
+__device__ __forceinline__ StatsUnit stats_unit(const Shape& sh, int u, int chunks, int chunk_tiles) {
+  StatsUnit s;
+  const int q_pairs = (sh.maxM + kQBlock - 1) / kQBlock;
+  s.chunk = u % chunks;
+  s.h = (u / chunks) % sh.H;
+  const int z = u / (chunks * sh.H);
+  const int r = z / q_pairs;
+  s.hk = s.h / sh.g;
+  s.p0 = sh.prompt_cu[r]; s.N = sh.prompt_cu[r + 1] - s.p0;
+  s.l0 = sh.live_cu[r]; s.M = sh.live_cu[r + 1] - s.l0;
+  s.q0 = (z % q_pairs) * kQBlock;
+  const int T = (s.N + kTile - 1) / kTile + (s.M + kTile - 1) / kTile;
+  s.t_begin = s.chunk * chunk_tiles;
+  s.nt = min(s.t_begin + chunk_tiles, T) - s.t_begin;
+  s.valid = s.q0 < s.M && s.nt > 0;
+  s.n_qtiles = (s.M - s.q0 > kTile) ? 2 : 1;
+  return s;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kp,
+               const __grid_constant__ CUtensorMap map_km, Shape sh, float2* __restrict__ part, int C, int chunks,
+               int chunk_tiles, int n_units, uint32_t* __restrict__ status) {
+  using S = Smem<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* base = align_1024(smem_raw);
+  const Bars bars = carve_bars(base, S::kBarOff);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + S::kMiscOff);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base + S::kMiscOff + 4);
+  block_setup(bars, 4, tmem_slot, abort_flag);
   const uint32_t tmem_base = *tmem_slot;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (warp == 0) {
     if (lane == 0) {
       prefetch_tmap(&map_q); prefetch_tmap(&map_kp); prefetch_tmap(&map_km);
-      mbar_expect_tx(bars.qfull, S::kQBytes);
-      for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kQBoxBytes, &map_q, bars.qfull, b * 64, h, l0 + q0);
-      int it = 0;
-      for (; it < nt; ++it) {
-        const int stage = it % kStages, use = it / kStages;
-        if (!mbar_wait(bars.empty + stage, (use & 1) ^ 1, abort_flag, status, 0x101)) break;
-        const KeyTile kt = key_tile(t_begin + it, p0, N, l0, M);
-        mbar_expect_tx(bars.full + stage, S::kKBytes);
-        for (int b = 0; b < S::kBoxes; ++b)
-          tma_load_3d(base + S::kKOff + stage * S::kKBytes + b * S::kKBoxBytes, kt.prompt ? &map_kp : &map_km, bars.full + stage,
-                      b * 64, hk, kt.token);
+      int kt_it = 0, q_it = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x) {
+        const StatsUnit s = stats_unit(sh, u, chunks, chunk_tiles);
+        if (!s.valid) continue;
+        if (!(ok = mbar_wait(bars.qempty, (q_it & 1) ^ 1, abort_flag, status, 0x100))) break;
+        mbar_expect_tx(bars.qfull, S::kQBytes);
+        for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kQBoxBytes, &map_q, bars.qfull, b * 64, s.h, s.l0 + s.q0);
+        ++q_it;
+        for (int it = 0; it < s.nt; ++it, ++kt_it) {
+          const int stage = kt_it % kStages, use = kt_it / kStages;
+          if (!(ok = mbar_wait(bars.empty + stage, (use & 1) ^ 1, abort_flag, status, 0x101))) break;
+          const KeyTile kt = key_tile(s.t_begin + it, s.p0, s.N, s.l0, s.M);
+          mbar_expect_tx(bars.full + stage, S::kKBytes);
+          for (int b = 0; b < S::kBoxes; ++b)
+            tma_load_3d(base + S::kKOff + stage * S::kKBytes + b * S::kKBoxBytes, kt.prompt ? &map_kp : &map_km, bars.full + stage,
+                        b * 64, s.hk, kt.token);
+        }
       }
-      if (it < nt) drain_loads(bars, it);
+      if (!ok) drain_loads(bars, kt_it);
     }
   } else if (warp == 1) {
     if (lane == 0) {
       const uint32_t idesc = idesc_bf16_f32(kTile, kTile);
-      bool ok = mbar_wait(bars.qfull, 0, abort_flag, status, 0x102);
-      tc_fence_after();
-      for (int it = 0; ok && it < nt; ++it) {
-        const int stage = it % kStages, use = it / kStages, buf = it & 1;
-        if (!(ok = mbar_wait(bars.full + stage, use & 1, abort_flag, status, 0x103))) break;
+      const uint32_t q_base = smem_u32(base + S::kQOff);
+      int kt_it = 0, q_it = 0;
+      uint32_t cnt[2] = {0u, 0u};                            // tiles issued per query tile
+      bool ok = true;
+      for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x) {
+        const StatsUnit s = stats_unit(sh, u, chunks, chunk_tiles);
+        if (!s.valid) continue;
+        if (!(ok = mbar_wait(bars.qfull, q_it & 1, abort_flag, status, 0x102))) break;
+        ++q_it;
         tc_fence_after();
-        const uint32_t k_addr = smem_u32(base + S::kKOff + stage * S::kKBytes);
-        for (int a = 0; a < n_qtiles; ++a) {
-          const int acc = a * 2 + buf;
-          if (!(ok = mbar_wait(bars.tempty + acc, ((it >> 1) & 1) ^ 1, abort_flag, status, 0x104))) break;
+        for (int it = 0; ok && it < s.nt; ++it, ++kt_it) {
+          const int stage = kt_it % kStages, use = kt_it / kStages;
+          if (!(ok = mbar_wait(bars.full + stage, use & 1, abort_flag, status, 0x103))) break;
           tc_fence_after();
-          const uint32_t q_addr = smem_u32(base + S::kQOff) + a * kTile * 128;
+          const uint32_t k_addr = smem_u32(base + S::kKOff + stage * S::kKBytes);
+          for (int a = 0; a < s.n_qtiles; ++a) {
+            const int acc = a * 2 + (cnt[a] & 1);
+            if (!(ok = mbar_wait(bars.tempty + acc, ((cnt[a] >> 1) & 1) ^ 1, abort_flag, status, 0x104))) break;
+            tc_fence_after();
+            const uint32_t q_addr = q_base + a * kTile * 128;
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint64_t adesc = smem_desc_sw128(q_addr + (kk >> 2) * S::kQBoxBytes + (kk & 3) * 32);
-            const uint64_t bdesc = smem_desc_sw128(k_addr + (kk >> 2) * S::kKBoxBytes + (kk & 3) * 32);
-            umma_ss(tmem_base + acc * kTile, adesc, bdesc, idesc, kk > 0);
+            for (int kk = 0; kk < D / 16; ++kk) {
+              const uint64_t adesc = smem_desc_sw128(q_addr + (kk >> 2) * S::kQBoxBytes + (kk & 3) * 32);
+              const uint64_t bdesc = smem_desc_sw128(k_addr + (kk >> 2) * S::kKBoxBytes + (kk & 3) * 32);
+              umma_ss(tmem_base + acc * kTile, adesc, bdesc, idesc, kk > 0);
+            }
+            umma_commit(bars.tfull + acc);
+            ++cnt[a];
           }
-          umma_commit(bars.tfull + acc);
+          umma_commit(bars.empty + stage);
         }
-        umma_commit(bars.empty + stage);
+        umma_commit(bars.qempty);
       }
     }
   } else {
-    const int wg = (warp - 2) >> 2;                         // warpgroup = query tile
+    // Four warpgroups: query tile a = wg >> 1, and of each 128-key accumulator the 64-column half (wg & 1).
+    // Each (row, half) keeps its own running (max, sum); the merge kernel combines the halves like any two chunks.
+    const int wg = (warp - 2) >> 2;
+    const int a = wg >> 1, half = wg & 1;
     const int lane_group = warp & 3;                        // TMEM lanes this warp may read
     const int row = lane_group * 32 + lane;                 // query inside the tile
-    if (wg < n_qtiles) {
-      const float cs = sh.scale * kLog2e;
+    const float cs = sh.scale * kLog2e;
+    uint32_t cnt = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x) {
+      const StatsUnit s = stats_unit(sh, u, chunks, chunk_tiles);
+      if (!s.valid || a >= s.n_qtiles) continue;
       float m = -INFINITY, l = 0.f;                         // m in raw (unscaled) logits
-      bool ok = true;
-      for (int it = 0; ok && it < nt; ++it) {
-        const int buf = it & 1, acc = wg * 2 + buf;
-        if (!(ok = mbar_wait(bars.tfull + acc, (it >> 1) & 1, abort_flag, status, 0x105))) break;
-        tc_fence_after();
-        const int valid = key_tile(t_begin + it, p0, N, l0, M).valid;
-        const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + acc * kTile;
-#pragma unroll 1
-        for (int cb = 0; cb < kTile / 32; ++cb) {
-          if (cb * 32 >= valid) break;
-          float v[32];
-          tmem_ld32(taddr + cb * 32, v);
-          tmem_ld_wait();
-          if (valid - cb * 32 < 32) {
+      auto absorb = [&](float* v, int col0, int valid) {
+        if (valid - col0 < 32) {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) if (cb * 32 + c >= valid) v[c] = -INFINITY;
-          }
-          float cmax = v[0];
-#pragma unroll
-          for (int c = 1; c < 32; ++c) cmax = fmaxf(cmax, v[c]);
-          if (cmax > m) { l *= ex2((m - cmax) * cs); m = cmax; }
-          const float neg = -m * cs;
-#pragma unroll
-          for (int c = 0; c < 32; ++c) l += ex2(fmaf(v[c], cs, neg));
+          for (int c = 0; c < 32; ++c) if (col0 + c >= valid) v[c] = -INFINITY;
         }
+        float cmax = fmaxf(v[0], v[1]);
+#pragma unroll
+        for (int c = 2; c < 32; c += 2) cmax = fmaxf(cmax, fmaxf(v[c], v[c + 1]));
+        if (cmax > m) { l *= ex2((m - cmax) * cs); m = cmax; }
+        const float neg = -m * cs;
+        float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) { l0 += ex2(fmaf(v[c], cs, neg)); l1 += ex2(fmaf(v[c + 1], cs, neg)); }
+        l += l0 + l1;
+      };
+      for (int it = 0; ok && it < s.nt; ++it, ++cnt) {
+        const int acc = a * 2 + (cnt & 1);
+        if (!(ok = mbar_wait(bars.tfull + acc, (cnt >> 1) & 1, abort_flag, status, 0x105))) break;
+        tc_fence_after();
+        const int valid = key_tile(s.t_begin + it, s.p0, s.N, s.l0, s.M).valid;
+        const int col0 = half * 64;
+        const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + acc * kTile + col0;
+        const int n_chunks = valid > col0 + 32 ? 2 : (valid > col0 ? 1 : 0);
+        float va[32], vb[32];
+        if (n_chunks > 0) tmem_ld32(taddr, va);
+        if (n_chunks > 1) tmem_ld32(taddr + 32, vb);
+        if (n_chunks > 0) tmem_ld_wait();
         tc_fence_before();
-        mbar_arrive(bars.tempty + acc);
+        mbar_arrive(bars.tempty + acc);                     // this thread's logits are in registers
+        if (n_chunks > 0) absorb(va, col0, valid);
+        if (n_chunks > 1) absorb(vb, col0 + 32, valid);
       }
-      const int i = q0 + wg * kTile + row;
-      if (ok && i < M) part[((long long)h * sh.sumM + l0 + i) * C + chunk] = make_float2(m * sh.scale, l);
+      const int i = s.q0 + a * kTile + row;
+      if (ok && i < s.M) part[((long long)s.h * sh.sumM + s.l0 + i) * C + s.chunk * 2 + half] = make_float2(m * sh.scale, l);
     }
   }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
+  block_teardown(tmem_base);
 }
 
 // =====================================================================================================
-// sweep 2: column sums.  grid (tile groups, H_kv, R).
+// sweep 2: column sums.  unit u -> (tile group, hk, r).
 // scores[hk][p0 + j] = sum over the group's query heads and mask rows of w_i * exp(s_ij - lse_i);
-// mass_part[(r*H_kv + hk)*Tmax + t] = (sum over the tile's prompt keys, sum over its mask keys).
+// mass_part[((r*H_kv + hk)*Tmax + t)*4 + w] = (sum over prompt keys, sum over mask keys) of tile t seen by warp w.
 // =====================================================================================================
+struct ColsumUnit { int hk, r, p0, N, l0, M, t_begin, nt, nqb, q_per_head; bool valid; };
+
+__device__ __forceinline__ ColsumUnit colsum_unit(const Shape& sh, int u, int groups, int tiles_per_unit) {
+  ColsumUnit c;
+  const int tg = u % groups;
+  c.hk = (u / groups) % sh.Hkv;
+  c.r = u / (groups * sh.Hkv);
+  c.p0 = sh.prompt_cu[c.r]; c.N = sh.prompt_cu[c.r + 1] - c.p0;
+  c.l0 = sh.live_cu[c.r]; c.M = sh.live_cu[c.r + 1] - c.l0;
+  const int T = (c.N + kTile - 1) / kTile + (c.M + kTile - 1) / kTile;
+  c.t_begin = tg * tiles_per_unit;
+  c.nt = min(c.t_begin + tiles_per_unit, T) - c.t_begin;
+  c.q_per_head = (c.M + kQBlock - 1) / kQBlock;
+  c.nqb = sh.g * c.q_per_head;
+  c.valid = c.nt > 0 && c.M > 0;
+  return c;
+}
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kp,
                 const __grid_constant__ CUtensorMap map_km, Shape sh, const float* __restrict__ lse,
                 const float* __restrict__ w, float* __restrict__ scores, float2* __restrict__ mass_part, int Tmax,
-                int tiles_per_cta, uint32_t* __restrict__ status) {
+                int groups, int tiles_per_unit, int n_units, uint32_t* __restrict__ status) {
   using S = Smem<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = align_1024(smem_raw);
   const Bars bars = carve_bars(base, S::kBarOff);
   float* accs = reinterpret_cast<float*>(base + S::kAccOff);
   float* c2s = reinterpret_cast<float*>(base + S::kC2Off);
-  float* red = reinterpret_cast<float*>(base + S::kRedOff);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + S::kMiscOff);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base + S::kMiscOff + 4);
-
-  const int r = blockIdx.z, hk = blockIdx.y;
-  const int p0 = sh.prompt_cu[r], N = sh.prompt_cu[r + 1] - p0;
-  const int l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
-  const int T = (N + kTile - 1) / kTile + (M + kTile - 1) / kTile;
-  const int t_begin = blockIdx.x * tiles_per_cta, t_end = min(t_begin + tiles_per_cta, T);
-  float2* mp = mass_part + (long long)(r * sh.Hkv + hk) * Tmax;
-  // tiles of this CTA's nominal range that the request does not have: their partials must read as zero
-  for (int t = max(t_begin, T) + (int)threadIdx.x; t < min(t_begin + tiles_per_cta, Tmax); t += kThreads) mp[t] = make_float2(0.f, 0.f);
-  if (t_begin >= t_end) return;
-  const int nt = t_end - t_begin;
-  if (M == 0) {                                             // no voters: every score of the range is zero
-    for (int e = threadIdx.x; e < nt * kTile; e += kThreads) {
-      const int j = t_begin * kTile + e;
-      if (j < N) scores[(long long)hk * sh.sumN + p0 + j] = 0.f;
-    }
-    for (int t = t_begin + (int)threadIdx.x; t < t_end; t += kThreads) mp[t] = make_float2(0.f, 0.f);
-    return;
-  }
-  const int q_per_head = (M + kQBlock - 1) / kQBlock;
-  const int nqb = sh.g * q_per_head;
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(bars.full + s, 1); mbar_init(bars.empty + s, 1); }
-    mbar_init(bars.qfull, 1); mbar_init(bars.qempty, 1);
-    for (int b = 0; b < 2; ++b) { mbar_init(bars.tfull + b, 1); mbar_init(bars.tempty + b, kTile); }
-    *abort_flag = 0u;
-    fence_barrier_init();
-  }
-  if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
+  block_setup(bars, 2, tmem_slot, abort_flag);
   const uint32_t tmem_base = *tmem_slot;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (warp == 0) {
     if (lane == 0) {
       prefetch_tmap(&map_q); prefetch_tmap(&map_kp); prefetch_tmap(&map_km);
-      int it = 0;
+      int kt_it = 0, q_it = 0;
       bool ok = true;
-      for (int qb = 0; ok && qb < nqb; ++qb) {
-        const int h = hk * sh.g + qb / q_per_head, q0 = (qb % q_per_head) * kQBlock;
-        if (!(ok = mbar_wait(bars.qempty, (qb & 1) ^ 1, abort_flag, status, 0x201))) break;
-        mbar_expect_tx(bars.qfull, S::kQBytes);
-        for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kQBoxBytes, &map_q, bars.qfull, b * 64, h, l0 + q0);
-        for (int tl = 0; tl < nt; ++tl, ++it) {
-          const int stage = it % kStages, use = it / kStages;
-          if (!(ok = mbar_wait(bars.empty + stage, (use & 1) ^ 1, abort_flag, status, 0x202))) break;
-          const KeyTile kt = key_tile(t_begin + tl, p0, N, l0, M);
-          mbar_expect_tx(bars.full + stage, S::kKBytes);
-          for (int b = 0; b < S::kBoxes; ++b)
-            tma_load_3d(base + S::kKOff + stage * S::kKBytes + b * S::kKBoxBytes, kt.prompt ? &map_kp : &map_km,
-                        bars.full + stage, b * 64, hk, kt.token);
+      for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x) {
+        const ColsumUnit c = colsum_unit(sh, u, groups, tiles_per_unit);
+        if (!c.valid) continue;
+        for (int qb = 0; ok && qb < c.nqb; ++qb, ++q_it) {
+          const int h = c.hk * sh.g + qb / c.q_per_head, q0 = (qb % c.q_per_head) * kQBlock;
+          if (!(ok = mbar_wait(bars.qempty, (q_it & 1) ^ 1, abort_flag, status, 0x201))) break;
+          mbar_expect_tx(bars.qfull, S::kQBytes);
+          for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kQBoxBytes, &map_q, bars.qfull, b * 64, h, c.l0 + q0);
+          for (int tl = 0; tl < c.nt; ++tl, ++kt_it) {
+            const int stage = kt_it % kStages, use = kt_it / kStages;
+            if (!(ok = mbar_wait(bars.empty + stage, (use & 1) ^ 1, abort_flag, status, 0x202))) break;
+            const KeyTile kt = key_tile(c.t_begin + tl, c.p0, c.N, c.l0, c.M);
+            mbar_expect_tx(bars.full + stage, S::kKBytes);
+            for (int b = 0; b < S::kBoxes; ++b)
+              tma_load_3d(base + S::kKOff + stage * S::kKBytes + b * S::kKBoxBytes, kt.prompt ? &map_kp : &map_km,
+                          bars.full + stage, b * 64, c.hk, kt.token);
+          }
         }
       }
-      if (!ok) drain_loads(bars, it);
+      if (!ok) drain_loads(bars, kt_it);
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      int it = 0;
+      int kt_it = 0, q_it = 0, base_par = 0;
       uint32_t uses[2] = {0u, 0u};
       bool ok = true;
       const uint32_t q_addr = smem_u32(base + S::kQOff);
-      for (int qb = 0; ok && qb < nqb; ++qb) {
-        const int q0 = (qb % q_per_head) * kQBlock;
-        const int n_mma = (min(kQBlock, M - q0) + 31) & ~31;           // columns the epilogue will read
-        const uint32_t idesc = idesc_bf16_f32(kTile, n_mma);
-        if (!(ok = mbar_wait(bars.qfull, qb & 1, abort_flag, status, 0x203))) break;
-        tc_fence_after();
-        for (int tl = 0; tl < nt; ++tl, ++it) {
-          const int stage = it % kStages, use = it / kStages, buf = tl & 1;
-          if (!(ok = mbar_wait(bars.full + stage, use & 1, abort_flag, status, 0x204))) break;
-          if (!(ok = mbar_wait(bars.tempty + buf, (uses[buf] & 1) ^ 1, abort_flag, status, 0x205))) break;
+      for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x) {
+        const ColsumUnit c = colsum_unit(sh, u, groups, tiles_per_unit);
+        if (!c.valid) continue;
+        for (int qb = 0; ok && qb < c.nqb; ++qb, ++q_it) {
+          const int q0 = (qb % c.q_per_head) * kQBlock;
+          const int n_mma = (min(kQBlock, c.M - q0) + 31) & ~31;           // columns the epilogue will read
+          const uint32_t idesc = idesc_bf16_f32(kTile, n_mma);
+          if (!(ok = mbar_wait(bars.qfull, q_it & 1, abort_flag, status, 0x203))) break;
           tc_fence_after();
-          const uint32_t k_addr = smem_u32(base + S::kKOff + stage * S::kKBytes);
+          for (int tl = 0; tl < c.nt; ++tl, ++kt_it) {
+            const int stage = kt_it % kStages, use = kt_it / kStages, buf = (tl + base_par) & 1;
+            if (!(ok = mbar_wait(bars.full + stage, use & 1, abort_flag, status, 0x204))) break;
+            if (!(ok = mbar_wait(bars.tempty + buf, (uses[buf] & 1) ^ 1, abort_flag, status, 0x205))) break;
+            tc_fence_after();
+            const uint32_t k_addr = smem_u32(base + S::kKOff + stage * S::kKBytes);
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint64_t adesc = smem_desc_sw128(k_addr + (kk >> 2) * S::kKBoxBytes + (kk & 3) * 32);
-            const uint64_t bdesc = smem_desc_sw128(q_addr + (kk >> 2) * S::kQBoxBytes + (kk & 3) * 32);
-            umma_ss(tmem_base + buf * kQBlock, adesc, bdesc, idesc, kk > 0);
+            for (int kk = 0; kk < D / 16; ++kk) {
+              const uint64_t adesc = smem_desc_sw128(k_addr + (kk >> 2) * S::kKBoxBytes + (kk & 3) * 32);
+              const uint64_t bdesc = smem_desc_sw128(q_addr + (kk >> 2) * S::kQBoxBytes + (kk & 3) * 32);
+              umma_ss(tmem_base + buf * kQBlock, adesc, bdesc, idesc, kk > 0);
+            }
+            umma_commit(bars.empty + stage);
+            umma_commit(bars.tfull + buf);
+            ++uses[buf];
           }
-          umma_commit(bars.empty + stage);
-          umma_commit(bars.tfull + buf);
-          ++uses[buf];
+          umma_commit(bars.qempty);
         }
-        umma_commit(bars.qempty);
+        base_par ^= c.nt & 1;
       }
     }
   } else {
-    const int wg = (warp - 2) >> 2;                         // warpgroup = accumulator = parity of the local tile index
+    // Four warpgroups: accumulator buf = wg >> 1, and of its (up to) 256 query columns the 128-column half (wg & 1).
+    // The two halves of a key's sum meet in shared memory (one named barrier per tile per pair); the half-0 thread
+    // owns the key from then on.  Inside a unit the tile -> accumulator map is fixed, (tl + base_par) & 1, so a key's
+    // running sum in shared memory always belongs to the same thread; base_par carries the alternation across units.
+    // After a failed wait a thread skips the arithmetic but still walks the loops, so that every thread reaches every
+    // named barrier.
+    const int wg = (warp - 2) >> 2;
+    const int buf = wg >> 1, half = wg & 1;
     const int lane_group = warp & 3;
     const int row = lane_group * 32 + lane;                 // key inside the tile
-    const int tid_wg = ((warp - 2) & 3) * 32 + lane;
-    float* c2 = c2s + wg * kQBlock;
     const float cs = sh.scale * kLog2e;
-    uint32_t uses = 0;
+    const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + buf * kQBlock + half * kTile;
+    float* xch = reinterpret_cast<float*>(base + S::kXchOff) + buf * 2 * kTile;
+    uint32_t uses = 0, c2_it = 0;
+    int base_par = 0;
     bool ok = true;
-    // After a failed wait a thread skips the work but still walks the loops, so that every thread of the
-    // warpgroup reaches every named barrier.
-    for (int qb = 0; qb < nqb; ++qb) {
-      const int h = hk * sh.g + qb / q_per_head, q0 = (qb % q_per_head) * kQBlock;
-      const int nq = min(kQBlock, M - q0);
-      named_barrier(1 + wg, kTile);                         // the previous block's constants are no longer read
-      for (int e = tid_wg; e < kQBlock; e += kTile) {
-        const int q = q0 + e;
-        float c = INFINITY;                                 // 2^(x - inf) = 0: rows that do not exist never vote
-        if (e < nq) c = lse[(long long)h * sh.sumM + l0 + q] * kLog2e - (w ? log2f(w[l0 + q]) : 0.f);
-        c2[e] = c;
-      }
-      named_barrier(1 + wg, kTile);
-      const int chunks = (nq + 31) >> 5;
-      for (int tl = wg; ok && tl < nt; tl += 2) {
-        if (!(ok = mbar_wait(bars.tfull + wg, uses & 1, abort_flag, status, 0x206))) break;
-        ++uses;
-        tc_fence_after();
-        const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + wg * kQBlock;
-        float a0 = 0.f, a1 = 0.f;
-#pragma unroll 1
-        for (int cb = 0; cb < chunks; ++cb) {
-          float v[32];
-          tmem_ld32(taddr + cb * 32, v);
-          tmem_ld_wait();
+    for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+      const ColsumUnit c = colsum_unit(sh, u, groups, tiles_per_unit);
+      if (!c.valid) continue;
+      const int seg = c.r * sh.Hkv + c.hk;
+      for (int qb = 0; qb < c.nqb; ++qb, ++c2_it) {
+        const int h = c.hk * sh.g + qb / c.q_per_head, q0 = (qb % c.q_per_head) * kQBlock + half * kTile;
+        const int nq = max(0, min(kTile, c.M - q0));        // voters in this warpgroup's half of the block
+        float* c2 = c2s + (wg * 2 + (c2_it & 1)) * kTile;
+        {
+          float cst = INFINITY;                             // 2^(x - inf) = 0: rows that do not exist never vote
+          if (row < nq) cst = lse[(long long)h * sh.sumM + c.l0 + q0 + row] * kLog2e - (w ? log2f(w[c.l0 + q0 + row]) : 0.f);
+          c2[row] = cst;
+        }
+        named_barrier(1 + wg, kTile);
+        const int chunks = (nq + 31) >> 5;
+        auto absorb = [&](const float* v, int cb, float& a0, float& a1) {
           const float4* cc = reinterpret_cast<const float4*>(c2 + cb * 32);
 #pragma unroll
           for (int c4 = 0; c4 < 8; ++c4) {
@@ -371,34 +414,56 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             a0 += ex2(fmaf(v[4 * c4 + 2], cs, -k4.z));
             a1 += ex2(fmaf(v[4 * c4 + 3], cs, -k4.w));
           }
+        };
+        for (int tl = (buf + base_par) & 1; tl < c.nt; tl += 2) {
+          float a0 = 0.f, a1 = 0.f;
+          if (ok) ok = mbar_wait(bars.tfull + buf, uses & 1, abort_flag, status, 0x206);
+          if (ok) {
+            tc_fence_after();
+            // four warps per scheduler hide the load latency: no register double-buffering here
+#pragma unroll 1
+            for (int cb = 0; cb < chunks; ++cb) {
+              float v[32];
+              tmem_ld32(taddr + cb * 32, v);
+              tmem_ld_wait();
+              if (cb + 1 == chunks) { tc_fence_before(); mbar_arrive(bars.tempty + buf); }   // last logits are in registers
+              absorb(v, cb, a0, a1);
+            }
+            if (chunks == 0) { tc_fence_before(); mbar_arrive(bars.tempty + buf); }
+          }
+          float* slot = xch + (uses & 1) * kTile;
+          ++uses;
+          if (half == 1) slot[row] = a0 + a1;
+          named_barrier(5 + buf, 2 * kTile);                // the pair's two halves of this tile are done
+          if (half == 1 || !ok) continue;
+          float acc = (a0 + a1) + slot[row];
+          if (c.nqb > 1) {                                  // grouped heads / more than 256 voters: sum over query blocks
+            if (qb > 0) acc += accs[tl * kTile + row];
+            if (qb + 1 < c.nqb) { accs[tl * kTile + row] = acc; continue; }
+          }
+          const KeyTile kt = key_tile(c.t_begin + tl, c.p0, c.N, c.l0, c.M);
+          if (row >= kt.valid) acc = 0.f;
+          if (kt.prompt && row < kt.valid) scores[(long long)c.hk * sh.sumN + kt.token + row] = acc;
+          acc = warp_sum(acc);
+          if (lane == 0)
+            mass_part[((long long)seg * Tmax + c.t_begin + tl) * 4 + lane_group] = kt.prompt ? make_float2(acc, 0.f) : make_float2(0.f, acc);
         }
-        tc_fence_before();
-        mbar_arrive(bars.tempty + wg);
-        const float acc = a0 + a1;
-        if (qb == 0) accs[tl * kTile + row] = acc; else accs[tl * kTile + row] += acc;
       }
-    }
-    named_barrier(3, 2 * kTile);                            // both warpgroups: all column sums are in shared memory
-    if (wg == 0 && !*abort_flag) {
-      for (int tl = 0; tl < nt; ++tl) {
-        const KeyTile kt = key_tile(t_begin + tl, p0, N, l0, M);
-        float v = accs[tl * kTile + tid_wg];
-        if (tid_wg >= kt.valid) v = 0.f;
-        if (kt.prompt && tid_wg < kt.valid) scores[(long long)hk * sh.sumN + kt.token + tid_wg] = v;
-        v = warp_sum(v);
-        if (lane == 0) red[(warp - 2) & 3] = v;
-        named_barrier(1, kTile);
-        if (tid_wg == 0) {
-          const float s = (red[0] + red[1]) + (red[2] + red[3]);
-          mp[t_begin + tl] = kt.prompt ? make_float2(s, 0.f) : make_float2(0.f, s);
-        }
-        named_barrier(1, kTile);
-      }
+      base_par ^= c.nt & 1;
     }
   }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
+  block_teardown(tmem_base);
+}
+
+// Requests without voters (M = 0): every score is zero and so are the masses.  grid (tiles, H_kv, R).
+__global__ void score_zero_fill(Shape sh, float* __restrict__ scores, float2* __restrict__ mass_part, int Tmax) {
+  const int t = blockIdx.x, hk = blockIdx.y, r = blockIdx.z;
+  const int p0 = sh.prompt_cu[r], N = sh.prompt_cu[r + 1] - p0;
+  const int M = sh.live_cu[r + 1] - sh.live_cu[r];
+  if (M > 0 || t * kTile >= N) return;
+  const int j = t * kTile + threadIdx.x;
+  if (j < N) scores[(long long)hk * sh.sumN + p0 + j] = 0.f;
+  if (threadIdx.x < 4) mass_part[((long long)(r * sh.Hkv + hk) * Tmax + t) * 4 + threadIdx.x] = make_float2(0.f, 0.f);
 }
 
 // =====================================================================================================
@@ -417,16 +482,16 @@ bool build_maps(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kp,
          make_tmap_rows(ctx->encode_tiled, &m->km, km, sh.d, sh.Hkv, sh.sumM, sh.kv_hs * 2, sh.kv_ts * 2, kTile);
 }
 
-// Tiles per CTA such that the grid is close to a whole number of waves over the SMs.
+// Tiles per unit: small enough that the persistent CTAs end within a few percent of each other, large enough
+// that the resident query block (reloaded per unit) is amortised.
 int pick_tiles(int tiles, long long units, int sm_count, int lo, int hi) {
   int best = lo;
-  double best_eff = -1.0;
+  double best_cost = 1e300;
   for (int tp = lo; tp <= hi; ++tp) {
-    const long long ctas = units * ((tiles + tp - 1) / tp);
-    const long long waves = (ctas + sm_count - 1) / sm_count;
-    // work is counted in tiles: the slowest SM processes `waves` CTAs of up to tp tiles (+1 for the query load)
-    const double eff = (double)units * tiles / ((double)waves * sm_count * (tp + 1.0));
-    if (eff > best_eff) { best_eff = eff; best = tp; }
+    const long long n = units * ((tiles + tp - 1) / tp);
+    const long long per_cta = (n + sm_count - 1) / sm_count;
+    const double cost = (double)per_cta * (tp + 1.5);      // +1.5 tiles: query load and pipeline refill per unit
+    if (cost < best_cost) { best_cost = cost; best = tp; }
   }
   return best;
 }
@@ -445,7 +510,7 @@ cudaError_t set_smem_attr() {
 
 int score_tc_max_chunks(const Shape& sh) {
   const int T = (sh.maxN + kTile - 1) / kTile + (sh.maxM + kTile - 1) / kTile;
-  return (T + 3) / 4;                                       // a chunk never has fewer than 4 tiles
+  return 2 * ((T + 3) / 4);                                 // a chunk never has fewer than 4 tiles and yields 2 partials per row
 }
 
 int score_tc_max_tiles(const Shape& sh) { return (sh.maxN + kTile - 1) / kTile + (sh.maxM + kTile - 1) / kTile; }
@@ -462,34 +527,45 @@ int launch_score_stats_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const
   const int T = score_tc_max_tiles(sh);
   const int q_pairs = (sh.maxM + kQBlock - 1) / kQBlock;
   int ct = pick_tiles(T, (long long)sh.H * sh.R * q_pairs, ctx->sm_count, 4, 32);
-  while ((T + ct - 1) / ct > C) ++ct;
+  while (2 * ((T + ct - 1) / ct) > C) ++ct;
   *chunk_tiles_out = ct;
-  dim3 grid((T + ct - 1) / ct, sh.H, sh.R * q_pairs);
+  const int chunks = (T + ct - 1) / ct;
+  const long long n_units = (long long)chunks * sh.H * sh.R * q_pairs;
+  if (n_units > 0x7fffffffLL) return 1;
+  const int grid = (int)(n_units < ctx->sm_count ? n_units : ctx->sm_count);
   if (sh.d == 128) {
     if (set_smem_attr<128>() != cudaSuccess) return 1;
-    score_stats_tc<128><<<grid, kThreads, Smem<128>::kDynamic, st>>>(m.q, m.kp, m.km, sh, part, C, ct, ctx->status_dev);
+    score_stats_tc<128><<<grid, kThreads, Smem<128>::kDynamic, st>>>(m.q, m.kp, m.km, sh, part, C, chunks, ct, (int)n_units, ctx->status_dev);
   } else {
     if (set_smem_attr<64>() != cudaSuccess) return 1;
-    score_stats_tc<64><<<grid, kThreads, Smem<64>::kDynamic, st>>>(m.q, m.kp, m.km, sh, part, C, ct, ctx->status_dev);
+    score_stats_tc<64><<<grid, kThreads, Smem<64>::kDynamic, st>>>(m.q, m.kp, m.km, sh, part, C, chunks, ct, (int)n_units, ctx->status_dev);
   }
   return 0;
 }
 
 int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kp, const void* km, const float* lse,
-                           const float* w, float* scores, float2* mass_part, int Tmax, cudaStream_t st) {
+                           const float* w, float* scores, float2* mass_part, int Tmax, bool any_without_voters,
+                           cudaStream_t st) {
   Maps m;
   if (!build_maps(ctx, sh, q, kp, km, &m)) return 1;
   const int T = score_tc_max_tiles(sh);
   const int tp = pick_tiles(T, (long long)sh.Hkv * sh.R, ctx->sm_count, 4, kColsumMaxTiles);
-  dim3 grid((T + tp - 1) / tp, sh.Hkv, sh.R);
+  const int groups = (T + tp - 1) / tp;
+  const long long n_units = (long long)groups * sh.Hkv * sh.R;
+  if (n_units > 0x7fffffffLL) return 1;
+  const int grid = (int)(n_units < ctx->sm_count ? n_units : ctx->sm_count);
+  if (any_without_voters) {
+    dim3 gz(T, sh.Hkv, sh.R);
+    score_zero_fill<<<gz, kTile, 0, st>>>(sh, scores, mass_part, Tmax);
+  }
   if (sh.d == 128) {
     if (set_smem_attr<128>() != cudaSuccess) return 1;
-    score_colsum_tc<128><<<grid, kThreads, Smem<128>::kDynamic, st>>>(m.q, m.kp, m.km, sh, lse, w, scores, mass_part, Tmax, tp,
-                                                                      ctx->status_dev);
+    score_colsum_tc<128><<<grid, kThreads, Smem<128>::kDynamic, st>>>(m.q, m.kp, m.km, sh, lse, w, scores, mass_part, Tmax, groups, tp,
+                                                                      (int)n_units, ctx->status_dev);
   } else {
     if (set_smem_attr<64>() != cudaSuccess) return 1;
-    score_colsum_tc<64><<<grid, kThreads, Smem<64>::kDynamic, st>>>(m.q, m.kp, m.km, sh, lse, w, scores, mass_part, Tmax, tp,
-                                                                     ctx->status_dev);
+    score_colsum_tc<64><<<grid, kThreads, Smem<64>::kDynamic, st>>>(m.q, m.kp, m.km, sh, lse, w, scores, mass_part, Tmax, groups, tp,
+                                                                     (int)n_units, ctx->status_dev);
   }
   return 0;
 }

@@ -16,7 +16,8 @@ int score_tc_max_tiles(const Shape& sh);
 int launch_score_stats_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kp, const void* km, float2* part,
                           int C, int* chunk_tiles_out, cudaStream_t st);
 int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kp, const void* km, const float* lse,
-                           const float* w, float* scores, float2* mass_part, int Tmax, cudaStream_t st);
+                           const float* w, float* scores, float2* mass_part, int Tmax, bool any_without_voters,
+                           cudaStream_t st);
 
 }  // namespace tc
 }  // namespace mkv
