@@ -16,7 +16,7 @@ LIB = os.path.join(PKG, "libmaskkv.so")
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC,-fvisibility=hidden", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-]
+] + os.environ.get("MASKKV_EXTRA_NVCC_FLAGS", "").split()
 
 
 def _nvcc() -> str:

@@ -213,7 +213,8 @@ int maskkv_create(maskkv_ctx** out, int device) {
       qres != cudaDriverEntryPointSuccess)
     ctx->encode_tiled = nullptr;
   if (const char* e = getenv("MASKKV_FORCE_SIMT")) ctx->force_simt = (unsigned)strtoul(e, nullptr, 0);
-  cudaFuncSetAttribute(mkv::select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - 2048);
+  cudaFuncSetAttribute(mkv::select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - mkv::kSelectStaticSmem);
+  cudaFuncSetAttribute(mkv::select_kernel_reg, cudaFuncAttributeMaxDynamicSharedMemorySize, mkv::kSelectRegKeys * 4);
   if (cudaGetLastError() != cudaSuccess) { cudaFree(ctx->status_dev); free(ctx); return MASKKV_E_CUDA; }
   *out = ctx;
   return MASKKV_OK;
@@ -352,7 +353,12 @@ int maskkv_select(maskkv_ctx* ctx, const maskkv_desc_t* desc, const float* score
   if (rc != MASKKV_OK) return rc;
   if (scores_dev == nullptr || budgets_dev == nullptr || offsets_dev == nullptr || kept_idx_dev == nullptr) return MASKKV_E_INVALID;
   DeviceGuard guard(ctx->device);
-  const int max_cache = (ctx->smem_optin - 2048) / 4;
+  if (sh.maxN <= mkv::kSelectRegKeys) {                  // every segment fits the register-resident kernel
+    mkv::select_kernel_reg<<<sh.R * sh.Hkv * mkv::kSelectCluster, mkv::kSelectRegThreads, (size_t)mkv::kSelectRegKeys * 4, static_cast<cudaStream_t>(stream)>>>(
+        sh, scores_dev, budgets_dev, offsets_dev, kept_idx_dev, ctx->status_dev);
+    return launch_status(ctx, 1);
+  }
+  const int max_cache = (ctx->smem_optin - mkv::kSelectStaticSmem) / 4;
   const int cache = sh.maxN <= max_cache ? sh.maxN : 0;   // segments that do not fit are read through L2
   mkv::select_kernel<<<sh.R * sh.Hkv, mkv::kSelectThreads, (size_t)cache * 4, static_cast<cudaStream_t>(stream)>>>(
       sh, scores_dev, budgets_dev, offsets_dev, kept_idx_dev, cache, ctx->status_dev);

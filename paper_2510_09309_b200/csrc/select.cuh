@@ -1,12 +1,14 @@
 // Top-k eviction (Eq. 16): an exact radix select per (request, head) segment.
 //
 // One block per segment.  The segment's scores are turned into order-preserving 32-bit keys and
-// (when they fit) staged once in shared memory; four 8-bit histogram passes then find the k-th
-// largest key exactly, and a last sweep emits the kept indices in ascending order, ties at the
+// (when they fit) staged once in shared memory; three histogram passes (11 + 11 + 10 bits) then find
+// the k-th largest key exactly, and a last sweep emits the kept indices in ascending order, ties at the
 // threshold going to the lowest indices.  Each warp owns a contiguous index range and walks it 32
 // consecutive elements at a time, so ranks inside a step come from a ballot and shared-memory
 // accesses are conflict-free.
 #pragma once
+
+#include <cooperative_groups.h>
 
 #include "common.cuh"
 
@@ -14,6 +16,7 @@ namespace mkv {
 
 constexpr int kSelectThreads = 1024;
 constexpr int kSelectWarps = kSelectThreads / 32;
+constexpr int kSelectStaticSmem = 10240;   // upper bound of the kernel's static shared memory (histogram, partials)
 
 // Larger float <=> larger key; NaN maps to 0 (below every number, -inf included).
 __device__ __forceinline__ uint32_t order_key(float f) {
@@ -23,15 +26,285 @@ __device__ __forceinline__ uint32_t order_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Finds the digit in which the `remaining`-th largest matching key falls, given the histogram of that digit
+// (at most 2048 bins; thread t of a THREADS-wide block owns 2048/THREADS consecutive bins).  Returns through
+// shared memory: the digit, and how many keys of that digit are still wanted.
+template <int THREADS>
+__device__ __forceinline__ void find_digit(const uint32_t* hist, int bins, uint32_t remaining, uint32_t* warp_tot,
+                                           uint32_t* out_digit, uint32_t* out_remaining) {
+  constexpr int BPT = 2048 / THREADS;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t c[BPT], mine = 0;
+#pragma unroll
+  for (int t = 0; t < BPT; ++t) { c[t] = BPT * tid + t < bins ? hist[BPT * tid + t] : 0u; mine += c[t]; }
+  uint32_t suf = mine;                                   // inclusive suffix sum inside the warp (higher lanes = higher digits)
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t v = __shfl_down_sync(0xffffffffu, suf, o);
+    if (lane + o < 32) suf += v;
+  }
+  if (lane == 0) warp_tot[warp] = suf;
+  __syncthreads();
+  uint32_t above = suf - mine;                           // keys with a higher digit
+  for (int w2 = warp + 1; w2 < THREADS / 32; ++w2) above += warp_tot[w2];
+#pragma unroll
+  for (int t = BPT - 1; t >= 0; --t) {                   // highest digit first
+    if (above < remaining && above + c[t] >= remaining) { *out_digit = BPT * tid + t; *out_remaining = remaining - above; }
+    above += c[t];
+  }
+  __syncthreads();
+}
+
+// Register-resident, four-CTA variant for segments of at most kSelectRegKeys scores.  A thread-block cluster of
+// four CTAs shares one segment: CTA q, warp w, lane l keeps key i of index ((q*16 + w)*16 + i)*32 + l in a
+// register.  Each CTA histograms its own keys; the four histograms are summed through distributed shared
+// memory, so every CTA derives the same digit.  Only the first radix pass looks at every key: the keys that
+// fall into its threshold bin are copied to a per-CTA candidate list; every CTA then collects all four lists
+// and finishes the search on its own (the lists are short unless the scores are nearly all equal).  The emit sweep visits only the 32-key rows that hold a kept key.  The work is integer issue
+// slots, which is why it is spread over four SMs per segment.
+constexpr int kSelectCluster = 4;
+constexpr int kSelectRegThreads = 512;
+constexpr int kSelectRegWarps = kSelectRegThreads / 32;
+constexpr int kSelectKeysPerThread = 16;
+constexpr int kSelectRegKeys = kSelectCluster * kSelectRegThreads * kSelectKeysPerThread;
+
+// Sum over the cluster of 4 consecutive histogram bins owned by this thread.
+__device__ __forceinline__ void cluster_bins(cooperative_groups::cluster_group& cluster, uint32_t* hist, int tid, uint32_t* c) {
+  c[0] = c[1] = c[2] = c[3] = 0u;
+#pragma unroll
+  for (int q = 0; q < kSelectCluster; ++q) {
+    const uint4 v = *reinterpret_cast<const uint4*>(cluster.map_shared_rank(hist, q) + 4 * tid);
+    c[0] += v.x; c[1] += v.y; c[2] += v.z; c[3] += v.w;
+  }
+}
+
+// Digit search on cluster-summed counts (thread t owns bins 4t..4t+3); every CTA computes the same answer.
+__device__ __forceinline__ void find_digit_counts(const uint32_t* c, uint32_t remaining, uint32_t* warp_tot,
+                                                  uint32_t* out_digit, uint32_t* out_remaining) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t mine = (c[0] + c[1]) + (c[2] + c[3]);
+  uint32_t suf = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t v = __shfl_down_sync(0xffffffffu, suf, o);
+    if (lane + o < 32) suf += v;
+  }
+  if (lane == 0) warp_tot[warp] = suf;
+  __syncthreads();
+  uint32_t above = suf - mine;
+  for (int w2 = warp + 1; w2 < kSelectRegWarps; ++w2) above += warp_tot[w2];
+#pragma unroll
+  for (int t = 3; t >= 0; --t) {
+    if (above < remaining && above + c[t] >= remaining) { *out_digit = 4 * tid + t; *out_remaining = remaining - above; }
+    above += c[t];
+  }
+  __syncthreads();
+}
+
+// grid = 4 * segments (cluster of 4 per segment); dynamic shared memory: uint32 cand[kSelectRegKeys]
+__global__ void __cluster_dims__(kSelectCluster, 1, 1) __launch_bounds__(kSelectRegThreads, 1)
+select_kernel_reg(Shape sh, const float* __restrict__ scores, const int32_t* __restrict__ budgets,
+                  const int32_t* __restrict__ offsets, int32_t* __restrict__ kept_idx, uint32_t* __restrict__ status) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  extern __shared__ __align__(16) uint32_t cand[];
+  __shared__ __align__(16) uint32_t hist[2048];
+  __shared__ uint32_t sh_digit, sh_remaining, sh_ncand;
+  __shared__ uint32_t warp_gt[kSelectRegWarps], warp_eq[kSelectRegWarps], warp_tot[kSelectRegWarps];
+  __shared__ uint32_t and_or[2];
+
+  const int s = blockIdx.x / kSelectCluster;
+  const int q = (int)cluster.block_rank();
+  const int r = s / sh.Hkv, hk = s % sh.Hkv;
+  const int p0 = sh.prompt_cu[r], N = sh.prompt_cu[r + 1] - p0;
+  const int out0 = offsets[s];
+  int k = budgets[s];
+  if (k > N) { k = N; if (threadIdx.x == 0 && q == 0) atomicOr(status, (uint32_t)MASKKV_FLAG_BOUNDS); }
+  if (k <= 0) return;                                    // uniform over the cluster
+  const float* seg = scores + (long long)hk * sh.sumN + p0;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (k == N) {                                          // nothing to evict (uniform over the cluster)
+    for (int j = q * kSelectRegThreads + tid; j < N; j += kSelectCluster * kSelectRegThreads) kept_idx[out0 + j] = j;
+    return;
+  }
+
+  const int jbase = (q * kSelectRegWarps + warp) * (32 * kSelectKeysPerThread) + lane;
+  uint32_t key[kSelectKeysPerThread];
+#pragma unroll
+  for (int i = 0; i < kSelectKeysPerThread; ++i) {        // all loads first: the whole segment is in flight at once
+    const int j = jbase + i * 32;
+    key[i] = j < N ? __float_as_uint(__ldg(seg + j)) : 0u;
+  }
+  uint32_t vmask = 0u;                                   // bit i: key i exists
+  uint32_t k_and = 0xffffffffu, k_or = 0u;
+#pragma unroll
+  for (int i = 0; i < kSelectKeysPerThread; ++i) {
+    key[i] = order_key(__uint_as_float(key[i]));
+    if (jbase + i * 32 < N) { vmask |= 1u << i; k_and &= key[i]; k_or |= key[i]; }
+  }
+  k_and = __reduce_and_sync(0xffffffffu, k_and);
+  k_or = __reduce_or_sync(0xffffffffu, k_or);
+  if (tid < 32) { warp_gt[tid & (kSelectRegWarps - 1)] = 0xffffffffu; warp_eq[tid & (kSelectRegWarps - 1)] = 0u; }
+  for (int b2 = tid; b2 < 2048; b2 += kSelectRegThreads) hist[b2] = 0;
+  if (tid == 0) sh_ncand = 0;
+  __syncthreads();
+  if (lane == 0) { warp_gt[warp] = k_and; warp_eq[warp] = k_or; }
+  __syncthreads();
+  if (warp == 0) {
+    k_and = __reduce_and_sync(0xffffffffu, warp_gt[lane & (kSelectRegWarps - 1)]);
+    k_or = __reduce_or_sync(0xffffffffu, warp_eq[lane & (kSelectRegWarps - 1)]);
+    if (lane == 0) { and_or[0] = k_and; and_or[1] = k_or; }
+  }
+  cluster.sync();
+  k_and = 0xffffffffu; k_or = 0u;
+#pragma unroll
+  for (int c = 0; c < kSelectCluster; ++c) {
+    const uint32_t* peer = cluster.map_shared_rank(and_or, c);
+    k_and &= peer[0];
+    k_or |= peer[1];
+  }
+  // Leading bits on which every key agrees carry no order information: the radix starts below them.
+  const int common = __clz(k_and ^ k_or);                // 32 when all keys are equal
+  int bits_left = 32 - common;
+  uint32_t have_mask = common == 0 ? 0u : (common == 32 ? 0xffffffffu : ~(0xffffffffu >> common));
+  uint32_t prefix = k_and & have_mask;
+  uint32_t remaining = (uint32_t)k;
+  uint32_t cnt4[4];
+
+  if (bits_left > 0) {
+    // first pass: every key (all of them match the common prefix)
+    const int width = bits_left >= 11 ? 11 : bits_left;
+    const int shift = bits_left - width;
+    const uint32_t dmask = (1u << width) - 1u;
+#pragma unroll
+    for (int i = 0; i < kSelectKeysPerThread; ++i)
+      if ((vmask >> i) & 1u) atomicAdd(&hist[(key[i] >> shift) & dmask], 1u);
+    cluster.sync();
+    cluster_bins(cluster, hist, tid, cnt4);
+    find_digit_counts(cnt4, remaining, warp_tot, &sh_digit, &sh_remaining);
+    prefix |= sh_digit << shift;
+    remaining = sh_remaining;
+    have_mask |= dmask << shift;
+    bits_left = shift;
+    if (bits_left > 0) {
+      // the keys of the threshold bin become this CTA's candidate list
+#pragma unroll
+      for (int i = 0; i < kSelectKeysPerThread; ++i) {
+        const bool m = ((vmask >> i) & 1u) && (key[i] & have_mask) == prefix;
+        const uint32_t bal = __ballot_sync(0xffffffffu, m);
+        if (bal) {
+          uint32_t pos = 0;
+          if (lane == 0) pos = atomicAdd(&sh_ncand, (uint32_t)__popc(bal));
+          pos = __shfl_sync(0xffffffffu, pos, 0);
+          if (m) cand[pos + __popc(bal & ((1u << lane) - 1u))] = key[i];
+        }
+      }
+    }
+    cluster.sync();                                      // peers are done with this CTA's histogram; candidates are complete
+    if (bits_left > 0) {
+      // Every CTA appends its peers' candidates to its own (through distributed shared memory) and finishes the
+      // search on its own: the same list in a different order gives the same histogram, hence the same threshold.
+      int ncand = (int)sh_ncand;
+      const int own = ncand;
+#pragma unroll
+      for (int c = 1; c < kSelectCluster; ++c) {
+        const int peer = (q + c) & (kSelectCluster - 1);
+        const int n_peer = (int)*cluster.map_shared_rank(&sh_ncand, peer);
+        const uint32_t* src = cluster.map_shared_rank(cand, peer);
+        for (int t = tid; t < n_peer; t += kSelectRegThreads) cand[ncand + t] = src[t];
+        ncand += n_peer;
+      }
+      (void)own;
+#pragma unroll 1
+      while (bits_left > 0) {
+        const int w2 = bits_left >= 11 ? 11 : bits_left;
+        const int sh2 = bits_left - w2;
+        const uint32_t dm2 = (1u << w2) - 1u;
+        for (int b2 = tid; b2 < 2048; b2 += kSelectRegThreads) hist[b2] = 0;
+        __syncthreads();
+        for (int t = tid; t < ncand; t += kSelectRegThreads) {
+          const uint32_t c = cand[t];
+          if ((c & have_mask) == prefix) atomicAdd(&hist[(c >> sh2) & dm2], 1u);
+        }
+        __syncthreads();
+        find_digit<kSelectRegThreads>(hist, 2048, remaining, warp_tot, &sh_digit, &sh_remaining);
+        prefix |= sh_digit << sh2;
+        remaining = sh_remaining;
+        have_mask |= dm2 << sh2;
+        bits_left = sh2;
+      }
+    }
+  }
+  const uint32_t thr = prefix;                           // threshold key; `remaining` ties are kept, lowest indices first
+
+  uint32_t gt_mask = 0u, eq_mask = 0u;
+#pragma unroll
+  for (int i = 0; i < kSelectKeysPerThread; ++i) {
+    if ((vmask >> i) & 1u) {
+      if (key[i] > thr) gt_mask |= 1u << i;
+      if (key[i] == thr) eq_mask |= 1u << i;
+    }
+  }
+  const uint32_t n_gt = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(gt_mask));
+  const uint32_t n_eq = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(eq_mask));
+  __syncthreads();                                       // warp_gt / warp_eq are reused
+  if (lane == 0) { warp_gt[warp] = n_gt; warp_eq[warp] = n_eq; }
+  __syncthreads();
+  if (warp == 0) {                                       // this CTA's totals, for the CTAs after it
+    const uint32_t g = __reduce_add_sync(0xffffffffu, lane < kSelectRegWarps ? warp_gt[lane] : 0u);
+    const uint32_t e = __reduce_add_sync(0xffffffffu, lane < kSelectRegWarps ? warp_eq[lane] : 0u);
+    if (lane == 0) { and_or[0] = g; and_or[1] = e; }
+  }
+  cluster.sync();
+  // ties / outputs that precede this warp: the lower CTAs as wholes, then the lower warps of this CTA
+  uint32_t eq_before = 0, out_before = 0;
+  {
+    uint32_t pg[kSelectCluster], pe[kSelectCluster];
+#pragma unroll
+    for (int c = 0; c < kSelectCluster; ++c) {
+      const uint32_t* peer = cluster.map_shared_rank(and_or, c);
+      pg[c] = c < q ? peer[0] : 0u;
+      pe[c] = c < q ? peer[1] : 0u;
+    }
+#pragma unroll
+    for (int c = 0; c < kSelectCluster; ++c) {
+      const uint32_t take = eq_before >= remaining ? 0u : min(pe[c], remaining - eq_before);
+      out_before += pg[c] + take;
+      eq_before += pe[c];
+    }
+    for (int w2 = 0; w2 < warp; ++w2) {
+      const uint32_t e2 = warp_eq[w2];
+      const uint32_t take = eq_before >= remaining ? 0u : min(e2, remaining - eq_before);
+      out_before += warp_gt[w2] + take;
+      eq_before += e2;
+    }
+  }
+  // rows of this warp that hold a key at or above the threshold, lowest row first
+  uint32_t rows = __reduce_or_sync(0xffffffffu, gt_mask | eq_mask);
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  while (rows) {
+    const int i = __ffs((int)rows) - 1;
+    rows &= rows - 1;
+    const bool gt = (gt_mask >> i) & 1u, eq = (eq_mask >> i) & 1u;
+    const uint32_t eq_bal = __ballot_sync(0xffffffffu, eq);
+    const bool take = gt || (eq && eq_before + __popc(eq_bal & lt_mask) < remaining);
+    const uint32_t take_bal = __ballot_sync(0xffffffffu, take);
+    if (take) kept_idx[out0 + out_before + __popc(take_bal & lt_mask)] = jbase + i * 32;
+    out_before += __popc(take_bal);
+    eq_before += __popc(eq_bal);
+  }
+  cluster.sync();                                        // no CTA leaves while a peer may still read its shared memory
+}
+
 // dynamic shared memory: uint32 keys[cache_elems] (cache_elems = 0 -> keys are re-read from global)
 __global__ void __launch_bounds__(kSelectThreads)
 select_kernel(Shape sh, const float* __restrict__ scores, const int32_t* __restrict__ budgets,
               const int32_t* __restrict__ offsets, int32_t* __restrict__ kept_idx, int cache_elems,
               uint32_t* __restrict__ status) {
   extern __shared__ __align__(16) uint32_t keys_smem[];
-  __shared__ uint32_t hist[256];
-  __shared__ uint32_t sh_prefix, sh_remaining;
-  __shared__ uint32_t warp_gt[kSelectWarps], warp_eq[kSelectWarps];
+  __shared__ uint32_t hist[2048];
+  __shared__ uint32_t sh_digit, sh_remaining;
+  __shared__ uint32_t warp_gt[kSelectWarps], warp_eq[kSelectWarps], warp_tot[kSelectWarps];
 
   const int s = blockIdx.x;
   const int r = s / sh.Hkv, hk = s % sh.Hkv;
@@ -48,57 +321,75 @@ select_kernel(Shape sh, const float* __restrict__ scores, const int32_t* __restr
     return;
   }
   const bool cached = N <= cache_elems;
-  if (cached) {
-    for (int j = tid; j < N; j += kSelectThreads) keys_smem[j] = order_key(seg[j]);
-    __syncthreads();
-  }
   auto key_at = [&](int j) -> uint32_t { return cached ? keys_smem[j] : order_key(__ldg(seg + j)); };
 
-  // --- k-th largest key: 4 passes over 8-bit digits, most significant first ---
-  uint32_t prefix = 0, have_mask = 0, remaining = (uint32_t)k;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    for (int b = tid; b < 256; b += kSelectThreads) hist[b] = 0;
-    __syncthreads();
-    for (int j0 = 0; j0 < N; j0 += kSelectThreads) {
-      const int j = j0 + tid;
-      const bool in = j < N;
-      const uint32_t key = in ? key_at(j) : 0u;
-      const bool match = in && ((key & have_mask) == prefix);
-      const uint32_t digit = (key >> shift) & 0xffu;
-      // aggregate equal digits inside the warp so that a crowded bin costs one atomic per warp
-      const uint32_t active = __ballot_sync(0xffffffffu, match);
-      if (match) {
-        const uint32_t peers = __match_any_sync(active, digit);
-        if (lane == (31 - __clz(peers))) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
+  // --- stage the keys and find the bits they all share ---
+  uint32_t k_and = 0xffffffffu, k_or = 0u;
+  auto stage = [&](int j, float f) {
+    const uint32_t key = order_key(f);
+    if (cached) keys_smem[j] = key;
+    k_and &= key;
+    k_or |= key;
+  };
+  {
+    // 16-byte loads, eight in flight per thread: the whole segment is requested before the first key is used
+    const int head = min(N, (int)((4 - (((long long)hk * sh.sumN + p0) & 3)) & 3));   // scalars up to the first aligned score
+    const int n4 = (N - head) >> 2;
+    const float4* seg4 = reinterpret_cast<const float4*>(seg + head);
+    for (int j = tid; j < head; j += kSelectThreads) stage(j, seg[j]);
+    for (int i0 = 0; i0 < n4; i0 += 8 * kSelectThreads) {
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int i = i0 + u * kSelectThreads + tid;
+        if (i < n4) v[u] = __ldg(seg4 + i);
       }
-    }
-    __syncthreads();
-    if (warp == 0) {
-      // lane owns digits [8*lane, 8*lane+8); suffix sums from the top digit down
-      uint32_t c[8], mine = 0;
 #pragma unroll
-      for (int t = 0; t < 8; ++t) { c[t] = hist[lane * 8 + t]; mine += c[t]; }
-      uint32_t above = mine;                             // inclusive suffix sum over lanes >= lane
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t v = __shfl_down_sync(0xffffffffu, above, o);
-        if (lane + o < 32) above += v;
-      }
-      above -= mine;                                     // keys with a digit in a higher lane
-      uint32_t acc = above;
-#pragma unroll
-      for (int t = 7; t >= 0; --t) {
-        if (acc < remaining && acc + c[t] >= remaining) {  // the k-th largest falls in this digit
-          sh_prefix = prefix | ((uint32_t)(lane * 8 + t) << shift);
-          sh_remaining = remaining - acc;
+      for (int u = 0; u < 8; ++u) {
+        const int i = i0 + u * kSelectThreads + tid;
+        if (i < n4) {
+          const int j = head + 4 * i;
+          stage(j, v[u].x); stage(j + 1, v[u].y); stage(j + 2, v[u].z); stage(j + 3, v[u].w);
         }
-        acc += c[t];
       }
     }
+    for (int j = head + 4 * n4 + tid; j < N; j += kSelectThreads) stage(j, seg[j]);
+  }
+  k_and = __reduce_and_sync(0xffffffffu, k_and);
+  k_or = __reduce_or_sync(0xffffffffu, k_or);
+  if (lane == 0) { warp_gt[warp] = k_and; warp_eq[warp] = k_or; }
+  __syncthreads();
+  k_and = warp_gt[lane];
+  k_or = warp_eq[lane];
+  k_and = __reduce_and_sync(0xffffffffu, k_and);
+  k_or = __reduce_or_sync(0xffffffffu, k_or);
+  __syncthreads();
+  // Leading bits on which every key agrees carry no order information: the radix starts below them, so the
+  // first digit is spread over its bins however narrow the range of the scores is.
+  const int common = __clz(k_and ^ k_or);                // 32 when all keys are equal
+  int bits_left = 32 - common;
+  uint32_t prefix = common == 0 ? 0u : (k_and & ~(0xffffffffu >> common));
+  uint32_t have_mask = common == 0 ? 0u : ~(0xffffffffu >> common);
+  if (common == 32) { prefix = k_and; have_mask = 0xffffffffu; }
+  uint32_t remaining = (uint32_t)k;
+
+  // --- k-th largest key: passes over 11-bit digits (the last one takes what is left), most significant first ---
+#pragma unroll 1
+  while (bits_left > 0) {
+    const int width = bits_left >= 11 ? 11 : bits_left;
+    const int shift = bits_left - width, bins = 1 << width;
+    for (int b = tid; b < bins; b += kSelectThreads) hist[b] = 0;
     __syncthreads();
-    prefix = sh_prefix;
+    for (int j = tid; j < N; j += kSelectThreads) {
+      const uint32_t key = key_at(j);
+      if ((key & have_mask) == prefix) atomicAdd(&hist[(key >> shift) & (uint32_t)(bins - 1)], 1u);
+    }
+    __syncthreads();
+    find_digit<kSelectThreads>(hist, bins, remaining, warp_tot, &sh_digit, &sh_remaining);
+    prefix |= sh_digit << shift;
     remaining = sh_remaining;
-    have_mask |= 0xffu << shift;
+    have_mask |= (uint32_t)(bins - 1) << shift;
+    bits_left = shift;
     __syncthreads();
   }
   // prefix = threshold key; `remaining` ties at the threshold are kept, lowest indices first.
@@ -123,6 +414,7 @@ select_kernel(Shape sh, const float* __restrict__ scores, const int32_t* __restr
     out_before += warp_gt[w2] + take;
     eq_before += e2;
   }
+  if (n_gt + n_eq == 0) return;                          // nothing of this warp's range is kept
   const uint32_t lt_mask = (1u << lane) - 1u;
   for (int j0 = wb; j0 < we; j0 += 32) {
     const int j = j0 + lane;

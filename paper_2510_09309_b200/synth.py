@@ -160,10 +160,13 @@ def layer_inputs(wl: Workload, layer: int = 0, device="cpu") -> Dict[str, torch.
     vm = _randn((sumM, Hkv, d), _gen(dev, wl, layer, _T_VM), dev)
 
     cu = wl.prompt_cu()
+    # mean mask-query direction per (request, KV head), taken BEFORE the head bias below is applied, so that the
+    # planted keys and the information/structure bias live in different directions and do not interact
+    u_dirs = [_unit(q[r * M:(r + 1) * M].view(M, Hkv, g, d).mean(dim=(0, 2))) for r in range(R)]
     if wl.head_recipe == "info_structure":
-        # Even heads lean on the prompt (target prompt mass 0.7), odd heads on the mask
-        # region (0.2): an exact logit offset t_h on the mask keys along a private
-        # direction w_h that every other row is made orthogonal to.
+        # Even heads lean on the prompt (target prompt mass 0.7 before planting), odd heads on the mask
+        # region (0.2): an exact logit offset t_h on the mask keys along a private direction w_h that every
+        # other row - and the planting direction - is made orthogonal to.
         assert g == 1, "info/structure recipe is defined for MHA shapes"
         w = _unit(_randn((H, d), _gen(dev, wl, layer, _T_W), dev))
         p_target = torch.where(torch.arange(H, device=dev) % 2 == 0, 0.7, 0.2).to(torch.float32)
@@ -174,6 +177,8 @@ def layer_inputs(wl: Workload, layer: int = 0, device="cpu") -> Dict[str, torch.
             t_h = torch.log(n_r * (1.0 - p_target) / (p_target * M))
             sl = slice(r * M, (r + 1) * M)
             q[sl] = _set_component(q[sl], w, t_h)
+            u_r = u_dirs[r]
+            u_dirs[r] = _unit(u_r - (u_r * w).sum(-1, keepdim=True) * w)
 
     planted = []
     gp = _gen(dev, wl, layer, _T_PLANT)
@@ -181,8 +186,7 @@ def layer_inputs(wl: Workload, layer: int = 0, device="cpu") -> Dict[str, torch.
         n_r = cu[r + 1] - cu[r]
         cnt = wl.planted_per_head if wl.planted_per_head is not None else max(1, int(round(wl.planted_frac * n_r)))
         cnt = min(cnt, n_r)
-        qr = q[r * M:(r + 1) * M]                                  # [M, H, d]
-        u = _unit(qr.view(M, Hkv, g, d).mean(dim=(0, 2)))          # [H_kv, d] mean mask-query direction
+        u = u_dirs[r]                                              # [H_kv, d] mean mask-query direction
         per_head = []
         for h in range(Hkv):
             idx = torch.randperm(n_r, generator=gp, device=dev)[:cnt]
