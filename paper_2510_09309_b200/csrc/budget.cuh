@@ -10,29 +10,33 @@
 
 namespace mkv {
 
-constexpr int kBudgetThreads = 1024;
-constexpr int kBudgetMaxSegments = 8192;
+constexpr int kBudgetThreads = 256;
+constexpr int kBudgetMaxSegments = 4096;
 
 __device__ __forceinline__ double prompt_preference(float sp, float sm) {
   const double a = (double)sp, b = (double)sm;
   return __ddiv_rn(a, __dadd_rn(a, b));                 // Eq. 14
 }
 
-// dynamic shared memory: double T[R] | int k[S]
+// dynamic shared memory: double P[S] | double T[R] | int k[S]
 __global__ void __launch_bounds__(kBudgetThreads)
 budget_kernel(Shape sh, int k_l, const int32_t* __restrict__ k_l_req, double alpha, double one_minus_alpha,
               const float* __restrict__ mass_p, const float* __restrict__ mass_m, long long capacity,
               int32_t* __restrict__ budgets, int32_t* __restrict__ offsets, uint32_t* __restrict__ status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  double* T = reinterpret_cast<double*>(smem_raw);
+  const int S = sh.R * sh.Hkv;
+  double* P = reinterpret_cast<double*>(smem_raw);
+  double* T = P + S;
   int* kbuf = reinterpret_cast<int*>(T + sh.R);
   __shared__ long long warp_tot[kBudgetThreads / 32];
-  const int S = sh.R * sh.Hkv;
   const int tid = threadIdx.x;
 
+  // the divisions are the slow part (double precision): all of them in parallel, then the sums in fixed order
+  for (int s = tid; s < S; s += kBudgetThreads) P[s] = prompt_preference(mass_p[s], mass_m[s]);
+  __syncthreads();
   for (int r = tid; r < sh.R; r += kBudgetThreads) {   // sum of preferences, ascending head order
     double t = 0.0;
-    for (int h = 0; h < sh.Hkv; ++h) t = __dadd_rn(t, prompt_preference(mass_p[r * sh.Hkv + h], mass_m[r * sh.Hkv + h]));
+    for (int h = 0; h < sh.Hkv; ++h) t = __dadd_rn(t, P[r * sh.Hkv + h]);
     T[r] = t;
   }
   __syncthreads();
@@ -40,7 +44,7 @@ budget_kernel(Shape sh, int k_l, const int32_t* __restrict__ k_l_req, double alp
     const int r = s / sh.Hkv;
     const int kl = k_l_req ? k_l_req[r] : k_l;
     const int n_r = sh.prompt_cu[r + 1] - sh.prompt_cu[r];
-    const double phat = __ddiv_rn(prompt_preference(mass_p[s], mass_m[s]), T[r]);
+    const double phat = __ddiv_rn(P[s], T[r]);
     const double x = __dadd_rn(__dmul_rn(alpha, (double)kl),
                                __dmul_rn(__dmul_rn(one_minus_alpha, (double)((long long)sh.Hkv * kl)), phat));  // Eq. 15
     long long k = 0;

@@ -17,14 +17,26 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   return v;
 }
 
+constexpr int kCompactSmemSegments = 2048;             // offsets[] is staged in shared memory up to this many segments
+
 // row_bytes = d * sizeof(T); strides in bytes.  grid-stride over the rows in use (offsets[S], read on the device).
 __global__ void __launch_bounds__(kCompactThreads)
 compact_kernel(Shape sh, int row_bytes, long long ts_bytes, long long hs_bytes, const unsigned char* __restrict__ kp,
                const unsigned char* __restrict__ vp, const int32_t* __restrict__ kept_idx,
                const int32_t* __restrict__ offsets, long long capacity, unsigned char* __restrict__ kc,
                unsigned char* __restrict__ vc, uint32_t* __restrict__ status) {
+  __shared__ int32_t off_s[kCompactSmemSegments + 1];
+  __shared__ int32_t pcu_s[kCompactSmemSegments + 1];
   const int S = sh.R * sh.Hkv;
-  long long total = offsets[S];
+  const bool staged = S <= kCompactSmemSegments;        // the search below then runs out of shared memory
+  if (staged) {
+    for (int e = threadIdx.x; e <= S; e += kCompactThreads) off_s[e] = offsets[e];
+    for (int e = threadIdx.x; e <= sh.R; e += kCompactThreads) pcu_s[e] = sh.prompt_cu[e];
+    __syncthreads();
+  }
+  const int32_t* off = staged ? off_s : offsets;
+  const int32_t* pcu = staged ? pcu_s : sh.prompt_cu;
+  long long total = off[S];
   if (total > capacity) total = capacity;
   const int lane = threadIdx.x & 31;
   const int warps_per_block = kCompactThreads / 32;
@@ -32,9 +44,9 @@ compact_kernel(Shape sh, int row_bytes, long long ts_bytes, long long hs_bytes, 
   const int pieces = 2 * vec_per_row;                   // K row then V row
   for (long long t = (long long)blockIdx.x * warps_per_block + (threadIdx.x >> 5); t < total;
        t += (long long)gridDim.x * warps_per_block) {
-    const int s = find_request(offsets, S, (int)t);     // segment that owns output row t
+    const int s = find_request(off, S, (int)t);         // segment that owns output row t
     const int r = s / sh.Hkv, hk = s % sh.Hkv;
-    const int p0 = sh.prompt_cu[r], N = sh.prompt_cu[r + 1] - p0;
+    const int p0 = pcu[r], N = pcu[r + 1] - p0;
     const int j = kept_idx[t];
     if (j < 0 || j >= N) {                              // never dereference a bad index
       if (lane == 0) atomicOr(status, (uint32_t)MASKKV_FLAG_BOUNDS);
@@ -44,9 +56,9 @@ compact_kernel(Shape sh, int row_bytes, long long ts_bytes, long long hs_bytes, 
     const long long dst = t * row_bytes;
     for (int e = lane; e < pieces; e += 32) {
       const bool is_v = e >= vec_per_row;
-      const int off = (is_v ? e - vec_per_row : e) * 16;
-      const uint4 v = ld_stream(reinterpret_cast<const uint4*>((is_v ? vp : kp) + src + off));
-      *reinterpret_cast<uint4*>((is_v ? vc : kc) + dst + off) = v;
+      const int o16 = (is_v ? e - vec_per_row : e) * 16;
+      const uint4 v = ld_stream(reinterpret_cast<const uint4*>((is_v ? vp : kp) + src + o16));
+      *reinterpret_cast<uint4*>((is_v ? vc : kc) + dst + o16) = v;
     }
   }
 }

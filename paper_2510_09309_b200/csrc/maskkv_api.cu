@@ -73,11 +73,11 @@ struct ScoreWorkspace {
   int C, Tmax;
 };
 
-ScoreWorkspace score_workspace(const Shape& sh) {
+ScoreWorkspace score_workspace(const maskkv_ctx* ctx, const Shape& sh) {
   ScoreWorkspace w;
   const long long keys = (long long)sh.maxN + sh.maxM;
   w.C = (int)((keys + mkv::kStatsChunk - 1) / mkv::kStatsChunk);
-  if (w.C < mkv::tc::score_tc_max_chunks(sh)) w.C = mkv::tc::score_tc_max_chunks(sh);
+  if (ctx != nullptr && w.C < mkv::tc::score_tc_max_chunks(ctx, sh)) w.C = mkv::tc::score_tc_max_chunks(ctx, sh);
   if (w.C < 1) w.C = 1;
   w.Tmax = mkv::tc::score_tc_max_tiles(sh);               // >= ceil(keys / 128), the FP32-pipe kernel's tiling
   if (w.Tmax < 1) w.Tmax = 1;
@@ -98,8 +98,8 @@ inline int launch_status(maskkv_ctx* ctx, int n) {
 // Scoring = sweep 1 (row statistics) + merge + sweep 2 (column sums) + mass reduction.  bf16 problems run the two
 // sweeps on the tensor cores; fp32 problems (and anything the tensor-core path cannot take) on the FP32 pipes.
 template <typename T, int D>
-int launch_score(maskkv_ctx* ctx, const Shape& sh, const ScoreWorkspace& w, bool any_without_voters, const void* q,
-                 const void* kp, const void* km, const float* rw, float* scores, float* mass_p, float* mass_m,
+int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, const ScoreWorkspace& w, bool any_without_voters,
+                 const void* q, const void* kp, const void* km, const float* rw, float* scores, float* mass_p, float* mass_m,
                  unsigned char* ws, cudaStream_t st) {
   float* lse = reinterpret_cast<float*>(ws + w.lse_off);
   float2* part = reinterpret_cast<float2*>(ws + w.part_off);
@@ -108,23 +108,23 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const ScoreWorkspace& w, bool
   const bool tc_ok = mkv::tc::score_tc_supported(ctx, sh);
   int n = 0;
   if (sh.sumM > 0) {
-    int chunk_tiles = 0;
     bool done = false;
-    if (tc_ok && !(ctx->force_simt & 1u)) done = mkv::tc::launch_score_stats_tc(ctx, sh, q, kp, km, part, w.C, &chunk_tiles, st) == 0;
+    if (tc_ok && !(ctx->force_simt & 1u))
+      done = mkv::tc::launch_score_stats_tc(ctx, sh, desc->prompt_cu, desc->live_cu, q, kp, km, part, w.C, lse, st) == 0;
     if (done) ++ctx->tc_launches;
     if (!done) {
-      chunk_tiles = 0;
       const int q_tiles = (sh.maxM + mkv::kSimtThreads - 1) / mkv::kSimtThreads;
       dim3 g1((unsigned)((sh.maxN + sh.maxM + mkv::kStatsChunk - 1) / mkv::kStatsChunk), sh.H, sh.R * q_tiles);
       mkv::score_stats_simt<T, D><<<g1, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, part, w.C);
+      const long long rows = (long long)sh.H * sh.sumM;
+      mkv::score_merge_stats<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(sh, part, w.C, lse);
     }
-    const long long rows = (long long)sh.H * sh.sumM;
-    mkv::score_merge_stats<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(sh, part, w.C, chunk_tiles, lse);
     n += 2;
   }
   bool done = false;
   if (tc_ok && !(ctx->force_simt & 2u)) {
-    done = mkv::tc::launch_score_colsum_tc(ctx, sh, q, kp, km, lse, rw, scores, mass_part, w.Tmax, any_without_voters, st) == 0;
+    done = mkv::tc::launch_score_colsum_tc(ctx, sh, desc->prompt_cu, desc->live_cu, q, kp, km, lse, rw, scores, mass_part, w.Tmax,
+                                           any_without_voters, st) == 0;
     if (done) { ++ctx->tc_launches; n += any_without_voters ? 1 : 0; }
   }
   if (!done) {
@@ -214,6 +214,7 @@ int maskkv_create(maskkv_ctx** out, int device) {
     ctx->encode_tiled = nullptr;
   if (const char* e = getenv("MASKKV_FORCE_SIMT")) ctx->force_simt = (unsigned)strtoul(e, nullptr, 0);
   cudaFuncSetAttribute(mkv::select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - mkv::kSelectStaticSmem);
+  cudaFuncSetAttribute(mkv::budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
   cudaFuncSetAttribute(mkv::select_kernel_reg, cudaFuncAttributeMaxDynamicSharedMemorySize, mkv::kSelectRegKeys * 4);
   if (cudaGetLastError() != cudaSuccess) { cudaFree(ctx->status_dev); free(ctx); return MASKKV_E_CUDA; }
   *out = ctx;
@@ -247,7 +248,7 @@ size_t maskkv_workspace_bytes(const maskkv_ctx* ctx, const maskkv_desc_t* desc) 
   (void)ctx;
   Shape sh;
   if (resolve(desc, &sh) != MASKKV_OK) return 0;
-  return score_workspace(sh).total;
+  return score_workspace(ctx, sh).total;
 }
 
 int maskkv_layer_budgets(int64_t k_p, double beta, int32_t n_layers, const double* importance_host,
@@ -291,14 +292,14 @@ int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_
   if (!aligned16(q_mask_dev) || !aligned16(k_prompt_dev) || !aligned16(k_mask_dev) || !aligned16(scores_dev) ||
       !aligned16(workspace_dev))
     return MASKKV_E_ALIGN;
-  const ScoreWorkspace w = score_workspace(sh);
+  const ScoreWorkspace w = score_workspace(ctx, sh);
   if (workspace_dev == nullptr || workspace_bytes < w.total) return MASKKV_E_WORKSPACE;
   DeviceGuard guard(ctx->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   unsigned char* ws = static_cast<unsigned char*>(workspace_dev);
   bool any_without_voters = false;
   for (int r = 0; r < sh.R; ++r) any_without_voters |= desc->live_cu[r + 1] == desc->live_cu[r];
-#define MKV_SCORE(T, D) launch_score<T, D>(ctx, sh, w, any_without_voters, q_mask_dev, k_prompt_dev, k_mask_dev, row_weights_dev, scores_dev, \
+#define MKV_SCORE(T, D) launch_score<T, D>(ctx, sh, desc, w, any_without_voters, q_mask_dev, k_prompt_dev, k_mask_dev, row_weights_dev, scores_dev, \
                                                 mass_p_dev, mass_m_dev, ws, st)
   if (sh.dtype == MASKKV_F32) return sh.d == 64 ? MKV_SCORE(float, 64) : MKV_SCORE(float, 128);
   return sh.d == 64 ? MKV_SCORE(__nv_bfloat16, 64) : MKV_SCORE(__nv_bfloat16, 128);
@@ -336,7 +337,7 @@ int maskkv_budget(maskkv_ctx* ctx, const maskkv_desc_t* desc, int32_t k_l, const
   const int S = sh.R * sh.Hkv;
   if (S > mkv::kBudgetMaxSegments) return MASKKV_E_UNSUPPORTED;
   DeviceGuard guard(ctx->device);
-  const size_t smem = sizeof(double) * sh.R + sizeof(int) * S;
+  const size_t smem = sizeof(double) * (S + sh.R) + sizeof(int) * S;
   mkv::budget_kernel<<<1, mkv::kBudgetThreads, smem, static_cast<cudaStream_t>(stream)>>>(
       sh, k_l, k_l_per_request_dev, alpha, 1.0 - alpha, mass_p_dev, mass_m_dev, (long long)capacity, budgets_dev,
       offsets_dev, ctx->status_dev);

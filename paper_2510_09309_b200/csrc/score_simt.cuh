@@ -86,16 +86,14 @@ score_stats_simt(Shape sh, const T* __restrict__ q, const T* __restrict__ kp, co
   if (valid) part[((long long)h * sh.sumM + l0 + i) * C + c] = make_float2(m, l);
 }
 
-// One thread per (h, row): lse[h*sumM + row] = ln sum_j exp(s_j).  chunk_tiles = 0: partials cover kStatsChunk
-// keys each; otherwise each chunk of chunk_tiles 128-key tiles of the [prompt tiles ; mask tiles] order has two.
-__global__ void score_merge_stats(Shape sh, const float2* __restrict__ part, int C, int chunk_tiles, float* __restrict__ lse) {
+// One thread per (h, row): lse[h*sumM + row] = ln sum_j exp(s_j), from partials that cover kStatsChunk keys each.
+__global__ void score_merge_stats(Shape sh, const float2* __restrict__ part, int C, float* __restrict__ lse) {
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= (long long)sh.H * sh.sumM) return;
   const int row = (int)(t % sh.sumM);
   const int r = find_request(sh.live_cu, sh.R, row);
   const int N = sh.prompt_cu[r + 1] - sh.prompt_cu[r], M = sh.live_cu[r + 1] - sh.live_cu[r];
-  const int tiles = (N + 127) / 128 + (M + 127) / 128;
-  const int chunks = chunk_tiles > 0 ? 2 * ((tiles + chunk_tiles - 1) / chunk_tiles) : (N + M + kStatsChunk - 1) / kStatsChunk;
+  const int chunks = (N + M + kStatsChunk - 1) / kStatsChunk;
   const float2* p = part + t * C;
   float m = -INFINITY;
   for (int c = 0; c < chunks; ++c) m = fmaxf(m, p[c].x);

@@ -13,8 +13,8 @@
 //                             A_ij = 2^(s_ij*c - lse2_i) and sums over i in a register - the column sum
 //                             needs no cross-thread reduction.
 //
-// Both kernels are persistent (one CTA per SM walks a strided list of units, its TMA / MMA / epilogue
-// pipelines running on across unit boundaries) and warp-specialised: warp 0 issues TMA loads (4-stage
+// Both kernels are persistent (one CTA per SM walks an equal, contiguous share of the sweep's tiles, its
+// TMA / MMA / epilogue pipelines running on across segment boundaries) and warp-specialised: warp 0 issues TMA loads (4-stage
 // ring of key tiles), warp 1 issues the MMAs, warps 2-17 are four epilogue warpgroups - two per
 // accumulator, each taking half of its columns - so that every scheduler has four warps of
 // exponentials to interleave while the tensor pipe fills the other accumulator.  Tensor memory: 512 columns
@@ -116,35 +116,66 @@ __device__ __forceinline__ void block_teardown(uint32_t tmem_base) {
 }
 
 // =====================================================================================================
-// sweep 1: per-row (max, sum of exp) over one chunk of key tiles.
-// unit u -> (chunk, h, r, query pair); part[(h*sumM + row)*C + chunk] = (max of scaled logits, sum of exp).
+// Work distribution.  The tiles of a sweep form one flat sequence ordered by (request, group, tile), where a
+// group is a (query head, 256-query block) in sweep 1 and a KV head in sweep 2.  CTA c of G takes the
+// contiguous share [c*F/G, (c+1)*F/G) of the F tiles - every CTA gets the same number of tiles to within one -
+// and walks it one segment (a run of tiles of one group) at a time.  Every role of the CTA runs the same walk.
 // =====================================================================================================
-struct StatsUnit { int chunk, h, hk, p0, N, l0, M, q0, t_begin, nt, n_qtiles; bool valid; };
+struct Seg { int r, g, t, len, p0, N, l0, M, T; long long unit_start; };
 
-__device__ __forceinline__ StatsUnit stats_unit(const Shape& sh, int u, int chunks, int chunk_tiles) {
-  StatsUnit s;
-  const int q_pairs = (sh.maxM + kQBlock - 1) / kQBlock;
-  s.chunk = u % chunks;
-  s.h = (u / chunks) % sh.H;
-  const int z = u / (chunks * sh.H);
-  const int r = z / q_pairs;
-  s.hk = s.h / sh.g;
-  s.p0 = sh.prompt_cu[r]; s.N = sh.prompt_cu[r + 1] - s.p0;
-  s.l0 = sh.live_cu[r]; s.M = sh.live_cu[r + 1] - s.l0;
-  s.q0 = (z % q_pairs) * kQBlock;
-  const int T = (s.N + kTile - 1) / kTile + (s.M + kTile - 1) / kTile;
-  s.t_begin = s.chunk * chunk_tiles;
-  s.nt = min(s.t_begin + chunk_tiles, T) - s.t_begin;
-  s.valid = s.q0 < s.M && s.nt > 0;
-  s.n_qtiles = (s.M - s.q0 > kTile) ? 2 : 1;
-  return s;
+struct Walker {
+  long long f, f_end, base;
+  int r;
+  bool stats;
+};
+
+__device__ __forceinline__ int walk_groups(const Shape& sh, bool stats, int M) {
+  return M <= 0 ? 0 : (stats ? sh.H * ((M + kQBlock - 1) / kQBlock) : sh.Hkv);
+}
+__device__ __forceinline__ int tiles_of(int N, int M) { return (N + kTile - 1) / kTile + (M + kTile - 1) / kTile; }
+
+__device__ __forceinline__ void walker_init(Walker& w, bool stats, long long F) {
+  w.stats = stats;
+  w.f = (long long)blockIdx.x * F / gridDim.x;
+  w.f_end = (long long)(blockIdx.x + 1) * F / gridDim.x;
+  w.base = 0;
+  w.r = 0;
 }
 
+__device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, int max_len, Seg& s) {
+  if (w.f >= w.f_end) return false;
+  for (;;) {
+    s.p0 = sh.prompt_cu[w.r]; s.N = sh.prompt_cu[w.r + 1] - s.p0;
+    s.l0 = sh.live_cu[w.r]; s.M = sh.live_cu[w.r + 1] - s.l0;
+    s.T = tiles_of(s.N, s.M);
+    const long long span = (long long)walk_groups(sh, w.stats, s.M) * s.T;
+    if (w.f < w.base + span) break;
+    w.base += span;
+    ++w.r;
+  }
+  const long long rel = w.f - w.base;
+  s.r = w.r;
+  s.g = (int)(rel / s.T);
+  s.t = (int)(rel % s.T);
+  const long long room = w.f_end - w.f;
+  s.len = min(min(s.T - s.t, max_len), (int)min(room, (long long)0x7fffffff));
+  s.unit_start = w.base + (long long)s.g * s.T;
+  w.f += s.len;
+  return true;
+}
+
+// CTA whose share contains flat tile f.
+__host__ __device__ __forceinline__ int cta_of(long long f, long long F, int G) { return (int)(((f + 1) * G - 1) / F); }
+
+// =====================================================================================================
+// sweep 1: per-row (max, sum of exp) over a segment of key tiles.
+// part[(h*sumM + row)*C + 2*(cta - first cta of the row's unit) + half] = (max of scaled logits, sum of exp).
+// =====================================================================================================
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kp,
-               const __grid_constant__ CUtensorMap map_km, Shape sh, float2* __restrict__ part, int C, int chunks,
-               int chunk_tiles, int n_units, uint32_t* __restrict__ status) {
+               const __grid_constant__ CUtensorMap map_km, Shape sh, float2* __restrict__ part, int C, long long F,
+               uint32_t* __restrict__ status) {
   using S = Smem<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = align_1024(smem_raw);
@@ -154,27 +185,30 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   block_setup(bars, 4, tmem_slot, abort_flag);
   const uint32_t tmem_base = *tmem_slot;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  Walker wk;
+  walker_init(wk, true, F);
+  Seg s;
 
   if (warp == 0) {
     if (lane == 0) {
       prefetch_tmap(&map_q); prefetch_tmap(&map_kp); prefetch_tmap(&map_km);
       int kt_it = 0, q_it = 0;
       bool ok = true;
-      for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x) {
-        const StatsUnit s = stats_unit(sh, u, chunks, chunk_tiles);
-        if (!s.valid) continue;
-        if (!(ok = mbar_wait(bars.qempty, (q_it & 1) ^ 1, abort_flag, status, 0x100))) break;
+      while (ok && walker_next(wk, sh, 0x7fffffff, s)) {
+        const int qp_n = (s.M + kQBlock - 1) / kQBlock;
+        const int h = s.g / qp_n, q0 = (s.g % qp_n) * kQBlock, hk = h / sh.g;
+        if (!(ok = mbar_wait(bars.qempty, q_it & 1, abort_flag, status, 0x100))) break;   // the MMA warp released the old block
         mbar_expect_tx(bars.qfull, S::kQBytes);
-        for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kQBoxBytes, &map_q, bars.qfull, b * 64, s.h, s.l0 + s.q0);
+        for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kQBoxBytes, &map_q, bars.qfull, b * 64, h, s.l0 + q0);
         ++q_it;
-        for (int it = 0; it < s.nt; ++it, ++kt_it) {
+        for (int it = 0; it < s.len; ++it, ++kt_it) {
           const int stage = kt_it % kStages, use = kt_it / kStages;
           if (!(ok = mbar_wait(bars.empty + stage, (use & 1) ^ 1, abort_flag, status, 0x101))) break;
-          const KeyTile kt = key_tile(s.t_begin + it, s.p0, s.N, s.l0, s.M);
+          const KeyTile kt = key_tile(s.t + it, s.p0, s.N, s.l0, s.M);
           mbar_expect_tx(bars.full + stage, S::kKBytes);
           for (int b = 0; b < S::kBoxes; ++b)
             tma_load_3d(base + S::kKOff + stage * S::kKBytes + b * S::kKBoxBytes, kt.prompt ? &map_kp : &map_km, bars.full + stage,
-                        b * 64, s.hk, kt.token);
+                        b * 64, hk, kt.token);
         }
       }
       if (!ok) drain_loads(bars, kt_it);
@@ -186,18 +220,20 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       int kt_it = 0, q_it = 0;
       uint32_t cnt[2] = {0u, 0u};                            // tiles issued per query tile
       bool ok = true;
-      for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x) {
-        const StatsUnit s = stats_unit(sh, u, chunks, chunk_tiles);
-        if (!s.valid) continue;
+      while (ok && walker_next(wk, sh, 0x7fffffff, s)) {
+        const int qp_n = (s.M + kQBlock - 1) / kQBlock;
+        const int q0 = (s.g % qp_n) * kQBlock;
+        const int n_qtiles = (s.M - q0 > kTile) ? 2 : 1;
+        umma_commit(bars.qempty);                            // every MMA that read the resident queries has been issued
         if (!(ok = mbar_wait(bars.qfull, q_it & 1, abort_flag, status, 0x102))) break;
         ++q_it;
         tc_fence_after();
-        for (int it = 0; ok && it < s.nt; ++it, ++kt_it) {
+        for (int it = 0; ok && it < s.len; ++it, ++kt_it) {
           const int stage = kt_it % kStages, use = kt_it / kStages;
           if (!(ok = mbar_wait(bars.full + stage, use & 1, abort_flag, status, 0x103))) break;
           tc_fence_after();
           const uint32_t k_addr = smem_u32(base + S::kKOff + stage * S::kKBytes);
-          for (int a = 0; a < s.n_qtiles; ++a) {
+          for (int a = 0; a < n_qtiles; ++a) {
             const int acc = a * 2 + (cnt[a] & 1);
             if (!(ok = mbar_wait(bars.tempty + acc, ((cnt[a] >> 1) & 1) ^ 1, abort_flag, status, 0x104))) break;
             tc_fence_after();
@@ -213,7 +249,6 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           }
           umma_commit(bars.empty + stage);
         }
-        umma_commit(bars.qempty);
       }
     }
   } else {
@@ -226,9 +261,11 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const float cs = sh.scale * kLog2e;
     uint32_t cnt = 0;
     bool ok = true;
-    for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x) {
-      const StatsUnit s = stats_unit(sh, u, chunks, chunk_tiles);
-      if (!s.valid || a >= s.n_qtiles) continue;
+    while (ok && walker_next(wk, sh, 0x7fffffff, s)) {
+      const int qp_n = (s.M + kQBlock - 1) / kQBlock;
+      const int h = s.g / qp_n, q0 = (s.g % qp_n) * kQBlock;
+      const int n_qtiles = (s.M - q0 > kTile) ? 2 : 1;
+      if (a >= n_qtiles) continue;
       float m = -INFINITY, l = 0.f;                         // m in raw (unscaled) logits
       auto absorb = [&](float* v, int col0, int valid) {
         if (valid - col0 < 32) {
@@ -245,11 +282,11 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         for (int c = 0; c < 32; c += 2) { l0 += ex2(fmaf(v[c], cs, neg)); l1 += ex2(fmaf(v[c + 1], cs, neg)); }
         l += l0 + l1;
       };
-      for (int it = 0; ok && it < s.nt; ++it, ++cnt) {
+      for (int it = 0; ok && it < s.len; ++it, ++cnt) {
         const int acc = a * 2 + (cnt & 1);
         if (!(ok = mbar_wait(bars.tfull + acc, (cnt >> 1) & 1, abort_flag, status, 0x105))) break;
         tc_fence_after();
-        const int valid = key_tile(s.t_begin + it, s.p0, s.N, s.l0, s.M).valid;
+        const int valid = key_tile(s.t + it, s.p0, s.N, s.l0, s.M).valid;
         const int col0 = half * 64;
         const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + acc * kTile + col0;
         const int n_chunks = valid > col0 + 32 ? 2 : (valid > col0 ? 1 : 0);
@@ -262,42 +299,49 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         if (n_chunks > 0) absorb(va, col0, valid);
         if (n_chunks > 1) absorb(vb, col0 + 32, valid);
       }
-      const int i = s.q0 + a * kTile + row;
-      if (ok && i < s.M) part[((long long)s.h * sh.sumM + s.l0 + i) * C + s.chunk * 2 + half] = make_float2(m * sh.scale, l);
+      const int i = q0 + a * kTile + row;
+      const int slot = 2 * ((int)blockIdx.x - cta_of(s.unit_start, F, gridDim.x)) + half;
+      if (ok && i < s.M) part[((long long)h * sh.sumM + s.l0 + i) * C + slot] = make_float2(m * sh.scale, l);
     }
   }
   block_teardown(tmem_base);
 }
 
+// One thread per (h, row): lse[h*sumM + row] = ln sum_j exp(s_j), from the partials the CTAs of sweep 1 left.
+__global__ void score_merge_stats_tc(Shape sh, const float2* __restrict__ part, int C, long long F, int G,
+                                     float* __restrict__ lse) {
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= (long long)sh.H * sh.sumM) return;
+  const int h = (int)(t / sh.sumM), row = (int)(t % sh.sumM);
+  const int r = find_request(sh.live_cu, sh.R, row);
+  long long base = 0;
+  for (int r2 = 0; r2 < r; ++r2) {
+    const int N2 = sh.prompt_cu[r2 + 1] - sh.prompt_cu[r2], M2 = sh.live_cu[r2 + 1] - sh.live_cu[r2];
+    base += (long long)walk_groups(sh, true, M2) * tiles_of(N2, M2);
+  }
+  const int N = sh.prompt_cu[r + 1] - sh.prompt_cu[r], l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
+  const int T = tiles_of(N, M), qp_n = (M + kQBlock - 1) / kQBlock;
+  const long long unit_start = base + ((long long)h * qp_n + (row - l0) / kQBlock) * T;
+  const int slots = 2 * (cta_of(unit_start + T - 1, F, G) - cta_of(unit_start, F, G) + 1);
+  const float2* p = part + t * C;
+  float m = -INFINITY;
+  for (int c = 0; c < slots; ++c) m = fmaxf(m, p[c].x);
+  float l = 0.f;
+  for (int c = 0; c < slots; ++c) l += p[c].y * expf(p[c].x - m);
+  lse[t] = m + logf(l);
+}
+
 // =====================================================================================================
-// sweep 2: column sums.  unit u -> (tile group, hk, r).
+// sweep 2: column sums.
 // scores[hk][p0 + j] = sum over the group's query heads and mask rows of w_i * exp(s_ij - lse_i);
 // mass_part[((r*H_kv + hk)*Tmax + t)*4 + w] = (sum over prompt keys, sum over mask keys) of tile t seen by warp w.
 // =====================================================================================================
-struct ColsumUnit { int hk, r, p0, N, l0, M, t_begin, nt, nqb, q_per_head; bool valid; };
-
-__device__ __forceinline__ ColsumUnit colsum_unit(const Shape& sh, int u, int groups, int tiles_per_unit) {
-  ColsumUnit c;
-  const int tg = u % groups;
-  c.hk = (u / groups) % sh.Hkv;
-  c.r = u / (groups * sh.Hkv);
-  c.p0 = sh.prompt_cu[c.r]; c.N = sh.prompt_cu[c.r + 1] - c.p0;
-  c.l0 = sh.live_cu[c.r]; c.M = sh.live_cu[c.r + 1] - c.l0;
-  const int T = (c.N + kTile - 1) / kTile + (c.M + kTile - 1) / kTile;
-  c.t_begin = tg * tiles_per_unit;
-  c.nt = min(c.t_begin + tiles_per_unit, T) - c.t_begin;
-  c.q_per_head = (c.M + kQBlock - 1) / kQBlock;
-  c.nqb = sh.g * c.q_per_head;
-  c.valid = c.nt > 0 && c.M > 0;
-  return c;
-}
-
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kp,
                 const __grid_constant__ CUtensorMap map_km, Shape sh, const float* __restrict__ lse,
                 const float* __restrict__ w, float* __restrict__ scores, float2* __restrict__ mass_part, int Tmax,
-                int groups, int tiles_per_unit, int n_units, uint32_t* __restrict__ status) {
+                long long F, uint32_t* __restrict__ status) {
   using S = Smem<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = align_1024(smem_raw);
@@ -309,28 +353,36 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   block_setup(bars, 2, tmem_slot, abort_flag);
   const uint32_t tmem_base = *tmem_slot;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  Walker wk;
+  walker_init(wk, false, F);
+  Seg s;
+  int last_r = -1, last_g = -1;                             // the (request, KV head) whose queries are resident
 
   if (warp == 0) {
     if (lane == 0) {
       prefetch_tmap(&map_q); prefetch_tmap(&map_kp); prefetch_tmap(&map_km);
       int kt_it = 0, q_it = 0;
       bool ok = true;
-      for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x) {
-        const ColsumUnit c = colsum_unit(sh, u, groups, tiles_per_unit);
-        if (!c.valid) continue;
-        for (int qb = 0; ok && qb < c.nqb; ++qb, ++q_it) {
-          const int h = c.hk * sh.g + qb / c.q_per_head, q0 = (qb % c.q_per_head) * kQBlock;
-          if (!(ok = mbar_wait(bars.qempty, (q_it & 1) ^ 1, abort_flag, status, 0x201))) break;
-          mbar_expect_tx(bars.qfull, S::kQBytes);
-          for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kQBoxBytes, &map_q, bars.qfull, b * 64, h, c.l0 + q0);
-          for (int tl = 0; tl < c.nt; ++tl, ++kt_it) {
+      while (ok && walker_next(wk, sh, kColsumMaxTiles, s)) {
+        const int q_per_head = (s.M + kQBlock - 1) / kQBlock, nqb = sh.g * q_per_head;
+        const bool reuse_q = nqb == 1 && s.r == last_r && s.g == last_g;
+        last_r = s.r; last_g = s.g;
+        for (int qb = 0; ok && qb < nqb; ++qb) {
+          if (!reuse_q) {
+            const int h = s.g * sh.g + qb / q_per_head, q0 = (qb % q_per_head) * kQBlock;
+            if (!(ok = mbar_wait(bars.qempty, q_it & 1, abort_flag, status, 0x201))) break;
+            mbar_expect_tx(bars.qfull, S::kQBytes);
+            for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kQBoxBytes, &map_q, bars.qfull, b * 64, h, s.l0 + q0);
+            ++q_it;
+          }
+          for (int tl = 0; tl < s.len; ++tl, ++kt_it) {
             const int stage = kt_it % kStages, use = kt_it / kStages;
             if (!(ok = mbar_wait(bars.empty + stage, (use & 1) ^ 1, abort_flag, status, 0x202))) break;
-            const KeyTile kt = key_tile(c.t_begin + tl, c.p0, c.N, c.l0, c.M);
+            const KeyTile kt = key_tile(s.t + tl, s.p0, s.N, s.l0, s.M);
             mbar_expect_tx(bars.full + stage, S::kKBytes);
             for (int b = 0; b < S::kBoxes; ++b)
               tma_load_3d(base + S::kKOff + stage * S::kKBytes + b * S::kKBoxBytes, kt.prompt ? &map_kp : &map_km,
-                          bars.full + stage, b * 64, c.hk, kt.token);
+                          bars.full + stage, b * 64, s.g, kt.token);
           }
         }
       }
@@ -342,16 +394,21 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       uint32_t uses[2] = {0u, 0u};
       bool ok = true;
       const uint32_t q_addr = smem_u32(base + S::kQOff);
-      for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x) {
-        const ColsumUnit c = colsum_unit(sh, u, groups, tiles_per_unit);
-        if (!c.valid) continue;
-        for (int qb = 0; ok && qb < c.nqb; ++qb, ++q_it) {
-          const int q0 = (qb % c.q_per_head) * kQBlock;
-          const int n_mma = (min(kQBlock, c.M - q0) + 31) & ~31;           // columns the epilogue will read
+      while (ok && walker_next(wk, sh, kColsumMaxTiles, s)) {
+        const int q_per_head = (s.M + kQBlock - 1) / kQBlock, nqb = sh.g * q_per_head;
+        const bool reuse_q = nqb == 1 && s.r == last_r && s.g == last_g;
+        last_r = s.r; last_g = s.g;
+        for (int qb = 0; ok && qb < nqb; ++qb) {
+          const int q0 = (qb % q_per_head) * kQBlock;
+          const int n_mma = (min(kQBlock, s.M - q0) + 31) & ~31;           // columns the epilogue will read
           const uint32_t idesc = idesc_bf16_f32(kTile, n_mma);
-          if (!(ok = mbar_wait(bars.qfull, q_it & 1, abort_flag, status, 0x203))) break;
-          tc_fence_after();
-          for (int tl = 0; tl < c.nt; ++tl, ++kt_it) {
+          if (!reuse_q) {
+            umma_commit(bars.qempty);                        // every MMA that read the resident queries has been issued
+            if (!(ok = mbar_wait(bars.qfull, q_it & 1, abort_flag, status, 0x203))) break;
+            ++q_it;
+            tc_fence_after();
+          }
+          for (int tl = 0; tl < s.len; ++tl, ++kt_it) {
             const int stage = kt_it % kStages, use = kt_it / kStages, buf = (tl + base_par) & 1;
             if (!(ok = mbar_wait(bars.full + stage, use & 1, abort_flag, status, 0x204))) break;
             if (!(ok = mbar_wait(bars.tempty + buf, (uses[buf] & 1) ^ 1, abort_flag, status, 0x205))) break;
@@ -367,18 +424,17 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             umma_commit(bars.tfull + buf);
             ++uses[buf];
           }
-          umma_commit(bars.qempty);
         }
-        base_par ^= c.nt & 1;
+        base_par ^= s.len & 1;
       }
     }
   } else {
     // Four warpgroups: accumulator buf = wg >> 1, and of its (up to) 256 query columns the 128-column half (wg & 1).
     // The two halves of a key's sum meet in shared memory (one named barrier per tile per pair); the half-0 thread
-    // owns the key from then on.  Inside a unit the tile -> accumulator map is fixed, (tl + base_par) & 1, so a key's
-    // running sum in shared memory always belongs to the same thread; base_par carries the alternation across units.
-    // After a failed wait a thread skips the arithmetic but still walks the loops, so that every thread reaches every
-    // named barrier.
+    // owns the key from then on.  Inside a segment the tile -> accumulator map is fixed, (tl + base_par) & 1, so a
+    // key's running sum in shared memory always belongs to the same thread; base_par carries the alternation across
+    // segments.  After a failed wait a thread skips the arithmetic but still walks the loops, so that every thread
+    // reaches every named barrier.
     const int wg = (warp - 2) >> 2;
     const int buf = wg >> 1, half = wg & 1;
     const int lane_group = warp & 3;
@@ -389,20 +445,24 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     uint32_t uses = 0, c2_it = 0;
     int base_par = 0;
     bool ok = true;
-    for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
-      const ColsumUnit c = colsum_unit(sh, u, groups, tiles_per_unit);
-      if (!c.valid) continue;
-      const int seg = c.r * sh.Hkv + c.hk;
-      for (int qb = 0; qb < c.nqb; ++qb, ++c2_it) {
-        const int h = c.hk * sh.g + qb / c.q_per_head, q0 = (qb % c.q_per_head) * kQBlock + half * kTile;
-        const int nq = max(0, min(kTile, c.M - q0));        // voters in this warpgroup's half of the block
-        float* c2 = c2s + (wg * 2 + (c2_it & 1)) * kTile;
-        {
+    const float* c2 = c2s;
+    while (walker_next(wk, sh, kColsumMaxTiles, s)) {
+      const int q_per_head = (s.M + kQBlock - 1) / kQBlock, nqb = sh.g * q_per_head;
+      const bool reuse_q = nqb == 1 && s.r == last_r && s.g == last_g;
+      last_r = s.r; last_g = s.g;
+      const int seg = s.r * sh.Hkv + s.g;
+      for (int qb = 0; qb < nqb; ++qb) {
+        const int h = s.g * sh.g + qb / q_per_head, q0 = (qb % q_per_head) * kQBlock + half * kTile;
+        const int nq = max(0, min(kTile, s.M - q0));        // voters in this warpgroup's half of the block
+        if (!reuse_q) {
+          float* c2w = c2s + (wg * 2 + (c2_it & 1)) * kTile;
+          ++c2_it;
           float cst = INFINITY;                             // 2^(x - inf) = 0: rows that do not exist never vote
-          if (row < nq) cst = lse[(long long)h * sh.sumM + c.l0 + q0 + row] * kLog2e - (w ? log2f(w[c.l0 + q0 + row]) : 0.f);
-          c2[row] = cst;
+          if (row < nq) cst = lse[(long long)h * sh.sumM + s.l0 + q0 + row] * kLog2e - (w ? log2f(w[s.l0 + q0 + row]) : 0.f);
+          c2w[row] = cst;
+          named_barrier(1 + wg, kTile);
+          c2 = c2w;
         }
-        named_barrier(1 + wg, kTile);
         const int chunks = (nq + 31) >> 5;
         auto absorb = [&](const float* v, int cb, float& a0, float& a1) {
           const float4* cc = reinterpret_cast<const float4*>(c2 + cb * 32);
@@ -415,7 +475,7 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             a1 += ex2(fmaf(v[4 * c4 + 3], cs, -k4.w));
           }
         };
-        for (int tl = (buf + base_par) & 1; tl < c.nt; tl += 2) {
+        for (int tl = (buf + base_par) & 1; tl < s.len; tl += 2) {
           float a0 = 0.f, a1 = 0.f;
           if (ok) ok = mbar_wait(bars.tfull + buf, uses & 1, abort_flag, status, 0x206);
           if (ok) {
@@ -437,19 +497,19 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           named_barrier(5 + buf, 2 * kTile);                // the pair's two halves of this tile are done
           if (half == 1 || !ok) continue;
           float acc = (a0 + a1) + slot[row];
-          if (c.nqb > 1) {                                  // grouped heads / more than 256 voters: sum over query blocks
+          if (nqb > 1) {                                    // grouped heads / more than 256 voters: sum over query blocks
             if (qb > 0) acc += accs[tl * kTile + row];
-            if (qb + 1 < c.nqb) { accs[tl * kTile + row] = acc; continue; }
+            if (qb + 1 < nqb) { accs[tl * kTile + row] = acc; continue; }
           }
-          const KeyTile kt = key_tile(c.t_begin + tl, c.p0, c.N, c.l0, c.M);
+          const KeyTile kt = key_tile(s.t + tl, s.p0, s.N, s.l0, s.M);
           if (row >= kt.valid) acc = 0.f;
-          if (kt.prompt && row < kt.valid) scores[(long long)c.hk * sh.sumN + kt.token + row] = acc;
+          if (kt.prompt && row < kt.valid) scores[(long long)s.g * sh.sumN + kt.token + row] = acc;
           acc = warp_sum(acc);
           if (lane == 0)
-            mass_part[((long long)seg * Tmax + c.t_begin + tl) * 4 + lane_group] = kt.prompt ? make_float2(acc, 0.f) : make_float2(0.f, acc);
+            mass_part[((long long)seg * Tmax + s.t + tl) * 4 + lane_group] = kt.prompt ? make_float2(acc, 0.f) : make_float2(0.f, acc);
         }
       }
-      base_par ^= c.nt & 1;
+      base_par ^= s.len & 1;
     }
   }
   block_teardown(tmem_base);
@@ -482,18 +542,16 @@ bool build_maps(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kp,
          make_tmap_rows(ctx->encode_tiled, &m->km, km, sh.d, sh.Hkv, sh.sumM, sh.kv_hs * 2, sh.kv_ts * 2, kTile);
 }
 
-// Tiles per unit: small enough that the persistent CTAs end within a few percent of each other, large enough
-// that the resident query block (reloaded per unit) is amortised.
-int pick_tiles(int tiles, long long units, int sm_count, int lo, int hi) {
-  int best = lo;
-  double best_cost = 1e300;
-  for (int tp = lo; tp <= hi; ++tp) {
-    const long long n = units * ((tiles + tp - 1) / tp);
-    const long long per_cta = (n + sm_count - 1) / sm_count;
-    const double cost = (double)per_cta * (tp + 1.5);      // +1.5 tiles: query load and pipeline refill per unit
-    if (cost < best_cost) { best_cost = cost; best = tp; }
+// F of the walk: tiles over all (request, group) pairs, from the host's copy of the lengths.
+long long flat_tiles(const Shape& sh, const int32_t* prompt_cu, const int32_t* live_cu, bool stats) {
+  long long F = 0;
+  for (int r = 0; r < sh.R; ++r) {
+    const int N = prompt_cu[r + 1] - prompt_cu[r], M = live_cu[r + 1] - live_cu[r];
+    if (M <= 0) continue;
+    const long long groups = stats ? (long long)sh.H * ((M + kQBlock - 1) / kQBlock) : sh.Hkv;
+    F += groups * ((N + kTile - 1) / kTile + (M + kTile - 1) / kTile);
   }
-  return best;
+  return F;
 }
 
 template <int D>
@@ -508,9 +566,13 @@ cudaError_t set_smem_attr() {
 
 }  // namespace
 
-int score_tc_max_chunks(const Shape& sh) {
+int score_tc_max_chunks(const maskkv_ctx* ctx, const Shape& sh) {
+  // partials per row in sweep 1: two per CTA that touches the row's unit.  A unit of T tiles lies inside a request
+  // that contributes at least H*T tiles to the walk, so a CTA's share is at least floor(H*T/G) >= H*T/(2G) tiles (or
+  // one tile) and the unit spans at most 2*ceil(G/H) + 1 shares - and never more than T.
   const int T = (sh.maxN + kTile - 1) / kTile + (sh.maxM + kTile - 1) / kTile;
-  return 2 * ((T + 3) / 4);                                 // a chunk never has fewer than 4 tiles and yields 2 partials per row
+  const int span = 2 * ((ctx->sm_count + sh.H - 1) / sh.H) + 2;
+  return 2 * (span < T ? span : T);
 }
 
 int score_tc_max_tiles(const Shape& sh) { return (sh.maxN + kTile - 1) / kTile + (sh.maxM + kTile - 1) / kTile; }
@@ -520,52 +582,45 @@ bool score_tc_supported(const maskkv_ctx* ctx, const Shape& sh) {
          ctx->smem_optin >= Smem<128>::kDynamic;
 }
 
-int launch_score_stats_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kp, const void* km, float2* part,
-                          int C, int* chunk_tiles_out, cudaStream_t st) {
+int launch_score_stats_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prompt_cu_host, const int32_t* live_cu_host,
+                          const void* q, const void* kp, const void* km, float2* part, int C, float* lse, cudaStream_t st) {
   Maps m;
   if (!build_maps(ctx, sh, q, kp, km, &m)) return 1;
-  const int T = score_tc_max_tiles(sh);
-  const int q_pairs = (sh.maxM + kQBlock - 1) / kQBlock;
-  int ct = pick_tiles(T, (long long)sh.H * sh.R * q_pairs, ctx->sm_count, 4, 32);
-  while (2 * ((T + ct - 1) / ct) > C) ++ct;
-  *chunk_tiles_out = ct;
-  const int chunks = (T + ct - 1) / ct;
-  const long long n_units = (long long)chunks * sh.H * sh.R * q_pairs;
-  if (n_units > 0x7fffffffLL) return 1;
-  const int grid = (int)(n_units < ctx->sm_count ? n_units : ctx->sm_count);
+  const long long F = flat_tiles(sh, prompt_cu_host, live_cu_host, true);
+  if (F <= 0) return 1;
+  const int grid = (int)(F < ctx->sm_count ? F : ctx->sm_count);
   if (sh.d == 128) {
     if (set_smem_attr<128>() != cudaSuccess) return 1;
-    score_stats_tc<128><<<grid, kThreads, Smem<128>::kDynamic, st>>>(m.q, m.kp, m.km, sh, part, C, chunks, ct, (int)n_units, ctx->status_dev);
+    score_stats_tc<128><<<grid, kThreads, Smem<128>::kDynamic, st>>>(m.q, m.kp, m.km, sh, part, C, F, ctx->status_dev);
   } else {
     if (set_smem_attr<64>() != cudaSuccess) return 1;
-    score_stats_tc<64><<<grid, kThreads, Smem<64>::kDynamic, st>>>(m.q, m.kp, m.km, sh, part, C, chunks, ct, (int)n_units, ctx->status_dev);
+    score_stats_tc<64><<<grid, kThreads, Smem<64>::kDynamic, st>>>(m.q, m.kp, m.km, sh, part, C, F, ctx->status_dev);
   }
+  const long long rows = (long long)sh.H * sh.sumM;
+  score_merge_stats_tc<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(sh, part, C, F, grid, lse);
   return 0;
 }
 
-int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kp, const void* km, const float* lse,
-                           const float* w, float* scores, float2* mass_part, int Tmax, bool any_without_voters,
-                           cudaStream_t st) {
+int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prompt_cu_host, const int32_t* live_cu_host,
+                           const void* q, const void* kp, const void* km, const float* lse, const float* w, float* scores,
+                           float2* mass_part, int Tmax, bool any_without_voters, cudaStream_t st) {
   Maps m;
   if (!build_maps(ctx, sh, q, kp, km, &m)) return 1;
-  const int T = score_tc_max_tiles(sh);
-  const int tp = pick_tiles(T, (long long)sh.Hkv * sh.R, ctx->sm_count, 4, kColsumMaxTiles);
-  const int groups = (T + tp - 1) / tp;
-  const long long n_units = (long long)groups * sh.Hkv * sh.R;
-  if (n_units > 0x7fffffffLL) return 1;
-  const int grid = (int)(n_units < ctx->sm_count ? n_units : ctx->sm_count);
+  const long long F = flat_tiles(sh, prompt_cu_host, live_cu_host, false);
+  if (F <= 0) return 1;
+  const int grid = (int)(F < ctx->sm_count ? F : ctx->sm_count);
   if (any_without_voters) {
-    dim3 gz(T, sh.Hkv, sh.R);
+    dim3 gz(score_tc_max_tiles(sh), sh.Hkv, sh.R);
     score_zero_fill<<<gz, kTile, 0, st>>>(sh, scores, mass_part, Tmax);
   }
   if (sh.d == 128) {
     if (set_smem_attr<128>() != cudaSuccess) return 1;
-    score_colsum_tc<128><<<grid, kThreads, Smem<128>::kDynamic, st>>>(m.q, m.kp, m.km, sh, lse, w, scores, mass_part, Tmax, groups, tp,
-                                                                      (int)n_units, ctx->status_dev);
+    score_colsum_tc<128><<<grid, kThreads, Smem<128>::kDynamic, st>>>(m.q, m.kp, m.km, sh, lse, w, scores, mass_part, Tmax, F,
+                                                                      ctx->status_dev);
   } else {
     if (set_smem_attr<64>() != cudaSuccess) return 1;
-    score_colsum_tc<64><<<grid, kThreads, Smem<64>::kDynamic, st>>>(m.q, m.kp, m.km, sh, lse, w, scores, mass_part, Tmax, groups, tp,
-                                                                     (int)n_units, ctx->status_dev);
+    score_colsum_tc<64><<<grid, kThreads, Smem<64>::kDynamic, st>>>(m.q, m.kp, m.km, sh, lse, w, scores, mass_part, Tmax, F,
+                                                                     ctx->status_dev);
   }
   return 0;
 }

@@ -9,15 +9,16 @@ namespace tc {
 // True when the tcgen05 path can serve this problem (bf16, tensor-map encoder resolved, voters present).
 bool score_tc_supported(const maskkv_ctx* ctx, const Shape& sh);
 // Upper bounds used to size the workspace: partials per row in sweep 1, key tiles per request in sweep 2.
-int score_tc_max_chunks(const Shape& sh);
+int score_tc_max_chunks(const maskkv_ctx* ctx, const Shape& sh);
 int score_tc_max_tiles(const Shape& sh);
 
-// Each returns 0 after a launch, 1 when nothing was launched (tensor map or attribute set-up failed).
-int launch_score_stats_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kp, const void* km, float2* part,
-                          int C, int* chunk_tiles_out, cudaStream_t st);
-int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kp, const void* km, const float* lse,
-                           const float* w, float* scores, float2* mass_part, int Tmax, bool any_without_voters,
-                           cudaStream_t st);
+// Each returns 0 after its launches, 1 when nothing was launched (tensor map or attribute set-up failed).
+// The *_host arrays are the descriptor's cumulative lengths.  Sweep 1 also launches its merge kernel (-> lse).
+int launch_score_stats_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prompt_cu_host, const int32_t* live_cu_host,
+                          const void* q, const void* kp, const void* km, float2* part, int C, float* lse, cudaStream_t st);
+int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prompt_cu_host, const int32_t* live_cu_host,
+                           const void* q, const void* kp, const void* km, const float* lse, const float* w, float* scores,
+                           float2* mass_part, int Tmax, bool any_without_voters, cudaStream_t st);
 
 }  // namespace tc
 }  // namespace mkv
