@@ -40,12 +40,9 @@ struct ASmem {
   static constexpr int kDynamic = kBytes + 1024;
 };
 
-// Shared-memory descriptor of an N-major (row = k index, 64 contiguous n per 128-byte row) operand with
-// 128-byte swizzle: 8-row groups 1024 bytes apart along k, the next 64 columns `n_stride` bytes away.
-__device__ __forceinline__ uint64_t smem_desc_sw128_nmajor(uint32_t saddr, uint32_t n_stride) {
-  return (uint64_t)((saddr & 0x3ffffu) >> 4) | ((uint64_t)(n_stride >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
-         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
+// The value operand V is row-major in shared memory (row = k index, 64 contiguous n per 128-byte row): an N-major
+// descriptor with 128-byte swizzle - 8-row groups 1024 bytes apart along k, the next 64 columns one box away
+// (that distance goes into the leading-byte-offset field of the low word).
 // bf16 x bf16 -> fp32, A K-major (tensor memory), B N-major.
 __device__ __forceinline__ uint32_t idesc_bf16_f32_bn(uint32_t m, uint32_t n) { return idesc_bf16_f32(m, n) | (1u << 16); }
 
@@ -183,19 +180,18 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     if (lane == 0) {
       const uint32_t idesc_qk = idesc_bf16_f32(kATile, kATile);
       const uint32_t idesc_pv = idesc_bf16_f32_bn(kATile, D);
-      const uint32_t q_addr = smem_u32(base + S::kQOff);
+      const uint32_t q_lo = smem_desc_lo(smem_u32(base + S::kQOff));
       bool ok = mbar_wait(bars.qfull, 0, abort_flag, status, 0x303);
       tc_fence_after();
       auto issue_qk = [&](int j) -> bool {
         const int stage = j % kAStages, use = j / kAStages;
         if (!mbar_wait(bars.kfull + stage, use & 1, abort_flag, status, 0x304)) return false;
         tc_fence_after();
-        const uint32_t k_addr = smem_u32(base + S::kKOff + stage * S::kTileBytes);
+        const uint32_t k_lo = smem_desc_lo(smem_u32(base + S::kKOff + stage * S::kTileBytes));
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint64_t adesc = smem_desc_sw128(q_addr + (kk >> 2) * S::kBoxBytes + (kk & 3) * 32);
-          const uint64_t bdesc = smem_desc_sw128(k_addr + (kk >> 2) * S::kBoxBytes + (kk & 3) * 32);
-          umma_ss(tm_s + (j & 1) * kATile, adesc, bdesc, idesc_qk, kk > 0);
+          const uint32_t o = ((kk >> 2) * S::kBoxBytes + (kk & 3) * 32) >> 4;
+          umma_ss(tm_s + (j & 1) * kATile, make_desc(q_lo + o, kDescHiSw128), make_desc(k_lo + o, kDescHiSw128), idesc_qk, kk > 0);
         }
         umma_commit(bars.sfull + (j & 1));
         umma_commit(bars.kempty + stage);
@@ -209,12 +205,11 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         if (!(ok = mbar_wait(bars.oempty + b, ((j >> 1) & 1) ^ 1, abort_flag, status, 0x306))) break;
         if (!(ok = mbar_wait(bars.pready + b, (j >> 1) & 1, abort_flag, status, 0x307))) break;
         tc_fence_after();
-        const uint32_t v_addr = smem_u32(base + S::kVOff + stage * S::kTileBytes);
+        // N-major descriptor: low word = address | (box stride between the two 64-column halves), high word as K-major
+        const uint32_t v_lo = ((smem_u32(base + S::kVOff + stage * S::kTileBytes) & 0x3ffffu) >> 4) | ((uint32_t)(S::kBoxBytes >> 4) << 16);
 #pragma unroll
-        for (int kk = 0; kk < kATile / 16; ++kk) {
-          const uint64_t bdesc = smem_desc_sw128_nmajor(v_addr + kk * 16 * 128, S::kBoxBytes);
-          umma_ts(tm_o + b * kATile, tm_s + b * kATile + kk * 8, bdesc, idesc_pv, kk > 0);
-        }
+        for (int kk = 0; kk < kATile / 16; ++kk)
+          umma_ts(tm_o + b * kATile, tm_s + b * kATile + kk * 8, make_desc(v_lo + ((kk * 16 * 128) >> 4), kDescHiSw128), idesc_pv, kk > 0);
         umma_commit(bars.ofull + b);
         umma_commit(bars.vempty + stage);
       }

@@ -121,12 +121,12 @@ __device__ __forceinline__ void block_teardown(uint32_t tmem_base) {
 // contiguous share [c*F/G, (c+1)*F/G) of the F tiles - every CTA gets the same number of tiles to within one -
 // and walks it one segment (a run of tiles of one group) at a time.  Every role of the CTA runs the same walk.
 // =====================================================================================================
-struct Seg { int r, g, t, len, p0, N, l0, M, T; long long unit_start; };
+struct Seg { int r, g, t, len, p0, N, l0, M, T, dir; long long unit_start; };   // tiles t, t+dir, ..., len of them
 
 struct Walker {
-  long long f, f_end, base;
+  long long f, f_end, base;   // forward: [f, f_end) still to do; reverse: [f_end, f) still to do, taken from the top
   int r;
-  bool stats;
+  bool stats, reverse;
 };
 
 __device__ __forceinline__ int walk_groups(const Shape& sh, bool stats, int M) {
@@ -134,33 +134,70 @@ __device__ __forceinline__ int walk_groups(const Shape& sh, bool stats, int M) {
 }
 __device__ __forceinline__ int tiles_of(int N, int M) { return (N + kTile - 1) / kTile + (M + kTile - 1) / kTile; }
 
-__device__ __forceinline__ void walker_init(Walker& w, bool stats, long long F) {
+// Sweep 2 walks every share backwards: it then starts on the tiles sweep 1 read last, which are the ones most
+// likely to be still in L2 (the key tensor of a long prompt is larger than L2, so a forward walk would miss all).
+__device__ __forceinline__ void walker_init(Walker& w, const Shape& sh, bool stats, bool reverse, long long F) {
   w.stats = stats;
-  w.f = (long long)blockIdx.x * F / gridDim.x;
-  w.f_end = (long long)(blockIdx.x + 1) * F / gridDim.x;
+  w.reverse = reverse;
+  const long long lo = (long long)blockIdx.x * F / gridDim.x, hi = (long long)(blockIdx.x + 1) * F / gridDim.x;
   w.base = 0;
   w.r = 0;
+  if (!reverse) { w.f = lo; w.f_end = hi; return; }
+  w.f = hi; w.f_end = lo;
+  // position (r, base) on the request that holds the last tile of the share
+  for (;;) {
+    const int N = sh.prompt_cu[w.r + 1] - sh.prompt_cu[w.r], M = sh.live_cu[w.r + 1] - sh.live_cu[w.r];
+    const long long span = (long long)walk_groups(sh, stats, M) * tiles_of(N, M);
+    if (hi <= lo || hi - 1 < w.base + span || w.r + 1 >= sh.R) break;
+    w.base += span;
+    ++w.r;
+  }
 }
 
 __device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, int max_len, Seg& s) {
-  if (w.f >= w.f_end) return false;
+  if (!w.reverse) {
+    if (w.f >= w.f_end) return false;
+    for (;;) {
+      s.p0 = sh.prompt_cu[w.r]; s.N = sh.prompt_cu[w.r + 1] - s.p0;
+      s.l0 = sh.live_cu[w.r]; s.M = sh.live_cu[w.r + 1] - s.l0;
+      s.T = tiles_of(s.N, s.M);
+      const long long span = (long long)walk_groups(sh, w.stats, s.M) * s.T;
+      if (w.f < w.base + span) break;
+      w.base += span;
+      ++w.r;
+    }
+    const long long rel = w.f - w.base;
+    s.r = w.r;
+    s.g = (int)(rel / s.T);
+    s.t = (int)(rel % s.T);
+    s.dir = 1;
+    const long long room = w.f_end - w.f;
+    s.len = min(min(s.T - s.t, max_len), (int)min(room, (long long)0x7fffffff));
+    s.unit_start = w.base + (long long)s.g * s.T;
+    w.f += s.len;
+    return true;
+  }
+  if (w.f <= w.f_end) return false;
+  const long long last = w.f - 1;                          // highest tile still to do
   for (;;) {
     s.p0 = sh.prompt_cu[w.r]; s.N = sh.prompt_cu[w.r + 1] - s.p0;
     s.l0 = sh.live_cu[w.r]; s.M = sh.live_cu[w.r + 1] - s.l0;
     s.T = tiles_of(s.N, s.M);
-    const long long span = (long long)walk_groups(sh, w.stats, s.M) * s.T;
-    if (w.f < w.base + span) break;
-    w.base += span;
-    ++w.r;
+    if (last >= w.base) break;
+    // step back to the previous request
+    --w.r;
+    const int N2 = sh.prompt_cu[w.r + 1] - sh.prompt_cu[w.r], M2 = sh.live_cu[w.r + 1] - sh.live_cu[w.r];
+    w.base -= (long long)walk_groups(sh, w.stats, M2) * tiles_of(N2, M2);
   }
-  const long long rel = w.f - w.base;
+  const long long rel = last - w.base;
   s.r = w.r;
   s.g = (int)(rel / s.T);
   s.t = (int)(rel % s.T);
-  const long long room = w.f_end - w.f;
-  s.len = min(min(s.T - s.t, max_len), (int)min(room, (long long)0x7fffffff));
+  s.dir = -1;
+  const long long room = w.f - w.f_end;
+  s.len = min(min(s.t + 1, max_len), (int)min(room, (long long)0x7fffffff));
   s.unit_start = w.base + (long long)s.g * s.T;
-  w.f += s.len;
+  w.f -= s.len;
   return true;
 }
 
@@ -186,7 +223,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const uint32_t tmem_base = *tmem_slot;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   Walker wk;
-  walker_init(wk, true, F);
+  walker_init(wk, sh, true, false, F);
   Seg s;
 
   if (warp == 0) {
@@ -216,7 +253,8 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   } else if (warp == 1) {
     if (lane == 0) {
       const uint32_t idesc = idesc_bf16_f32(kTile, kTile);
-      const uint32_t q_base = smem_u32(base + S::kQOff);
+      const uint32_t q_lo_base = smem_desc_lo(smem_u32(base + S::kQOff));
+      const uint32_t k_lo_base = smem_desc_lo(smem_u32(base + S::kKOff));
       int kt_it = 0, q_it = 0;
       uint32_t cnt[2] = {0u, 0u};                            // tiles issued per query tile
       bool ok = true;
@@ -232,17 +270,17 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           const int stage = kt_it % kStages, use = kt_it / kStages;
           if (!(ok = mbar_wait(bars.full + stage, use & 1, abort_flag, status, 0x103))) break;
           tc_fence_after();
-          const uint32_t k_addr = smem_u32(base + S::kKOff + stage * S::kKBytes);
+          const uint32_t k_lo = k_lo_base + stage * (S::kKBytes >> 4);
           for (int a = 0; a < n_qtiles; ++a) {
             const int acc = a * 2 + (cnt[a] & 1);
             if (!(ok = mbar_wait(bars.tempty + acc, ((cnt[a] >> 1) & 1) ^ 1, abort_flag, status, 0x104))) break;
             tc_fence_after();
-            const uint32_t q_addr = q_base + a * kTile * 128;
+            const uint32_t q_lo = q_lo_base + ((a * kTile * 128) >> 4);
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
-              const uint64_t adesc = smem_desc_sw128(q_addr + (kk >> 2) * S::kQBoxBytes + (kk & 3) * 32);
-              const uint64_t bdesc = smem_desc_sw128(k_addr + (kk >> 2) * S::kKBoxBytes + (kk & 3) * 32);
-              umma_ss(tmem_base + acc * kTile, adesc, bdesc, idesc, kk > 0);
+              const uint32_t qo = ((kk >> 2) * S::kQBoxBytes + (kk & 3) * 32) >> 4;
+              const uint32_t ko = ((kk >> 2) * S::kKBoxBytes + (kk & 3) * 32) >> 4;
+              umma_ss(tmem_base + acc * kTile, make_desc(q_lo + qo, kDescHiSw128), make_desc(k_lo + ko, kDescHiSw128), idesc, kk > 0);
             }
             umma_commit(bars.tfull + acc);
             ++cnt[a];
@@ -274,12 +312,19 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
         float cmax = fmaxf(v[0], v[1]);
 #pragma unroll
-        for (int c = 2; c < 32; c += 2) cmax = fmaxf(cmax, fmaxf(v[c], v[c + 1]));
+        for (int c = 2; c < 32; c += 2) cmax = max3(cmax, v[c], v[c + 1]);
         if (cmax > m) { l *= ex2((m - cmax) * cs); m = cmax; }
         const float neg = -m * cs;
-        float l0 = 0.f, l1 = 0.f;
+        const uint64_t cs2 = pack2(cs, cs), neg2 = pack2(neg, neg);
+        uint64_t acc2 = pack2(0.f, 0.f);
 #pragma unroll
-        for (int c = 0; c < 32; c += 2) { l0 += ex2(fmaf(v[c], cs, neg)); l1 += ex2(fmaf(v[c + 1], cs, neg)); }
+        for (int c = 0; c < 32; c += 2) {
+          float x0, x1;
+          unpack2(fma2(pack2(v[c], v[c + 1]), cs2, neg2), x0, x1);
+          acc2 = add2(acc2, pack2(ex2(x0), ex2(x1)));
+        }
+        float l0, l1;
+        unpack2(acc2, l0, l1);
         l += l0 + l1;
       };
       for (int it = 0; ok && it < s.len; ++it, ++cnt) {
@@ -354,7 +399,7 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   const uint32_t tmem_base = *tmem_slot;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   Walker wk;
-  walker_init(wk, false, F);
+  walker_init(wk, sh, false, true, F);
   Seg s;
   int last_r = -1, last_g = -1;                             // the (request, KV head) whose queries are resident
 
@@ -378,7 +423,7 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           for (int tl = 0; tl < s.len; ++tl, ++kt_it) {
             const int stage = kt_it % kStages, use = kt_it / kStages;
             if (!(ok = mbar_wait(bars.empty + stage, (use & 1) ^ 1, abort_flag, status, 0x202))) break;
-            const KeyTile kt = key_tile(s.t + tl, s.p0, s.N, s.l0, s.M);
+            const KeyTile kt = key_tile(s.t + s.dir * tl, s.p0, s.N, s.l0, s.M);
             mbar_expect_tx(bars.full + stage, S::kKBytes);
             for (int b = 0; b < S::kBoxes; ++b)
               tma_load_3d(base + S::kKOff + stage * S::kKBytes + b * S::kKBoxBytes, kt.prompt ? &map_kp : &map_km,
@@ -393,7 +438,8 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       int kt_it = 0, q_it = 0, base_par = 0;
       uint32_t uses[2] = {0u, 0u};
       bool ok = true;
-      const uint32_t q_addr = smem_u32(base + S::kQOff);
+      const uint32_t q_lo_base = smem_desc_lo(smem_u32(base + S::kQOff));
+      const uint32_t k_lo_base = smem_desc_lo(smem_u32(base + S::kKOff));
       while (ok && walker_next(wk, sh, kColsumMaxTiles, s)) {
         const int q_per_head = (s.M + kQBlock - 1) / kQBlock, nqb = sh.g * q_per_head;
         const bool reuse_q = nqb == 1 && s.r == last_r && s.g == last_g;
@@ -413,12 +459,12 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (!(ok = mbar_wait(bars.full + stage, use & 1, abort_flag, status, 0x204))) break;
             if (!(ok = mbar_wait(bars.tempty + buf, (uses[buf] & 1) ^ 1, abort_flag, status, 0x205))) break;
             tc_fence_after();
-            const uint32_t k_addr = smem_u32(base + S::kKOff + stage * S::kKBytes);
+            const uint32_t k_lo = k_lo_base + stage * (S::kKBytes >> 4);
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
-              const uint64_t adesc = smem_desc_sw128(k_addr + (kk >> 2) * S::kKBoxBytes + (kk & 3) * 32);
-              const uint64_t bdesc = smem_desc_sw128(q_addr + (kk >> 2) * S::kQBoxBytes + (kk & 3) * 32);
-              umma_ss(tmem_base + buf * kQBlock, adesc, bdesc, idesc, kk > 0);
+              const uint32_t ko = ((kk >> 2) * S::kKBoxBytes + (kk & 3) * 32) >> 4;
+              const uint32_t qo = ((kk >> 2) * S::kQBoxBytes + (kk & 3) * 32) >> 4;
+              umma_ss(tmem_base + buf * kQBlock, make_desc(k_lo + ko, kDescHiSw128), make_desc(q_lo_base + qo, kDescHiSw128), idesc, kk > 0);
             }
             umma_commit(bars.empty + stage);
             umma_commit(bars.tfull + buf);
@@ -457,26 +503,28 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (!reuse_q) {
           float* c2w = c2s + (wg * 2 + (c2_it & 1)) * kTile;
           ++c2_it;
-          float cst = INFINITY;                             // 2^(x - inf) = 0: rows that do not exist never vote
-          if (row < nq) cst = lse[(long long)h * sh.sumM + s.l0 + q0 + row] * kLog2e - (w ? log2f(w[s.l0 + q0 + row]) : 0.f);
-          c2w[row] = cst;
+          float cst = -INFINITY;                            // 2^(x - inf) = 0: rows that do not exist never vote
+          if (row < nq) cst = (w ? log2f(w[s.l0 + q0 + row]) : 0.f) - lse[(long long)h * sh.sumM + s.l0 + q0 + row] * kLog2e;
+          c2w[row] = cst;                                   // stored negated: x = s*c + cst
           named_barrier(1 + wg, kTile);
           c2 = c2w;
         }
         const int chunks = (nq + 31) >> 5;
-        auto absorb = [&](const float* v, int cb, float& a0, float& a1) {
-          const float4* cc = reinterpret_cast<const float4*>(c2 + cb * 32);
+        auto absorb = [&](const float* v, int cb, uint64_t& acc2) {
+          const float4* cc = reinterpret_cast<const float4*>(c2 + cb * 32);   // negated constants
+          const uint64_t cs2 = pack2(cs, cs);
 #pragma unroll
           for (int c4 = 0; c4 < 8; ++c4) {
             const float4 k4 = cc[c4];
-            a0 += ex2(fmaf(v[4 * c4], cs, -k4.x));
-            a1 += ex2(fmaf(v[4 * c4 + 1], cs, -k4.y));
-            a0 += ex2(fmaf(v[4 * c4 + 2], cs, -k4.z));
-            a1 += ex2(fmaf(v[4 * c4 + 3], cs, -k4.w));
+            float x0, x1, x2, x3;
+            unpack2(fma2(pack2(v[4 * c4], v[4 * c4 + 1]), cs2, pack2(k4.x, k4.y)), x0, x1);
+            unpack2(fma2(pack2(v[4 * c4 + 2], v[4 * c4 + 3]), cs2, pack2(k4.z, k4.w)), x2, x3);
+            acc2 = add2(acc2, pack2(ex2(x0), ex2(x1)));
+            acc2 = add2(acc2, pack2(ex2(x2), ex2(x3)));
           }
         };
         for (int tl = (buf + base_par) & 1; tl < s.len; tl += 2) {
-          float a0 = 0.f, a1 = 0.f;
+          uint64_t acc2 = pack2(0.f, 0.f);
           if (ok) ok = mbar_wait(bars.tfull + buf, uses & 1, abort_flag, status, 0x206);
           if (ok) {
             tc_fence_after();
@@ -487,10 +535,12 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               tmem_ld32(taddr + cb * 32, v);
               tmem_ld_wait();
               if (cb + 1 == chunks) { tc_fence_before(); mbar_arrive(bars.tempty + buf); }   // last logits are in registers
-              absorb(v, cb, a0, a1);
+              absorb(v, cb, acc2);
             }
             if (chunks == 0) { tc_fence_before(); mbar_arrive(bars.tempty + buf); }
           }
+          float a0, a1;
+          unpack2(acc2, a0, a1);
           float* slot = xch + (uses & 1) * kTile;
           ++uses;
           if (half == 1) slot[row] = a0 + a1;
@@ -501,12 +551,12 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (qb > 0) acc += accs[tl * kTile + row];
             if (qb + 1 < nqb) { accs[tl * kTile + row] = acc; continue; }
           }
-          const KeyTile kt = key_tile(s.t + tl, s.p0, s.N, s.l0, s.M);
+          const KeyTile kt = key_tile(s.t + s.dir * tl, s.p0, s.N, s.l0, s.M);
           if (row >= kt.valid) acc = 0.f;
           if (kt.prompt && row < kt.valid) scores[(long long)s.g * sh.sumN + kt.token + row] = acc;
           acc = warp_sum(acc);
           if (lane == 0)
-            mass_part[((long long)seg * Tmax + s.t + tl) * 4 + lane_group] = kt.prompt ? make_float2(acc, 0.f) : make_float2(0.f, acc);
+            mass_part[((long long)seg * Tmax + s.t + s.dir * tl) * 4 + lane_group] = kt.prompt ? make_float2(acc, 0.f) : make_float2(0.f, acc);
         }
       }
       base_par ^= s.len & 1;
