@@ -151,10 +151,23 @@ def run_layer(ctx, buf, x, live, k_l, alpha, events=None):
     if events: events[5].record()
 
 
-def algorithmic_work(wl):
+# DRAM bytes (read + write) of one maskkv_score call at this workload, from the ncu capture summarised in
+# profiles/score_tc_llada32k_ncu.md: sweep 1 282.5 MB + sweep 2 283.4 MB (the key tensor is read once per sweep).
+SCORE_DRAM_TRAFFIC_BYTES = 565.9e6
+
+
+def algorithmic_work(wl, mean_kept_per_head):
     """Per layer: flops of the one Q K^T product scoring needs, and the bytes each HBM-bound call must move."""
-    N, M, H, d = wl.prompt_lens[0], wl.n_mask, wl.n_q_heads, wl.head_dim
-    return {"score_flops": 2.0 * M * (N + M) * d * H}
+    N, M, H, Hkv, d = wl.prompt_lens[0], wl.n_mask, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
+    k = mean_kept_per_head
+    return {
+        "score_flops": 2.0 * M * (N + M) * d * H,                       # one Q K^T over prompt + mask keys
+        "score_bytes": 2.0 * d * (N + M) * Hkv + 2.0 * d * M * H + 4.0 * N * Hkv,
+        "select_bytes": 4.0 * N * Hkv + 4.0 * k * Hkv,                  # read every score once, write kept indices
+        "compact_bytes": (4 * d * 2 + 4.0) * k * Hkv,                   # K and V row read + written, plus the index
+        "attend_flops": 4.0 * M * (k + M) * d * H,
+        "attend_bytes": 2.0 * (2 * M * H * d) + 2.0 * 2 * d * (k + M) * Hkv,
+    }
 
 
 def bench_ours(args):
@@ -193,12 +206,10 @@ def bench_ours(args):
         torch.cuda.synchronize()
 
     # ---- device-resident timing
+    sampler = ClockSampler(local_rank) if rank == 0 else None   # samples through warm-up, the timed region and the e2e leg
     for i in range(args.warmup):
         step(i)
     barrier()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    if sampler:
-        time.sleep(0.25)
     per_call = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
     launches0 = ctx.maskkv_launch_count()
     barrier()
@@ -210,7 +221,7 @@ def bench_ours(args):
     barrier()
     launches = ctx.maskkv_launch_count() - launches0
     elapsed_ms = max_over_ranks(t0.elapsed_time(t1), device)
-    clocks = sampler.stop() if sampler else {}
+    mean_kept = float(buf.offsets[-1].item()) / wl.n_kv_heads
     call_us = {name: 1e3 * statistics.mean(ev[c].elapsed_time(ev[c + 1]) for ev in per_call) for c, name in enumerate(CALLS)}
     flags = ctx.maskkv_check_status()
 
@@ -235,7 +246,7 @@ def bench_ours(args):
         host_out.copy_(buf.out, non_blocking=True)
         host_bud.copy_(buf.budgets, non_blocking=True)
 
-    e2e_steps = max(3, min(args.steps, 20))
+    e2e_steps = max(3, min(args.steps, 50))
     for i in range(2):
         e2e_step(i)
     barrier()
@@ -246,6 +257,7 @@ def bench_ours(args):
     e1.record()
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), device)
+    clocks = sampler.stop() if sampler else {}
 
     if world > 1:
         dist.destroy_process_group()
@@ -255,10 +267,20 @@ def bench_ours(args):
     ms_per_step = elapsed_ms / args.steps
     value = world * N / (ms_per_step * 1e-3)
     peaks = load_peaks()
-    work = algorithmic_work(wl)
+    work = algorithmic_work(wl, mean_kept)
     score_s = call_us["score"] * 1e-6
     achieved_tf = work["score_flops"] / score_s / 1e12
     peak_tf = peaks["bf16_tflops_sustained"]
+    hbm = peaks["hbm_gbs"]
+    other = {
+        "score_hbm": {"bound": "hbm", "achieved": work["score_bytes"] / score_s / 1e9, "peak": hbm, "unit": "GB/s"},
+        "select": {"bound": "hbm", "achieved": work["select_bytes"] / (call_us["select"] * 1e-6) / 1e9, "peak": hbm, "unit": "GB/s"},
+        "compact": {"bound": "hbm", "achieved": work["compact_bytes"] / (call_us["compact"] * 1e-6) / 1e9, "peak": hbm, "unit": "GB/s"},
+        "attend": {"bound": "hbm", "achieved": work["attend_bytes"] / (call_us["attend"] * 1e-6) / 1e9, "peak": hbm, "unit": "GB/s",
+                   "tflops": work["attend_flops"] / (call_us["attend"] * 1e-6) / 1e12},
+    }
+    for v in other.values():
+        v["frac"] = v["achieved"] / v["peak"]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -276,7 +298,10 @@ def bench_ours(args):
         "status_flags": flags,
         "roofline": {"kernel": "maskkv_score (all its kernels; one Q K^T product counted)", "bound": "tensor",
                      "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
-                     "peak_source": peaks["source"] + " (sustained bf16)", "traffic": None},
+                     "peak_source": peaks["source"] + " (sustained bf16; the kernels run inside a long step)",
+                     "traffic": SCORE_DRAM_TRAFFIC_BYTES, "executed_over_algorithmic_flops": 2.0},
+        "roofline_other_calls": other,
+        "mean_kept_per_head": mean_kept,
     }
     line["cpu_baseline"] = oracle_baseline(wl, budget_s=15.0)
     return line
@@ -367,7 +392,7 @@ def main():
         args.warmup = 1 if args.warmup is None else max(0, args.warmup)
         line = bench_reference(args)
     else:
-        args.steps = 40 if args.steps is None else max(1, args.steps)
+        args.steps = 1000 if args.steps is None else max(1, args.steps)
         args.warmup = 5 if args.warmup is None else max(3, args.warmup)
         line = bench_ours(args)
     if line is not None:

@@ -1,0 +1,63 @@
+"""The multi-rank plumbing of bench.py on CPU: two gloo ranks shard the layers (every layer exactly once,
+no data-path collective) and agree on the slowest rank's time.  No GPU involved."""
+import os
+import socket
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank))
+    import bench
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        assert bench.rank_world() == (rank, world, rank)
+        mine = bench.shard_layers(32, rank, world)
+        gathered = [None] * world
+        dist.all_gather_object(gathered, mine)
+        slowest = bench.max_over_ranks(10.0 + 5.0 * rank)
+        total = bench.sum_over_ranks(float(len(mine)))
+        out.put((rank, gathered, slowest, total))
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.timeout(120)
+def test_two_ranks_shard_layers_and_reduce_times():
+    world = 2
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    results = [out.get(timeout=90) for _ in range(world)]
+    for p in procs:
+        p.join(timeout=30)
+        assert p.exitcode == 0
+    for rank, gathered, slowest, total in results:
+        layers = sorted(l for part in gathered for l in part)
+        assert layers == list(range(32))                       # every layer once
+        assert set(gathered[0]).isdisjoint(gathered[1])
+        assert slowest == 15.0                                 # the max over ranks, on every rank
+        assert total == 32.0
+
+
+def test_single_process_helpers_are_no_ops():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.shard_layers(5, 0, 1) == [0, 1, 2, 3, 4]
+    assert bench.max_over_ranks(3.5) == 3.5 and bench.sum_over_ranks(2.0) == 2.0
