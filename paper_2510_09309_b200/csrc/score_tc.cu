@@ -327,26 +327,42 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         unpack2(acc2, l0, l1);
         l += l0 + l1;
       };
+      // Rolling double buffer over the chunk stream (tile 0: c0, c1; tile 1: c0, c1; ...): while one 32-column chunk
+      // is being exponentiated the next one - possibly of the next tile - is already on its way from tensor memory.
+      const int col0 = half * 64;
+      const uint32_t lane_addr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + col0;
+      float va[32], vb[32];
+      int valid = 0;
+      if (s.len > 0) {
+        if ((ok = mbar_wait(bars.tfull + a * 2 + (cnt & 1), (cnt >> 1) & 1, abort_flag, status, 0x105))) {
+          tc_fence_after();
+          valid = key_tile(s.t, s.p0, s.N, s.l0, s.M).valid;
+          tmem_ld32(lane_addr + (a * 2 + (cnt & 1)) * kTile, va);
+        }
+      }
       for (int it = 0; ok && it < s.len; ++it, ++cnt) {
         const int acc = a * 2 + (cnt & 1);
-        if (!(ok = mbar_wait(bars.tfull + acc, (cnt >> 1) & 1, abort_flag, status, 0x105))) break;
-        tc_fence_after();
-        const int valid = key_tile(s.t + it, s.p0, s.N, s.l0, s.M).valid;
-        const int col0 = half * 64;
-        const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + acc * kTile + col0;
-        const int n_chunks = valid > col0 + 32 ? 2 : (valid > col0 ? 1 : 0);
-        float va[32], vb[32];
-        if (n_chunks > 0) tmem_ld32(taddr, va);
-        if (n_chunks > 1) tmem_ld32(taddr + 32, vb);
-        if (n_chunks > 0) tmem_ld_wait();
+        // chunk 0 of this tile is in flight (into va); start chunk 1 behind it
+        tmem_ld_wait();
+        tmem_ld32(lane_addr + acc * kTile + 32, vb);
+        if (valid > col0) absorb(va, col0, valid);
+        tmem_ld_wait();
         tc_fence_before();
-        mbar_arrive(bars.tempty + acc);                     // this thread's logits are in registers
-        if (n_chunks > 0) absorb(va, col0, valid);
-        if (n_chunks > 1) absorb(vb, col0 + 32, valid);
+        mbar_arrive(bars.tempty + acc);                     // both chunks of this thread are in registers
+        const int valid_now = valid;
+        if (it + 1 < s.len) {                               // chunk 0 of the next tile goes out before chunk 1 is processed
+          const uint32_t c2n = cnt + 1;
+          if (!(ok = mbar_wait(bars.tfull + a * 2 + (c2n & 1), (c2n >> 1) & 1, abort_flag, status, 0x105))) break;
+          tc_fence_after();
+          valid = key_tile(s.t + it + 1, s.p0, s.N, s.l0, s.M).valid;
+          tmem_ld32(lane_addr + (a * 2 + (c2n & 1)) * kTile, va);
+        }
+        if (valid_now > col0 + 32) absorb(vb, col0 + 32, valid_now);
       }
+      if (!ok) continue;
       const int i = q0 + a * kTile + row;
       const int slot = 2 * ((int)blockIdx.x - cta_of(s.unit_start, F, gridDim.x)) + half;
-      if (ok && i < s.M) part[((long long)h * sh.sumM + s.l0 + i) * C + slot] = make_float2(m * sh.scale, l);
+      if (i < s.M) part[((long long)h * sh.sumM + s.l0 + i) * C + slot] = make_float2(m * sh.scale, l);
     }
   }
   block_teardown(tmem_base);
