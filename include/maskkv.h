@@ -87,6 +87,9 @@ const char* maskkv_status_string(int code);
  * MASKKV_E_CUDA if the stream reported an error, else MASKKV_OK. */
 int maskkv_check_status(maskkv_ctx* ctx, void* stream, uint32_t* flags_out);
 
+/* Text of the most recent CUDA runtime error behind a MASKKV_E_CUDA return of this context ("" if none). */
+const char* maskkv_last_cuda_error(const maskkv_ctx* ctx);
+
 /* Number of kernels this context has launched so far (host counter; for benchmarks and for checking
  * that a failed validation launched nothing). */
 uint64_t maskkv_launch_count(const maskkv_ctx* ctx);

@@ -22,7 +22,7 @@ MASKKV_F32, MASKKV_BF16 = 0, 1
 MASKKV_FLAG_TIMEOUT, MASKKV_FLAG_CAPACITY, MASKKV_FLAG_BOUNDS = 1, 2, 4
 
 EXPORTS = (
-    "maskkv_create", "maskkv_destroy", "maskkv_status_string", "maskkv_check_status", "maskkv_launch_count",
+    "maskkv_create", "maskkv_destroy", "maskkv_status_string", "maskkv_check_status", "maskkv_launch_count", "maskkv_last_cuda_error",
     "maskkv_tensor_core_launch_count",
     "maskkv_workspace_bytes",
     "maskkv_layer_budgets", "maskkv_score", "maskkv_score_noalloc", "maskkv_score_noalloc_max_bytes", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend",
@@ -59,6 +59,8 @@ def _load() -> C.CDLL:
     lib.maskkv_status_string.argtypes = [C.c_int]
     lib.maskkv_status_string.restype = C.c_char_p
     lib.maskkv_check_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
+    lib.maskkv_last_cuda_error.argtypes = [vp]
+    lib.maskkv_last_cuda_error.restype = C.c_char_p
     lib.maskkv_launch_count.argtypes = [vp]
     lib.maskkv_launch_count.restype = C.c_uint64
     lib.maskkv_tensor_core_launch_count.argtypes = [vp]
@@ -76,7 +78,7 @@ def _load() -> C.CDLL:
     lib.maskkv_attend.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("maskkv_status_string", "maskkv_workspace_bytes", "maskkv_launch_count", "maskkv_tensor_core_launch_count",
-                        "maskkv_score_noalloc_max_bytes"):
+                        "maskkv_score_noalloc_max_bytes", "maskkv_last_cuda_error"):
             getattr(lib, name).restype = C.c_int
     return lib
 
@@ -88,8 +90,10 @@ def status_string(code: int) -> str:
     return lib.maskkv_status_string(code).decode()
 
 
-def _check(code: int, what: str) -> None:
+def _check(code: int, what: str, handle=None) -> None:
     if code != MASKKV_OK:
+        if code == MASKKV_E_CUDA and handle:
+            what = f"{what} [{lib.maskkv_last_cuda_error(handle).decode()}]"
         raise MaskKVError(code, what)
 
 
@@ -174,7 +178,7 @@ class Context:
         _check(lib.maskkv_score(self._h, C.byref(p.desc), _ptr(q_mask), _ptr(k_prompt), _ptr(k_mask), _ptr(row_weights),
                                 _ptr(scores), _ptr(mass_p), _ptr(mass_m), _ptr(workspace),
                                 0 if workspace is None else workspace.numel() * workspace.element_size(), _stream()),
-               "maskkv_score")
+               "maskkv_score", self._h)
 
     def maskkv_score_noalloc(self, p: Problem, q_mask, k_prompt, k_mask, scores, mass_p, mass_m, row_weights=None):
         """maskkv_score without a workspace argument, for callers that may not allocate device memory: the
@@ -182,22 +186,22 @@ class Context:
         the first call and on overlapping calls)."""
         _check(lib.maskkv_score_noalloc(self._h, C.byref(p.desc), _ptr(q_mask), _ptr(k_prompt), _ptr(k_mask),
                                         _ptr(row_weights), _ptr(scores), _ptr(mass_p), _ptr(mass_m), _stream()),
-               "maskkv_score_noalloc")
+               "maskkv_score_noalloc", self._h)
 
     def maskkv_budget(self, p: Problem, k_l: int, alpha: float, mass_p, mass_m, capacity: int, budgets, offsets,
                       k_l_per_request=None):
         _check(lib.maskkv_budget(self._h, C.byref(p.desc), int(k_l), _ptr(k_l_per_request), float(alpha), _ptr(mass_p),
-                                 _ptr(mass_m), int(capacity), _ptr(budgets), _ptr(offsets), _stream()), "maskkv_budget")
+                                 _ptr(mass_m), int(capacity), _ptr(budgets), _ptr(offsets), _stream()), "maskkv_budget", self._h)
 
     def maskkv_select(self, p: Problem, scores, budgets, offsets, kept_idx, workspace=None):
         _check(lib.maskkv_select(self._h, C.byref(p.desc), _ptr(scores), _ptr(budgets), _ptr(offsets), _ptr(kept_idx),
                                  _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
-                                 _stream()), "maskkv_select")
+                                 _stream()), "maskkv_select", self._h)
 
     def maskkv_compact(self, p: Problem, k_prompt, v_prompt, kept_idx, offsets, capacity: int, kc, vc):
         _check(lib.maskkv_compact(self._h, C.byref(p.desc), _ptr(k_prompt), _ptr(v_prompt), _ptr(kept_idx), _ptr(offsets),
-                                  int(capacity), _ptr(kc), _ptr(vc), _stream()), "maskkv_compact")
+                                  int(capacity), _ptr(kc), _ptr(vc), _stream()), "maskkv_compact", self._h)
 
     def maskkv_attend(self, p: Problem, q_live, k_live, v_live, kc, vc, offsets, capacity: int, out, lse=None):
         _check(lib.maskkv_attend(self._h, C.byref(p.desc), _ptr(q_live), _ptr(k_live), _ptr(v_live), _ptr(kc), _ptr(vc),
-                                 _ptr(offsets), int(capacity), _ptr(out), _ptr(lse), _stream()), "maskkv_attend")
+                                 _ptr(offsets), int(capacity), _ptr(out), _ptr(lse), _stream()), "maskkv_attend", self._h)

@@ -5,13 +5,15 @@
 // head's ragged segment of the compacted cache (rows [offsets[s], offsets[s+1]) of kc / vc), then over
 // the request's live rows.  Per tile:
 //     S = Q K^T            tcgen05.mma, operands in shared memory (TMA, 128-byte swizzle), S in tensor memory
-//     P = 2^(S*c - m*c)    one thread per query row: online max / sum in fp32, P rounded to bf16 and
-//                          written back into tensor memory over S
+//     P = 2^(S*c - m*c)    NW threads per query row (128/NW key columns each; NW = 2): online max / sum in
+//                          fp32, P rounded to bf16 and written back into tensor memory over S
 //     PV = P V             tcgen05.mma with P read from tensor memory and V (row-major, i.e. N-major) from
 //                          shared memory, into a fresh accumulator
-//     O = O*corr + PV      in registers of the row's thread (no rescaling pass over tensor memory)
+//     O = O*corr + PV      in registers, d/NW output columns per thread (no rescaling pass over tensor memory)
 // S/P and PV are double-buffered (4 x 128 columns of tensor memory) so the next tile's Q K^T overlaps the
-// softmax.  Columns of a ragged tile's tail are masked to -inf, and the matching V rows are zeroed in
+// softmax; key and value tiles come through separate TMA rings (3 and 2 stages) and tiles beyond the rings are
+// requested into L2 ahead of time.  The kernel is a latency chain (3-8 dependent tiles per CTA), not a
+// throughput kernel: measured per tile, about 0.4 us goes to issuing the two MMA groups from one thread.  Columns of a ragged tile's tail are masked to -inf, and the matching V rows are zeroed in
 // shared memory so that stale cache rows can never leak a NaN into the product.
 #include "attend_tc.h"
 
@@ -20,9 +22,14 @@
 namespace mkv {
 namespace tc {
 
-constexpr int kAThreads = 192;         // warp 0: TMA, warp 1: MMA, warps 2-5: softmax (one thread per query row)
+// warp 0: TMA, warp 1: MMA, then NW softmax warpgroups (thread = one query row, 128/NW key columns, d/NW output columns)
+#ifndef MKV_ATTEND_NW
+#define MKV_ATTEND_NW 2
+#endif
+template <int D> struct AWgs { static constexpr int kNW = MKV_ATTEND_NW; static constexpr int kThreads = 64 + 128 * kNW; };
 constexpr int kATile = 128;
-constexpr int kAStages = 3;
+constexpr int kAKStages = 3;            // key tiles in flight (the next Q K^T is issued a tile ahead)
+constexpr int kAVStages = 2;            // value tiles in flight
 constexpr float kALog2e = 1.4426950408889634f;
 
 template <int D>
@@ -32,11 +39,13 @@ struct ASmem {
   static constexpr int kTileBytes = kBoxes * kBoxBytes;
   static constexpr int kQOff = 0;
   static constexpr int kKOff = kTileBytes;
-  static constexpr int kVOff = kKOff + kAStages * kTileBytes;
-  static constexpr int kBarOff = kVOff + kAStages * kTileBytes;
-  static constexpr int kNumBars = 1 + 4 * kAStages + 8;
+  static constexpr int kVOff = kKOff + kAKStages * kTileBytes;
+  static constexpr int kBarOff = kVOff + kAVStages * kTileBytes;
+  static constexpr int kNumBars = 1 + 2 * kAKStages + 2 * kAVStages + 8;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
-  static constexpr int kBytes = kMiscOff + 16;
+  static constexpr int kMxOff = kMiscOff + 16;                             // float [2 tiles][4 warpgroups][128]: partial row maxima
+  static constexpr int kLxOff = kMxOff + 8 * kATile * 4;                   // float [4 warpgroups][128]: partial row sums
+  static constexpr int kBytes = kLxOff + 4 * kATile * 4;
   static constexpr int kDynamic = kBytes + 1024;
 };
 
@@ -67,6 +76,13 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* u) {
         "r"(u[27]), "r"(u[28]), "r"(u[29]), "r"(u[30]), "r"(u[31])
       : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* u) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(u[0]), "r"(u[1]), "r"(u[2]), "r"(u[3]), "r"(u[4]), "r"(u[5]), "r"(u[6]), "r"(u[7]), "r"(u[8]),
+        "r"(u[9]), "r"(u[10]), "r"(u[11]), "r"(u[12]), "r"(u[13]), "r"(u[14]), "r"(u[15])
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
@@ -76,14 +92,15 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 struct ABars {
   uint64_t* qfull;
-  uint64_t *kfull, *kempty, *vfull, *vempty;   // [kAStages]
+  uint64_t *kfull, *kempty;                    // [kAKStages]
+  uint64_t *vfull, *vempty;                    // [kAVStages]
   uint64_t *sfull, *pready, *ofull, *oempty;   // [2]
 };
 __device__ __forceinline__ ABars carve_abars(uint8_t* base, int off) {
   uint64_t* b = reinterpret_cast<uint64_t*>(base + off);
   ABars r;
-  r.qfull = b; r.kfull = b + 1; r.kempty = r.kfull + kAStages; r.vfull = r.kempty + kAStages; r.vempty = r.vfull + kAStages;
-  r.sfull = r.vempty + kAStages; r.pready = r.sfull + 2; r.ofull = r.pready + 2; r.oempty = r.ofull + 2;
+  r.qfull = b; r.kfull = b + 1; r.kempty = r.kfull + kAKStages; r.vfull = r.kempty + kAKStages; r.vempty = r.vfull + kAVStages;
+  r.sfull = r.vempty + kAVStages; r.pready = r.sfull + 2; r.ofull = r.pready + 2; r.oempty = r.ofull + 2;
   return r;
 }
 
@@ -101,7 +118,7 @@ __device__ __forceinline__ ATile a_tile(int j, int c0, int nc, int l0, int M) {
 
 // grid (q tiles, H, R)
 template <int D>
-__global__ void __launch_bounds__(kAThreads, 1)
+__global__ void __launch_bounds__(AWgs<D>::kThreads, 1)
 attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kl,
           const __grid_constant__ CUtensorMap map_vl, const __grid_constant__ CUtensorMap map_kc,
           const __grid_constant__ CUtensorMap map_vc, Shape sh, const int32_t* __restrict__ offsets,
@@ -124,11 +141,10 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     mbar_init(bars.qfull, 1);
-    for (int s = 0; s < kAStages; ++s) {
-      mbar_init(bars.kfull + s, 1); mbar_init(bars.kempty + s, 1); mbar_init(bars.vfull + s, 1); mbar_init(bars.vempty + s, 1);
-    }
+    for (int s = 0; s < kAKStages; ++s) { mbar_init(bars.kfull + s, 1); mbar_init(bars.kempty + s, 1); }
+    for (int s = 0; s < kAVStages; ++s) { mbar_init(bars.vfull + s, 1); mbar_init(bars.vempty + s, 1); }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(bars.sfull + b, 1); mbar_init(bars.pready + b, kATile); mbar_init(bars.ofull + b, 1); mbar_init(bars.oempty + b, kATile);
+      mbar_init(bars.sfull + b, 1); mbar_init(bars.pready + b, AWgs<D>::kNW * kATile); mbar_init(bars.ofull + b, 1); mbar_init(bars.oempty + b, AWgs<D>::kNW * kATile);
     }
     *abort_flag = 0u;
     fence_barrier_init();
@@ -145,35 +161,61 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       prefetch_tmap(&map_q); prefetch_tmap(&map_kl); prefetch_tmap(&map_vl); prefetch_tmap(&map_kc); prefetch_tmap(&map_vc);
       mbar_expect_tx(bars.qfull, S::kTileBytes);
       for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kBoxBytes, &map_q, bars.qfull, b * 64, h, l0 + q0);
-      bool ok = true;
+      // two independent rings (keys, values): whichever has a free stage gets its next tile, keys first
       int jk = 0, jv = 0;
-      // keys run ahead of values: the Q K^T of tile j+1 is issued before the P V of tile j
-      while (ok && (jk < nt || jv < nt)) {
-        if (jk < nt && jk <= jv + 1) {
-          const int stage = jk % kAStages, use = jk / kAStages;
-          if (!(ok = mbar_wait(bars.kempty + stage, (use & 1) ^ 1, abort_flag, status, 0x301))) break;
-          const ATile t = a_tile(jk, c0, nc, l0, M);
-          mbar_expect_tx(bars.kfull + stage, S::kTileBytes);
-          for (int b = 0; b < S::kBoxes; ++b)
-            tma_load_3d(base + S::kKOff + stage * S::kTileBytes + b * S::kBoxBytes, t.cache ? &map_kc : &map_kl, bars.kfull + stage,
-                        b * 64, t.cache ? 0 : hk, t.row);
-          ++jk;
-        } else {
-          const int stage = jv % kAStages, use = jv / kAStages;
-          if (!(ok = mbar_wait(bars.vempty + stage, (use & 1) ^ 1, abort_flag, status, 0x302))) break;
-          const ATile t = a_tile(jv, c0, nc, l0, M);
-          mbar_expect_tx(bars.vfull + stage, S::kTileBytes);
-          for (int b = 0; b < S::kBoxes; ++b)
-            tma_load_3d(base + S::kVOff + stage * S::kTileBytes + b * S::kBoxBytes, t.cache ? &map_vc : &map_vl, bars.vfull + stage,
-                        b * 64, t.cache ? 0 : hk, t.row);
-          ++jv;
+      const unsigned long long t_start = global_ns();
+      uint32_t spins = 0;
+      bool ok = true, prefetched = false;
+      while (jk < nt || jv < nt) {
+        bool issued = false;
+        if (jk < nt) {
+          const int stage = jk % kAKStages, use = jk / kAKStages;
+          if (mbar_try_wait(bars.kempty + stage, (use & 1) ^ 1)) {
+            const ATile t = a_tile(jk, c0, nc, l0, M);
+            mbar_expect_tx(bars.kfull + stage, S::kTileBytes);
+            for (int b = 0; b < S::kBoxes; ++b)
+              tma_load_3d(base + S::kKOff + stage * S::kTileBytes + b * S::kBoxBytes, t.cache ? &map_kc : &map_kl,
+                          bars.kfull + stage, b * 64, t.cache ? 0 : hk, t.row);
+            ++jk;
+            issued = true;
+          }
+        }
+        if (jv < nt) {
+          const int stage = jv % kAVStages, use = jv / kAVStages;
+          if (mbar_try_wait(bars.vempty + stage, (use & 1) ^ 1)) {
+            const ATile t = a_tile(jv, c0, nc, l0, M);
+            mbar_expect_tx(bars.vfull + stage, S::kTileBytes);
+            for (int b = 0; b < S::kBoxes; ++b)
+              tma_load_3d(base + S::kVOff + stage * S::kTileBytes + b * S::kBoxBytes, t.cache ? &map_vc : &map_vl,
+                          bars.vfull + stage, b * 64, t.cache ? 0 : hk, t.row);
+            ++jv;
+            issued = true;
+          }
+        }
+        if (!prefetched && jk >= min(nt, kAKStages) && jv >= min(nt, kAVStages)) {
+          // the rings are full: ask for the later tiles to be brought into L2, so that their ring loads pay L2 latency only
+          for (int j = kAVStages; j < nt; ++j) {
+            const ATile t = a_tile(j, c0, nc, l0, M);
+            for (int b = 0; b < S::kBoxes; ++b) {
+              if (j >= kAKStages) tma_prefetch_l2_3d(t.cache ? &map_kc : &map_kl, b * 64, t.cache ? 0 : hk, t.row);
+              tma_prefetch_l2_3d(t.cache ? &map_vc : &map_vl, b * 64, t.cache ? 0 : hk, t.row);
+            }
+          }
+          prefetched = true;
+        }
+        if (!issued && (++spins & 255u) == 0u) {             // bounded like every other wait
+          if (*abort_flag) { ok = false; break; }
+          if (global_ns() - t_start > kWaitLimitNs) {
+            *abort_flag = 1u; atomicOr(status, (uint32_t)MASKKV_FLAG_TIMEOUT); atomicExch(status + 1, 0x301u);
+            ok = false; break;
+          }
         }
       }
       if (!ok) {   // wait (bounded) for the copies already issued
-        for (int i = max(0, jk - kAStages); i < jk; ++i)
-          for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(bars.kfull + i % kAStages, (i / kAStages) & 1); ++it) __nanosleep(64);
-        for (int i = max(0, jv - kAStages); i < jv; ++i)
-          for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(bars.vfull + i % kAStages, (i / kAStages) & 1); ++it) __nanosleep(64);
+        for (int i = max(0, jk - kAKStages); i < jk; ++i)
+          for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(bars.kfull + i % kAKStages, (i / kAKStages) & 1); ++it) __nanosleep(64);
+        for (int i = max(0, jv - kAVStages); i < jv; ++i)
+          for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(bars.vfull + i % kAVStages, (i / kAVStages) & 1); ++it) __nanosleep(64);
       }
     }
   } else if (warp == 1) {
@@ -184,7 +226,7 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       bool ok = mbar_wait(bars.qfull, 0, abort_flag, status, 0x303);
       tc_fence_after();
       auto issue_qk = [&](int j) -> bool {
-        const int stage = j % kAStages, use = j / kAStages;
+        const int stage = j % kAKStages, use = j / kAKStages;
         if (!mbar_wait(bars.kfull + stage, use & 1, abort_flag, status, 0x304)) return false;
         tc_fence_after();
         const uint32_t k_lo = smem_desc_lo(smem_u32(base + S::kKOff + stage * S::kTileBytes));
@@ -200,7 +242,7 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       if (ok) ok = issue_qk(0);
       for (int j = 0; ok && j < nt; ++j) {
         if (j + 1 < nt && !(ok = issue_qk(j + 1))) break;
-        const int b = j & 1, stage = j % kAStages, use = j / kAStages;
+        const int b = j & 1, stage = j % kAVStages, use = j / kAVStages;
         if (!(ok = mbar_wait(bars.vfull + stage, use & 1, abort_flag, status, 0x305))) break;
         if (!(ok = mbar_wait(bars.oempty + b, ((j >> 1) & 1) ^ 1, abort_flag, status, 0x306))) break;
         if (!(ok = mbar_wait(bars.pready + b, (j >> 1) & 1, abort_flag, status, 0x307))) break;
@@ -209,113 +251,125 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         const uint32_t v_lo = ((smem_u32(base + S::kVOff + stage * S::kTileBytes) & 0x3ffffu) >> 4) | ((uint32_t)(S::kBoxBytes >> 4) << 16);
 #pragma unroll
         for (int kk = 0; kk < kATile / 16; ++kk)
-          umma_ts(tm_o + b * kATile, tm_s + b * kATile + kk * 8, make_desc(v_lo + ((kk * 16 * 128) >> 4), kDescHiSw128), idesc_pv, kk > 0);
+          // P of keys [SC*w, SC*w + SC) sits in packed columns [SC*w, SC*w + SC/2), SC = 128 / NW key columns per thread
+          umma_ts(tm_o + b * kATile, tm_s + b * kATile + (16 * kk / (kATile / AWgs<D>::kNW)) * (kATile / AWgs<D>::kNW) + (16 * kk % (kATile / AWgs<D>::kNW)) / 2,
+                  make_desc(v_lo + ((kk * 16 * 128) >> 4), kDescHiSw128), idesc_pv, kk > 0);
         umma_commit(bars.ofull + b);
         umma_commit(bars.vempty + stage);
       }
     }
   } else {
+    // NW softmax warpgroups share every tile: thread (wg, row) owns S columns [SC wg, SC wg + SC) of its query row
+    // (SC = 128 / NW) and the output columns [32 wg, 32 wg + 32).  The row maximum is the only thing they exchange per
+    // tile (shared memory + one named barrier); P of the thread's keys is written over the S columns the same thread
+    // has just read (packed columns SC wg .. SC wg + SC/2 - 1), so the warpgroups never touch each other's columns.
+    constexpr int NW = AWgs<D>::kNW;
+    constexpr int SC = kATile / NW;                         // 32 or 64
+    const int wg = (warp - 2) >> 2;
     const int lane_group = warp & 3;
     const int row = lane_group * 32 + lane;                 // query inside the tile
-    const int tid = (warp - 2) * 32 + lane;                 // 0..127, used for cooperative shared-memory work
+    const int tid_all = wg * kATile + ((warp - 2) & 3) * 32 + lane;   // 0 .. NW*128-1 over the softmax warpgroups
     const uint32_t lane_addr = (uint32_t)(lane_group * 32) << 16;
     const float cs = sh.scale * kALog2e;
-    float o[D];
+    float* mx = reinterpret_cast<float*>(base + S::kMxOff);
+    float* lx = reinterpret_cast<float*>(base + S::kLxOff);
+    constexpr int OC = D / NW;                              // output columns per thread
+    float o[OC];
 #pragma unroll
-    for (int c = 0; c < D; ++c) o[c] = 0.f;
+    for (int c = 0; c < OC; ++c) o[c] = 0.f;
     float m = -INFINITY, l = 0.f, corr_prev = 0.f;
     bool ok = true;
 
-    auto consume_pv = [&](int j, float corr) -> bool {      // O = O*corr + PV(j)
+    auto consume_pv = [&](int j, float corr) {               // O = O*corr + PV(j), this thread's 32 output columns
       const int b = j & 1;
-      if (!mbar_wait(bars.ofull + b, (j >> 1) & 1, abort_flag, status, 0x308)) return false;
+      if (ok) ok = mbar_wait(bars.ofull + b, (j >> 1) & 1, abort_flag, status, 0x308);
+      if (!ok) return;
       tc_fence_after();
 #pragma unroll
-      for (int cb = 0; cb < D / 32; ++cb) {
+      for (int cb = 0; cb < OC / 32; ++cb) {
         float v[32];
-        tmem_ld32(tm_o + lane_addr + b * kATile + cb * 32, v);
+        tmem_ld32(tm_o + lane_addr + b * kATile + wg * OC + cb * 32, v);
         tmem_ld_wait();
+        if (cb + 1 == OC / 32) { tc_fence_before(); mbar_arrive(bars.oempty + b); }
 #pragma unroll
         for (int c = 0; c < 32; ++c) o[cb * 32 + c] = fmaf(o[cb * 32 + c], corr, v[c]);
       }
-      tc_fence_before();
-      mbar_arrive(bars.oempty + b);
-      return true;
     };
 
-    for (int j = 0; ok && j < nt; ++j) {
+    // After a failed wait a thread skips the tensor-memory work but still reaches every named barrier.
+    for (int j = 0; j < nt; ++j) {
       const int b = j & 1;
       const ATile t = a_tile(j, c0, nc, l0, M);
-      if (t.valid < kATile) {
+      const int my_valid = min(SC, max(0, t.valid - wg * SC));   // valid columns among this thread's SC
+      if (ok && t.valid < kATile) {
         // ragged tail: zero the value rows that do not belong to this tile (every thread clears a slice)
-        const int stage = j % kAStages, use = j / kAStages;
-        if (!(ok = mbar_wait(bars.vfull + stage, use & 1, abort_flag, status, 0x309))) break;
-        uint8_t* v_tile = base + S::kVOff + stage * S::kTileBytes;
-        const int n16 = (kATile - t.valid) * 8;             // 16-byte pieces per box
-        for (int bx = 0; bx < S::kBoxes; ++bx) {
-          uint4* dst = reinterpret_cast<uint4*>(v_tile + bx * S::kBoxBytes + t.valid * 128);
-          for (int e = tid; e < n16; e += kATile) dst[e] = make_uint4(0u, 0u, 0u, 0u);
+        const int stage = j % kAVStages, su = j / kAVStages;
+        if ((ok = mbar_wait(bars.vfull + stage, su & 1, abort_flag, status, 0x309))) {
+          uint8_t* v_tile = base + S::kVOff + stage * S::kTileBytes;
+          const int n16 = (kATile - t.valid) * 8;           // 16-byte pieces per box
+          for (int bx = 0; bx < S::kBoxes; ++bx) {
+            uint4* dst = reinterpret_cast<uint4*>(v_tile + bx * S::kBoxBytes + t.valid * 128);
+            for (int e = tid_all; e < n16; e += NW * kATile) dst[e] = make_uint4(0u, 0u, 0u, 0u);
+          }
+          fence_async_smem();
         }
-        fence_async_smem();
       }
-      if (!(ok = mbar_wait(bars.sfull + b, (j >> 1) & 1, abort_flag, status, 0x30a))) break;
-      tc_fence_after();
-      const uint32_t s_addr = tm_s + lane_addr + b * kATile;
-      // pass 1 over the tile: row maximum
+      if (ok) ok = mbar_wait(bars.sfull + b, (j >> 1) & 1, abort_flag, status, 0x30a);
+      const uint32_t s_addr = tm_s + lane_addr + b * kATile + wg * SC;
+      // the thread's logits are read once and stay in registers for both passes
+      float v[SC];
       float tmax = -INFINITY;
-#pragma unroll 1
-      for (int cb = 0; cb < kATile / 32; ++cb) {
-        if (cb * 32 >= t.valid) break;
-        float v[32];
-        tmem_ld32(s_addr + cb * 32, v);
-        tmem_ld_wait();
+      if (ok) {
+        tc_fence_after();
 #pragma unroll
-        for (int c = 0; c < 32; ++c) if (cb * 32 + c < t.valid) tmax = fmaxf(tmax, v[c]);
+        for (int cb = 0; cb < SC / 32; ++cb) tmem_ld32(s_addr + cb * 32, v + cb * 32);
+        tmem_ld_wait();
+        if (my_valid < SC) {                                 // masked columns of a ragged tile do not take part
+#pragma unroll
+          for (int c = 0; c < SC; ++c) if (c >= my_valid) v[c] = -INFINITY;
+        }
+#pragma unroll
+        for (int c = 0; c < SC; c += 2) tmax = max3(tmax, v[c], v[c + 1]);
       }
-      const float m_new = fmaxf(m, tmax);
+      mx[(b * NW + wg) * kATile + row] = tmax;
+      named_barrier(1, NW * kATile);
+#pragma unroll
+      for (int w2 = 0; w2 < NW; ++w2) tmax = fmaxf(tmax, mx[(b * NW + w2) * kATile + row]);
+      const float m_new = fmaxf(m, tmax);                    // the same value in every warpgroup
       const float corr = ex2((m - m_new) * cs);
       const float neg = -m_new * cs;
       float rs = 0.f;
-      // pass 2: P = 2^(s*c - m*c), packed to bf16 and written over S (64 packed columns)
-#pragma unroll 1
-      for (int half = 0; half < 2; ++half) {
-        uint32_t packed[32];
+      if (ok) {
+        // P = 2^(s*c - m*c) as bf16 pairs (a masked column gives 2^-inf = 0), written over the columns just read
+        uint32_t packed[SC / 2];
 #pragma unroll
-        for (int sub = 0; sub < 2; ++sub) {
-          const int cb = half * 2 + sub;
-          float v[32];
-          if (cb * 32 < t.valid) {
-            tmem_ld32(s_addr + cb * 32, v);
-            tmem_ld_wait();
-          }
-#pragma unroll
-          for (int c = 0; c < 32; c += 2) {
-            float p0 = 0.f, p1 = 0.f;
-            if (cb * 32 + c < t.valid) p0 = ex2(fmaf(v[c], cs, neg));
-            if (cb * 32 + c + 1 < t.valid) p1 = ex2(fmaf(v[c + 1], cs, neg));
-            rs += p0 + p1;
-            packed[sub * 16 + c / 2] = pack_bf16(p0, p1);
-          }
+        for (int c = 0; c < SC; c += 2) {
+          const float p0 = ex2(fmaf(v[c], cs, neg)), p1 = ex2(fmaf(v[c + 1], cs, neg));
+          rs += p0 + p1;
+          packed[c / 2] = pack_bf16(p0, p1);
         }
-        // all four chunks of S must be in registers before P overwrites columns 0..63: half 0 writes P columns
-        // 0..31 (keys 0..63) after reading S columns 0..63; half 1 reads S columns 64..127 which P never touches
-        tmem_st32(s_addr + half * 32, packed);
+        if (SC == 64) tmem_st32(s_addr, packed); else tmem_st16(s_addr, packed);
+        tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive(bars.pready + b);
       }
-      tmem_st_wait();
       l = l * corr + rs;
       m = m_new;
-      tc_fence_before();
-      mbar_arrive(bars.pready + b);
-      if (j > 0 && !(ok = consume_pv(j - 1, corr_prev))) break;
+      if (j > 0) consume_pv(j - 1, corr_prev);
       corr_prev = corr;
     }
-    if (ok && nt > 0) ok = consume_pv(nt - 1, corr_prev);
-    const int i = q0 + row;
-    if (ok && i < M) {
-      const float inv = 1.f / l;
-      __nv_bfloat16* dst = out + (long long)(l0 + i) * sh.q_ts + (long long)h * sh.q_hs;
+    if (nt > 0) consume_pv(nt - 1, corr_prev);
+    lx[wg * kATile + row] = l;
+    named_barrier(1, NW * kATile);
+    l = 0.f;
 #pragma unroll
-      for (int c = 0; c < D; c += 8) {
+    for (int w2 = 0; w2 < NW; ++w2) l += lx[w2 * kATile + row];
+    const int i = q0 + row;
+    if (ok && !*abort_flag && i < M) {
+      const float inv = 1.f / l;
+      __nv_bfloat16* dst = out + (long long)(l0 + i) * sh.q_ts + (long long)h * sh.q_hs + wg * OC;
+#pragma unroll
+      for (int c = 0; c < OC; c += 8) {
         uint4 w;
         w.x = pack_bf16(o[c] * inv, o[c + 1] * inv);
         w.y = pack_bf16(o[c + 2] * inv, o[c + 3] * inv);
@@ -323,7 +377,7 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         w.w = pack_bf16(o[c + 6] * inv, o[c + 7] * inv);
         *reinterpret_cast<uint4*>(dst + c) = w;
       }
-      if (lse != nullptr) lse[(long long)h * sh.sumM + l0 + i] = m * sh.scale + logf(l);
+      if (wg == 0 && lse != nullptr) lse[(long long)h * sh.sumM + l0 + i] = m * sh.scale + logf(l);
     }
   }
   tc_fence_before();
@@ -362,11 +416,11 @@ int launch_attend_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const void
   dim3 grid((sh.maxM + kATile - 1) / kATile, sh.H, sh.R);
   if (sh.d == 128) {
     if (set_attend_attr<128>() != cudaSuccess) return 1;
-    attend_tc<128><<<grid, kAThreads, ASmem<128>::kDynamic, st>>>(mq, mkl, mvl, mkc, mvc, sh, offsets, (__nv_bfloat16*)out, lse,
+    attend_tc<128><<<grid, AWgs<128>::kThreads, ASmem<128>::kDynamic, st>>>(mq, mkl, mvl, mkc, mvc, sh, offsets, (__nv_bfloat16*)out, lse,
                                                                   ctx->status_dev);
   } else {
     if (set_attend_attr<64>() != cudaSuccess) return 1;
-    attend_tc<64><<<grid, kAThreads, ASmem<64>::kDynamic, st>>>(mq, mkl, mvl, mkc, mvc, sh, offsets, (__nv_bfloat16*)out, lse,
+    attend_tc<64><<<grid, AWgs<64>::kThreads, ASmem<64>::kDynamic, st>>>(mq, mkl, mvl, mkc, mvc, sh, offsets, (__nv_bfloat16*)out, lse,
                                                                 ctx->status_dev);
   }
   return 0;

@@ -92,7 +92,9 @@ ScoreWorkspace score_workspace(const maskkv_ctx* ctx, const Shape& sh) {
 // Adds `n` launches to the context's counter and maps the runtime's launch status to a return code.
 inline int launch_status(maskkv_ctx* ctx, int n) {
   ctx->launches += (unsigned long long)n;
-  return cudaGetLastError() == cudaSuccess ? MASKKV_OK : MASKKV_E_CUDA;
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) ctx->last_cuda_error = (int)e;
+  return e == cudaSuccess ? MASKKV_OK : MASKKV_E_CUDA;
 }
 
 // Scoring = sweep 1 (row statistics) + merge + sweep 2 (column sums) + mass reduction.  bf16 problems run the two
@@ -242,6 +244,9 @@ int maskkv_check_status(maskkv_ctx* ctx, void* stream, uint32_t* flags_out) {
 }
 
 uint64_t maskkv_launch_count(const maskkv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+const char* maskkv_last_cuda_error(const maskkv_ctx* ctx) {
+  return ctx && ctx->last_cuda_error ? cudaGetErrorString((cudaError_t)ctx->last_cuda_error) : "";
+}
 uint64_t maskkv_tensor_core_launch_count(const maskkv_ctx* ctx) { return ctx ? ctx->tc_launches : 0; }
 
 size_t maskkv_workspace_bytes(const maskkv_ctx* ctx, const maskkv_desc_t* desc) {

@@ -6,7 +6,7 @@
 //   * Operand tiles are [rows][64] bf16 boxes (128 bytes per row) written by TMA with the 128-byte
 //     swizzle; a head_dim of 128 is two such boxes.  Tile bases are 1024-byte aligned, groups of 8
 //     rows are 1024 bytes apart, and the k-th 16-element slice of a box starts 32*k bytes in.
-//   * Every wait on an mbarrier gives up after a bounded number of polls, raises
+//   * Every wait on an mbarrier gives up after a bounded time (about one second), raises
 //     MASKKV_FLAG_TIMEOUT in the status word and makes the whole block leave its loops; nothing
 //     in these kernels can spin forever.
 #pragma once
@@ -18,7 +18,7 @@
 namespace mkv {
 namespace tc {
 
-constexpr uint32_t kMaxPolls = 1u << 24;   // with the back-off below: on the order of a second
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // a wait gives up after about a second
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -50,13 +50,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 
 // Block-wide abort protocol: `abort_flag` lives in shared memory; once set every role stops waiting.
 // Returns false when the wait was abandoned (by this thread's limit or by another thread's).
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
                                           uint32_t* status, uint32_t where) {
-  for (uint32_t it = 0; it < kMaxPolls; ++it) {
+  // No sleeping between polls: try_wait already blocks for a short, hardware-chosen time, and the kernels that use
+  // this are latency chains.  The limit is wall time (kWaitLimitNs), checked every 256 polls.
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (it >= 128) {
-      __nanosleep(64);
+    if ((it & 255u) == 255u) {
       if (*abort_flag) return false;
+      const unsigned long long now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) break;
     }
   }
   *abort_flag = 1u;
@@ -71,6 +81,10 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
+}
+// Brings the tile into L2 only (no shared memory, no barrier): hides the DRAM latency of a later tma_load_3d.
+__device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap* map, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
