@@ -24,6 +24,7 @@ Readings taken where the paper is silent (each is also listed in the design note
     * Budgets are clamped to [0, N]; budget lost to floors or clamping stays unallocated.
     * argtopk uses the total order (score descending, index ascending); kept indices are
       reported in ascending index order.  NaN scores rank below every number.
+    * Eq. 8 (layer importance): a zero hidden-state row counts as cosine 0.
 
 Pins: tests/test_oracle_*.py (brute force, closed forms, invariants, library special cases,
 hand-derived budget examples under tests/golden/).  No function here is "parity unpinned".
@@ -92,6 +93,21 @@ def score(q_mask, k_prompt, k_mask, prompt_cu: Sequence[int], live_cu: Sequence[
             mass_p[r, hk] = imp.sum()                                # mask-to-prompt attention
             mass_m[r, hk] = sm
     return scores, mass_p, mass_m
+
+
+def layer_importance(h_in, h_out) -> float:
+    """Eq. 8: I^(l) = 1 - (1/n) sum_i cos_sim(h_in_i, h_out_i) over the n token rows of one layer.
+
+    h_in, h_out [n, hidden]: hidden states entering and leaving the layer's attention sub-layer (whether h_out carries
+    the residual is the caller's choice; the paper does not say).  Reading for a zero row, where the cosine is
+    undefined: it counts as cosine 0."""
+    a, b = _f64(h_in), _f64(h_out)
+    dot = (a * b).sum(axis=1)
+    na = np.sqrt((a * a).sum(axis=1))
+    nb = np.sqrt((b * b).sum(axis=1))
+    den = na * nb
+    cos = np.where(den > 0, dot / np.where(den > 0, den, 1.0), 0.0)
+    return float(1.0 - cos.sum() / a.shape[0])
 
 
 def guarded_floor(x: float) -> int:
