@@ -259,6 +259,31 @@ def bench_ours(args):
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), device)
     clocks = sampler.stop() if sampler else {}
 
+    # ---- calibration step of the budget rule (Eq. 8), outside the timed step: a streaming reduction bound by HBM
+    importance = None
+    if rank == 0:
+        n_tok, hidden = N + wl.n_mask, 4096                       # one LLaDA-8B-shaped layer: 541 MB read per call
+        g = torch.Generator(device=device); g.manual_seed(synth.BASE_SEED + 8)
+        h_in = torch.randn(n_tok, hidden, generator=g, device=device).bfloat16()
+        h_out = (h_in.float() + 0.5 * torch.randn(n_tok, hidden, generator=g, device=device)).bfloat16()
+        imp_out = torch.zeros(1, dtype=torch.float32, device=device)
+        imp_ws = ctx.maskkv_layer_importance(h_in, h_out, imp_out)
+        reps = 20
+        for _ in range(3):
+            ctx.maskkv_layer_importance(h_in, h_out, imp_out, imp_ws)
+        torch.cuda.synchronize()
+        i0, i1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        i0.record()
+        for _ in range(reps):
+            ctx.maskkv_layer_importance(h_in, h_out, imp_out, imp_ws)
+        i1.record()
+        torch.cuda.synchronize()
+        imp_us = 1e3 * i0.elapsed_time(i1) / reps
+        imp_bytes = 2.0 * n_tok * hidden * 2
+        importance = {"workload": f"{n_tok} tokens x hidden {hidden}, bf16", "us": imp_us, "bytes": imp_bytes,
+                      "value": float(imp_out.item())}
+        del h_in, h_out
+
     if world > 1:
         dist.destroy_process_group()
     if rank != 0:
@@ -303,6 +328,10 @@ def bench_ours(args):
         "roofline_other_calls": other,
         "mean_kept_per_head": mean_kept,
     }
+    if importance is not None:
+        gbs = importance["bytes"] / (importance["us"] * 1e-6) / 1e9
+        line["layer_importance"] = {"workload": importance["workload"], "us": round(importance["us"], 2),
+                                    "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm}}
     line["cpu_baseline"] = oracle_baseline(wl, budget_s=15.0)
     return line
 

@@ -123,6 +123,18 @@ size_t maskkv_workspace_bytes(const maskkv_ctx* ctx, const maskkv_desc_t* desc);
 int maskkv_layer_budgets(int64_t k_p, double beta, int32_t n_layers, const double* importance_host,
                          const uint8_t* is_boundary_host, int32_t* k_l_out_host);
 
+/* Eq. 8, the calibration step that produces the offline profile consumed by maskkv_layer_budgets:
+ *   importance = 1 - (1/n) sum_i cos_sim(h_in[i], h_out[i])
+ * over the n_tokens rows of one layer's attention sub-layer input / output hidden states (T = dtype, [n_tokens][hidden],
+ * row strides in elements, 0 = packed; hidden * sizeof(T) and the strides must be multiples of 16 bytes).  A row with a
+ * zero vector counts as cosine 0.  Writes one float to importance_out_dev.  Needs
+ * maskkv_layer_importance_workspace_bytes(ctx) bytes of scratch (8-byte aligned).  Deterministic: the same inputs
+ * give the same bits on every call. */
+size_t maskkv_layer_importance_workspace_bytes(const maskkv_ctx* ctx);
+int maskkv_layer_importance(maskkv_ctx* ctx, int32_t dtype, const void* h_in_dev, const void* h_out_dev,
+                            int64_t n_tokens, int32_t hidden, int64_t in_row_stride, int64_t out_row_stride,
+                            float* importance_out_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
+
 /* Eq. 6-7 and the sums of Eq. 14.  For every request r and KV head h: softmax (fp32) of
  * scale * q_i . k_j over the request's N_r prompt keys followed by its M_r mask keys, for each of the
  * H/H_kv query heads that share h; scores[h][prompt_cu[r] + j] = sum over those heads and mask rows i of

@@ -25,7 +25,7 @@ EXPORTS = (
     "maskkv_create", "maskkv_destroy", "maskkv_status_string", "maskkv_check_status", "maskkv_launch_count", "maskkv_last_cuda_error",
     "maskkv_tensor_core_launch_count",
     "maskkv_workspace_bytes",
-    "maskkv_layer_budgets", "maskkv_score", "maskkv_score_noalloc", "maskkv_score_noalloc_max_bytes", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend",
+    "maskkv_layer_budgets", "maskkv_layer_importance", "maskkv_layer_importance_workspace_bytes", "maskkv_score", "maskkv_score_noalloc", "maskkv_score_noalloc_max_bytes", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend",
 )
 
 
@@ -68,6 +68,9 @@ def _load() -> C.CDLL:
     lib.maskkv_workspace_bytes.argtypes = [vp, dp]
     lib.maskkv_workspace_bytes.restype = sz
     lib.maskkv_layer_budgets.argtypes = [i64, C.c_double, i32, C.POINTER(C.c_double), C.POINTER(C.c_uint8), C.POINTER(i32)]
+    lib.maskkv_layer_importance_workspace_bytes.argtypes = [vp]
+    lib.maskkv_layer_importance_workspace_bytes.restype = sz
+    lib.maskkv_layer_importance.argtypes = [vp, i32, vp, vp, i64, i32, i64, i64, vp, vp, sz, vp]
     lib.maskkv_score.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.maskkv_score_noalloc.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.maskkv_score_noalloc_max_bytes.argtypes = []
@@ -78,7 +81,8 @@ def _load() -> C.CDLL:
     lib.maskkv_attend.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("maskkv_status_string", "maskkv_workspace_bytes", "maskkv_launch_count", "maskkv_tensor_core_launch_count",
-                        "maskkv_score_noalloc_max_bytes", "maskkv_last_cuda_error"):
+                        "maskkv_score_noalloc_max_bytes", "maskkv_last_cuda_error",
+                        "maskkv_layer_importance_workspace_bytes"):
             getattr(lib, name).restype = C.c_int
     return lib
 
@@ -173,6 +177,16 @@ class Context:
         if rc not in (MASKKV_OK, MASKKV_E_TIMEOUT):
             _check(rc, "maskkv_check_status")
         return int(flags.value)
+
+    def maskkv_layer_importance(self, h_in, h_out, out, workspace=None):
+        """Eq. 8 for one layer: h_in, h_out [n_tokens, hidden] (bf16 or fp32, rows may be strided), out a 1-element fp32 tensor."""
+        if workspace is None:
+            workspace = torch.empty(int(lib.maskkv_layer_importance_workspace_bytes(self._h)), dtype=torch.uint8, device=h_in.device)
+        dt = MASKKV_F32 if h_in.dtype == torch.float32 else MASKKV_BF16
+        _check(lib.maskkv_layer_importance(self._h, dt, _ptr(h_in), _ptr(h_out), h_in.shape[0], h_in.shape[1], h_in.stride(0),
+                                           h_out.stride(0), _ptr(out), _ptr(workspace), workspace.numel(), _stream()),
+               "maskkv_layer_importance", self._h)
+        return workspace
 
     def maskkv_score(self, p: Problem, q_mask, k_prompt, k_mask, scores, mass_p, mass_m, workspace, row_weights=None):
         _check(lib.maskkv_score(self._h, C.byref(p.desc), _ptr(q_mask), _ptr(k_prompt), _ptr(k_mask), _ptr(row_weights),

@@ -9,6 +9,7 @@
 #include "budget.cuh"
 #include "common.cuh"
 #include "compact.cuh"
+#include "importance.cuh"
 #include "score_simt.cuh"
 #include "score_tc.h"
 #include "select.cuh"
@@ -282,6 +283,43 @@ int maskkv_layer_budgets(int64_t k_p, double beta, int32_t n_layers, const doubl
     k_l_out_host[l] = (int32_t)(k_base + (long long)floor(share + 1e-6));
   }
   return MASKKV_OK;
+}
+
+size_t maskkv_layer_importance_workspace_bytes(const maskkv_ctx* ctx) {
+  return ctx ? sizeof(double) * (size_t)ctx->sm_count * mkv::kImpBlocksPerSm : 0;
+}
+
+int maskkv_layer_importance(maskkv_ctx* ctx, int32_t dtype, const void* h_in_dev, const void* h_out_dev, int64_t n_tokens,
+                            int32_t hidden, int64_t in_row_stride, int64_t out_row_stride, float* importance_out_dev,
+                            void* workspace_dev, size_t workspace_bytes, void* stream) {
+  if (ctx == nullptr || importance_out_dev == nullptr || n_tokens < 0 || hidden <= 0) return MASKKV_E_INVALID;
+  if (dtype != MASKKV_F32 && dtype != MASKKV_BF16) return MASKKV_E_UNSUPPORTED;
+  if (n_tokens > 0 && (h_in_dev == nullptr || h_out_dev == nullptr)) return MASKKV_E_INVALID;
+  const int es = elem_size(dtype);
+  if (in_row_stride <= 0) in_row_stride = hidden;
+  if (out_row_stride <= 0) out_row_stride = hidden;
+  if (in_row_stride < hidden || out_row_stride < hidden) return MASKKV_E_INVALID;
+  if (((long long)hidden * es) % 16 || (in_row_stride * es) % 16 || (out_row_stride * es) % 16 || !aligned16(h_in_dev) ||
+      !aligned16(h_out_dev) || (reinterpret_cast<uintptr_t>(workspace_dev) & 7u))
+    return MASKKV_E_ALIGN;
+  if (workspace_dev == nullptr || workspace_bytes < maskkv_layer_importance_workspace_bytes(ctx)) return MASKKV_E_WORKSPACE;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int rows_per_block = mkv::kImpThreads / 32;
+  long long blocks = (n_tokens + rows_per_block - 1) / rows_per_block;
+  const long long max_blocks = (long long)ctx->sm_count * mkv::kImpBlocksPerSm;
+  if (blocks > max_blocks) blocks = max_blocks;
+  if (blocks < 1) blocks = 1;
+  double* partial = static_cast<double*>(workspace_dev);
+  if (dtype == MASKKV_F32)
+    mkv::importance_partial_kernel<float><<<(unsigned)blocks, mkv::kImpThreads, 0, st>>>(
+        static_cast<const float*>(h_in_dev), static_cast<const float*>(h_out_dev), n_tokens, hidden, in_row_stride, out_row_stride, partial);
+  else
+    mkv::importance_partial_kernel<__nv_bfloat16><<<(unsigned)blocks, mkv::kImpThreads, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(h_in_dev), static_cast<const __nv_bfloat16*>(h_out_dev), n_tokens, hidden, in_row_stride,
+        out_row_stride, partial);
+  mkv::importance_final_kernel<<<1, 32, 0, st>>>(partial, (int)blocks, n_tokens, importance_out_dev);
+  return launch_status(ctx, 2);
 }
 
 int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_dev, const void* k_prompt_dev,

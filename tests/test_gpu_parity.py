@@ -82,12 +82,21 @@ def test_score_row_weights(case):
         pytest.skip("covered on the smaller cases")
     g = torch.Generator().manual_seed(11)
     w = torch.rand(wl.n_requests * wl.n_mask, generator=g) * 2
+    w[: wl.n_mask // 2] = 0.0        # position-aware voting: the front half of the first request's mask rows does not vote
     sc, mp, mm = O.score(case["x"]["q_mask"], case["x"]["k_prompt"], case["x"]["k_mask"], wl.prompt_cu(), wl.live_cu(),
                          row_weights=w.numpy())
     run.score(case["xd"], row_weights=to_dev(w))
     torch.cuda.synchronize()
     assert_scores_close(run.scores.cpu().numpy(), sc)
     assert_scores_close(run.mass_m.cpu().numpy(), mm, what="mass_m")
+    # voting with the back half only = scoring with 0/1 weights (the mask-position ablation of the paper)
+    if wl.n_requests == 1:
+        w01 = torch.zeros(wl.n_mask); w01[wl.n_mask // 2:] = 1.0
+        sc2, _, _ = O.score(case["x"]["q_mask"], case["x"]["k_prompt"], case["x"]["k_mask"], wl.prompt_cu(), wl.live_cu(),
+                            row_weights=w01.numpy())
+        run.score(case["xd"], row_weights=to_dev(w01))
+        torch.cuda.synchronize()
+        assert_scores_close(run.scores.cpu().numpy(), sc2)
 
 
 def test_budget_bit_exact(case):
