@@ -210,17 +210,22 @@ def bench_ours(args):
     for i in range(args.warmup):
         step(i)
     barrier()
-    per_call = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
     launches0 = ctx.maskkv_launch_count()
     barrier()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
     for i in range(args.steps):
-        step(args.warmup + i, per_call[i])
+        step(args.warmup + i)
     t1.record()
     barrier()
     launches = ctx.maskkv_launch_count() - launches0
     elapsed_ms = max_over_ranks(t0.elapsed_time(t1), device)
+    # Per-call breakdown from a separate pass: an event between every two calls costs a few microseconds of
+    # serialisation per step, which does not belong in the headline number.
+    per_call = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(min(args.steps, 200))]
+    for i, ev in enumerate(per_call):
+        step(args.warmup + i, ev)
+    barrier()
     mean_kept = float(buf.offsets[-1].item()) / wl.n_kv_heads
     call_us = {name: 1e3 * statistics.mean(ev[c].elapsed_time(ev[c + 1]) for ev in per_call) for c, name in enumerate(CALLS)}
     flags = ctx.maskkv_check_status()

@@ -70,7 +70,7 @@ int resolve(const maskkv_desc_t* d, Shape* sh) {
 }
 
 struct ScoreWorkspace {
-  size_t lse_off, part_off, mass_off, total;
+  size_t lse_off, part_off, mass_off, cnt_off, total;
   int C, Tmax;
 };
 
@@ -85,7 +85,8 @@ ScoreWorkspace score_workspace(const maskkv_ctx* ctx, const Shape& sh) {
   size_t off = 0;
   w.lse_off = off;  off = align_up(off + sizeof(float) * (size_t)sh.H * sh.sumM, 256);
   w.part_off = off; off = align_up(off + sizeof(float2) * (size_t)sh.H * sh.sumM * w.C, 256);
-  w.mass_off = off; off = align_up(off + sizeof(float2) * (size_t)sh.R * sh.Hkv * w.Tmax * 4, 256);
+  w.mass_off = off; off = align_up(off + sizeof(float2) * (size_t)sh.R * sh.Hkv * w.Tmax * 8, 256);
+  w.cnt_off = off;  off = align_up(off + sizeof(uint32_t) * (size_t)sh.R * sh.Hkv, 256);
   w.total = off;
   return w;
 }
@@ -107,36 +108,42 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, co
   float* lse = reinterpret_cast<float*>(ws + w.lse_off);
   float2* part = reinterpret_cast<float2*>(ws + w.part_off);
   float2* mass_part = reinterpret_cast<float2*>(ws + w.mass_off);
+  uint32_t* seg_cnt = reinterpret_cast<uint32_t*>(ws + w.cnt_off);
   const int S = sh.R * sh.Hkv;
   const bool tc_ok = mkv::tc::score_tc_supported(ctx, sh);
+  const bool want_tc2 = tc_ok && !(ctx->force_simt & 2u);
   int n = 0;
+  bool tc1 = false;                                          // sweep 1 ran on the tensor cores: `part` has its layout
   if (sh.sumM > 0) {
-    bool done = false;
     if (tc_ok && !(ctx->force_simt & 1u))
-      done = mkv::tc::launch_score_stats_tc(ctx, sh, desc->prompt_cu, desc->live_cu, q, kp, km, part, w.C, lse, st) == 0;
-    if (done) ++ctx->tc_launches;
-    if (!done) {
+      tc1 = mkv::tc::launch_score_stats_tc(ctx, sh, desc->prompt_cu, desc->live_cu, q, kp, km, part, w.C, seg_cnt, st) == 0;
+    if (tc1) { ++ctx->tc_launches; ++n; }
+    if (!tc1) {
       const int q_tiles = (sh.maxM + mkv::kSimtThreads - 1) / mkv::kSimtThreads;
       dim3 g1((unsigned)((sh.maxN + sh.maxM + mkv::kStatsChunk - 1) / mkv::kStatsChunk), sh.H, sh.R * q_tiles);
       mkv::score_stats_simt<T, D><<<g1, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, part, w.C);
       const long long rows = (long long)sh.H * sh.sumM;
       mkv::score_merge_stats<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(sh, part, w.C, lse);
+      n += 2;
+      if (want_tc2 && cudaMemsetAsync(seg_cnt, 0, sizeof(uint32_t) * (size_t)S, st) != cudaSuccess) return launch_status(ctx, n);
     }
-    n += 2;
   }
-  bool done = false;
-  if (tc_ok && !(ctx->force_simt & 2u)) {
-    done = mkv::tc::launch_score_colsum_tc(ctx, sh, desc->prompt_cu, desc->live_cu, q, kp, km, lse, rw, scores, mass_part, w.Tmax,
-                                           any_without_voters, st) == 0;
-    if (done) { ++ctx->tc_launches; n += any_without_voters ? 1 : 0; }
+  bool tc2 = false;
+  if (want_tc2) {
+    // after a tensor-core sweep 1 the kernel merges the partials itself; otherwise it reads lse
+    tc2 = mkv::tc::launch_score_colsum_tc(ctx, sh, desc->prompt_cu, desc->live_cu, q, kp, km, lse, tc1 ? part : nullptr, w.C, rw,
+                                          scores, mass_part, w.Tmax, seg_cnt, mass_p, mass_m, any_without_voters, st) == 0;
+    if (tc2) { ++ctx->tc_launches; n += any_without_voters ? 2 : 1; }
   }
-  if (!done) {
+  if (!tc2) {
+    if (tc1) { mkv::tc::launch_score_merge_tc(ctx, sh, desc->prompt_cu, desc->live_cu, part, w.C, lse, st); ++n; }
     dim3 g2(w.Tmax, sh.Hkv, sh.R);
     mkv::score_colsum_simt<T, D><<<g2, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, lse, rw,
                                                                     scores, mass_part, w.Tmax);
+    mkv::score_mass_reduce<<<(S + 3) / 4, 128, 0, st>>>(sh, mass_part, w.Tmax, mass_p, mass_m);
+    n += 2;
   }
-  mkv::score_mass_reduce<<<(S + 3) / 4, 128, 0, st>>>(sh, mass_part, w.Tmax, mass_p, mass_m);
-  return launch_status(ctx, n + 2);
+  return launch_status(ctx, n);
 }
 
 template <typename T, int D>

@@ -206,19 +206,23 @@ __host__ __device__ __forceinline__ int cta_of(long long f, long long F, int G) 
 
 // =====================================================================================================
 // sweep 1: per-row (max, sum of exp) over a segment of key tiles.
-// part[(h*sumM + row)*C + 2*(cta - first cta of the row's unit) + half] = (max of scaled logits, sum of exp).
+// part[(h*C + slot)*sumM + row] = (max of scaled logits, sum of exp), slot = 2*(cta - first cta of the row's unit) + half:
+// neighbouring rows are neighbours in memory, so a warp's 32 rows of one slot are one 256-byte access.
 // =====================================================================================================
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kp,
                const __grid_constant__ CUtensorMap map_km, Shape sh, float2* __restrict__ part, int C, long long F,
-               uint32_t* __restrict__ status) {
+               uint32_t* __restrict__ seg_cnt, uint32_t* __restrict__ status) {
   using S = Smem<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = align_1024(smem_raw);
   const Bars bars = carve_bars(base, S::kBarOff);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + S::kMiscOff);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base + S::kMiscOff + 4);
+  // sweep 2 counts finished mass partials per segment in seg_cnt; it starts after this grid has ended
+  if (blockIdx.x == 0 && seg_cnt != nullptr)
+    for (int i = threadIdx.x; i < sh.R * sh.Hkv; i += blockDim.x) seg_cnt[i] = 0u;
   block_setup(bars, 4, tmem_slot, abort_flag);
   const uint32_t tmem_base = *tmem_slot;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -305,27 +309,42 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const int n_qtiles = (s.M - q0 > kTile) ? 2 : 1;
       if (a >= n_qtiles) continue;
       float m = -INFINITY, l = 0.f;                         // m in raw (unscaled) logits
+      // The reference m of the running sum l = sum 2^((s - m) * cs) is only moved when a logit exceeds it by more
+      // than 2^kSlack: the exponentials of a chunk then do not wait for the chunk's maximum (which is found beside
+      // them), and l stays far inside the fp32 range (each term <= 2^kSlack, at most 2^31 terms).  (m, l) is as good a
+      // pair for the later log-sum-exp merge as (true maximum, sum) - only ln l + m * scale is ever used.
+      constexpr float kSlack = 64.f;
+      auto chunk_max = [&](const float* v) {
+        float t[11];
+#pragma unroll
+        for (int c = 0; c < 10; ++c) t[c] = max3(v[3 * c], v[3 * c + 1], v[3 * c + 2]);
+        t[10] = fmaxf(v[30], v[31]);
+        return fmaxf(max3(max3(t[0], t[1], t[2]), max3(t[3], t[4], t[5]), max3(t[6], t[7], t[8])), fmaxf(t[9], t[10]));
+      };
+      auto chunk_sum = [&](const float* v, float ref) {
+        const float neg = -ref * cs;
+        const uint64_t cs2 = pack2(cs, cs), neg2 = pack2(neg, neg);
+        uint64_t acc_a = pack2(0.f, 0.f), acc_b = pack2(0.f, 0.f);
+#pragma unroll
+        for (int c = 0; c < 32; c += 4) {
+          float x0, x1, x2, x3;
+          unpack2(fma2(pack2(v[c], v[c + 1]), cs2, neg2), x0, x1);
+          unpack2(fma2(pack2(v[c + 2], v[c + 3]), cs2, neg2), x2, x3);
+          acc_a = add2(acc_a, pack2(ex2(x0), ex2(x1)));
+          acc_b = add2(acc_b, pack2(ex2(x2), ex2(x3)));
+        }
+        float l0, l1;
+        unpack2(add2(acc_a, acc_b), l0, l1);
+        return l0 + l1;
+      };
       auto absorb = [&](float* v, int col0, int valid) {
         if (valid - col0 < 32) {
 #pragma unroll
           for (int c = 0; c < 32; ++c) if (col0 + c >= valid) v[c] = -INFINITY;
         }
-        float cmax = fmaxf(v[0], v[1]);
-#pragma unroll
-        for (int c = 2; c < 32; c += 2) cmax = max3(cmax, v[c], v[c + 1]);
+        const float cmax = chunk_max(v);
         if (cmax > m) { l *= ex2((m - cmax) * cs); m = cmax; }
-        const float neg = -m * cs;
-        const uint64_t cs2 = pack2(cs, cs), neg2 = pack2(neg, neg);
-        uint64_t acc2 = pack2(0.f, 0.f);
-#pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          float x0, x1;
-          unpack2(fma2(pack2(v[c], v[c + 1]), cs2, neg2), x0, x1);
-          acc2 = add2(acc2, pack2(ex2(x0), ex2(x1)));
-        }
-        float l0, l1;
-        unpack2(acc2, l0, l1);
-        l += l0 + l1;
+        l += chunk_sum(v, m);
       };
       // Rolling double buffer over the chunk stream (tile 0: c0, c1; tile 1: c0, c1; ...): while one 32-column chunk
       // is being exponentiated the next one - possibly of the next tile - is already on its way from tensor memory.
@@ -362,46 +381,68 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (!ok) continue;
       const int i = q0 + a * kTile + row;
       const int slot = 2 * ((int)blockIdx.x - cta_of(s.unit_start, F, gridDim.x)) + half;
-      if (i < s.M) part[((long long)h * sh.sumM + s.l0 + i) * C + slot] = make_float2(m * sh.scale, l);
+      if (i < s.M) part[((long long)h * C + slot) * sh.sumM + s.l0 + i] = make_float2(m * sh.scale, l);
     }
   }
   block_teardown(tmem_base);
 }
 
-// One thread per (h, row): lse[h*sumM + row] = ln sum_j exp(s_j), from the partials the CTAs of sweep 1 left.
+// ln sum_j exp(s_j) of query row `row` (index over all requests) of head h, which lies in 256-query block `qblock` of
+// request r: log-sum-exp merge of the partials the CTAs of sweep 1 left.  F1, G1: flat tile count and grid of sweep 1.
+__device__ __noinline__ float merged_lse(const Shape& sh, const float2* __restrict__ part, int C, long long F1, int G1,
+                                            int r, int h, int qblock, int row) {
+  long long base = 0;
+  for (int r2 = 0; r2 < r; ++r2) {
+    const int N2 = sh.prompt_cu[r2 + 1] - sh.prompt_cu[r2], M2 = sh.live_cu[r2 + 1] - sh.live_cu[r2];
+    base += (long long)walk_groups(sh, true, M2) * tiles_of(N2, M2);
+  }
+  const int N = sh.prompt_cu[r + 1] - sh.prompt_cu[r], M = sh.live_cu[r + 1] - sh.live_cu[r];
+  const int T = tiles_of(N, M), qp_n = (M + kQBlock - 1) / kQBlock;
+  const long long unit_start = base + ((long long)h * qp_n + qblock) * T;
+  const int slots = 2 * (cta_of(unit_start + T - 1, F1, G1) - cta_of(unit_start, F1, G1) + 1);
+  const float2* p = part + (long long)h * C * sh.sumM + row;      // slot c at p[c * sumM]
+  // the loads of a batch are issued together (a row has 4 to 8 partials on a long prompt)
+  float m = -INFINITY, l = 0.f;
+  for (int c0 = 0; c0 < slots; c0 += 8) {
+    float2 v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v[k] = c0 + k < slots ? p[(long long)(c0 + k) * sh.sumM] : make_float2(-INFINITY, 0.f);
+    float bm = m;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) bm = fmaxf(bm, v[k].x);
+    if (bm == -INFINITY) continue;
+    l *= expf(m - bm);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) l += v[k].y * expf(v[k].x - bm);
+    m = bm;
+  }
+  return m + logf(l);
+}
+
+// One thread per (h, row): lse[h*sumM + row].  Only launched when sweep 2 does not run on the tensor-core kernel
+// (which merges the partials itself).
 __global__ void score_merge_stats_tc(Shape sh, const float2* __restrict__ part, int C, long long F, int G,
                                      float* __restrict__ lse) {
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= (long long)sh.H * sh.sumM) return;
   const int h = (int)(t / sh.sumM), row = (int)(t % sh.sumM);
   const int r = find_request(sh.live_cu, sh.R, row);
-  long long base = 0;
-  for (int r2 = 0; r2 < r; ++r2) {
-    const int N2 = sh.prompt_cu[r2 + 1] - sh.prompt_cu[r2], M2 = sh.live_cu[r2 + 1] - sh.live_cu[r2];
-    base += (long long)walk_groups(sh, true, M2) * tiles_of(N2, M2);
-  }
-  const int N = sh.prompt_cu[r + 1] - sh.prompt_cu[r], l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
-  const int T = tiles_of(N, M), qp_n = (M + kQBlock - 1) / kQBlock;
-  const long long unit_start = base + ((long long)h * qp_n + (row - l0) / kQBlock) * T;
-  const int slots = 2 * (cta_of(unit_start + T - 1, F, G) - cta_of(unit_start, F, G) + 1);
-  const float2* p = part + t * C;
-  float m = -INFINITY;
-  for (int c = 0; c < slots; ++c) m = fmaxf(m, p[c].x);
-  float l = 0.f;
-  for (int c = 0; c < slots; ++c) l += p[c].y * expf(p[c].x - m);
-  lse[t] = m + logf(l);
+  lse[t] = merged_lse(sh, part, C, F, G, r, h, (row - sh.live_cu[r]) / kQBlock, row);
 }
 
 // =====================================================================================================
 // sweep 2: column sums.
 // scores[hk][p0 + j] = sum over the group's query heads and mask rows of w_i * exp(s_ij - lse_i);
-// mass_part[((r*H_kv + hk)*Tmax + t)*4 + w] = (sum over prompt keys, sum over mask keys) of tile t seen by warp w.
+// mass_part[(r*H_kv + hk)*Tmax*8 + slot] = (sum over prompt keys, sum over mask keys) one warp of one CTA saw;
+// mass_p / mass_m [r*H_kv + hk] = their sums, written by the warp that completes the segment.
 // =====================================================================================================
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kp,
                 const __grid_constant__ CUtensorMap map_km, Shape sh, const float* __restrict__ lse,
+                const float2* __restrict__ part, int C, long long F1, int G1,
                 const float* __restrict__ w, float* __restrict__ scores, float2* __restrict__ mass_part, int Tmax,
+                uint32_t* __restrict__ seg_cnt, float* __restrict__ mass_p, float* __restrict__ mass_m,
                 long long F, uint32_t* __restrict__ status) {
   using S = Smem<D>;
   extern __shared__ uint8_t smem_raw[];
@@ -508,11 +549,46 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     int base_par = 0;
     bool ok = true;
     const float* c2 = c2s;
+    // Attention mass of the segment in hand, summed over the tiles this warp finished (half-0 warps only).  When the
+    // walk leaves the segment the warp stores its pair in slot (CTA - first CTA of the segment) * 8 + warp and
+    // counts itself in; the warp that completes the count adds the slots up, always in slot order.
+    int cur_seg = -1, cur_T = 0;
+    long long cur_start = 0;
+    float run_p = 0.f, run_m = 0.f;
+    auto flush = [&]() {
+      if (cur_seg < 0 || half != 0) return;
+      const int first = cta_of(cur_start, F, gridDim.x);
+      const unsigned slots = 8u * (unsigned)(cta_of(cur_start + cur_T - 1, F, gridDim.x) - first + 1);
+      float2* mp = mass_part + (long long)cur_seg * Tmax * 8;
+      unsigned last = 0;
+      if (lane == 0) {
+        mp[((int)blockIdx.x - first) * 8 + buf * 4 + lane_group] = make_float2(run_p, run_m);
+        __threadfence();
+        last = atomicAdd(seg_cnt + cur_seg, 1u) + 1u == slots;
+      }
+      if (__shfl_sync(0xffffffffu, last, 0)) {
+        __threadfence();
+        float sum_p = 0.f, sum_m = 0.f;
+        for (unsigned t = lane; t < slots; t += 32) {
+          const float2 v = __ldcg(mp + t);
+          sum_p += v.x;
+          sum_m += v.y;
+        }
+        sum_p = warp_sum(sum_p);
+        sum_m = warp_sum(sum_m);
+        if (lane == 0) { mass_p[cur_seg] = sum_p; mass_m[cur_seg] = sum_m; }
+      }
+    };
     while (walker_next(wk, sh, kColsumMaxTiles, s)) {
       const int q_per_head = (s.M + kQBlock - 1) / kQBlock, nqb = sh.g * q_per_head;
       const bool reuse_q = nqb == 1 && s.r == last_r && s.g == last_g;
       last_r = s.r; last_g = s.g;
       const int seg = s.r * sh.Hkv + s.g;
+      if (seg != cur_seg) {
+        flush();
+        cur_seg = seg; cur_T = s.T; cur_start = s.unit_start;
+        run_p = run_m = 0.f;
+      }
       for (int qb = 0; qb < nqb; ++qb) {
         const int h = s.g * sh.g + qb / q_per_head, q0 = (qb % q_per_head) * kQBlock + half * kTile;
         const int nq = max(0, min(kTile, s.M - q0));        // voters in this warpgroup's half of the block
@@ -520,7 +596,12 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           float* c2w = c2s + (wg * 2 + (c2_it & 1)) * kTile;
           ++c2_it;
           float cst = -INFINITY;                            // 2^(x - inf) = 0: rows that do not exist never vote
-          if (row < nq) cst = (w ? log2f(w[s.l0 + q0 + row]) : 0.f) - lse[(long long)h * sh.sumM + s.l0 + q0 + row] * kLog2e;
+          if (row < nq) {
+            const int i = s.l0 + q0 + row;
+            const float ln_z = part != nullptr ? merged_lse(sh, part, C, F1, G1, s.r, h, qb % q_per_head, i)
+                                               : lse[(long long)h * sh.sumM + i];
+            cst = (w ? log2f(w[i]) : 0.f) - ln_z * kLog2e;
+          }
           c2w[row] = cst;                                   // stored negated: x = s*c + cst
           named_barrier(1 + wg, kTile);
           c2 = c2w;
@@ -571,25 +652,26 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           if (row >= kt.valid) acc = 0.f;
           if (kt.prompt && row < kt.valid) scores[(long long)s.g * sh.sumN + kt.token + row] = acc;
           acc = warp_sum(acc);
-          if (lane == 0)
-            mass_part[((long long)seg * Tmax + s.t + s.dir * tl) * 4 + lane_group] = kt.prompt ? make_float2(acc, 0.f) : make_float2(0.f, acc);
+          if (kt.prompt) run_p += acc; else run_m += acc;
         }
       }
       base_par ^= s.len & 1;
     }
+    flush();
   }
   block_teardown(tmem_base);
 }
 
 // Requests without voters (M = 0): every score is zero and so are the masses.  grid (tiles, H_kv, R).
-__global__ void score_zero_fill(Shape sh, float* __restrict__ scores, float2* __restrict__ mass_part, int Tmax) {
+__global__ void score_zero_fill(Shape sh, float* __restrict__ scores, float* __restrict__ mass_p, float* __restrict__ mass_m) {
   const int t = blockIdx.x, hk = blockIdx.y, r = blockIdx.z;
   const int p0 = sh.prompt_cu[r], N = sh.prompt_cu[r + 1] - p0;
   const int M = sh.live_cu[r + 1] - sh.live_cu[r];
-  if (M > 0 || t * kTile >= N) return;
+  if (M > 0) return;
+  if (t == 0 && threadIdx.x == 0) { mass_p[r * sh.Hkv + hk] = 0.f; mass_m[r * sh.Hkv + hk] = 0.f; }
+  if (t * kTile >= N) return;
   const int j = t * kTile + threadIdx.x;
   if (j < N) scores[(long long)hk * sh.sumN + p0 + j] = 0.f;
-  if (threadIdx.x < 4) mass_part[((long long)(r * sh.Hkv + hk) * Tmax + t) * 4 + threadIdx.x] = make_float2(0.f, 0.f);
 }
 
 // =====================================================================================================
@@ -649,7 +731,7 @@ bool score_tc_supported(const maskkv_ctx* ctx, const Shape& sh) {
 }
 
 int launch_score_stats_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prompt_cu_host, const int32_t* live_cu_host,
-                          const void* q, const void* kp, const void* km, float2* part, int C, float* lse, cudaStream_t st) {
+                          const void* q, const void* kp, const void* km, float2* part, int C, uint32_t* seg_cnt, cudaStream_t st) {
   Maps m;
   if (!build_maps(ctx, sh, q, kp, km, &m)) return 1;
   const long long F = flat_tiles(sh, prompt_cu_host, live_cu_host, true);
@@ -657,37 +739,44 @@ int launch_score_stats_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* promp
   const int grid = (int)(F < ctx->sm_count ? F : ctx->sm_count);
   if (sh.d == 128) {
     if (set_smem_attr<128>() != cudaSuccess) return 1;
-    score_stats_tc<128><<<grid, kThreads, Smem<128>::kDynamic, st>>>(m.q, m.kp, m.km, sh, part, C, F, ctx->status_dev);
+    score_stats_tc<128><<<grid, kThreads, Smem<128>::kDynamic, st>>>(m.q, m.kp, m.km, sh, part, C, F, seg_cnt, ctx->status_dev);
   } else {
     if (set_smem_attr<64>() != cudaSuccess) return 1;
-    score_stats_tc<64><<<grid, kThreads, Smem<64>::kDynamic, st>>>(m.q, m.kp, m.km, sh, part, C, F, ctx->status_dev);
+    score_stats_tc<64><<<grid, kThreads, Smem<64>::kDynamic, st>>>(m.q, m.kp, m.km, sh, part, C, F, seg_cnt, ctx->status_dev);
   }
-  const long long rows = (long long)sh.H * sh.sumM;
-  score_merge_stats_tc<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(sh, part, C, F, grid, lse);
   return 0;
 }
 
+void launch_score_merge_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prompt_cu_host, const int32_t* live_cu_host,
+                           const float2* part, int C, float* lse, cudaStream_t st) {
+  const long long F = flat_tiles(sh, prompt_cu_host, live_cu_host, true);
+  const int grid = (int)(F < ctx->sm_count ? F : ctx->sm_count);
+  const long long rows = (long long)sh.H * sh.sumM;
+  score_merge_stats_tc<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(sh, part, C, F, grid, lse);
+}
+
 int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prompt_cu_host, const int32_t* live_cu_host,
-                           const void* q, const void* kp, const void* km, const float* lse, const float* w, float* scores,
-                           float2* mass_part, int Tmax, bool any_without_voters, cudaStream_t st) {
+                           const void* q, const void* kp, const void* km, const float* lse, const float2* part, int C,
+                           const float* w, float* scores, float2* mass_part, int Tmax, uint32_t* seg_cnt, float* mass_p,
+                           float* mass_m, bool any_without_voters, cudaStream_t st) {
   Maps m;
   if (!build_maps(ctx, sh, q, kp, km, &m)) return 1;
   const long long F = flat_tiles(sh, prompt_cu_host, live_cu_host, false);
   if (F <= 0) return 1;
   const int grid = (int)(F < ctx->sm_count ? F : ctx->sm_count);
+  const long long F1 = flat_tiles(sh, prompt_cu_host, live_cu_host, true);     // sweep 1's walk, for its partials
+  const int G1 = (int)(F1 < ctx->sm_count ? F1 : ctx->sm_count);
+  if (sh.d == 128 ? set_smem_attr<128>() != cudaSuccess : set_smem_attr<64>() != cudaSuccess) return 1;
   if (any_without_voters) {
     dim3 gz(score_tc_max_tiles(sh), sh.Hkv, sh.R);
-    score_zero_fill<<<gz, kTile, 0, st>>>(sh, scores, mass_part, Tmax);
+    score_zero_fill<<<gz, kTile, 0, st>>>(sh, scores, mass_p, mass_m);
   }
-  if (sh.d == 128) {
-    if (set_smem_attr<128>() != cudaSuccess) return 1;
-    score_colsum_tc<128><<<grid, kThreads, Smem<128>::kDynamic, st>>>(m.q, m.kp, m.km, sh, lse, w, scores, mass_part, Tmax, F,
-                                                                      ctx->status_dev);
-  } else {
-    if (set_smem_attr<64>() != cudaSuccess) return 1;
-    score_colsum_tc<64><<<grid, kThreads, Smem<64>::kDynamic, st>>>(m.q, m.kp, m.km, sh, lse, w, scores, mass_part, Tmax, F,
-                                                                     ctx->status_dev);
-  }
+  if (sh.d == 128)
+    score_colsum_tc<128><<<grid, kThreads, Smem<128>::kDynamic, st>>>(m.q, m.kp, m.km, sh, lse, part, C, F1, G1, w, scores, mass_part,
+                                                                      Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
+  else
+    score_colsum_tc<64><<<grid, kThreads, Smem<64>::kDynamic, st>>>(m.q, m.kp, m.km, sh, lse, part, C, F1, G1, w, scores, mass_part,
+                                                                     Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
   return 0;
 }
 
