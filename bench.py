@@ -18,9 +18,9 @@ import argparse
 import json
 import os
 import statistics
-import subprocess
+
 import sys
-import tempfile
+import threading
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -68,53 +68,71 @@ def sum_over_ranks(value: float, device=None) -> float:
 
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Reads SM clock, power and the clock-event reasons of one GPU every 10 ms through NVML (read-only queries) on a
+    thread of its own.  mark() brackets the timed region; stop() reports the medians inside it."""
 
     def __init__(self, gpu_index: int):
-        self.path = tempfile.mktemp(prefix="maskkv_clocks_", suffix=".csv")
-        self.proc = None
+        self.samples = []            # (time, sm_mhz, power_w, reasons bitmask)
+        self.marks = {}
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
         try:
-            self.f = open(self.path, "w")
-            self.proc = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
-                                         stderr=subprocess.DEVNULL)
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            uuid = torch.cuda.get_device_properties(gpu_index).uuid      # CUDA_VISIBLE_DEVICES may renumber the GPUs
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(gpu_index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
         except Exception:
-            self.proc = None
+            self._thread = None
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                mhz = float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                watts = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                reasons = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                self.samples.append((time.perf_counter(), mhz, watts, reasons))
+            except Exception:
+                pass
+            self._stop.wait(0.01)
+
+    def mark(self, name: str):
+        self.marks[name] = time.perf_counter()
 
     def stop(self) -> dict:
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.proc is None:
+        out = {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        if self._thread is None:
             return out
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        self.f.close()
-        sm, mx, reasons = [], [], set()
-        try:
-            for ln in open(self.path):
-                p = [x.strip() for x in ln.split(",")]
-                if len(p) < 9:
-                    continue
-                try:
-                    sm.append(float(p[1])); mx.append(float(p[2]))
-                except ValueError:
-                    continue
-                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
-                    if val.lower().startswith("active"):
-                        reasons.add(name)
-            os.unlink(self.path)
-        except Exception:
-            pass
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
-        out["reasons"] = sorted(reasons)
+        self._stop.set()
+        self._thread.join(timeout=2)
+        nv = self.nv
+        t0, t1 = self.marks.get("timed_start"), self.marks.get("timed_end")
+        inside = [x for x in self.samples if t0 is not None and t1 is not None and t0 <= x[0] <= t1]
+        region = "timed steps"
+        if len(inside) < 3:
+            inside, region = self.samples, "whole run"
+        if not inside:
+            return out
+        bits = 0
+        for x in inside:
+            bits |= x[3]
+        names = (("hw_slowdown", nv.nvmlClocksEventReasonHwSlowdown), ("hw_thermal_slowdown", nv.nvmlClocksEventReasonHwThermalSlowdown),
+                 ("sw_thermal_slowdown", nv.nvmlClocksEventReasonSwThermalSlowdown), ("sw_power_cap", nv.nvmlClocksEventReasonSwPowerCap),
+                 ("hw_power_brake", nv.nvmlClocksEventReasonHwPowerBrakeSlowdown))
+        out.update(sm_mhz=statistics.median(x[1] for x in inside), power_w=round(statistics.median(x[2] for x in inside), 1),
+                   samples=len(inside), region=region, reasons=[n for n, b in names if bits & b])
         return out
 
 
-# ----------------------------------------------------------------------------- our arm
+
 class LayerBuffers:
     """Device-side outputs and scratch shared by all layers of the workload (one layer in flight at a time)."""
 
@@ -213,11 +231,13 @@ def bench_ours(args):
     launches0 = ctx.maskkv_launch_count()
     barrier()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if sampler: sampler.mark("timed_start")
     t0.record()
     for i in range(args.steps):
         step(args.warmup + i)
     t1.record()
     barrier()
+    if sampler: sampler.mark("timed_end")
     launches = ctx.maskkv_launch_count() - launches0
     elapsed_ms = max_over_ranks(t0.elapsed_time(t1), device)
     # Per-call breakdown from a separate pass: an event between every two calls costs a few microseconds of
@@ -426,7 +446,7 @@ def main():
         args.warmup = 1 if args.warmup is None else max(0, args.warmup)
         line = bench_reference(args)
     else:
-        args.steps = 1000 if args.steps is None else max(1, args.steps)
+        args.steps = 2000 if args.steps is None else max(1, args.steps)
         args.warmup = 5 if args.warmup is None else max(3, args.warmup)
         line = bench_ours(args)
     if line is not None:
