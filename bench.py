@@ -350,6 +350,7 @@ def bench_ours(args):
                      "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
                      "peak_source": peaks["source"] + " (sustained bf16; the kernels run inside a long step)",
                      "traffic": SCORE_DRAM_TRAFFIC_BYTES, "executed_over_algorithmic_flops": 2.0},
+        "roofline_alu": exp_roofline(wl, call_us["score"], clocks.get("sm_max_mhz") or 1965.0),
         "roofline_other_calls": other,
         "mean_kept_per_head": mean_kept,
     }
@@ -359,6 +360,18 @@ def bench_ours(args):
                                     "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm}}
     line["cpu_baseline"] = oracle_baseline(wl, budget_s=15.0)
     return line
+
+
+def exp_roofline(wl, score_us, sm_max_mhz):
+    """The unit that actually bounds maskkv_score: every logit is exponentiated once per sweep (row statistics, then
+    weights) on the special-function unit, 16 results per clock per SM on 148 SMs; the peak takes the maximum SM
+    clock, which the kernels do not hold under load."""
+    N, M, H = wl.prompt_lens[0], wl.n_mask, wl.n_q_heads
+    exps = 2.0 * M * (N + M) * H
+    achieved = exps / (score_us * 1e-6) / 1e12
+    peak = 148 * 16 * sm_max_mhz * 1e6 / 1e12
+    return {"kernel": "maskkv_score", "bound": "alu", "achieved": achieved, "peak": peak, "unit": "Texp/s",
+            "frac": achieved / peak, "peak_source": "148 SMs x 16 ex2 per clock x max SM clock (nominal unit count)"}
 
 
 # ----------------------------------------------------------------------------- peaks and the CPU oracle

@@ -3,7 +3,7 @@
 // hidden-state tensors is read exactly once, 16 bytes per lane per access, eight accesses per tensor in flight.
 //
 // One warp per token row (grid-stride); a warp adds the cosines of its rows in row order into a double, the block
-// adds its warps in warp order, and a second one-block kernel adds the block partials in block order: the result
+// adds its warps in warp order, and a second one-block kernel adds the block partials in a fixed tree: the result
 // does not depend on scheduling.  A row with a zero vector counts as cosine 0.
 #pragma once
 
@@ -87,12 +87,22 @@ importance_partial_kernel(const T* __restrict__ h_in, const T* __restrict__ h_ou
   }
 }
 
-__global__ void importance_final_kernel(const double* __restrict__ partial, int n_blocks, long long n_tokens,
-                                        float* __restrict__ out) {
-  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+// One block: thread t adds partial[t], partial[t + 256], ... in that order, the warp adds its lanes through a fixed
+// shuffle tree, thread 0 adds the warps in warp order.
+__global__ void __launch_bounds__(kImpThreads)
+importance_final_kernel(const double* __restrict__ partial, int n_blocks, long long n_tokens, float* __restrict__ out) {
+  __shared__ double warp_sum_s[kImpThreads / 32];
   double s = 0.0;
-  for (int b = 0; b < n_blocks; ++b) s += partial[b];
-  *out = n_tokens > 0 ? (float)(1.0 - s / (double)n_tokens) : 0.f;
+  for (int b = threadIdx.x; b < n_blocks; b += kImpThreads) s += partial[b];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if ((threadIdx.x & 31) == 0) warp_sum_s[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int w = 0; w < kImpThreads / 32; ++w) t += warp_sum_s[w];
+    *out = n_tokens > 0 ? (float)(1.0 - t / (double)n_tokens) : 0.f;
+  }
 }
 
 }  // namespace mkv

@@ -325,7 +325,7 @@ int maskkv_layer_importance(maskkv_ctx* ctx, int32_t dtype, const void* h_in_dev
     mkv::importance_partial_kernel<__nv_bfloat16><<<(unsigned)blocks, mkv::kImpThreads, 0, st>>>(
         static_cast<const __nv_bfloat16*>(h_in_dev), static_cast<const __nv_bfloat16*>(h_out_dev), n_tokens, hidden, in_row_stride,
         out_row_stride, partial);
-  mkv::importance_final_kernel<<<1, 32, 0, st>>>(partial, (int)blocks, n_tokens, importance_out_dev);
+  mkv::importance_final_kernel<<<1, mkv::kImpThreads, 0, st>>>(partial, (int)blocks, n_tokens, importance_out_dev);
   return launch_status(ctx, 2);
 }
 
