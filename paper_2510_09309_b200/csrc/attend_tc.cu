@@ -130,14 +130,8 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + S::kMiscOff);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base + S::kMiscOff + 4);
 
-  const int qt = blockIdx.x, h = blockIdx.y, r = blockIdx.z, hk = h / sh.g;
-  const int l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
-  const int q0 = qt * kATile;
-  if (q0 >= M) return;
-  const int seg = r * sh.Hkv + hk;
-  const int c0 = offsets[seg], nc = offsets[seg + 1] - c0;
-  const int nt = (nc + kATile - 1) / kATile + (M + kATile - 1) / kATile;
-
+  // Set-up that touches no global memory runs before the wait for the previous kernel of the stream.
+  pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     mbar_init(bars.qfull, 1);
@@ -154,6 +148,19 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();
+
+  const int qt = blockIdx.x, h = blockIdx.y, r = blockIdx.z, hk = h / sh.g;
+  const int l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
+  const int q0 = qt * kATile;
+  if (q0 >= M) {                                           // uniform over the block: nothing to do for this tile
+    if (warp == 1) tmem_dealloc(tmem_base, 512);
+    return;
+  }
+  const int seg = r * sh.Hkv + hk;
+  const int c0 = offsets[seg], nc = offsets[seg + 1] - c0;
+  const int nt = (nc + kATile - 1) / kATile + (M + kATile - 1) / kATile;
+
   const uint32_t tm_s = tmem_base, tm_o = tmem_base + 256;   // S/P buffers at columns 0 / 128, PV buffers at 256 / 384
 
   if (warp == 0) {
@@ -416,12 +423,12 @@ int launch_attend_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const void
   dim3 grid((sh.maxM + kATile - 1) / kATile, sh.H, sh.R);
   if (sh.d == 128) {
     if (set_attend_attr<128>() != cudaSuccess) return 1;
-    attend_tc<128><<<grid, AWgs<128>::kThreads, ASmem<128>::kDynamic, st>>>(mq, mkl, mvl, mkc, mvc, sh, offsets, (__nv_bfloat16*)out, lse,
-                                                                  ctx->status_dev);
+    launch_overlapped(attend_tc<128>, grid, dim3(AWgs<128>::kThreads), ASmem<128>::kDynamic, st, mq, mkl, mvl, mkc, mvc, sh, offsets,
+                      (__nv_bfloat16*)out, lse, ctx->status_dev);
   } else {
     if (set_attend_attr<64>() != cudaSuccess) return 1;
-    attend_tc<64><<<grid, AWgs<64>::kThreads, ASmem<64>::kDynamic, st>>>(mq, mkl, mvl, mkc, mvc, sh, offsets, (__nv_bfloat16*)out, lse,
-                                                                ctx->status_dev);
+    launch_overlapped(attend_tc<64>, grid, dim3(AWgs<64>::kThreads), ASmem<64>::kDynamic, st, mq, mkl, mvl, mkc, mvc, sh, offsets,
+                      (__nv_bfloat16*)out, lse, ctx->status_dev);
   }
   return 0;
 }

@@ -30,6 +30,8 @@ budget_kernel(Shape sh, int k_l, const int32_t* __restrict__ k_l_req, double alp
   int* kbuf = reinterpret_cast<int*>(T + sh.R);
   __shared__ long long warp_tot[kBudgetThreads / 32];
   const int tid = threadIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
 
   // the divisions are the slow part (double precision): all of them in parallel, then the sums in fixed order
   for (int s = tid; s < S; s += kBudgetThreads) P[s] = prompt_preference(mass_p[s], mass_m[s]);

@@ -5,6 +5,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
 
 #include "maskkv.h"
 
@@ -31,6 +32,31 @@ struct Shape {
 };
 
 namespace mkv {
+
+// Programmatic dependent launch.  Every kernel of the layer path is launched with launch_overlapped(): its blocks may
+// be scheduled while the previous kernel of the stream is still running, which hides the launch latency and the
+// block's own set-up.  A kernel first lets its own successor go (pdl_launch_dependents), does whatever touches no
+// global memory, then calls pdl_wait(), which returns once the previous kernel has completed and its writes are
+// visible; every thread calls it before its first global access, so completion is transitive along the stream.
+// Both are no-ops in a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  static const int serial = [] { const char* e = getenv("MASKKV_SERIAL_LAUNCH"); return e != nullptr && e[0] == '1'; }();
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = serial ? 0 : 1;   // MASKKV_SERIAL_LAUNCH=1: ordinary stream order
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }

@@ -29,6 +29,8 @@ compact_kernel(Shape sh, int row_bytes, long long ts_bytes, long long hs_bytes, 
   __shared__ int32_t pcu_s[kCompactSmemSegments + 1];
   const int S = sh.R * sh.Hkv;
   const bool staged = S <= kCompactSmemSegments;        // the search below then runs out of shared memory
+  pdl_launch_dependents();
+  pdl_wait();
   if (staged) {
     for (int e = threadIdx.x; e <= S; e += kCompactThreads) off_s[e] = offsets[e];
     for (int e = threadIdx.x; e <= sh.R; e += kCompactThreads) pcu_s[e] = sh.prompt_cu[e];

@@ -388,9 +388,9 @@ int maskkv_budget(maskkv_ctx* ctx, const maskkv_desc_t* desc, int32_t k_l, const
   if (S > mkv::kBudgetMaxSegments) return MASKKV_E_UNSUPPORTED;
   DeviceGuard guard(ctx->device);
   const size_t smem = sizeof(double) * (S + sh.R) + sizeof(int) * S;
-  mkv::budget_kernel<<<1, mkv::kBudgetThreads, smem, static_cast<cudaStream_t>(stream)>>>(
-      sh, k_l, k_l_per_request_dev, alpha, 1.0 - alpha, mass_p_dev, mass_m_dev, (long long)capacity, budgets_dev,
-      offsets_dev, ctx->status_dev);
+  mkv::launch_overlapped(mkv::budget_kernel, dim3(1), dim3(mkv::kBudgetThreads), smem, static_cast<cudaStream_t>(stream),
+                         sh, k_l, k_l_per_request_dev, alpha, 1.0 - alpha, mass_p_dev, mass_m_dev, (long long)capacity, budgets_dev,
+                         offsets_dev, ctx->status_dev);
   return launch_status(ctx, 1);
 }
 
@@ -405,8 +405,9 @@ int maskkv_select(maskkv_ctx* ctx, const maskkv_desc_t* desc, const float* score
   if (scores_dev == nullptr || budgets_dev == nullptr || offsets_dev == nullptr || kept_idx_dev == nullptr) return MASKKV_E_INVALID;
   DeviceGuard guard(ctx->device);
   if (sh.maxN <= mkv::kSelectRegKeys) {                  // every segment fits the register-resident kernel
-    mkv::select_kernel_reg<<<sh.R * sh.Hkv * mkv::kSelectCluster, mkv::kSelectRegThreads, (size_t)mkv::kSelectRegKeys * 4, static_cast<cudaStream_t>(stream)>>>(
-        sh, scores_dev, budgets_dev, offsets_dev, kept_idx_dev, ctx->status_dev);
+    mkv::launch_overlapped(mkv::select_kernel_reg, dim3(sh.R * sh.Hkv * mkv::kSelectCluster), dim3(mkv::kSelectRegThreads),
+                           (size_t)mkv::kSelectRegKeys * 4, static_cast<cudaStream_t>(stream), sh, scores_dev, budgets_dev, offsets_dev,
+                           kept_idx_dev, ctx->status_dev);
     return launch_status(ctx, 1);
   }
   const int max_cache = (ctx->smem_optin - mkv::kSelectStaticSmem) / 4;
@@ -433,10 +434,10 @@ int maskkv_compact(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* k_pro
   long long blocks = (warps + (mkv::kCompactThreads / 32) - 1) / (mkv::kCompactThreads / 32);
   const long long max_blocks = (long long)ctx->sm_count * 8;
   if (blocks > max_blocks) blocks = max_blocks;
-  mkv::compact_kernel<<<(unsigned)blocks, mkv::kCompactThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-      sh, sh.d * es, sh.kv_ts * es, sh.kv_hs * es, static_cast<const unsigned char*>(k_prompt_dev),
-      static_cast<const unsigned char*>(v_prompt_dev), kept_idx_dev, offsets_dev, (long long)capacity,
-      static_cast<unsigned char*>(kc_dev), static_cast<unsigned char*>(vc_dev), ctx->status_dev);
+  mkv::launch_overlapped(mkv::compact_kernel, dim3((unsigned)blocks), dim3(mkv::kCompactThreads), 0, static_cast<cudaStream_t>(stream),
+                         sh, sh.d * es, sh.kv_ts * es, sh.kv_hs * es, static_cast<const unsigned char*>(k_prompt_dev),
+                         static_cast<const unsigned char*>(v_prompt_dev), kept_idx_dev, offsets_dev, (long long)capacity,
+                         static_cast<unsigned char*>(kc_dev), static_cast<unsigned char*>(vc_dev), ctx->status_dev);
   return launch_status(ctx, 1);
 }
 

@@ -220,10 +220,12 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const Bars bars = carve_bars(base, S::kBarOff);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + S::kMiscOff);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base + S::kMiscOff + 4);
-  // sweep 2 counts finished mass partials per segment in seg_cnt; it starts after this grid has ended
+  pdl_launch_dependents();
+  block_setup(bars, 4, tmem_slot, abort_flag);
+  pdl_wait();
+  // sweep 2 counts finished mass partials per segment in seg_cnt; it reads them after this grid has ended
   if (blockIdx.x == 0 && seg_cnt != nullptr)
     for (int i = threadIdx.x; i < sh.R * sh.Hkv; i += blockDim.x) seg_cnt[i] = 0u;
-  block_setup(bars, 4, tmem_slot, abort_flag);
   const uint32_t tmem_base = *tmem_slot;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   Walker wk;
@@ -309,11 +311,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const int n_qtiles = (s.M - q0 > kTile) ? 2 : 1;
       if (a >= n_qtiles) continue;
       float m = -INFINITY, l = 0.f;                         // m in raw (unscaled) logits
-      // The reference m of the running sum l = sum 2^((s - m) * cs) is only moved when a logit exceeds it by more
-      // than 2^kSlack: the exponentials of a chunk then do not wait for the chunk's maximum (which is found beside
-      // them), and l stays far inside the fp32 range (each term <= 2^kSlack, at most 2^31 terms).  (m, l) is as good a
-      // pair for the later log-sum-exp merge as (true maximum, sum) - only ln l + m * scale is ever used.
-      constexpr float kSlack = 64.f;
+      // running maximum m and l = sum 2^((s - m) * cs); a chunk's maximum is a tree of 3-input max
       auto chunk_max = [&](const float* v) {
         float t[11];
 #pragma unroll
@@ -452,7 +450,9 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   float* c2s = reinterpret_cast<float*>(base + S::kC2Off);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + S::kMiscOff);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base + S::kMiscOff + 4);
+  pdl_launch_dependents();
   block_setup(bars, 2, tmem_slot, abort_flag);
+  pdl_wait();
   const uint32_t tmem_base = *tmem_slot;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   Walker wk;
@@ -739,10 +739,12 @@ int launch_score_stats_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* promp
   const int grid = (int)(F < ctx->sm_count ? F : ctx->sm_count);
   if (sh.d == 128) {
     if (set_smem_attr<128>() != cudaSuccess) return 1;
-    score_stats_tc<128><<<grid, kThreads, Smem<128>::kDynamic, st>>>(m.q, m.kp, m.km, sh, part, C, F, seg_cnt, ctx->status_dev);
+    launch_overlapped(score_stats_tc<128>, dim3(grid), dim3(kThreads), Smem<128>::kDynamic, st, m.q, m.kp, m.km, sh, part, C, F, seg_cnt,
+                      ctx->status_dev);
   } else {
     if (set_smem_attr<64>() != cudaSuccess) return 1;
-    score_stats_tc<64><<<grid, kThreads, Smem<64>::kDynamic, st>>>(m.q, m.kp, m.km, sh, part, C, F, seg_cnt, ctx->status_dev);
+    launch_overlapped(score_stats_tc<64>, dim3(grid), dim3(kThreads), Smem<64>::kDynamic, st, m.q, m.kp, m.km, sh, part, C, F, seg_cnt,
+                      ctx->status_dev);
   }
   return 0;
 }
@@ -772,11 +774,11 @@ int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prom
     score_zero_fill<<<gz, kTile, 0, st>>>(sh, scores, mass_p, mass_m);
   }
   if (sh.d == 128)
-    score_colsum_tc<128><<<grid, kThreads, Smem<128>::kDynamic, st>>>(m.q, m.kp, m.km, sh, lse, part, C, F1, G1, w, scores, mass_part,
-                                                                      Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
+    launch_overlapped(score_colsum_tc<128>, dim3(grid), dim3(kThreads), Smem<128>::kDynamic, st, m.q, m.kp, m.km, sh, lse, part, C, F1, G1,
+                      w, scores, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
   else
-    score_colsum_tc<64><<<grid, kThreads, Smem<64>::kDynamic, st>>>(m.q, m.kp, m.km, sh, lse, part, C, F1, G1, w, scores, mass_part,
-                                                                     Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
+    launch_overlapped(score_colsum_tc<64>, dim3(grid), dim3(kThreads), Smem<64>::kDynamic, st, m.q, m.kp, m.km, sh, lse, part, C, F1, G1,
+                      w, scores, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
   return 0;
 }
 

@@ -116,6 +116,8 @@ select_kernel_reg(Shape sh, const float* __restrict__ scores, const int32_t* __r
   const int s = blockIdx.x / kSelectCluster;
   const int q = (int)cluster.block_rank();
   const int r = s / sh.Hkv, hk = s % sh.Hkv;
+  pdl_launch_dependents();
+  pdl_wait();
   const int p0 = sh.prompt_cu[r], N = sh.prompt_cu[r + 1] - p0;
   const int out0 = offsets[s];
   int k = budgets[s];
