@@ -156,7 +156,7 @@ int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_
  * The scratch is instead a fixed array of maskkv_score_noalloc_max_bytes() = 8 MiB that is part of the
  * library image: each GPU that loads the library reserves those bytes until the process exits, used or not.
  * The call allocates nothing and frees nothing.  If maskkv_workspace_bytes(desc) exceeds the array the call
- * returns MASKKV_E_WORKSPACE and launches nothing (8 MiB covers a single request of up to about 60k prompt
+ * returns MASKKV_E_WORKSPACE and launches nothing (8 MiB covers a single request of up to about 57,000 prompt
  * keys at 32 heads x 256 mask rows; batches need the regular call).
  *
  * The first call on each device looks up the array's device address (a one-time, host-side set-up step);

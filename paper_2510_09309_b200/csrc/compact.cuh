@@ -1,7 +1,7 @@
-// Gather of the kept K/V rows into the ragged per-head cache: a pure byte copy, one warp per kept
-// row, 16 bytes per lane per access (K row on the lower half-warp, V row on the upper one when a row
-// is 256 bytes).  Bound by HBM; the source rows are scattered 256-byte pieces, the destination is
-// contiguous.
+// Gather of the kept K/V rows into the ragged per-head cache: a pure byte copy, two consecutive kept
+// rows per warp and step, 16 bytes per lane per access (K row on the lower half-warp, V row on the
+// upper one when a row is 256 bytes).  Bound by HBM; the source rows are scattered 256-byte pieces
+// (one DRAM row each), the destination is contiguous.
 #pragma once
 
 #include "common.cuh"
@@ -9,6 +9,7 @@
 namespace mkv {
 
 constexpr int kCompactThreads = 256;
+constexpr int kCompactBlocksPerSm = 8;                 // grid cap: about what is resident at once; the blocks loop
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   uint4 v;
@@ -17,9 +18,12 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   return v;
 }
 
+constexpr int kCompactRows = 2;                         // output rows a warp moves per step
 constexpr int kCompactSmemSegments = 2048;             // offsets[] is staged in shared memory up to this many segments
 
 // row_bytes = d * sizeof(T); strides in bytes.  grid-stride over the rows in use (offsets[S], read on the device).
+// PP = 16-byte pieces per lane per row (K row + V row): 1 up to 256-byte rows, 2 for 512-byte rows.
+template <int PP>
 __global__ void __launch_bounds__(kCompactThreads)
 compact_kernel(Shape sh, int row_bytes, long long ts_bytes, long long hs_bytes, const unsigned char* __restrict__ kp,
                const unsigned char* __restrict__ vp, const int32_t* __restrict__ kept_idx,
@@ -44,23 +48,50 @@ compact_kernel(Shape sh, int row_bytes, long long ts_bytes, long long hs_bytes, 
   const int warps_per_block = kCompactThreads / 32;
   const int vec_per_row = row_bytes / 16;               // 16-byte pieces per row (8, 16 or 32)
   const int pieces = 2 * vec_per_row;                   // K row then V row
-  for (long long t = (long long)blockIdx.x * warps_per_block + (threadIdx.x >> 5); t < total;
-       t += (long long)gridDim.x * warps_per_block) {
-    const int s = find_request(off, S, (int)t);         // segment that owns output row t
-    const int r = s / sh.Hkv, hk = s % sh.Hkv;
-    const int p0 = pcu[r], N = pcu[r + 1] - p0;
-    const int j = kept_idx[t];
-    if (j < 0 || j >= N) {                              // never dereference a bad index
-      if (lane == 0) atomicOr(status, (uint32_t)MASKKV_FLAG_BOUNDS);
-      continue;
+  // kCompactRows consecutive output rows per warp and step: their index loads go out together, then all their row
+  // pieces, then the stores - three dependent round trips per step instead of per row.
+  const long long warp_id = (long long)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+  const long long warps_total = (long long)gridDim.x * warps_per_block;
+  for (long long t0 = warp_id * kCompactRows; t0 < total; t0 += warps_total * kCompactRows) {
+    int j[kCompactRows];
+#pragma unroll
+    for (int u = 0; u < kCompactRows; ++u) j[u] = t0 + u < total ? __ldg(kept_idx + t0 + u) : -1;
+    long long src[kCompactRows];
+#pragma unroll
+    for (int u = 0; u < kCompactRows; ++u) {
+      src[u] = -1;
+      if (t0 + u >= total) continue;
+      const int s = find_request(off, S, (int)(t0 + u));  // segment that owns output row t0 + u
+      const int r = s / sh.Hkv, hk = s % sh.Hkv;
+      const int p0 = pcu[r], N = pcu[r + 1] - p0;
+      if (j[u] < 0 || j[u] >= N) {                        // never dereference a bad index
+        if (lane == 0) atomicOr(status, (uint32_t)MASKKV_FLAG_BOUNDS);
+        continue;
+      }
+      src[u] = (long long)(p0 + j[u]) * ts_bytes + (long long)hk * hs_bytes;
     }
-    const long long src = (long long)(p0 + j) * ts_bytes + (long long)hk * hs_bytes;
-    const long long dst = t * row_bytes;
-    for (int e = lane; e < pieces; e += 32) {
-      const bool is_v = e >= vec_per_row;
-      const int o16 = (is_v ? e - vec_per_row : e) * 16;
-      const uint4 v = ld_stream(reinterpret_cast<const uint4*>((is_v ? vp : kp) + src + o16));
-      *reinterpret_cast<uint4*>((is_v ? vc : kc) + dst + o16) = v;
+    uint4 v[kCompactRows][PP];
+#pragma unroll
+    for (int u = 0; u < kCompactRows; ++u) {
+#pragma unroll
+      for (int c = 0; c < PP; ++c) {
+        const int e = lane + 32 * c;
+        if (src[u] < 0 || e >= pieces) continue;
+        const bool is_v = e >= vec_per_row;
+        const int o16 = (is_v ? e - vec_per_row : e) * 16;
+        v[u][c] = ld_stream(reinterpret_cast<const uint4*>((is_v ? vp : kp) + src[u] + o16));
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kCompactRows; ++u) {
+#pragma unroll
+      for (int c = 0; c < PP; ++c) {
+        const int e = lane + 32 * c;
+        if (src[u] < 0 || e >= pieces) continue;
+        const bool is_v = e >= vec_per_row;
+        const int o16 = (is_v ? e - vec_per_row : e) * 16;
+        *reinterpret_cast<uint4*>((is_v ? vc : kc) + (t0 + u) * row_bytes + o16) = v[u][c];
+      }
     }
   }
 }

@@ -430,11 +430,12 @@ int maskkv_compact(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* k_pro
   if (!aligned16(k_prompt_dev) || !aligned16(v_prompt_dev) || !aligned16(kc_dev) || !aligned16(vc_dev)) return MASKKV_E_ALIGN;
   DeviceGuard guard(ctx->device);
   const int es = elem_size(sh.dtype);
-  const long long warps = capacity;
+  const long long warps = (capacity + mkv::kCompactRows - 1) / mkv::kCompactRows;
   long long blocks = (warps + (mkv::kCompactThreads / 32) - 1) / (mkv::kCompactThreads / 32);
-  const long long max_blocks = (long long)ctx->sm_count * 8;
+  const long long max_blocks = (long long)ctx->sm_count * mkv::kCompactBlocksPerSm;
   if (blocks > max_blocks) blocks = max_blocks;
-  mkv::launch_overlapped(mkv::compact_kernel, dim3((unsigned)blocks), dim3(mkv::kCompactThreads), 0, static_cast<cudaStream_t>(stream),
+  auto kernel = 2 * sh.d * es / 16 <= 32 ? mkv::compact_kernel<1> : mkv::compact_kernel<2>;
+  mkv::launch_overlapped(kernel, dim3((unsigned)blocks), dim3(mkv::kCompactThreads), 0, static_cast<cudaStream_t>(stream),
                          sh, sh.d * es, sh.kv_ts * es, sh.kv_hs * es, static_cast<const unsigned char*>(k_prompt_dev),
                          static_cast<const unsigned char*>(v_prompt_dev), kept_idx_dev, offsets_dev, (long long)capacity,
                          static_cast<unsigned char*>(kc_dev), static_cast<unsigned char*>(vc_dev), ctx->status_dev);

@@ -281,6 +281,7 @@ select_kernel_reg(Shape sh, const float* __restrict__ scores, const int32_t* __r
       eq_before += e2;
     }
   }
+  cluster.barrier_arrive();                              // done reading the peers' shared memory (waited for at the end)
   // rows of this warp that hold a key at or above the threshold, lowest row first
   uint32_t rows = __reduce_or_sync(0xffffffffu, gt_mask | eq_mask);
   const uint32_t lt_mask = (1u << lane) - 1u;
@@ -295,7 +296,7 @@ select_kernel_reg(Shape sh, const float* __restrict__ scores, const int32_t* __r
     out_before += __popc(take_bal);
     eq_before += __popc(eq_bal);
   }
-  cluster.sync();                                        // no CTA leaves while a peer may still read its shared memory
+  cluster.barrier_wait();                                // no CTA leaves while a peer may still read its shared memory
 }
 
 // dynamic shared memory: uint32 keys[cache_elems] (cache_elems = 0 -> keys are re-read from global)
