@@ -11,25 +11,39 @@
 //                          shared memory, into a fresh accumulator
 //     O = O*corr + PV      in registers, d/NW output columns per thread (no rescaling pass over tensor memory)
 // S/P and PV are double-buffered (4 x 128 columns of tensor memory) so the next tile's Q K^T overlaps the
-// softmax; key and value tiles come through separate TMA rings (3 and 2 stages) and tiles beyond the rings are
-// requested into L2 ahead of time.  The kernel is a latency chain (3-8 dependent tiles per CTA), not a
-// throughput kernel: measured per tile, about 0.4 us goes to issuing the two MMA groups from one thread.  Columns of a ragged tile's tail are masked to -inf, and the matching V rows are zeroed in
-// shared memory so that stale cache rows can never leak a NaN into the product.
+// softmax; Q K^T and P V are issued by two different threads; key and value tiles come through separate TMA rings
+// (3 and 2 stages) and tiles beyond the rings are requested into L2 ahead of time.  Columns of a ragged tile's tail
+// are masked to -inf, and the matching V rows are zeroed in shared memory so that stale cache rows can never leak a
+// NaN into the product.  The output tile leaves through shared memory as whole rows.
+//
+// The kernel is a latency chain (3-8 dependent tiles per CTA), not a throughput kernel.  Cycle stamps of one CTA:
+// 2.6k cycles until the tile loop starts (set-up, wait for the previous kernel, segment offsets), 2.9k more until the
+// first S is ready (tensor maps, Q and K from L2, first MMA group), then about 2.6k per tile - 0.35k reading S and
+// finding the row maximum, 1.4k for the exchange of the maximum, the 128 x 128 exponentials (1,024 cycles of the
+// special-function unit by themselves), packing and the store of P, 0.45k adding the previous tile's P V - and 1-3k
+// to normalise and store.  When units are few and their key segments long, a cluster of two CTAs shares a unit: each
+// walks half of the tiles and CTA 1 hands its (max, sum, output) to CTA 0 through distributed shared memory; that
+// merge costs about three tiles' time, so it is used from eight tiles per unit on.
 #include "attend_tc.h"
+
+#include <cooperative_groups.h>
 
 #include "tc_common.cuh"
 
 namespace mkv {
 namespace tc {
 
-// warp 0: TMA, warp 1: MMA, then NW softmax warpgroups (thread = one query row, 128/NW key columns, d/NW output columns)
+// warp 0: TMA, warp 1: issues Q K^T, then NW softmax warpgroups (thread = one query row, 128/NW key columns, d/NW output
+// columns), last warp: issues P V.  Two issuing threads, because issuing a group of eight MMAs costs one thread
+// about 0.2 us and the two groups of a tile would otherwise queue behind each other.
 #ifndef MKV_ATTEND_NW
 #define MKV_ATTEND_NW 2
 #endif
-template <int D> struct AWgs { static constexpr int kNW = MKV_ATTEND_NW; static constexpr int kThreads = 64 + 128 * kNW; };
+template <int D> struct AWgs { static constexpr int kNW = MKV_ATTEND_NW; static constexpr int kThreads = 96 + 128 * kNW; static constexpr int kPvWarp = 2 + 4 * kNW; };
 constexpr int kATile = 128;
 constexpr int kAKStages = 3;            // key tiles in flight (the next Q K^T is issued a tile ahead)
 constexpr int kAVStages = 2;            // value tiles in flight
+constexpr int kASplitMinTiles = 8;      // key tiles per unit from which two CTAs share a unit
 constexpr float kALog2e = 1.4426950408889634f;
 
 template <int D>
@@ -84,6 +98,11 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* u) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// Cluster-wide barrier, every thread of every CTA of the cluster once per phase (no convergence requirement);
+// release / acquire order the distributed-shared-memory stores made before it against the loads after it.
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -150,7 +169,11 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   const uint32_t tmem_base = *tmem_slot;
   pdl_wait();
 
-  const int qt = blockIdx.x, h = blockIdx.y, r = blockIdx.z, hk = h / sh.g;
+  // A cluster of `nsplit` CTAs (1 or 2) shares one (query tile, head): CTA `part` walks its contiguous share of
+  // the key tiles; the partial (max, sum, output) of CTA 1 is merged into CTA 0's through distributed shared memory.
+  cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
+  const int nsplit = (int)cluster.num_blocks(), part = (int)cluster.block_rank();
+  const int qt = blockIdx.x / nsplit, h = blockIdx.y, r = blockIdx.z, hk = h / sh.g;
   const int l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
   const int q0 = qt * kATile;
   if (q0 >= M) {                                           // uniform over the block: nothing to do for this tile
@@ -159,7 +182,10 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   }
   const int seg = r * sh.Hkv + hk;
   const int c0 = offsets[seg], nc = offsets[seg + 1] - c0;
-  const int nt = (nc + kATile - 1) / kATile + (M + kATile - 1) / kATile;
+  const int nt_all = (nc + kATile - 1) / kATile + (M + kATile - 1) / kATile;
+  const int per_part = (nt_all + nsplit - 1) / nsplit;
+  const int j_first = part * per_part;                     // this CTA walks tiles [j_first, j_first + nt)
+  const int nt = max(0, min(per_part, nt_all - j_first));
 
   const uint32_t tm_s = tmem_base, tm_o = tmem_base + 256;   // S/P buffers at columns 0 / 128, PV buffers at 256 / 384
 
@@ -178,7 +204,7 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         if (jk < nt) {
           const int stage = jk % kAKStages, use = jk / kAKStages;
           if (mbar_try_wait(bars.kempty + stage, (use & 1) ^ 1)) {
-            const ATile t = a_tile(jk, c0, nc, l0, M);
+            const ATile t = a_tile(j_first + jk, c0, nc, l0, M);
             mbar_expect_tx(bars.kfull + stage, S::kTileBytes);
             for (int b = 0; b < S::kBoxes; ++b)
               tma_load_3d(base + S::kKOff + stage * S::kTileBytes + b * S::kBoxBytes, t.cache ? &map_kc : &map_kl,
@@ -190,7 +216,7 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         if (jv < nt) {
           const int stage = jv % kAVStages, use = jv / kAVStages;
           if (mbar_try_wait(bars.vempty + stage, (use & 1) ^ 1)) {
-            const ATile t = a_tile(jv, c0, nc, l0, M);
+            const ATile t = a_tile(j_first + jv, c0, nc, l0, M);
             mbar_expect_tx(bars.vfull + stage, S::kTileBytes);
             for (int b = 0; b < S::kBoxes; ++b)
               tma_load_3d(base + S::kVOff + stage * S::kTileBytes + b * S::kBoxBytes, t.cache ? &map_vc : &map_vl,
@@ -202,7 +228,7 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         if (!prefetched && jk >= min(nt, kAKStages) && jv >= min(nt, kAVStages)) {
           // the rings are full: ask for the later tiles to be brought into L2, so that their ring loads pay L2 latency only
           for (int j = kAVStages; j < nt; ++j) {
-            const ATile t = a_tile(j, c0, nc, l0, M);
+            const ATile t = a_tile(j_first + j, c0, nc, l0, M);
             for (int b = 0; b < S::kBoxes; ++b) {
               if (j >= kAKStages) tma_prefetch_l2_3d(t.cache ? &map_kc : &map_kl, b * 64, t.cache ? 0 : hk, t.row);
               tma_prefetch_l2_3d(t.cache ? &map_vc : &map_vl, b * 64, t.cache ? 0 : hk, t.row);
@@ -225,16 +251,18 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
           for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(bars.vfull + i % kAVStages, (i / kAVStages) & 1); ++it) __nanosleep(64);
       }
     }
+    if (nsplit > 1) { cluster_barrier(); cluster_barrier(); }   // the two phases of the merge below
   } else if (warp == 1) {
     if (lane == 0) {
       const uint32_t idesc_qk = idesc_bf16_f32(kATile, kATile);
-      const uint32_t idesc_pv = idesc_bf16_f32_bn(kATile, D);
       const uint32_t q_lo = smem_desc_lo(smem_u32(base + S::kQOff));
       bool ok = mbar_wait(bars.qfull, 0, abort_flag, status, 0x303);
       tc_fence_after();
-      auto issue_qk = [&](int j) -> bool {
+      for (int j = 0; ok && j < nt; ++j) {
         const int stage = j % kAKStages, use = j / kAKStages;
-        if (!mbar_wait(bars.kfull + stage, use & 1, abort_flag, status, 0x304)) return false;
+        if (!(ok = mbar_wait(bars.kfull + stage, use & 1, abort_flag, status, 0x304))) break;
+        // S/P buffer j & 1 is free once P V of tile j - 2 has read P from it
+        if (j >= 2 && !(ok = mbar_wait(bars.ofull + (j & 1), ((j - 2) >> 1) & 1, abort_flag, status, 0x30b))) break;
         tc_fence_after();
         const uint32_t k_lo = smem_desc_lo(smem_u32(base + S::kKOff + stage * S::kTileBytes));
 #pragma unroll
@@ -244,11 +272,14 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         }
         umma_commit(bars.sfull + (j & 1));
         umma_commit(bars.kempty + stage);
-        return true;
-      };
-      if (ok) ok = issue_qk(0);
+      }
+    }
+    if (nsplit > 1) { cluster_barrier(); cluster_barrier(); }
+  } else if (warp == AWgs<D>::kPvWarp) {
+    if (lane == 0) {
+      const uint32_t idesc_pv = idesc_bf16_f32_bn(kATile, D);
+      bool ok = true;
       for (int j = 0; ok && j < nt; ++j) {
-        if (j + 1 < nt && !(ok = issue_qk(j + 1))) break;
         const int b = j & 1, stage = j % kAVStages, use = j / kAVStages;
         if (!(ok = mbar_wait(bars.vfull + stage, use & 1, abort_flag, status, 0x305))) break;
         if (!(ok = mbar_wait(bars.oempty + b, ((j >> 1) & 1) ^ 1, abort_flag, status, 0x306))) break;
@@ -265,6 +296,7 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         umma_commit(bars.vempty + stage);
       }
     }
+    if (nsplit > 1) { cluster_barrier(); cluster_barrier(); }
   } else {
     // NW softmax warpgroups share every tile: thread (wg, row) owns S columns [SC wg, SC wg + SC) of its query row
     // (SC = 128 / NW) and the output columns [32 wg, 32 wg + 32).  The row maximum is the only thing they exchange per
@@ -306,7 +338,7 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     // After a failed wait a thread skips the tensor-memory work but still reaches every named barrier.
     for (int j = 0; j < nt; ++j) {
       const int b = j & 1;
-      const ATile t = a_tile(j, c0, nc, l0, M);
+      const ATile t = a_tile(j_first + j, c0, nc, l0, M);
       const int my_valid = min(SC, max(0, t.valid - wg * SC));   // valid columns among this thread's SC
       if (ok && t.valid < kATile) {
         // ragged tail: zero the value rows that do not belong to this tile (every thread clears a slice)
@@ -371,10 +403,45 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     l = 0.f;
 #pragma unroll
     for (int w2 = 0; w2 < NW; ++w2) l += lx[w2 * kATile + row];
+    if (nsplit > 1) {
+      // Exchange area in CTA 0: its key ring, free once both CTAs have finished their tiles (first barrier).
+      // xo4[column group of 4][row] as float4 (a warp's 32 rows of a group are 512 contiguous bytes, for the remote
+      // stores as for the loads), then xm[row], xl[row].
+      float4* xo4 = reinterpret_cast<float4*>(base + S::kKOff);
+      float* xm = reinterpret_cast<float*>(xo4 + (D / 4) * kATile);
+      float* xl = xm + kATile;
+      cluster_barrier();
+      if (part == 1) {
+        float4* ro = cluster.map_shared_rank(xo4, 0) + (wg * OC / 4) * kATile + row;
+#pragma unroll
+        for (int c = 0; c < OC; c += 4) ro[(c / 4) * kATile] = make_float4(o[c], o[c + 1], o[c + 2], o[c + 3]);
+        if (wg == 0) { cluster.map_shared_rank(xm, 0)[row] = m; cluster.map_shared_rank(xl, 0)[row] = l; }
+      }
+      cluster_barrier();
+      if (part == 0) {
+        const float m1 = xm[row], l1 = xl[row];
+        const float m_all = fmaxf(m, m1);
+        const float a0 = ex2((m - m_all) * cs), a1 = ex2((m1 - m_all) * cs);   // an empty share has m1 = -inf: a1 = 0
+        l = l * a0 + l1 * a1;
+        const float4* po = xo4 + (wg * OC / 4) * kATile + row;
+#pragma unroll
+        for (int c = 0; c < OC; c += 4) {
+          const float4 v4 = po[(c / 4) * kATile];
+          o[c] = o[c] * a0 + v4.x * a1; o[c + 1] = o[c + 1] * a0 + v4.y * a1;
+          o[c + 2] = o[c + 2] * a0 + v4.z * a1; o[c + 3] = o[c + 3] * a0 + v4.w * a1;
+        }
+        m = m_all;
+      }
+    }
+    // Output: a thread holds D/NW columns of one row, which would make every store instruction touch 32 rows.  The
+    // tile goes through shared memory instead (the value ring, free now; rows padded by 16 bytes against bank
+    // conflicts) and leaves as whole 2*D-byte rows, 16 bytes per lane.
     const int i = q0 + row;
-    if (ok && !*abort_flag && i < M) {
+    uint8_t* stage_o = base + S::kVOff;
+    constexpr int RS = D * 2 + 16;
+    if (ok && part == 0) {
       const float inv = 1.f / l;
-      __nv_bfloat16* dst = out + (long long)(l0 + i) * sh.q_ts + (long long)h * sh.q_hs + wg * OC;
+      uint4* dst = reinterpret_cast<uint4*>(stage_o + row * RS + wg * OC * 2);
 #pragma unroll
       for (int c = 0; c < OC; c += 8) {
         uint4 w;
@@ -382,9 +449,20 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         w.y = pack_bf16(o[c + 2] * inv, o[c + 3] * inv);
         w.z = pack_bf16(o[c + 4] * inv, o[c + 5] * inv);
         w.w = pack_bf16(o[c + 6] * inv, o[c + 7] * inv);
-        *reinterpret_cast<uint4*>(dst + c) = w;
+        dst[c / 8] = w;
       }
-      if (wg == 0 && lse != nullptr) lse[(long long)h * sh.sumM + l0 + i] = m * sh.scale + logf(l);
+      if (wg == 0 && lse != nullptr && i < M && !*abort_flag) lse[(long long)h * sh.sumM + l0 + i] = m * sh.scale + logf(l);
+    }
+    named_barrier(1, NW * kATile);
+    if (part == 0 && !*abort_flag) {
+      constexpr int PPR = D * 2 / 16;                        // 16-byte pieces per row
+      const int pieces = min(kATile, M - q0) * PPR;
+      uint8_t* out_tile = reinterpret_cast<uint8_t*>(out + (long long)(l0 + q0) * sh.q_ts + (long long)h * sh.q_hs);
+      for (int e = tid_all; e < pieces; e += NW * kATile) {
+        const int rr = e / PPR, pc = e % PPR;
+        *reinterpret_cast<uint4*>(out_tile + (long long)rr * sh.q_ts * 2 + pc * 16) =
+            *reinterpret_cast<const uint4*>(stage_o + rr * RS + pc * 16);
+      }
     }
   }
   tc_fence_before();
@@ -420,16 +498,26 @@ int launch_attend_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const void
                   make_tmap_rows(ctx->encode_tiled, &mkc, kc_base, sh.d, 1, rows, (uint64_t)sh.d * 2, (uint64_t)sh.d * 2, kATile) &&
                   make_tmap_rows(ctx->encode_tiled, &mvc, vc_base, sh.d, 1, rows, (uint64_t)sh.d * 2, (uint64_t)sh.d * 2, kATile);
   if (!ok) return 1;
-  dim3 grid((sh.maxM + kATile - 1) / kATile, sh.H, sh.R);
+  // Few (query tile, head, request) units leave most SMs idle and every CTA with a long chain of dependent tiles:
+  // then two CTAs share a unit (cluster of 2 along x).  The merge costs about as much as three tiles (64 KB through
+  // distributed shared memory), so the split only pays for long chains - eight tiles or more at the mean segment
+  // length the capacity allows; with enough units it only adds set-up cost.
+  const unsigned q_tiles = (unsigned)((sh.maxM + kATile - 1) / kATile);
+  const long long units = (long long)q_tiles * sh.H * sh.R;
+  const long long mean_rows = cache_rows / ((long long)sh.R * sh.Hkv);
+  const long long chain = (mean_rows + kATile - 1) / kATile + q_tiles;
+  const unsigned nsplit = (2 * units <= ctx->sm_count && chain >= kASplitMinTiles) ? 2u : 1u;
+  dim3 grid(q_tiles * nsplit, sh.H, sh.R);
   if (sh.d == 128) {
     if (set_attend_attr<128>() != cudaSuccess) return 1;
-    launch_overlapped(attend_tc<128>, grid, dim3(AWgs<128>::kThreads), ASmem<128>::kDynamic, st, mq, mkl, mvl, mkc, mvc, sh, offsets,
-                      (__nv_bfloat16*)out, lse, ctx->status_dev);
+    (void)launch_overlapped_cluster(attend_tc<128>, grid, dim3(AWgs<128>::kThreads), ASmem<128>::kDynamic, st, nsplit, mq, mkl, mvl, mkc, mvc,
+                                  sh, offsets, (__nv_bfloat16*)out, lse, ctx->status_dev);
   } else {
     if (set_attend_attr<64>() != cudaSuccess) return 1;
-    launch_overlapped(attend_tc<64>, grid, dim3(AWgs<64>::kThreads), ASmem<64>::kDynamic, st, mq, mkl, mvl, mkc, mvc, sh, offsets,
-                      (__nv_bfloat16*)out, lse, ctx->status_dev);
+    (void)launch_overlapped_cluster(attend_tc<64>, grid, dim3(AWgs<64>::kThreads), ASmem<64>::kDynamic, st, nsplit, mq, mkl, mvl, mkc, mvc,
+                                  sh, offsets, (__nv_bfloat16*)out, lse, ctx->status_dev);
   }
+  // a failed launch is reported by the caller through cudaGetLastError
   return 0;
 }
 

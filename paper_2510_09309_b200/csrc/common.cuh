@@ -42,20 +42,33 @@ namespace mkv {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// cluster_x > 1: thread-block clusters of that many CTAs along x (grid.x must be a multiple of it).
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+inline cudaError_t launch_overlapped_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                             unsigned cluster_x, Args&&... args) {
+  static const int serial = [] { const char* e = getenv("MASKKV_SERIAL_LAUNCH"); return e != nullptr && e[0] == '1'; }();
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  static const int serial = [] { const char* e = getenv("MASKKV_SERIAL_LAUNCH"); return e != nullptr && e[0] == '1'; }();
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = serial ? 0 : 1;   // MASKKV_SERIAL_LAUNCH=1: ordinary stream order
-  cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (cluster_x > 1) {
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = cluster_x;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+  }
+  cfg.attrs = attr;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  return launch_overlapped_cluster(kernel, grid, block, smem, st, 1u, static_cast<Args&&>(args)...);
 }
 
 __device__ __forceinline__ float to_f32(float x) { return x; }

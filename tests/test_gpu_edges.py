@@ -160,3 +160,28 @@ def test_validation_launches_nothing(ctx):
     assert B.lib.maskkv_attend(None, ctypes.byref(p.desc), *([f.data_ptr()] * 6), 16, f.data_ptr(), f.data_ptr(), None) == B.MASKKV_E_INVALID
     torch.cuda.synchronize()
     assert (f == 0).all() and ctx.maskkv_check_status() == 0
+
+
+@pytest.mark.parametrize("d,n_mask", [(128, 256), (64, 130)])
+def test_attend_long_segments_shared_by_two_ctas(ctx, d, n_mask):
+    """Few (query tile, head) units with long kept segments: two CTAs of a cluster split the key tiles of a unit and
+    merge their partial softmax through distributed shared memory.  Uneven shares, ragged tails and segments of very
+    different length (one of them empty) included."""
+    wl = synth.scaled(synth.config(2), "long_segments", dtype="bf16", prompt_lens=(4096,), n_mask=n_mask, n_q_heads=4,
+                      n_kv_heads=4, head_dim=d, mean_budget=1536)
+    x = synth.layer_inputs(wl, 0, "cpu"); live = synth.live_inputs(wl, 0, 0, "cpu")
+    xd = {k: to_dev(v) for k, v in x.items() if torch.is_tensor(v)}; ld = {k: to_dev(v) for k, v in live.items()}
+    run = GpuRun(ctx, wl, capacity=4 * 1536, k_l=1536)
+    budgets = torch.tensor([[1536, 0, 2999, 1609]], dtype=torch.int32)      # 12 / 0 / 24 / 13 key tiles + the live ones
+    offsets = torch.tensor([0, 1536, 1536, 4535, 6144], dtype=torch.int32)
+    run.score(xd)
+    run.select(budgets=to_dev(budgets), offsets=to_dev(offsets)); run.compact(xd, offsets=to_dev(offsets))
+    run.attend(ld, offsets=to_dev(offsets))
+    torch.cuda.synchronize()
+    kept = run.kept.cpu().numpy(); offd = offsets.numpy()
+    kc, vc = O.compact(x["k_prompt"], x["v_prompt"], kept, offd, wl.prompt_cu())
+    assert torch.equal(run.kc.cpu(), kc)
+    out, lse = O.attend(live["q_live"], live["k_live"], live["v_live"], kc, vc, offd, wl.live_cu(), wl.n_kv_heads)
+    assert np.abs(run.out.float().cpu().numpy() - out).max() <= ATTEND_ATOL["bf16"]
+    assert np.abs(run.lse.cpu().numpy() - lse).max() <= 1e-3
+    assert ctx.maskkv_check_status() == 0
