@@ -248,6 +248,30 @@ def bench_ours(args):
     barrier()
     mean_kept = float(buf.offsets[-1].item()) / wl.n_kv_heads
     call_us = {name: 1e3 * statistics.mean(ev[c].elapsed_time(ev[c + 1]) for ev in per_call) for c, name in enumerate(CALLS)}
+    # ---- the later denoising steps: maskkv_attend alone, back to back, as the per-step loop of a layer would issue it.
+    # The compacted cache is cloned until the copies exceed twice the L2, and the loop cycles through them.
+    cache_bytes = 2 * buf.kc.numel() * buf.kc.element_size()
+    n_copies = max(2, int(-(-2 * 126e6 // cache_bytes)))
+    caches = [(buf.kc.clone(), buf.vc.clone()) for _ in range(n_copies)]
+    p = buf.p
+
+    def attend_step(i):
+        kc, vc = caches[i % n_copies]
+        live = lives[i % len(lives)]
+        ctx.maskkv_attend(p, live["q_live"], live["k_live"], live["v_live"], kc, vc, buf.offsets, buf.capacity, buf.out)
+
+    for i in range(5):
+        attend_step(i)
+    barrier()
+    a_steps = min(max(args.steps, 50), 400)
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record()
+    for i in range(a_steps):
+        attend_step(i)
+    a1.record()
+    barrier()
+    attend_loop_us = 1e3 * max_over_ranks(a0.elapsed_time(a1), device) / a_steps
+    del caches
     flags = ctx.maskkv_check_status()
 
     # ---- end to end: the layer's inputs start in pinned host memory, results end in host memory
@@ -339,7 +363,9 @@ def bench_ours(args):
                                "adaptive budgets (k_l 512/238, alpha=0.1)", "layers_resident": len(resident),
                    "l2": "inputs 545 MB per step > 126 MB L2; resident layers are cycled", "calls": list(CALLS)},
         "call_us": {k: round(v, 2) for k, v in call_us.items()},
-        "attend_step_us": round(call_us["attend"], 2),
+        "attend_step_us": round(attend_loop_us, 2),
+        "attend_step": {"us": round(attend_loop_us, 2), "steps": a_steps, "mean_kept_per_head": mean_kept,
+                        "l2": f"{n_copies} copies of the compacted cache ({cache_bytes * n_copies / 1e6:.0f} MB) cycled"},
         "compress_tokens_per_s": N / (1e-6 * (call_us["score"] + call_us["budget"] + call_us["select"] + call_us["compact"])),
         "e2e": {"value": world * N / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
