@@ -110,6 +110,23 @@ def layer_importance(h_in, h_out) -> float:
     return float(1.0 - cos.sum() / a.shape[0])
 
 
+def refresh_set(v_cur, v_prev, delta: float, step: Optional[int] = None, t_r: Optional[int] = None):
+    """Response-token refresh rule of the feature cache the method builds on (appendix, "Response tokens"):
+    S_shift = { i : cos(V_i^(t), V_i^(t-1)) < delta },  S_period = all rows when t mod T_r = 0,  S = S_period U S_shift.
+
+    v_cur, v_prev [n, width]: the value features of the n response tokens at this step and the previous one (all heads
+    of a token side by side).  Returns (cos [n] float64, refresh [n] bool, indices of the refreshed rows, ascending).
+    Reading for a zero row, where the cosine is undefined: cosine 0, as in layer_importance."""
+    a, b = _f64(v_cur), _f64(v_prev)
+    dot = (a * b).sum(axis=1)
+    den = np.sqrt((a * a).sum(axis=1)) * np.sqrt((b * b).sum(axis=1))
+    cos = np.where(den > 0, dot / np.where(den > 0, den, 1.0), 0.0)
+    refresh = cos < delta
+    if step is not None and t_r is not None and t_r > 0 and step % t_r == 0:
+        refresh = np.ones_like(refresh)
+    return cos, refresh, np.nonzero(refresh)[0].astype(np.int32)
+
+
 def guarded_floor(x: float) -> int:
     return int(math.floor(x + 1e-6))
 
