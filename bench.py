@@ -331,6 +331,27 @@ def bench_ours(args):
         imp_bytes = 2.0 * n_tok * hidden * 2
         importance = {"workload": f"{n_tok} tokens x hidden {hidden}, bf16", "us": imp_us, "bytes": imp_bytes,
                       "value": float(imp_out.item())}
+        # the response-token refresh test of the per-step loop: cos(V_t, V_t-1) < delta over the live rows of one
+        # layer (256 x 4096: a latency-bound pair of launches) and over the same big tensors (HBM-bound)
+        r_idx = torch.zeros(n_tok, dtype=torch.int32, device=device)
+        r_cnt = torch.zeros(1, dtype=torch.int32, device=device)
+        refresh = {}
+        for name, rows, reps in (("one_layer_256_rows", wl.n_mask, 200), ("33k_rows", n_tok, 20)):
+            a, b = h_in[:rows], h_out[:rows]
+            for _ in range(3):
+                ctx.maskkv_refresh_set(a, b, 0.9, r_idx, r_cnt)
+            torch.cuda.synchronize()
+            r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            r0.record()
+            for _ in range(reps):
+                ctx.maskkv_refresh_set(a, b, 0.9, r_idx, r_cnt)
+            r1.record()
+            torch.cuda.synchronize()
+            us = 1e3 * r0.elapsed_time(r1) / reps
+            gbs = 2.0 * rows * hidden * 2 / (us * 1e-6) / 1e9
+            refresh[name] = {"us": round(us, 2), "GB/s": round(gbs, 1), "frac_of_hbm_peak": round(gbs / load_peaks()["hbm_gbs"], 3),
+                             "refreshed": int(r_cnt.item())}
+        importance["refresh_set"] = refresh
         del h_in, h_out
 
     if world > 1:
@@ -382,6 +403,7 @@ def bench_ours(args):
     }
     if importance is not None:
         gbs = importance["bytes"] / (importance["us"] * 1e-6) / 1e9
+        line["refresh_set"] = importance.pop("refresh_set", None)
         line["layer_importance"] = {"workload": importance["workload"], "us": round(importance["us"], 2),
                                     "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm}}
     line["cpu_baseline"] = oracle_baseline(wl, budget_s=15.0)

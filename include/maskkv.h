@@ -135,6 +135,19 @@ int maskkv_layer_importance(maskkv_ctx* ctx, int32_t dtype, const void* h_in_dev
                             int64_t n_tokens, int32_t hidden, int64_t in_row_stride, int64_t out_row_stride,
                             float* importance_out_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
 
+/* The response-token refresh rule of the feature cache the method is built on (appendix, "Response tokens"): which of
+ * the n_tokens response rows must be recomputed at this denoising step,
+ *   S_shift = { i : cos_sim(v_cur[i], v_prev[i]) < delta },
+ * v_cur / v_prev = the value features of the rows at this step and the previous one (T = dtype, [n_tokens][width], all
+ * heads of a token side by side; row strides in elements, 0 = packed; width * sizeof(T) and the strides multiples of
+ * 16 bytes).  refresh_all != 0 marks a periodic-refresh step (t mod T_r = 0, decided by the caller): every row is
+ * taken.  A row with a zero vector counts as cosine 0.  Outputs: idx_out_dev [n_tokens] receives the refreshed row
+ * numbers in ascending order (entries past the count are unspecified), count_out_dev [1] their number, cos_out_dev
+ * [n_tokens] the cosines (optional, may be NULL).  The comparison is made on the fp32 cosine.  No workspace. */
+int maskkv_refresh_set(maskkv_ctx* ctx, int32_t dtype, const void* v_cur_dev, const void* v_prev_dev, int64_t n_tokens,
+                       int32_t width, int64_t cur_row_stride, int64_t prev_row_stride, float delta, int32_t refresh_all,
+                       float* cos_out_dev, int32_t* idx_out_dev, int32_t* count_out_dev, void* stream);
+
 /* Eq. 6-7 and the sums of Eq. 14.  For every request r and KV head h: softmax (fp32) of
  * scale * q_i . k_j over the request's N_r prompt keys followed by its M_r mask keys, for each of the
  * H/H_kv query heads that share h; scores[h][prompt_cu[r] + j] = sum over those heads and mask rows i of

@@ -25,7 +25,7 @@ EXPORTS = (
     "maskkv_create", "maskkv_destroy", "maskkv_status_string", "maskkv_check_status", "maskkv_launch_count", "maskkv_last_cuda_error",
     "maskkv_tensor_core_launch_count",
     "maskkv_workspace_bytes",
-    "maskkv_layer_budgets", "maskkv_layer_importance", "maskkv_layer_importance_workspace_bytes", "maskkv_score", "maskkv_score_noalloc", "maskkv_score_noalloc_max_bytes", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend",
+    "maskkv_layer_budgets", "maskkv_layer_importance", "maskkv_layer_importance_workspace_bytes", "maskkv_refresh_set", "maskkv_score", "maskkv_score_noalloc", "maskkv_score_noalloc_max_bytes", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend",
 )
 
 
@@ -71,6 +71,7 @@ def _load() -> C.CDLL:
     lib.maskkv_layer_importance_workspace_bytes.argtypes = [vp]
     lib.maskkv_layer_importance_workspace_bytes.restype = sz
     lib.maskkv_layer_importance.argtypes = [vp, i32, vp, vp, i64, i32, i64, i64, vp, vp, sz, vp]
+    lib.maskkv_refresh_set.argtypes = [vp, i32, vp, vp, i64, i32, i64, i64, C.c_float, i32, vp, vp, vp, vp]
     lib.maskkv_score.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.maskkv_score_noalloc.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.maskkv_score_noalloc_max_bytes.argtypes = []
@@ -187,6 +188,16 @@ class Context:
                                            h_out.stride(0), _ptr(out), _ptr(workspace), workspace.numel(), _stream()),
                "maskkv_layer_importance", self._h)
         return workspace
+
+    def maskkv_refresh_set(self, v_cur, v_prev, delta: float, idx_out, count_out, refresh_all: bool = False, cos_out=None):
+        """Response-token refresh rule: v_cur, v_prev [n_tokens, width] (bf16 or fp32, rows may be strided); idx_out int32
+        [n_tokens] receives the ascending row numbers with cos < delta (all rows when refresh_all), count_out int32 [1]
+        their number, cos_out fp32 [n_tokens] (optional) the cosines."""
+        dt = MASKKV_F32 if v_cur.dtype == torch.float32 else MASKKV_BF16
+        n, width = (v_cur.shape[0], v_cur.shape[1]) if v_cur.dim() == 2 else (0, 0)
+        _check(lib.maskkv_refresh_set(self._h, dt, _ptr(v_cur), _ptr(v_prev), n, width, v_cur.stride(0) if n else 0,
+                                      v_prev.stride(0) if n else 0, float(delta), 1 if refresh_all else 0, _ptr(cos_out),
+                                      _ptr(idx_out), _ptr(count_out), _stream()), "maskkv_refresh_set", self._h)
 
     def maskkv_score(self, p: Problem, q_mask, k_prompt, k_mask, scores, mass_p, mass_m, workspace, row_weights=None):
         _check(lib.maskkv_score(self._h, C.byref(p.desc), _ptr(q_mask), _ptr(k_prompt), _ptr(k_mask), _ptr(row_weights),

@@ -10,6 +10,7 @@
 #include "common.cuh"
 #include "compact.cuh"
 #include "importance.cuh"
+#include "refresh.cuh"
 #include "score_simt.cuh"
 #include "score_tc.h"
 #include "select.cuh"
@@ -327,6 +328,46 @@ int maskkv_layer_importance(maskkv_ctx* ctx, int32_t dtype, const void* h_in_dev
         out_row_stride, partial);
   mkv::importance_final_kernel<<<1, mkv::kImpThreads, 0, st>>>(partial, (int)blocks, n_tokens, importance_out_dev);
   return launch_status(ctx, 2);
+}
+
+int maskkv_refresh_set(maskkv_ctx* ctx, int32_t dtype, const void* v_cur_dev, const void* v_prev_dev, int64_t n_tokens,
+                       int32_t width, int64_t cur_row_stride, int64_t prev_row_stride, float delta, int32_t refresh_all,
+                       float* cos_out_dev, int32_t* idx_out_dev, int32_t* count_out_dev, void* stream) {
+  if (ctx == nullptr || idx_out_dev == nullptr || count_out_dev == nullptr) return MASKKV_E_INVALID;
+  if (dtype != MASKKV_F32 && dtype != MASKKV_BF16) return MASKKV_E_UNSUPPORTED;
+  if (n_tokens < 0 || n_tokens > 0x7fffffffLL || width <= 0 || !(delta == delta)) return MASKKV_E_INVALID;
+  const int es = elem_size(dtype);
+  if (cur_row_stride == 0) cur_row_stride = width;
+  if (prev_row_stride == 0) prev_row_stride = width;
+  if (cur_row_stride < width || prev_row_stride < width) return MASKKV_E_INVALID;
+  const bool reads = !refresh_all || cos_out_dev != nullptr;
+  if (reads && n_tokens > 0) {
+    if (v_cur_dev == nullptr || v_prev_dev == nullptr) return MASKKV_E_INVALID;
+    if (((long long)width * es) % 16 != 0 || (cur_row_stride * es) % 16 != 0 || (prev_row_stride * es) % 16 != 0 ||
+        !aligned16(v_cur_dev) || !aligned16(v_prev_dev))
+      return MASKKV_E_ALIGN;
+  }
+  DeviceGuard guard(ctx->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int n = 0;
+  if (n_tokens > 0) {
+    const int rows_per_block = mkv::kRefreshThreads / 32;
+    long long blocks = (n_tokens + rows_per_block - 1) / rows_per_block;
+    const long long max_blocks = (long long)ctx->sm_count * 8;
+    if (blocks > max_blocks) blocks = max_blocks;
+    if (dtype == MASKKV_F32)
+      mkv::refresh_flag_kernel<float><<<(unsigned)blocks, mkv::kRefreshThreads, 0, st>>>(
+          static_cast<const float*>(v_cur_dev), static_cast<const float*>(v_prev_dev), n_tokens, width, cur_row_stride,
+          prev_row_stride, delta, refresh_all ? 1 : 0, cos_out_dev, idx_out_dev);
+    else
+      mkv::refresh_flag_kernel<__nv_bfloat16><<<(unsigned)blocks, mkv::kRefreshThreads, 0, st>>>(
+          static_cast<const __nv_bfloat16*>(v_cur_dev), static_cast<const __nv_bfloat16*>(v_prev_dev), n_tokens, width,
+          cur_row_stride, prev_row_stride, delta, refresh_all ? 1 : 0, cos_out_dev, idx_out_dev);
+    ++n;
+  }
+  mkv::launch_overlapped(mkv::refresh_compact_kernel, dim3(1), dim3(mkv::kRefreshScanThreads), 0, st, (long long)n_tokens, idx_out_dev,
+                         count_out_dev);
+  return launch_status(ctx, n + 1);
 }
 
 int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_dev, const void* k_prompt_dev,
