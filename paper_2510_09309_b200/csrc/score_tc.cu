@@ -154,6 +154,14 @@ __device__ __forceinline__ void walker_init(Walker& w, const Shape& sh, bool sta
   }
 }
 
+// Longest run of tiles one segment may have.  Sweep 2 only has to cut a run when a key's sum passes through the
+// shared-memory accumulators, i.e. when more than one query block votes on a KV head (grouped heads, or more than
+// 256 voters); otherwise a run is as long as the CTA's share allows and the per-run costs are paid once.
+__device__ __forceinline__ int seg_cap(const Shape& sh, bool stats, int M, int max_len) {
+  if (stats) return max_len;
+  return sh.g * ((M + kQBlock - 1) / kQBlock) == 1 ? 0x7fffffff : max_len;
+}
+
 __device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, int max_len, Seg& s) {
   if (!w.reverse) {
     if (w.f >= w.f_end) return false;
@@ -172,7 +180,7 @@ __device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, int max_
     s.t = (int)(rel % s.T);
     s.dir = 1;
     const long long room = w.f_end - w.f;
-    s.len = min(min(s.T - s.t, max_len), (int)min(room, (long long)0x7fffffff));
+    s.len = min(min(s.T - s.t, seg_cap(sh, w.stats, s.M, max_len)), (int)min(room, (long long)0x7fffffff));
     s.unit_start = w.base + (long long)s.g * s.T;
     w.f += s.len;
     return true;
@@ -195,7 +203,7 @@ __device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, int max_
   s.t = (int)(rel % s.T);
   s.dir = -1;
   const long long room = w.f - w.f_end;
-  s.len = min(min(s.t + 1, max_len), (int)min(room, (long long)0x7fffffff));
+  s.len = min(min(s.t + 1, seg_cap(sh, w.stats, s.M, max_len)), (int)min(room, (long long)0x7fffffff));
   s.unit_start = w.base + (long long)s.g * s.T;
   w.f -= s.len;
   return true;
