@@ -71,7 +71,7 @@ int resolve(const maskkv_desc_t* d, Shape* sh) {
 }
 
 struct ScoreWorkspace {
-  size_t lse_off, part_off, mass_off, cnt_off, total;
+  size_t lse_off, part_off, mass_off, cnt_off, col_off, total;
   int C, Tmax;
 };
 
@@ -88,6 +88,7 @@ ScoreWorkspace score_workspace(const maskkv_ctx* ctx, const Shape& sh) {
   w.part_off = off; off = align_up(off + sizeof(float2) * (size_t)sh.H * sh.sumM * w.C, 256);
   w.mass_off = off; off = align_up(off + sizeof(float2) * (size_t)sh.R * sh.Hkv * w.Tmax * 8, 256);
   w.cnt_off = off;  off = align_up(off + sizeof(uint32_t) * (size_t)sh.R * sh.Hkv, 256);
+  w.col_off = off;  off = align_up(off + mkv::tc::score_tc_colpart_bytes(sh), 256);   // per-block column sums (grouped heads)
   w.total = off;
   return w;
 }
@@ -132,9 +133,19 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, co
   bool tc2 = false;
   if (want_tc2) {
     // after a tensor-core sweep 1 the kernel merges the partials itself; otherwise it reads lse
+    int launched = 0;
+    float* colpart = reinterpret_cast<float*>(ws + w.col_off);
     tc2 = mkv::tc::launch_score_colsum_tc(ctx, sh, desc->prompt_cu, desc->live_cu, q, kp, km, lse, tc1 ? part : nullptr, w.C, rw,
-                                          scores, mass_part, w.Tmax, seg_cnt, mass_p, mass_m, any_without_voters, st) == 0;
-    if (tc2) { ++ctx->tc_launches; n += any_without_voters ? 2 : 1; }
+                                          scores, colpart, mass_part, w.Tmax, seg_cnt, mass_p, mass_m, any_without_voters, st,
+                                          &launched) == 0;
+    if (tc2) {
+      ++ctx->tc_launches;
+      n += launched;
+      if (mkv::tc::score_tc_split_blocks(sh)) {              // the masses of the per-block path are summed here
+        mkv::score_mass_reduce<<<(S + 3) / 4, 128, 0, st>>>(sh, mass_part, w.Tmax, mass_p, mass_m);
+        ++n;
+      }
+    }
   }
   if (!tc2) {
     if (tc1) { mkv::tc::launch_score_merge_tc(ctx, sh, desc->prompt_cu, desc->live_cu, part, w.C, lse, st); ++n; }

@@ -31,7 +31,6 @@ constexpr int kEpiThreadsPerAcc = 256; // two epilogue warpgroups share one accu
 constexpr int kStages = 4;
 constexpr int kTile = 128;             // keys per tile (both sweeps), queries per accumulator (sweep 1)
 constexpr int kQBlock = 256;           // queries resident per CTA
-constexpr int kColsumMaxTiles = 16;    // key tiles per unit in sweep 2 (bounded by the shared-memory accumulators)
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int D>
@@ -43,8 +42,7 @@ struct Smem {
   static constexpr int kKBytes = kBoxes * kKBoxBytes;
   static constexpr int kQOff = 0;
   static constexpr int kKOff = kQBytes;
-  static constexpr int kAccOff = kKOff + kStages * kKBytes;               // float [kColsumMaxTiles][128]
-  static constexpr int kC2Off = kAccOff + kColsumMaxTiles * kTile * 4;     // float [4 warpgroups][2][128]
+  static constexpr int kC2Off = kKOff + kStages * kKBytes;                 // float [4 warpgroups][2][128]
   static constexpr int kXchOff = kC2Off + 4 * kQBlock * 4;                 // float [2 accumulators][2][128]
   static constexpr int kBarOff = kXchOff + 4 * kTile * 4;                  // mbarriers
   static constexpr int kNumBars = 2 * kStages + 2 + 4 + 4;
@@ -123,21 +121,25 @@ __device__ __forceinline__ void block_teardown(uint32_t tmem_base) {
 // =====================================================================================================
 struct Seg { int r, g, t, len, p0, N, l0, M, T, dir; long long unit_start; };   // tiles t, t+dir, ..., len of them
 
+// mode of a walk: sweep 1 (groups = query head x 256-query block), sweep 2 with one query block per KV head (groups =
+// KV heads), sweep 2 with several (groups = query head x block again; the blocks' column sums meet in a later kernel)
+enum { kWalkStats = 0, kWalkColsum = 1, kWalkColsumSplit = 2 };
+
 struct Walker {
   long long f, f_end, base;   // forward: [f, f_end) still to do; reverse: [f_end, f) still to do, taken from the top
-  int r;
-  bool stats, reverse;
+  int r, mode;
+  bool reverse;
 };
 
-__device__ __forceinline__ int walk_groups(const Shape& sh, bool stats, int M) {
-  return M <= 0 ? 0 : (stats ? sh.H * ((M + kQBlock - 1) / kQBlock) : sh.Hkv);
+__host__ __device__ __forceinline__ int walk_groups(const Shape& sh, int mode, int M) {
+  return M <= 0 ? 0 : (mode == kWalkColsum ? sh.Hkv : sh.H * ((M + kQBlock - 1) / kQBlock));
 }
 __device__ __forceinline__ int tiles_of(int N, int M) { return (N + kTile - 1) / kTile + (M + kTile - 1) / kTile; }
 
 // Sweep 2 walks every share backwards: it then starts on the tiles sweep 1 read last, which are the ones most
 // likely to be still in L2 (the key tensor of a long prompt is larger than L2, so a forward walk would miss all).
-__device__ __forceinline__ void walker_init(Walker& w, const Shape& sh, bool stats, bool reverse, long long F) {
-  w.stats = stats;
+__device__ __forceinline__ void walker_init(Walker& w, const Shape& sh, int mode, bool reverse, long long F) {
+  w.mode = mode;
   w.reverse = reverse;
   const long long lo = (long long)blockIdx.x * F / gridDim.x, hi = (long long)(blockIdx.x + 1) * F / gridDim.x;
   w.base = 0;
@@ -147,29 +149,21 @@ __device__ __forceinline__ void walker_init(Walker& w, const Shape& sh, bool sta
   // position (r, base) on the request that holds the last tile of the share
   for (;;) {
     const int N = sh.prompt_cu[w.r + 1] - sh.prompt_cu[w.r], M = sh.live_cu[w.r + 1] - sh.live_cu[w.r];
-    const long long span = (long long)walk_groups(sh, stats, M) * tiles_of(N, M);
+    const long long span = (long long)walk_groups(sh, mode, M) * tiles_of(N, M);
     if (hi <= lo || hi - 1 < w.base + span || w.r + 1 >= sh.R) break;
     w.base += span;
     ++w.r;
   }
 }
 
-// Longest run of tiles one segment may have.  Sweep 2 only has to cut a run when a key's sum passes through the
-// shared-memory accumulators, i.e. when more than one query block votes on a KV head (grouped heads, or more than
-// 256 voters); otherwise a run is as long as the CTA's share allows and the per-run costs are paid once.
-__device__ __forceinline__ int seg_cap(const Shape& sh, bool stats, int M, int max_len) {
-  if (stats) return max_len;
-  return sh.g * ((M + kQBlock - 1) / kQBlock) == 1 ? 0x7fffffff : max_len;
-}
-
-__device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, int max_len, Seg& s) {
+__device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, Seg& s) {
   if (!w.reverse) {
     if (w.f >= w.f_end) return false;
     for (;;) {
       s.p0 = sh.prompt_cu[w.r]; s.N = sh.prompt_cu[w.r + 1] - s.p0;
       s.l0 = sh.live_cu[w.r]; s.M = sh.live_cu[w.r + 1] - s.l0;
       s.T = tiles_of(s.N, s.M);
-      const long long span = (long long)walk_groups(sh, w.stats, s.M) * s.T;
+      const long long span = (long long)walk_groups(sh, w.mode, s.M) * s.T;
       if (w.f < w.base + span) break;
       w.base += span;
       ++w.r;
@@ -180,7 +174,7 @@ __device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, int max_
     s.t = (int)(rel % s.T);
     s.dir = 1;
     const long long room = w.f_end - w.f;
-    s.len = min(min(s.T - s.t, seg_cap(sh, w.stats, s.M, max_len)), (int)min(room, (long long)0x7fffffff));
+    s.len = (int)min((long long)(s.T - s.t), room);
     s.unit_start = w.base + (long long)s.g * s.T;
     w.f += s.len;
     return true;
@@ -195,7 +189,7 @@ __device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, int max_
     // step back to the previous request
     --w.r;
     const int N2 = sh.prompt_cu[w.r + 1] - sh.prompt_cu[w.r], M2 = sh.live_cu[w.r + 1] - sh.live_cu[w.r];
-    w.base -= (long long)walk_groups(sh, w.stats, M2) * tiles_of(N2, M2);
+    w.base -= (long long)walk_groups(sh, w.mode, M2) * tiles_of(N2, M2);
   }
   const long long rel = last - w.base;
   s.r = w.r;
@@ -203,7 +197,7 @@ __device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, int max_
   s.t = (int)(rel % s.T);
   s.dir = -1;
   const long long room = w.f - w.f_end;
-  s.len = min(min(s.t + 1, seg_cap(sh, w.stats, s.M, max_len)), (int)min(room, (long long)0x7fffffff));
+  s.len = (int)min((long long)(s.t + 1), room);
   s.unit_start = w.base + (long long)s.g * s.T;
   w.f -= s.len;
   return true;
@@ -237,7 +231,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const uint32_t tmem_base = *tmem_slot;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   Walker wk;
-  walker_init(wk, sh, true, false, F);
+  walker_init(wk, sh, kWalkStats, false, F);
   Seg s;
 
   if (warp == 0) {
@@ -245,7 +239,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       prefetch_tmap(&map_q); prefetch_tmap(&map_kp); prefetch_tmap(&map_km);
       int kt_it = 0, q_it = 0;
       bool ok = true;
-      while (ok && walker_next(wk, sh, 0x7fffffff, s)) {
+      while (ok && walker_next(wk, sh, s)) {
         const int qp_n = (s.M + kQBlock - 1) / kQBlock;
         const int h = s.g / qp_n, q0 = (s.g % qp_n) * kQBlock, hk = h / sh.g;
         if (!(ok = mbar_wait(bars.qempty, q_it & 1, abort_flag, status, 0x100))) break;   // the MMA warp released the old block
@@ -272,7 +266,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       int kt_it = 0, q_it = 0;
       uint32_t cnt[2] = {0u, 0u};                            // tiles issued per query tile
       bool ok = true;
-      while (ok && walker_next(wk, sh, 0x7fffffff, s)) {
+      while (ok && walker_next(wk, sh, s)) {
         const int qp_n = (s.M + kQBlock - 1) / kQBlock;
         const int q0 = (s.g % qp_n) * kQBlock;
         const int n_qtiles = (s.M - q0 > kTile) ? 2 : 1;
@@ -313,7 +307,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const float cs = sh.scale * kLog2e;
     uint32_t cnt = 0;
     bool ok = true;
-    while (ok && walker_next(wk, sh, 0x7fffffff, s)) {
+    while (ok && walker_next(wk, sh, s)) {
       const int qp_n = (s.M + kQBlock - 1) / kQBlock;
       const int h = s.g / qp_n, q0 = (s.g % qp_n) * kQBlock;
       const int n_qtiles = (s.M - q0 > kTile) ? 2 : 1;
@@ -400,7 +394,7 @@ __device__ __noinline__ float merged_lse(const Shape& sh, const float2* __restri
   long long base = 0;
   for (int r2 = 0; r2 < r; ++r2) {
     const int N2 = sh.prompt_cu[r2 + 1] - sh.prompt_cu[r2], M2 = sh.live_cu[r2 + 1] - sh.live_cu[r2];
-    base += (long long)walk_groups(sh, true, M2) * tiles_of(N2, M2);
+    base += (long long)walk_groups(sh, kWalkStats, M2) * tiles_of(N2, M2);
   }
   const int N = sh.prompt_cu[r + 1] - sh.prompt_cu[r], M = sh.live_cu[r + 1] - sh.live_cu[r];
   const int T = tiles_of(N, M), qp_n = (M + kQBlock - 1) / kQBlock;
@@ -437,24 +431,30 @@ __global__ void score_merge_stats_tc(Shape sh, const float2* __restrict__ part, 
 }
 
 // =====================================================================================================
-// sweep 2: column sums.
-// scores[hk][p0 + j] = sum over the group's query heads and mask rows of w_i * exp(s_ij - lse_i);
-// mass_part[(r*H_kv + hk)*Tmax*8 + slot] = (sum over prompt keys, sum over mask keys) one warp of one CTA saw;
-// mass_p / mass_m [r*H_kv + hk] = their sums, written by the warp that completes the segment.
+// sweep 2: column sums, a thread per key.
+//
+// One query block (at most 256 voters) per KV head in every request (colpart == nullptr): the walk's groups are the KV
+// heads, and scores[hk][p0 + j] = sum over the block's rows of w_i * exp(s_ij - lse_i) is final.  The attention masses
+// are summed on the way: mass_part[(r*H_kv + hk)*Tmax*8 + slot] = (sum over prompt keys, sum over mask keys) one warp
+// of one CTA saw, and the warp that completes a segment's count adds the slots into mass_p / mass_m [r*H_kv + hk].
+//
+// Several query blocks per KV head (grouped heads, more than 256 voters): the walk's groups are (query head, block) as
+// in sweep 1, so a CTA keeps one block of queries resident over a long run of key tiles, and block b of KV head hk
+// leaves its column sums in colpart[(b*H_kv + hk)*(sum_N + sum_M) + key] (mask keys behind the prompt keys);
+// score_group_reduce adds the blocks up in block order and forms the masses.
 // =====================================================================================================
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kp,
                 const __grid_constant__ CUtensorMap map_km, Shape sh, const float* __restrict__ lse,
                 const float2* __restrict__ part, int C, long long F1, int G1,
-                const float* __restrict__ w, float* __restrict__ scores, float2* __restrict__ mass_part, int Tmax,
-                uint32_t* __restrict__ seg_cnt, float* __restrict__ mass_p, float* __restrict__ mass_m,
-                long long F, uint32_t* __restrict__ status) {
+                const float* __restrict__ w, float* __restrict__ scores, float* __restrict__ colpart,
+                float2* __restrict__ mass_part, int Tmax, uint32_t* __restrict__ seg_cnt, float* __restrict__ mass_p,
+                float* __restrict__ mass_m, long long F, uint32_t* __restrict__ status) {
   using S = Smem<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = align_1024(smem_raw);
   const Bars bars = carve_bars(base, S::kBarOff);
-  float* accs = reinterpret_cast<float*>(base + S::kAccOff);
   float* c2s = reinterpret_cast<float*>(base + S::kC2Off);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + S::kMiscOff);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base + S::kMiscOff + 4);
@@ -463,37 +463,41 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   pdl_wait();
   const uint32_t tmem_base = *tmem_slot;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const bool split = colpart != nullptr;
   Walker wk;
-  walker_init(wk, sh, false, true, F);
+  walker_init(wk, sh, split ? kWalkColsumSplit : kWalkColsum, true, F);
   Seg s;
-  int last_r = -1, last_g = -1;                             // the (request, KV head) whose queries are resident
+  int last_r = -1, last_g = -1;                             // the (request, group) whose queries are resident
+  // group of a run -> query head, KV head, first query of the block, index of the block among the KV head's blocks
+  auto unit_of = [&](const Seg& sg, int& h, int& hk, int& q0, int& blk) {
+    if (!split) { h = hk = sg.g; q0 = 0; blk = 0; return; }
+    const int qp_n = (sg.M + kQBlock - 1) / kQBlock;
+    h = sg.g / qp_n; hk = h / sh.g; q0 = (sg.g % qp_n) * kQBlock; blk = (h % sh.g) * qp_n + sg.g % qp_n;
+  };
 
   if (warp == 0) {
     if (lane == 0) {
       prefetch_tmap(&map_q); prefetch_tmap(&map_kp); prefetch_tmap(&map_km);
       int kt_it = 0, q_it = 0;
       bool ok = true;
-      while (ok && walker_next(wk, sh, kColsumMaxTiles, s)) {
-        const int q_per_head = (s.M + kQBlock - 1) / kQBlock, nqb = sh.g * q_per_head;
-        const bool reuse_q = nqb == 1 && s.r == last_r && s.g == last_g;
+      while (ok && walker_next(wk, sh, s)) {
+        int h, hk, q0, blk;
+        unit_of(s, h, hk, q0, blk);
+        if (s.r != last_r || s.g != last_g) {
+          if (!(ok = mbar_wait(bars.qempty, q_it & 1, abort_flag, status, 0x201))) break;
+          mbar_expect_tx(bars.qfull, S::kQBytes);
+          for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kQBoxBytes, &map_q, bars.qfull, b * 64, h, s.l0 + q0);
+          ++q_it;
+        }
         last_r = s.r; last_g = s.g;
-        for (int qb = 0; ok && qb < nqb; ++qb) {
-          if (!reuse_q) {
-            const int h = s.g * sh.g + qb / q_per_head, q0 = (qb % q_per_head) * kQBlock;
-            if (!(ok = mbar_wait(bars.qempty, q_it & 1, abort_flag, status, 0x201))) break;
-            mbar_expect_tx(bars.qfull, S::kQBytes);
-            for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kQBoxBytes, &map_q, bars.qfull, b * 64, h, s.l0 + q0);
-            ++q_it;
-          }
-          for (int tl = 0; tl < s.len; ++tl, ++kt_it) {
-            const int stage = kt_it % kStages, use = kt_it / kStages;
-            if (!(ok = mbar_wait(bars.empty + stage, (use & 1) ^ 1, abort_flag, status, 0x202))) break;
-            const KeyTile kt = key_tile(s.t + s.dir * tl, s.p0, s.N, s.l0, s.M);
-            mbar_expect_tx(bars.full + stage, S::kKBytes);
-            for (int b = 0; b < S::kBoxes; ++b)
-              tma_load_3d(base + S::kKOff + stage * S::kKBytes + b * S::kKBoxBytes, kt.prompt ? &map_kp : &map_km,
-                          bars.full + stage, b * 64, s.g, kt.token);
-          }
+        for (int tl = 0; tl < s.len; ++tl, ++kt_it) {
+          const int stage = kt_it % kStages, use = kt_it / kStages;
+          if (!(ok = mbar_wait(bars.empty + stage, (use & 1) ^ 1, abort_flag, status, 0x202))) break;
+          const KeyTile kt = key_tile(s.t + s.dir * tl, s.p0, s.N, s.l0, s.M);
+          mbar_expect_tx(bars.full + stage, S::kKBytes);
+          for (int b = 0; b < S::kBoxes; ++b)
+            tma_load_3d(base + S::kKOff + stage * S::kKBytes + b * S::kKBoxBytes, kt.prompt ? &map_kp : &map_km,
+                        bars.full + stage, b * 64, hk, kt.token);
         }
       }
       if (!ok) drain_loads(bars, kt_it);
@@ -505,36 +509,33 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       bool ok = true;
       const uint32_t q_lo_base = smem_desc_lo(smem_u32(base + S::kQOff));
       const uint32_t k_lo_base = smem_desc_lo(smem_u32(base + S::kKOff));
-      while (ok && walker_next(wk, sh, kColsumMaxTiles, s)) {
-        const int q_per_head = (s.M + kQBlock - 1) / kQBlock, nqb = sh.g * q_per_head;
-        const bool reuse_q = nqb == 1 && s.r == last_r && s.g == last_g;
+      while (ok && walker_next(wk, sh, s)) {
+        int h, hk, q0, blk;
+        unit_of(s, h, hk, q0, blk);
+        const int n_mma = (min(kQBlock, s.M - q0) + 31) & ~31;             // columns the epilogue will read
+        const uint32_t idesc = idesc_bf16_f32(kTile, n_mma);
+        if (s.r != last_r || s.g != last_g) {
+          umma_commit(bars.qempty);                          // every MMA that read the resident queries has been issued
+          if (!(ok = mbar_wait(bars.qfull, q_it & 1, abort_flag, status, 0x203))) break;
+          ++q_it;
+          tc_fence_after();
+        }
         last_r = s.r; last_g = s.g;
-        for (int qb = 0; ok && qb < nqb; ++qb) {
-          const int q0 = (qb % q_per_head) * kQBlock;
-          const int n_mma = (min(kQBlock, s.M - q0) + 31) & ~31;           // columns the epilogue will read
-          const uint32_t idesc = idesc_bf16_f32(kTile, n_mma);
-          if (!reuse_q) {
-            umma_commit(bars.qempty);                        // every MMA that read the resident queries has been issued
-            if (!(ok = mbar_wait(bars.qfull, q_it & 1, abort_flag, status, 0x203))) break;
-            ++q_it;
-            tc_fence_after();
-          }
-          for (int tl = 0; tl < s.len; ++tl, ++kt_it) {
-            const int stage = kt_it % kStages, use = kt_it / kStages, buf = (tl + base_par) & 1;
-            if (!(ok = mbar_wait(bars.full + stage, use & 1, abort_flag, status, 0x204))) break;
-            if (!(ok = mbar_wait(bars.tempty + buf, (uses[buf] & 1) ^ 1, abort_flag, status, 0x205))) break;
-            tc_fence_after();
-            const uint32_t k_lo = k_lo_base + stage * (S::kKBytes >> 4);
+        for (int tl = 0; tl < s.len; ++tl, ++kt_it) {
+          const int stage = kt_it % kStages, use = kt_it / kStages, buf = (tl + base_par) & 1;
+          if (!(ok = mbar_wait(bars.full + stage, use & 1, abort_flag, status, 0x204))) break;
+          if (!(ok = mbar_wait(bars.tempty + buf, (uses[buf] & 1) ^ 1, abort_flag, status, 0x205))) break;
+          tc_fence_after();
+          const uint32_t k_lo = k_lo_base + stage * (S::kKBytes >> 4);
 #pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-              const uint32_t ko = ((kk >> 2) * S::kKBoxBytes + (kk & 3) * 32) >> 4;
-              const uint32_t qo = ((kk >> 2) * S::kQBoxBytes + (kk & 3) * 32) >> 4;
-              umma_ss(tmem_base + buf * kQBlock, make_desc(k_lo + ko, kDescHiSw128), make_desc(q_lo_base + qo, kDescHiSw128), idesc, kk > 0);
-            }
-            umma_commit(bars.empty + stage);
-            umma_commit(bars.tfull + buf);
-            ++uses[buf];
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t ko = ((kk >> 2) * S::kKBoxBytes + (kk & 3) * 32) >> 4;
+            const uint32_t qo = ((kk >> 2) * S::kQBoxBytes + (kk & 3) * 32) >> 4;
+            umma_ss(tmem_base + buf * kQBlock, make_desc(k_lo + ko, kDescHiSw128), make_desc(q_lo_base + qo, kDescHiSw128), idesc, kk > 0);
           }
+          umma_commit(bars.empty + stage);
+          umma_commit(bars.tfull + buf);
+          ++uses[buf];
         }
         base_par ^= s.len & 1;
       }
@@ -542,10 +543,9 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   } else {
     // Four warpgroups: accumulator buf = wg >> 1, and of its (up to) 256 query columns the 128-column half (wg & 1).
     // The two halves of a key's sum meet in shared memory (one named barrier per tile per pair); the half-0 thread
-    // owns the key from then on.  Inside a segment the tile -> accumulator map is fixed, (tl + base_par) & 1, so a
-    // key's running sum in shared memory always belongs to the same thread; base_par carries the alternation across
-    // segments.  After a failed wait a thread skips the arithmetic but still walks the loops, so that every thread
-    // reaches every named barrier.
+    // owns the key from then on.  Inside a run the tile -> accumulator map is fixed, (tl + base_par) & 1; base_par
+    // carries the alternation across runs.  After a failed wait a thread skips the arithmetic but still walks the
+    // loops, so that every thread reaches every named barrier.
     const int wg = (warp - 2) >> 2;
     const int buf = wg >> 1, half = wg & 1;
     const int lane_group = warp & 3;
@@ -553,13 +553,15 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const float cs = sh.scale * kLog2e;
     const uint32_t taddr = tmem_base + ((uint32_t)(lane_group * 32) << 16) + buf * kQBlock + half * kTile;
     float* xch = reinterpret_cast<float*>(base + S::kXchOff) + buf * 2 * kTile;
+    const long long keys_total = (long long)sh.sumN + sh.sumM;
     uint32_t uses = 0, c2_it = 0;
     int base_par = 0;
     bool ok = true;
     const float* c2 = c2s;
-    // Attention mass of the segment in hand, summed over the tiles this warp finished (half-0 warps only).  When the
-    // walk leaves the segment the warp stores its pair in slot (CTA - first CTA of the segment) * 8 + warp and
-    // counts itself in; the warp that completes the count adds the slots up, always in slot order.
+    // Attention mass of the segment in hand (one query block per KV head only), summed over the tiles this warp
+    // finished (half-0 warps).  When the walk leaves the segment the warp stores its pair in slot
+    // (CTA - first CTA of the segment) * 8 + warp and counts itself in; the warp that completes the count adds the slots
+    // up, always in slot order.
     int cur_seg = -1, cur_T = 0;
     long long cur_start = 0;
     float run_p = 0.f, run_m = 0.f;
@@ -587,87 +589,113 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (lane == 0) { mass_p[cur_seg] = sum_p; mass_m[cur_seg] = sum_m; }
       }
     };
-    while (walker_next(wk, sh, kColsumMaxTiles, s)) {
-      const int q_per_head = (s.M + kQBlock - 1) / kQBlock, nqb = sh.g * q_per_head;
-      const bool reuse_q = nqb == 1 && s.r == last_r && s.g == last_g;
+    while (walker_next(wk, sh, s)) {
+      int h, hk, q0, blk;
+      unit_of(s, h, hk, q0, blk);
+      const bool new_q = s.r != last_r || s.g != last_g;
       last_r = s.r; last_g = s.g;
-      const int seg = s.r * sh.Hkv + s.g;
-      if (seg != cur_seg) {
-        flush();
-        cur_seg = seg; cur_T = s.T; cur_start = s.unit_start;
-        run_p = run_m = 0.f;
+      if (!split) {
+        const int seg = s.r * sh.Hkv + hk;
+        if (seg != cur_seg) {
+          flush();
+          cur_seg = seg; cur_T = s.T; cur_start = s.unit_start;
+          run_p = run_m = 0.f;
+        }
       }
-      for (int qb = 0; qb < nqb; ++qb) {
-        const int h = s.g * sh.g + qb / q_per_head, q0 = (qb % q_per_head) * kQBlock + half * kTile;
-        const int nq = max(0, min(kTile, s.M - q0));        // voters in this warpgroup's half of the block
-        if (!reuse_q) {
-          float* c2w = c2s + (wg * 2 + (c2_it & 1)) * kTile;
-          ++c2_it;
-          float cst = -INFINITY;                            // 2^(x - inf) = 0: rows that do not exist never vote
-          if (row < nq) {
-            const int i = s.l0 + q0 + row;
-            const float ln_z = part != nullptr ? merged_lse(sh, part, C, F1, G1, s.r, h, qb % q_per_head, i)
-                                               : lse[(long long)h * sh.sumM + i];
-            cst = (w ? log2f(w[i]) : 0.f) - ln_z * kLog2e;
-          }
-          c2w[row] = cst;                                   // stored negated: x = s*c + cst
-          named_barrier(1 + wg, kTile);
-          c2 = c2w;
+      const int qh0 = q0 + half * kTile;                    // first voter of this warpgroup's half of the block
+      const int nq = max(0, min(kTile, s.M - qh0));
+      if (new_q) {
+        float* c2w = c2s + (wg * 2 + (c2_it & 1)) * kTile;
+        ++c2_it;
+        float cst = -INFINITY;                              // 2^(x - inf) = 0: rows that do not exist never vote
+        if (row < nq) {
+          const int i = s.l0 + qh0 + row;
+          const float ln_z = part != nullptr ? merged_lse(sh, part, C, F1, G1, s.r, h, q0 / kQBlock, i)
+                                             : lse[(long long)h * sh.sumM + i];
+          cst = (w ? log2f(w[i]) : 0.f) - ln_z * kLog2e;
         }
-        const int chunks = (nq + 31) >> 5;
-        auto absorb = [&](const float* v, int cb, uint64_t& acc2) {
-          const float4* cc = reinterpret_cast<const float4*>(c2 + cb * 32);   // negated constants
-          const uint64_t cs2 = pack2(cs, cs);
+        c2w[row] = cst;                                     // stored negated: x = s*c + cst
+        named_barrier(1 + wg, kTile);
+        c2 = c2w;
+      }
+      const int chunks = (nq + 31) >> 5;
+      auto absorb = [&](const float* v, int cb, uint64_t& acc2) {
+        const float4* cc = reinterpret_cast<const float4*>(c2 + cb * 32);   // negated constants
+        const uint64_t cs2 = pack2(cs, cs);
 #pragma unroll
-          for (int c4 = 0; c4 < 8; ++c4) {
-            const float4 k4 = cc[c4];
-            float x0, x1, x2, x3;
-            unpack2(fma2(pack2(v[4 * c4], v[4 * c4 + 1]), cs2, pack2(k4.x, k4.y)), x0, x1);
-            unpack2(fma2(pack2(v[4 * c4 + 2], v[4 * c4 + 3]), cs2, pack2(k4.z, k4.w)), x2, x3);
-            acc2 = add2(acc2, pack2(ex2(x0), ex2(x1)));
-            acc2 = add2(acc2, pack2(ex2(x2), ex2(x3)));
-          }
-        };
-        for (int tl = (buf + base_par) & 1; tl < s.len; tl += 2) {
-          uint64_t acc2 = pack2(0.f, 0.f);
-          if (ok) ok = mbar_wait(bars.tfull + buf, uses & 1, abort_flag, status, 0x206);
-          if (ok) {
-            tc_fence_after();
-            // four warps per scheduler hide the load latency: no register double-buffering here
-#pragma unroll 1
-            for (int cb = 0; cb < chunks; ++cb) {
-              float v[32];
-              tmem_ld32(taddr + cb * 32, v);
-              tmem_ld_wait();
-              if (cb + 1 == chunks) { tc_fence_before(); mbar_arrive(bars.tempty + buf); }   // last logits are in registers
-              absorb(v, cb, acc2);
-            }
-            if (chunks == 0) { tc_fence_before(); mbar_arrive(bars.tempty + buf); }
-          }
-          float a0, a1;
-          unpack2(acc2, a0, a1);
-          float* slot = xch + (uses & 1) * kTile;
-          ++uses;
-          if (half == 1) slot[row] = a0 + a1;
-          named_barrier(5 + buf, 2 * kTile);                // the pair's two halves of this tile are done
-          if (half == 1 || !ok) continue;
-          float acc = (a0 + a1) + slot[row];
-          if (nqb > 1) {                                    // grouped heads / more than 256 voters: sum over query blocks
-            if (qb > 0) acc += accs[tl * kTile + row];
-            if (qb + 1 < nqb) { accs[tl * kTile + row] = acc; continue; }
-          }
-          const KeyTile kt = key_tile(s.t + s.dir * tl, s.p0, s.N, s.l0, s.M);
-          if (row >= kt.valid) acc = 0.f;
-          if (kt.prompt && row < kt.valid) scores[(long long)s.g * sh.sumN + kt.token + row] = acc;
-          acc = warp_sum(acc);
-          if (kt.prompt) run_p += acc; else run_m += acc;
+        for (int c4 = 0; c4 < 8; ++c4) {
+          const float4 k4 = cc[c4];
+          float x0, x1, x2, x3;
+          unpack2(fma2(pack2(v[4 * c4], v[4 * c4 + 1]), cs2, pack2(k4.x, k4.y)), x0, x1);
+          unpack2(fma2(pack2(v[4 * c4 + 2], v[4 * c4 + 3]), cs2, pack2(k4.z, k4.w)), x2, x3);
+          acc2 = add2(acc2, pack2(ex2(x0), ex2(x1)));
+          acc2 = add2(acc2, pack2(ex2(x2), ex2(x3)));
         }
+      };
+      float* out_row = split ? colpart + ((long long)blk * sh.Hkv + hk) * keys_total : scores + (long long)hk * sh.sumN;
+      for (int tl = (buf + base_par) & 1; tl < s.len; tl += 2) {
+        uint64_t acc2 = pack2(0.f, 0.f);
+        if (ok) ok = mbar_wait(bars.tfull + buf, uses & 1, abort_flag, status, 0x206);
+        if (ok) {
+          tc_fence_after();
+          // four warps per scheduler hide the load latency: no register double-buffering here
+#pragma unroll 1
+          for (int cb = 0; cb < chunks; ++cb) {
+            float v[32];
+            tmem_ld32(taddr + cb * 32, v);
+            tmem_ld_wait();
+            if (cb + 1 == chunks) { tc_fence_before(); mbar_arrive(bars.tempty + buf); }   // last logits are in registers
+            absorb(v, cb, acc2);
+          }
+          if (chunks == 0) { tc_fence_before(); mbar_arrive(bars.tempty + buf); }
+        }
+        float a0, a1;
+        unpack2(acc2, a0, a1);
+        float* slot = xch + (uses & 1) * kTile;
+        ++uses;
+        if (half == 1) slot[row] = a0 + a1;
+        named_barrier(5 + buf, 2 * kTile);                  // the pair's two halves of this tile are done
+        if (half == 1 || !ok) continue;
+        float acc = (a0 + a1) + slot[row];
+        const KeyTile kt = key_tile(s.t + s.dir * tl, s.p0, s.N, s.l0, s.M);
+        if (split) {                                        // prompt keys, then mask keys, of every request
+          if (row < kt.valid) out_row[(kt.prompt ? 0 : sh.sumN) + kt.token + row] = acc;
+          continue;
+        }
+        if (row >= kt.valid) acc = 0.f;
+        if (kt.prompt && row < kt.valid) out_row[kt.token + row] = acc;
+        acc = warp_sum(acc);
+        if (kt.prompt) run_p += acc; else run_m += acc;
       }
       base_par ^= s.len & 1;
     }
     flush();
   }
   block_teardown(tmem_base);
+}
+
+// Several query blocks per KV head: scores[hk][p0 + j] = sum over the blocks, in block order, of their column sums, and
+// the tile's share of the attention masses as the FP32-pipe sweep leaves it (mass_part[((r*H_kv + hk)*Tmax + t)*4 + warp],
+// summed by score_mass_reduce).  A request without voters has no blocks: zeros.  grid (Tmax, H_kv, R), 128 threads.
+__global__ void score_group_reduce(Shape sh, const float* __restrict__ colpart, float* __restrict__ scores,
+                                   float2* __restrict__ mass_part, int Tmax) {
+  const int t = blockIdx.x, hk = blockIdx.y, r = blockIdx.z;
+  const int p0 = sh.prompt_cu[r], N = sh.prompt_cu[r + 1] - p0;
+  const int l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
+  if (t >= tiles_of(N, M)) return;
+  const KeyTile kt = key_tile(t, p0, N, l0, M);
+  const int blocks = M <= 0 ? 0 : sh.g * ((M + kQBlock - 1) / kQBlock);
+  const long long keys_total = (long long)sh.sumN + sh.sumM;
+  const int j = threadIdx.x;
+  float acc = 0.f;
+  if (j < kt.valid) {
+    const float* src = colpart + (long long)hk * keys_total + (kt.prompt ? 0 : sh.sumN) + kt.token + j;
+    for (int b = 0; b < blocks; ++b) acc += src[(long long)b * sh.Hkv * keys_total];
+    if (kt.prompt) scores[(long long)hk * sh.sumN + kt.token + j] = acc;
+  }
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0)
+    mass_part[((long long)(r * sh.Hkv + hk) * Tmax + t) * 4 + (threadIdx.x >> 5)] = kt.prompt ? make_float2(acc, 0.f) : make_float2(0.f, acc);
 }
 
 // Requests without voters (M = 0): every score is zero and so are the masses.  grid (tiles, H_kv, R).
@@ -699,13 +727,11 @@ bool build_maps(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kp,
 }
 
 // F of the walk: tiles over all (request, group) pairs, from the host's copy of the lengths.
-long long flat_tiles(const Shape& sh, const int32_t* prompt_cu, const int32_t* live_cu, bool stats) {
+long long flat_tiles(const Shape& sh, const int32_t* prompt_cu, const int32_t* live_cu, int mode) {
   long long F = 0;
   for (int r = 0; r < sh.R; ++r) {
     const int N = prompt_cu[r + 1] - prompt_cu[r], M = live_cu[r + 1] - live_cu[r];
-    if (M <= 0) continue;
-    const long long groups = stats ? (long long)sh.H * ((M + kQBlock - 1) / kQBlock) : sh.Hkv;
-    F += groups * ((N + kTile - 1) / kTile + (M + kTile - 1) / kTile);
+    F += (long long)walk_groups(sh, mode, M) * ((N + kTile - 1) / kTile + (M + kTile - 1) / kTile);
   }
   return F;
 }
@@ -742,7 +768,7 @@ int launch_score_stats_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* promp
                           const void* q, const void* kp, const void* km, float2* part, int C, uint32_t* seg_cnt, cudaStream_t st) {
   Maps m;
   if (!build_maps(ctx, sh, q, kp, km, &m)) return 1;
-  const long long F = flat_tiles(sh, prompt_cu_host, live_cu_host, true);
+  const long long F = flat_tiles(sh, prompt_cu_host, live_cu_host, kWalkStats);
   if (F <= 0) return 1;
   const int grid = (int)(F < ctx->sm_count ? F : ctx->sm_count);
   if (sh.d == 128) {
@@ -759,34 +785,53 @@ int launch_score_stats_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* promp
 
 void launch_score_merge_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prompt_cu_host, const int32_t* live_cu_host,
                            const float2* part, int C, float* lse, cudaStream_t st) {
-  const long long F = flat_tiles(sh, prompt_cu_host, live_cu_host, true);
+  const long long F = flat_tiles(sh, prompt_cu_host, live_cu_host, kWalkStats);
   const int grid = (int)(F < ctx->sm_count ? F : ctx->sm_count);
   const long long rows = (long long)sh.H * sh.sumM;
   score_merge_stats_tc<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(sh, part, C, F, grid, lse);
 }
 
+bool score_tc_split_blocks(const Shape& sh) { return sh.g > 1 || sh.maxM > kQBlock; }
+
+size_t score_tc_colpart_bytes(const Shape& sh) {
+  if (!score_tc_split_blocks(sh)) return 0;
+  const size_t blocks = (size_t)sh.g * (size_t)((sh.maxM + kQBlock - 1) / kQBlock);
+  return sizeof(float) * blocks * (size_t)sh.Hkv * ((size_t)sh.sumN + (size_t)sh.sumM);
+}
+
 int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prompt_cu_host, const int32_t* live_cu_host,
                            const void* q, const void* kp, const void* km, const float* lse, const float2* part, int C,
-                           const float* w, float* scores, float2* mass_part, int Tmax, uint32_t* seg_cnt, float* mass_p,
-                           float* mass_m, bool any_without_voters, cudaStream_t st) {
+                           const float* w, float* scores, float* colpart, float2* mass_part, int Tmax, uint32_t* seg_cnt,
+                           float* mass_p, float* mass_m, bool any_without_voters, cudaStream_t st, int* launches) {
   Maps m;
   if (!build_maps(ctx, sh, q, kp, km, &m)) return 1;
-  const long long F = flat_tiles(sh, prompt_cu_host, live_cu_host, false);
+  const bool split = score_tc_split_blocks(sh);
+  if (split && colpart == nullptr) return 1;
+  const long long F = flat_tiles(sh, prompt_cu_host, live_cu_host, split ? kWalkColsumSplit : kWalkColsum);
   if (F <= 0) return 1;
   const int grid = (int)(F < ctx->sm_count ? F : ctx->sm_count);
-  const long long F1 = flat_tiles(sh, prompt_cu_host, live_cu_host, true);     // sweep 1's walk, for its partials
+  const long long F1 = flat_tiles(sh, prompt_cu_host, live_cu_host, kWalkStats);   // sweep 1's walk, for its partials
   const int G1 = (int)(F1 < ctx->sm_count ? F1 : ctx->sm_count);
   if (sh.d == 128 ? set_smem_attr<128>() != cudaSuccess : set_smem_attr<64>() != cudaSuccess) return 1;
-  if (any_without_voters) {
+  *launches = 0;
+  if (any_without_voters && !split) {                      // with several query blocks the reduce kernel writes the zeros
     dim3 gz(score_tc_max_tiles(sh), sh.Hkv, sh.R);
     score_zero_fill<<<gz, kTile, 0, st>>>(sh, scores, mass_p, mass_m);
+    ++*launches;
   }
+  float* cp = split ? colpart : nullptr;
   if (sh.d == 128)
     launch_overlapped(score_colsum_tc<128>, dim3(grid), dim3(kThreads), Smem<128>::kDynamic, st, m.q, m.kp, m.km, sh, lse, part, C, F1, G1,
-                      w, scores, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
+                      w, scores, cp, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
   else
     launch_overlapped(score_colsum_tc<64>, dim3(grid), dim3(kThreads), Smem<64>::kDynamic, st, m.q, m.kp, m.km, sh, lse, part, C, F1, G1,
-                      w, scores, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
+                      w, scores, cp, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
+  ++*launches;
+  if (split) {
+    dim3 gr(Tmax, sh.Hkv, sh.R);
+    score_group_reduce<<<gr, kTile, 0, st>>>(sh, colpart, scores, mass_part, Tmax);
+    ++*launches;
+  }
   return 0;
 }
 
