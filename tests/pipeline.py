@@ -23,7 +23,7 @@ def to_dev(x, device="cuda"):
     return x.to(device).contiguous()
 
 
-class GpuRun:
+class LayerRun:
     """Owns the device buffers of one layer's pass through the five calls."""
 
     def __init__(self, ctx, wl: synth.Workload, capacity: Optional[int] = None, k_l: Optional[int] = None):

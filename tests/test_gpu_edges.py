@@ -8,7 +8,7 @@ import torch
 
 from oracle import maskkv_oracle as O
 from paper_2510_09309_b200 import synth
-from pipeline import ATTEND_ATOL, GpuRun, assert_scores_close, to_dev
+from pipeline import ATTEND_ATOL, LayerRun, assert_scores_close, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -98,7 +98,7 @@ def test_empty_and_degenerate_segments(ctx, dtype):
     x = synth.layer_inputs(wl, 0, "cpu"); live = synth.live_inputs(wl, 0, 0, "cpu")
     xd = {k: to_dev(v) for k, v in x.items() if torch.is_tensor(v)}; ld = {k: to_dev(v) for k, v in live.items()}
     for k_l in (0, 1, 300):
-        run = GpuRun(ctx, wl, capacity=2000, k_l=k_l)
+        run = LayerRun(ctx, wl, capacity=2000, k_l=k_l)
         run.score(xd); run.budget(alpha=1.0); run.select(); run.compact(xd); run.attend(ld)
         torch.cuda.synchronize()
         sc, mp, mm = O.score(x["q_mask"], x["k_prompt"], x["k_mask"], wl.prompt_cu(), wl.live_cu())
@@ -171,7 +171,7 @@ def test_attend_long_segments_shared_by_two_ctas(ctx, d, n_mask):
                       n_kv_heads=4, head_dim=d, mean_budget=1536)
     x = synth.layer_inputs(wl, 0, "cpu"); live = synth.live_inputs(wl, 0, 0, "cpu")
     xd = {k: to_dev(v) for k, v in x.items() if torch.is_tensor(v)}; ld = {k: to_dev(v) for k, v in live.items()}
-    run = GpuRun(ctx, wl, capacity=4 * 1536, k_l=1536)
+    run = LayerRun(ctx, wl, capacity=4 * 1536, k_l=1536)
     budgets = torch.tensor([[1536, 0, 2999, 1609]], dtype=torch.int32)      # 12 / 0 / 24 / 13 key tiles + the live ones
     offsets = torch.tensor([0, 1536, 1536, 4535, 6144], dtype=torch.int32)
     run.score(xd)

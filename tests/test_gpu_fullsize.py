@@ -12,7 +12,7 @@ import torch
 
 from oracle import maskkv_oracle as O
 from paper_2510_09309_b200 import synth
-from pipeline import ATTEND_ATOL, GpuRun, assert_kept_within_band, assert_scores_close
+from pipeline import ATTEND_ATOL, LayerRun, assert_kept_within_band, assert_scores_close
 
 pytestmark = pytest.mark.gpu
 
@@ -28,7 +28,7 @@ def ctx():
 def _run_and_check(ctx, wl, layer, k_l, alpha, sample, attend_steps=1):
     """sample: list of (request, kv_head)."""
     x = synth.layer_inputs(wl, layer, "cuda")
-    run = GpuRun(ctx, wl, k_l=k_l)
+    run = LayerRun(ctx, wl, k_l=k_l)
     run.score(x)
     run.budget(alpha=alpha)
     run.select()

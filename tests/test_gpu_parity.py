@@ -9,7 +9,7 @@ import torch
 
 from oracle import maskkv_oracle as O
 from paper_2510_09309_b200 import synth
-from pipeline import (ATTEND_ATOL, GpuRun, assert_kept_within_band, assert_scores_close, oracle_layer, to_dev)
+from pipeline import (ATTEND_ATOL, LayerRun, assert_kept_within_band, assert_scores_close, oracle_layer, to_dev)
 
 pytestmark = pytest.mark.gpu
 
@@ -56,7 +56,7 @@ def case(request, ctx):
     ref = oracle_layer(wl, x, live, k_l, wl.alpha)
     xd = {k: to_dev(v) for k, v in x.items() if torch.is_tensor(v)}
     ld = {k: to_dev(v) for k, v in live.items()}
-    return dict(wl=wl, x=x, live=live, xd=xd, ld=ld, ref=ref, k_l=k_l, run=GpuRun(ctx, wl, k_l=k_l))
+    return dict(wl=wl, x=x, live=live, xd=xd, ld=ld, ref=ref, k_l=k_l, run=LayerRun(ctx, wl, k_l=k_l))
 
 
 def test_score(case):
@@ -191,7 +191,7 @@ def test_full_budget_equals_full_attention(ctx):
                       mean_budget=256)
     x = synth.layer_inputs(wl, 0, "cpu"); live = synth.live_inputs(wl, 0, 0, "cpu")
     xd = {k: to_dev(v) for k, v in x.items() if torch.is_tensor(v)}; ld = {k: to_dev(v) for k, v in live.items()}
-    run = GpuRun(ctx, wl)
+    run = LayerRun(ctx, wl)
     run.score(xd); run.budget(alpha=1.0); run.select(); run.compact(xd); run.attend(ld)
     torch.cuda.synchronize()
     assert run.budgets.cpu().tolist() == [[200, 200], [64, 64]]
