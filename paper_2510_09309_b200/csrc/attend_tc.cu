@@ -5,25 +5,26 @@
 // head's ragged segment of the compacted cache (rows [offsets[s], offsets[s+1]) of kc / vc), then over
 // the request's live rows.  Per tile:
 //     S = Q K^T            tcgen05.mma, operands in shared memory (TMA, 128-byte swizzle), S in tensor memory
-//     P = 2^(S*c - m*c)    NW threads per query row (128/NW key columns each; NW = 2): online max / sum in
-//                          fp32, P rounded to bf16 and written back into tensor memory over S
-//     PV = P V             tcgen05.mma with P read from tensor memory and V (row-major, i.e. N-major) from
-//                          shared memory, into a fresh accumulator
-//     O = O*corr + PV      in registers, d/NW output columns per thread (no rescaling pass over tensor memory)
-// S/P and PV are double-buffered (4 x 128 columns of tensor memory) so the next tile's Q K^T overlaps the
-// softmax; Q K^T and P V are issued by two different threads; key and value tiles come through separate TMA rings
-// (3 and 2 stages) and tiles beyond the rings are requested into L2 ahead of time.  Columns of a ragged tile's tail
+//     P = 2^(S*c - m*c)    two threads per query row, 64 key columns each, each with an online softmax of its own
+//                          (reference m, sum l) in fp32; P rounded to bf16 and written back over S
+//     O_w += P_w V_w       tcgen05.mma with P read from tensor memory and V (row-major, i.e. N-major) from shared
+//                          memory, accumulated over all tiles in the warpgroup's own 128 columns of tensor memory
+// S/P is double-buffered so the next tile's Q K^T overlaps the softmax; Q K^T and the two P V streams are issued by
+// three different threads; key and value tiles come through separate TMA rings (3 and 2 stages) and tiles beyond
+// the rings are requested into L2 ahead of time.  A reference only moves when a logit exceeds it by more than 2^8
+// (then the thread rescales its row of O_w in tensor memory), so nothing per tile waits for a P V product or for the
+// other warpgroup; the two partial softmaxes are merged once, after the last tile.  Columns of a ragged tile's tail
 // are masked to -inf, and the matching V rows are zeroed in shared memory so that stale cache rows can never leak a
 // NaN into the product.  The output tile leaves through shared memory as whole rows.
 //
 // The kernel is a latency chain (3-8 dependent tiles per CTA), not a throughput kernel.  Cycle stamps of one CTA:
-// 2.6k cycles until the tile loop starts (set-up, wait for the previous kernel, segment offsets), 2.9k more until the
-// first S is ready (tensor maps, Q and K from L2, first MMA group), then about 2.6k per tile - 0.35k reading S and
-// finding the row maximum, 1.4k for the exchange of the maximum, the 128 x 128 exponentials (1,024 cycles of the
-// special-function unit by themselves), packing and the store of P, 0.45k adding the previous tile's P V - and 1-3k
-// to normalise and store.  When units are few and their key segments long, a cluster of two CTAs shares a unit: each
-// walks half of the tiles and CTA 1 hands its (max, sum, output) to CTA 0 through distributed shared memory; that
-// merge costs about three tiles' time, so it is used from eight tiles per unit on.
+// 2.6k cycles until the tile loop starts (set-up, wait for the previous kernel, segment offsets), 2.3k more until the
+// first S is ready (tensor maps, Q and K from L2, first MMA group), then about 2.0k per tile - 0.3k reading S and
+// finding the row maximum, 1.4k for the 128 x 128 exponentials (1,024 cycles of the special-function unit by
+// themselves; the two warpgroups stay in phase because the S buffers are shared), packing and the store of P - and
+// 3.5k to merge, normalise and store.  When units are few and their key segments long, a cluster of two CTAs shares a
+// unit: each walks half of the tiles and CTA 1 hands its (max, sum, output) to CTA 0 through distributed shared
+// memory; that merge costs about three tiles' time, so it is used from eight tiles per unit on.
 #include "attend_tc.h"
 
 #include <cooperative_groups.h>
@@ -33,13 +34,9 @@
 namespace mkv {
 namespace tc {
 
-// warp 0: TMA, warp 1: issues Q K^T, then NW softmax warpgroups (thread = one query row, 128/NW key columns, d/NW output
-// columns), last warp: issues P V.  Two issuing threads, because issuing a group of eight MMAs costs one thread
-// about 0.2 us and the two groups of a tile would otherwise queue behind each other.
-#ifndef MKV_ATTEND_NW
-#define MKV_ATTEND_NW 2
-#endif
-template <int D> struct AWgs { static constexpr int kNW = MKV_ATTEND_NW; static constexpr int kThreads = 96 + 128 * kNW; static constexpr int kPvWarp = 2 + 4 * kNW; };
+// warp 0: TMA; warp 1: issues Q K^T; warps 2-9: two softmax warpgroups (thread = one query row, 64 key columns of every
+// tile); warps 10, 11: issue P V of warpgroup 0 / 1.
+template <int D> struct AWgs { static constexpr int kNW = 2; static constexpr int kThreads = 64 + 128 * kNW + 32 * kNW; static constexpr int kPvWarp = 2 + 4 * kNW; };
 constexpr int kATile = 128;
 constexpr int kAKStages = 3;            // key tiles in flight (the next Q K^T is issued a tile ahead)
 constexpr int kAVStages = 2;            // value tiles in flight
@@ -55,11 +52,11 @@ struct ASmem {
   static constexpr int kKOff = kTileBytes;
   static constexpr int kVOff = kKOff + kAKStages * kTileBytes;
   static constexpr int kBarOff = kVOff + kAVStages * kTileBytes;
-  static constexpr int kNumBars = 1 + 2 * kAKStages + 2 * kAVStages + 8;
+  static constexpr int kNumBars = 1 + 2 * kAKStages + 2 * kAVStages + 10;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
-  static constexpr int kMxOff = kMiscOff + 16;                             // float [2 tiles][4 warpgroups][128]: partial row maxima
-  static constexpr int kLxOff = kMxOff + 8 * kATile * 4;                   // float [4 warpgroups][128]: partial row sums
-  static constexpr int kBytes = kLxOff + 4 * kATile * 4;
+  static constexpr int kMxOff = kMiscOff + 16;                             // float [2 warpgroups][128]: row references
+  static constexpr int kLxOff = kMxOff + 2 * kATile * 4;                   // float [2 warpgroups][128]: row sums
+  static constexpr int kBytes = kLxOff + 2 * kATile * 4;
   static constexpr int kDynamic = kBytes + 1024;
 };
 
@@ -113,13 +110,14 @@ struct ABars {
   uint64_t* qfull;
   uint64_t *kfull, *kempty;                    // [kAKStages]
   uint64_t *vfull, *vempty;                    // [kAVStages]
-  uint64_t *sfull, *pready, *ofull, *oempty;   // [2]
+  uint64_t* sfull;                             // [2 buffers]
+  uint64_t *pready, *odone;                    // [2 buffers][2 warpgroups]
 };
 __device__ __forceinline__ ABars carve_abars(uint8_t* base, int off) {
   uint64_t* b = reinterpret_cast<uint64_t*>(base + off);
   ABars r;
   r.qfull = b; r.kfull = b + 1; r.kempty = r.kfull + kAKStages; r.vfull = r.kempty + kAKStages; r.vempty = r.vfull + kAVStages;
-  r.sfull = r.vempty + kAVStages; r.pready = r.sfull + 2; r.ofull = r.pready + 2; r.oempty = r.ofull + 2;
+  r.sfull = r.vempty + kAVStages; r.pready = r.sfull + 2; r.odone = r.pready + 4;
   return r;
 }
 
@@ -155,9 +153,10 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   if (threadIdx.x == 0) {
     mbar_init(bars.qfull, 1);
     for (int s = 0; s < kAKStages; ++s) { mbar_init(bars.kfull + s, 1); mbar_init(bars.kempty + s, 1); }
-    for (int s = 0; s < kAVStages; ++s) { mbar_init(bars.vfull + s, 1); mbar_init(bars.vempty + s, 1); }
+    for (int s = 0; s < kAVStages; ++s) { mbar_init(bars.vfull + s, 1); mbar_init(bars.vempty + s, 2); }   // both P V issuers release a stage
     for (int b = 0; b < 2; ++b) {
-      mbar_init(bars.sfull + b, 1); mbar_init(bars.pready + b, AWgs<D>::kNW * kATile); mbar_init(bars.ofull + b, 1); mbar_init(bars.oempty + b, AWgs<D>::kNW * kATile);
+      mbar_init(bars.sfull + b, 1);
+      for (int w = 0; w < 2; ++w) { mbar_init(bars.pready + 2 * b + w, kATile); mbar_init(bars.odone + 2 * b + w, 1); }
     }
     *abort_flag = 0u;
     fence_barrier_init();
@@ -187,7 +186,7 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   const int j_first = part * per_part;                     // this CTA walks tiles [j_first, j_first + nt)
   const int nt = max(0, min(per_part, nt_all - j_first));
 
-  const uint32_t tm_s = tmem_base, tm_o = tmem_base + 256;   // S/P buffers at columns 0 / 128, PV buffers at 256 / 384
+  const uint32_t tm_s = tmem_base, tm_o = tmem_base + 256;   // S/P buffers at columns 0 / 128, the warpgroups' outputs at 256 / 384
 
   if (warp == 0) {
     if (lane == 0) {
@@ -259,150 +258,196 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       bool ok = mbar_wait(bars.qfull, 0, abort_flag, status, 0x303);
       tc_fence_after();
       for (int j = 0; ok && j < nt; ++j) {
-        const int stage = j % kAKStages, use = j / kAKStages;
+        const int b = j & 1, stage = j % kAKStages, use = j / kAKStages;
         if (!(ok = mbar_wait(bars.kfull + stage, use & 1, abort_flag, status, 0x304))) break;
-        // S/P buffer j & 1 is free once P V of tile j - 2 has read P from it
-        if (j >= 2 && !(ok = mbar_wait(bars.ofull + (j & 1), ((j - 2) >> 1) & 1, abort_flag, status, 0x30b))) break;
+        // S/P buffer b is free once both P V products of tile j - 2 have read P from it
+        if (j >= 2) {
+          if (!(ok = mbar_wait(bars.odone + 2 * b, ((j - 2) >> 1) & 1, abort_flag, status, 0x30b))) break;
+          if (!(ok = mbar_wait(bars.odone + 2 * b + 1, ((j - 2) >> 1) & 1, abort_flag, status, 0x30c))) break;
+        }
         tc_fence_after();
         const uint32_t k_lo = smem_desc_lo(smem_u32(base + S::kKOff + stage * S::kTileBytes));
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t o = ((kk >> 2) * S::kBoxBytes + (kk & 3) * 32) >> 4;
-          umma_ss(tm_s + (j & 1) * kATile, make_desc(q_lo + o, kDescHiSw128), make_desc(k_lo + o, kDescHiSw128), idesc_qk, kk > 0);
+          umma_ss(tm_s + b * kATile, make_desc(q_lo + o, kDescHiSw128), make_desc(k_lo + o, kDescHiSw128), idesc_qk, kk > 0);
         }
-        umma_commit(bars.sfull + (j & 1));
+        umma_commit(bars.sfull + b);
         umma_commit(bars.kempty + stage);
       }
     }
     if (nsplit > 1) { cluster_barrier(); cluster_barrier(); }
-  } else if (warp == AWgs<D>::kPvWarp) {
+  } else if (warp >= AWgs<D>::kPvWarp) {
+    // P V of warpgroup w: O_w += P[:, 64w .. 64w+63] V[64w .. 64w+63, :], four k-steps, accumulated in tensor memory
+    // over all tiles (the warpgroup rescales O_w itself in the rare case its reference moves).
+    const int w = warp - AWgs<D>::kPvWarp;
     if (lane == 0) {
       const uint32_t idesc_pv = idesc_bf16_f32_bn(kATile, D);
       bool ok = true;
       for (int j = 0; ok && j < nt; ++j) {
         const int b = j & 1, stage = j % kAVStages, use = j / kAVStages;
         if (!(ok = mbar_wait(bars.vfull + stage, use & 1, abort_flag, status, 0x305))) break;
-        if (!(ok = mbar_wait(bars.oempty + b, ((j >> 1) & 1) ^ 1, abort_flag, status, 0x306))) break;
-        if (!(ok = mbar_wait(bars.pready + b, (j >> 1) & 1, abort_flag, status, 0x307))) break;
+        if (!(ok = mbar_wait(bars.pready + 2 * b + w, (j >> 1) & 1, abort_flag, status, 0x307))) break;
         tc_fence_after();
         // N-major descriptor: low word = address | (box stride between the two 64-column halves), high word as K-major
         const uint32_t v_lo = ((smem_u32(base + S::kVOff + stage * S::kTileBytes) & 0x3ffffu) >> 4) | ((uint32_t)(S::kBoxBytes >> 4) << 16);
 #pragma unroll
-        for (int kk = 0; kk < kATile / 16; ++kk)
-          // P of keys [SC*w, SC*w + SC) sits in packed columns [SC*w, SC*w + SC/2), SC = 128 / NW key columns per thread
-          umma_ts(tm_o + b * kATile, tm_s + b * kATile + (16 * kk / (kATile / AWgs<D>::kNW)) * (kATile / AWgs<D>::kNW) + (16 * kk % (kATile / AWgs<D>::kNW)) / 2,
-                  make_desc(v_lo + ((kk * 16 * 128) >> 4), kDescHiSw128), idesc_pv, kk > 0);
-        umma_commit(bars.ofull + b);
+        for (int kk = 0; kk < 4; ++kk)
+          // P of keys [64w, 64w + 64) sits in packed columns [64w, 64w + 32) of the S/P buffer
+          umma_ts(tm_o + w * kATile, tm_s + b * kATile + 64 * w + 8 * kk, make_desc(v_lo + (((4 * w + kk) * 16 * 128) >> 4), kDescHiSw128),
+                  idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
+        umma_commit(bars.odone + 2 * b + w);
         umma_commit(bars.vempty + stage);
       }
     }
     if (nsplit > 1) { cluster_barrier(); cluster_barrier(); }
   } else {
-    // NW softmax warpgroups share every tile: thread (wg, row) owns S columns [SC wg, SC wg + SC) of its query row
-    // (SC = 128 / NW) and the output columns [32 wg, 32 wg + 32).  The row maximum is the only thing they exchange per
-    // tile (shared memory + one named barrier); P of the thread's keys is written over the S columns the same thread
-    // has just read (packed columns SC wg .. SC wg + SC/2 - 1), so the warpgroups never touch each other's columns.
+    // Two softmax warpgroups, each an online softmax of its own over "its" 64 keys of every tile: thread (wg, row)
+    // owns S columns [64 wg, 64 wg + 64) of its query row, keeps its own reference m and sum l, writes P over the columns
+    // it has just read, and its P V accumulates in the warpgroup's own output O_wg in tensor memory.  Nothing is
+    // exchanged per tile, so the two groups drift apart and one's exponentials overlap the other's tensor-memory
+    // traffic.  m only moves when a logit exceeds it by more than 2^kSlack (P <= 2^kSlack is harmless in bf16 and
+    // fp32); then the thread rescales its row of O_wg in tensor memory.  The groups meet once, after the last tile.
     constexpr int NW = AWgs<D>::kNW;
-    constexpr int SC = kATile / NW;                         // 32 or 64
+    constexpr int SC = kATile / NW;                         // 64 key columns of a tile per thread
+    constexpr float kSlack = 8.f;
     const int wg = (warp - 2) >> 2;
     const int lane_group = warp & 3;
     const int row = lane_group * 32 + lane;                 // query inside the tile
-    const int tid_all = wg * kATile + ((warp - 2) & 3) * 32 + lane;   // 0 .. NW*128-1 over the softmax warpgroups
+    const int tid_all = wg * kATile + ((warp - 2) & 3) * 32 + lane;   // 0 .. 255 over the softmax warpgroups
     const uint32_t lane_addr = (uint32_t)(lane_group * 32) << 16;
+    const uint32_t o_addr = tm_o + lane_addr + wg * kATile;  // this row of O_wg
     const float cs = sh.scale * kALog2e;
     float* mx = reinterpret_cast<float*>(base + S::kMxOff);
     float* lx = reinterpret_cast<float*>(base + S::kLxOff);
-    constexpr int OC = D / NW;                              // output columns per thread
-    float o[OC];
-#pragma unroll
-    for (int c = 0; c < OC; ++c) o[c] = 0.f;
-    float m = -INFINITY, l = 0.f, corr_prev = 0.f;
+    constexpr int OC = D / NW;                              // output columns per thread after the groups have met
+    float m = -INFINITY, l = 0.f;
     bool ok = true;
-
-    auto consume_pv = [&](int j, float corr) {               // O = O*corr + PV(j), this thread's 32 output columns
-      const int b = j & 1;
-      if (ok) ok = mbar_wait(bars.ofull + b, (j >> 1) & 1, abort_flag, status, 0x308);
-      if (!ok) return;
-      tc_fence_after();
-#pragma unroll
-      for (int cb = 0; cb < OC / 32; ++cb) {
-        float v[32];
-        tmem_ld32(tm_o + lane_addr + b * kATile + wg * OC + cb * 32, v);
-        tmem_ld_wait();
-        if (cb + 1 == OC / 32) { tc_fence_before(); mbar_arrive(bars.oempty + b); }
-#pragma unroll
-        for (int c = 0; c < 32; ++c) o[cb * 32 + c] = fmaf(o[cb * 32 + c], corr, v[c]);
-      }
-    };
 
     // After a failed wait a thread skips the tensor-memory work but still reaches every named barrier.
     for (int j = 0; j < nt; ++j) {
       const int b = j & 1;
       const ATile t = a_tile(j_first + j, c0, nc, l0, M);
-      const int my_valid = min(SC, max(0, t.valid - wg * SC));   // valid columns among this thread's SC
+      const int my_valid = min(SC, max(0, t.valid - wg * SC));   // valid columns among this thread's 64
       if (ok && t.valid < kATile) {
-        // ragged tail: zero the value rows that do not belong to this tile (every thread clears a slice)
+        // ragged tail: zero the value rows that do not belong to this tile.  Each warpgroup clears all of them (its
+        // own P V is released by its own threads only, so it may not rely on the other group's stores).
         const int stage = j % kAVStages, su = j / kAVStages;
         if ((ok = mbar_wait(bars.vfull + stage, su & 1, abort_flag, status, 0x309))) {
           uint8_t* v_tile = base + S::kVOff + stage * S::kTileBytes;
           const int n16 = (kATile - t.valid) * 8;           // 16-byte pieces per box
           for (int bx = 0; bx < S::kBoxes; ++bx) {
             uint4* dst = reinterpret_cast<uint4*>(v_tile + bx * S::kBoxBytes + t.valid * 128);
-            for (int e = tid_all; e < n16; e += NW * kATile) dst[e] = make_uint4(0u, 0u, 0u, 0u);
+            for (int e = tid_all & (kATile - 1); e < n16; e += kATile) dst[e] = make_uint4(0u, 0u, 0u, 0u);
           }
           fence_async_smem();
         }
       }
       if (ok) ok = mbar_wait(bars.sfull + b, (j >> 1) & 1, abort_flag, status, 0x30a);
+      ok = __all_sync(0xffffffffu, ok);                     // the tensor-memory instructions below are warp-wide
+      if (!ok) continue;
+      tc_fence_after();
       const uint32_t s_addr = tm_s + lane_addr + b * kATile + wg * SC;
-      // the thread's logits are read once and stay in registers for both passes
-      float v[SC];
-      float tmax = -INFINITY;
-      if (ok) {
-        tc_fence_after();
+      float v[SC];                                          // the thread's logits, read once
 #pragma unroll
-        for (int cb = 0; cb < SC / 32; ++cb) tmem_ld32(s_addr + cb * 32, v + cb * 32);
-        tmem_ld_wait();
-        if (my_valid < SC) {                                 // masked columns of a ragged tile do not take part
+      for (int cb = 0; cb < SC / 32; ++cb) tmem_ld32(s_addr + cb * 32, v + cb * 32);
+      tmem_ld_wait();
+      if (my_valid < SC) {                                   // masked columns of a ragged tile do not take part
 #pragma unroll
-          for (int c = 0; c < SC; ++c) if (c >= my_valid) v[c] = -INFINITY;
-        }
-#pragma unroll
-        for (int c = 0; c < SC; c += 2) tmax = max3(tmax, v[c], v[c + 1]);
+        for (int c = 0; c < SC; ++c) if (c >= my_valid) v[c] = -INFINITY;
       }
-      mx[(b * NW + wg) * kATile + row] = tmax;
-      named_barrier(1, NW * kATile);
+      float tmax = -INFINITY;
 #pragma unroll
-      for (int w2 = 0; w2 < NW; ++w2) tmax = fmaxf(tmax, mx[(b * NW + w2) * kATile + row]);
-      const float m_new = fmaxf(m, tmax);                    // the same value in every warpgroup
-      const float corr = ex2((m - m_new) * cs);
-      const float neg = -m_new * cs;
+      for (int c = 0; c < SC; c += 2) tmax = max3(tmax, v[c], v[c + 1]);
+      // The reference moves up when a logit exceeds it by more than 2^kSlack: the sum and this row of O_wg are rescaled,
+      // once the previous tile's P V has landed.  Tensor-memory loads and stores are warp-wide instructions, so the whole
+      // warp goes through them as soon as one row needs it (factor 1 for the others).
+      const bool grow = m != -INFINITY && (tmax - m) * cs > kSlack;
+      const float f = grow ? ex2((m - tmax) * cs) : 1.f;
+      if (__any_sync(0xffffffffu, grow)) {
+        ok = __all_sync(0xffffffffu, mbar_wait(bars.odone + 2 * ((j - 1) & 1) + wg, ((j - 1) >> 1) & 1, abort_flag, status, 0x308));
+        if (ok) {
+          tc_fence_after();
+#pragma unroll
+          for (int cb = 0; cb < D / 32; ++cb) {
+            float ov[32];
+            tmem_ld32(o_addr + cb * 32, ov);
+            tmem_ld_wait();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) ov[c] *= f;
+            tmem_st32(o_addr + cb * 32, reinterpret_cast<const uint32_t*>(ov));
+          }
+          tmem_st_wait();
+        }
+      }
+      if (grow) { l *= f; m = tmax; }
+      else if (m == -INFINITY) m = tmax;                    // nothing accumulated so far (O_wg is zero or not yet written)
+      if (!ok) continue;
+      // P = 2^(s*c - m*c) as bf16 pairs (a masked column gives 2^-inf = 0), written over the columns just read
+      uint32_t packed[SC / 2];
       float rs = 0.f;
-      if (ok) {
-        // P = 2^(s*c - m*c) as bf16 pairs (a masked column gives 2^-inf = 0), written over the columns just read
-        uint32_t packed[SC / 2];
+      if (m == -INFINITY) {                                  // not a single valid column yet: P = 0
+#pragma unroll
+        for (int c = 0; c < SC / 2; ++c) packed[c] = 0u;
+      } else {
+        const float neg = -m * cs;
 #pragma unroll
         for (int c = 0; c < SC; c += 2) {
           const float p0 = ex2(fmaf(v[c], cs, neg)), p1 = ex2(fmaf(v[c + 1], cs, neg));
           rs += p0 + p1;
           packed[c / 2] = pack_bf16(p0, p1);
         }
-        if (SC == 64) tmem_st32(s_addr, packed); else tmem_st16(s_addr, packed);
-        tmem_st_wait();
-        tc_fence_before();
-        mbar_arrive(bars.pready + b);
       }
-      l = l * corr + rs;
-      m = m_new;
-      if (j > 0) consume_pv(j - 1, corr_prev);
-      corr_prev = corr;
+      tmem_st32(s_addr, packed);
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(bars.pready + 2 * b + wg);
+      l += rs;
     }
-    if (nt > 0) consume_pv(nt - 1, corr_prev);
+    // The groups meet: common reference, total sum, and each group's O scaled onto the common reference.  Thread
+    // (wg, row) ends up with output columns [OC wg, OC wg + OC) of its row: it keeps that half of its own O_wg and
+    // passes the other half to its partner through shared memory (the key ring, free by now), 16 bytes per access.
+    if (ok && nt > 0) ok = mbar_wait(bars.odone + 2 * ((nt - 1) & 1) + wg, ((nt - 1) >> 1) & 1, abort_flag, status, 0x30d);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) tc_fence_after();
+    mx[wg * kATile + row] = m;
     lx[wg * kATile + row] = l;
     named_barrier(1, NW * kATile);
-    l = 0.f;
+    const float m_other = mx[(wg ^ 1) * kATile + row], l_other = lx[(wg ^ 1) * kATile + row];
+    const float m_all = fmaxf(m, m_other);
+    const float a_me = m == -INFINITY ? 0.f : ex2((m - m_all) * cs);
+    const float a_other = m_other == -INFINITY ? 0.f : ex2((m_other - m_all) * cs);
+    float o[OC];
+    float4* xg = reinterpret_cast<float4*>(base + S::kKOff);   // [writer group][column group of 4][row] as float4
 #pragma unroll
-    for (int w2 = 0; w2 < NW; ++w2) l += lx[w2 * kATile + row];
+    for (int cb = 0; cb < D / 32; ++cb) {
+      float ov[32];
+      if (ok && nt > 0) {                                    // warp-uniform; a group that never saw a valid key holds exact zeros
+        tmem_ld32(o_addr + cb * 32, ov);
+        tmem_ld_wait();
+      } else {
+#pragma unroll
+        for (int c = 0; c < 32; ++c) ov[c] = 0.f;
+      }
+      if ((cb * 32) / OC == wg) {                            // a chunk of my own half
+#pragma unroll
+        for (int c = 0; c < 32; ++c) o[cb * 32 - wg * OC + c] = ov[c] * a_me;
+      } else {                                               // my partner's half
+        const int c_rel = cb * 32 - (wg ^ 1) * OC;           // column inside the partner's half
+#pragma unroll
+        for (int c = 0; c < 32; c += 4)
+          xg[(wg * (OC / 4) + (c_rel + c) / 4) * kATile + row] = make_float4(ov[c] * a_me, ov[c + 1] * a_me, ov[c + 2] * a_me, ov[c + 3] * a_me);
+      }
+    }
+    named_barrier(1, NW * kATile);
+#pragma unroll
+    for (int c = 0; c < OC; c += 4) {
+      const float4 x4 = xg[((wg ^ 1) * (OC / 4) + c / 4) * kATile + row];
+      o[c] += x4.x; o[c + 1] += x4.y; o[c + 2] += x4.z; o[c + 3] += x4.w;
+    }
+    l = l * a_me + l_other * a_other;
+    m = m_all;
+    named_barrier(1, NW * kATile);                           // the exchange area is reused below
     if (nsplit > 1) {
       // Exchange area in CTA 0: its key ring, free once both CTAs have finished their tiles (first barrier).
       // xo4[column group of 4][row] as float4 (a warp's 32 rows of a group are 512 contiguous bytes, for the remote
