@@ -166,6 +166,9 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) {                                  // kernel parameters: may be fetched before the wait
+    prefetch_tmap(&map_q); prefetch_tmap(&map_kl); prefetch_tmap(&map_vl); prefetch_tmap(&map_kc); prefetch_tmap(&map_vc);
+  }
   pdl_wait();
 
   // A cluster of `nsplit` CTAs (1 or 2) shares one (query tile, head): CTA `part` walks its contiguous share of
@@ -173,14 +176,15 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
   const int nsplit = (int)cluster.num_blocks(), part = (int)cluster.block_rank();
   const int qt = blockIdx.x / nsplit, h = blockIdx.y, r = blockIdx.z, hk = h / sh.g;
-  const int l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
+  const int seg = r * sh.Hkv + hk;
+  // the four loads go out together (they are independent, and nothing can start before them)
+  const int l0 = sh.live_cu[r], l1 = sh.live_cu[r + 1], c0 = offsets[seg], c1 = offsets[seg + 1];
+  const int M = l1 - l0, nc = c1 - c0;
   const int q0 = qt * kATile;
   if (q0 >= M) {                                           // uniform over the block: nothing to do for this tile
     if (warp == 1) tmem_dealloc(tmem_base, 512);
     return;
   }
-  const int seg = r * sh.Hkv + hk;
-  const int c0 = offsets[seg], nc = offsets[seg + 1] - c0;
   const int nt_all = (nc + kATile - 1) / kATile + (M + kATile - 1) / kATile;
   const int per_part = (nt_all + nsplit - 1) / nsplit;
   const int j_first = part * per_part;                     // this CTA walks tiles [j_first, j_first + nt)
@@ -190,7 +194,6 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
 
   if (warp == 0) {
     if (lane == 0) {
-      prefetch_tmap(&map_q); prefetch_tmap(&map_kl); prefetch_tmap(&map_vl); prefetch_tmap(&map_kc); prefetch_tmap(&map_vc);
       mbar_expect_tx(bars.qfull, S::kTileBytes);
       for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kBoxBytes, &map_q, bars.qfull, b * 64, h, l0 + q0);
       // two independent rings (keys, values): whichever has a free stage gets its next tile, keys first
