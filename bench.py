@@ -306,6 +306,47 @@ def bench_ours(args):
     e1.record()
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), device)
+
+    # ---- the same, with the prompt values left in pinned host memory: only the kept rows of V are ever needed on the
+    # device (maskkv_compact is the one reader of v_prompt), so the gather reads them straight from host memory and the
+    # evicted rows never cross the bus.  Reported next to the standard number, not instead of it.
+    def e2e_lazy_step(i):
+        for k in keys_in:
+            if k != "v_prompt":
+                dev_x[k].copy_(host_x[k], non_blocking=True)
+        for k in keys_live:
+            dev_l[k].copy_(host_l[k], non_blocking=True)
+        p = buf.p
+        ctx.maskkv_score(p, dev_x["q_mask"], dev_x["k_prompt"], dev_x["k_mask"], buf.scores, buf.mass_p, buf.mass_m, buf.ws)
+        ctx.maskkv_budget(p, k_layers[resident[0]], wl.alpha, buf.mass_p, buf.mass_m, buf.capacity, buf.budgets, buf.offsets)
+        ctx.maskkv_select(p, buf.scores, buf.budgets, buf.offsets, buf.kept, buf.ws)
+        ctx.maskkv_compact(p, dev_x["k_prompt"], host_x["v_prompt"], buf.kept, buf.offsets, buf.capacity, buf.kc, buf.vc)
+        ctx.maskkv_attend(p, dev_l["q_live"], dev_l["k_live"], dev_l["v_live"], buf.kc, buf.vc, buf.offsets, buf.capacity, buf.out)
+        host_out.copy_(buf.out, non_blocking=True)
+        host_bud.copy_(buf.budgets, non_blocking=True)
+
+    e2e_lazy = None
+    try:
+        ref_out = buf.out.clone()
+        for i in range(2):
+            e2e_lazy_step(i)
+        barrier()
+        same = bool(torch.equal(ref_out, buf.out))
+        z0, z1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        z0.record()
+        for i in range(e2e_steps):
+            e2e_lazy_step(i)
+        z1.record()
+        barrier()
+        lazy_ms = max_over_ranks(z0.elapsed_time(z1), device)
+        v_bytes = host_x["v_prompt"].numel() * host_x["v_prompt"].element_size()
+        kept_v_bytes = int(buf.offsets[-1].item()) * wl.head_dim * host_x["v_prompt"].element_size()
+        e2e_lazy = {"value": world * N / (lazy_ms / e2e_steps * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": h2d - v_bytes + kept_v_bytes, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                    "same_output_as_copied_v": same,
+                    "note": "v_prompt stays in pinned host memory; maskkv_compact reads the kept rows from there"}
+    except Exception as exc:                                           # a platform without device access to pinned memory
+        e2e_lazy = {"unavailable": str(exc)[:120]}
     clocks = sampler.stop() if sampler else {}
 
     # ---- calibration step of the budget rule (Eq. 8), outside the timed step: a streaming reduction bound by HBM
@@ -390,6 +431,7 @@ def bench_ours(args):
         "compress_tokens_per_s": N / (1e-6 * (call_us["score"] + call_us["budget"] + call_us["select"] + call_us["compact"])),
         "e2e": {"value": world * N / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "e2e_v_in_host_memory": e2e_lazy,
         "gpu_launches": int(launches),
         "clocks": clocks,
         "status_flags": flags,

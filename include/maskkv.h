@@ -204,7 +204,10 @@ int maskkv_select(maskkv_ctx* ctx, const maskkv_desc_t* desc, const float* score
                   void* workspace_dev, size_t workspace_bytes, void* stream);
 
 /* kc[offsets[s] + t] = k_prompt[prompt_cu[r] + kept_idx[offsets[s] + t]][h][:], same for v: a byte copy.
- * `capacity` is the number of rows kc/vc/kept_idx hold; rows at or beyond it are never touched. */
+ * `capacity` is the number of rows kc/vc/kept_idx hold; rows at or beyond it are never touched.
+ * k_prompt_dev / v_prompt_dev only have to be addresses the device can read: this call is the path's only reader of
+ * v_prompt, so a caller whose prompt values live in pinned (device-mapped) host memory can pass that pointer and have
+ * the kept rows alone cross the bus. */
 int maskkv_compact(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* k_prompt_dev,
                    const void* v_prompt_dev, const int32_t* kept_idx_dev, const int32_t* offsets_dev,
                    int64_t capacity, void* kc_dev, void* vc_dev, void* stream);
