@@ -228,18 +228,55 @@ def bench_ours(args):
     for i in range(args.warmup):
         step(i)
     barrier()
+    # The five calls of a layer allocate nothing and never synchronise, so a layer's step is captured once into a CUDA
+    # graph (one per resident layer: the pointers differ) and the timed loop replays the graphs - what a serving loop
+    # would do, and it removes the launch gaps between the six kernels.  --no-graph times plain calls instead.
+    graphs, launches_per_step = None, None
+    if not args.no_graph:
+        side = torch.cuda.Stream(device=device)
+        side.wait_stream(torch.cuda.current_stream())
+        graphs = []
+        with torch.cuda.stream(side):
+            for j in range(len(resident)):
+                before = ctx.maskkv_launch_count()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    step(j)
+                launches_per_step = ctx.maskkv_launch_count() - before
+                graphs.append(g)
+        torch.cuda.current_stream().wait_stream(side)
+        for j in range(len(resident)):                                # one replay each, untimed
+            graphs[j].replay()
+        barrier()
+
+    def timed_step(i):
+        if graphs is not None:
+            graphs[i % len(resident)].replay()
+        else:
+            step(i)
+
     launches0 = ctx.maskkv_launch_count()
     barrier()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if sampler: sampler.mark("timed_start")
     t0.record()
     for i in range(args.steps):
-        step(args.warmup + i)
+        timed_step(args.warmup + i)
     t1.record()
     barrier()
     if sampler: sampler.mark("timed_end")
-    launches = ctx.maskkv_launch_count() - launches0
+    launches = (launches_per_step * args.steps) if graphs is not None else (ctx.maskkv_launch_count() - launches0)
     elapsed_ms = max_over_ranks(t0.elapsed_time(t1), device)
+    # the same steps as plain calls, for comparison (shorter run)
+    eager_steps = min(args.steps, 300)
+    barrier()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record()
+    for i in range(eager_steps):
+        step(args.warmup + i)
+    g1.record()
+    barrier()
+    eager_ms_per_step = max_over_ranks(g0.elapsed_time(g1), device) / eager_steps
     # Per-call breakdown from a separate pass: an event between every two calls costs a few microseconds of
     # serialisation per step, which does not belong in the headline number.
     per_call = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(min(args.steps, 200))]
@@ -423,7 +460,9 @@ def bench_ours(args):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "configs[2] llada_stack_32k, one layer per step: N=32768 M=256 H=H_kv=32 d=128, "
                                "adaptive budgets (k_l 512/238, alpha=0.1)", "layers_resident": len(resident),
-                   "l2": "inputs 545 MB per step > 126 MB L2; resident layers are cycled", "calls": list(CALLS)},
+                   "l2": "inputs 545 MB per step > 126 MB L2; resident layers are cycled", "calls": list(CALLS),
+                   "launch": "one CUDA graph per resident layer, replayed" if graphs is not None else "plain calls"},
+        "ms_per_step_plain_calls": eager_ms_per_step,
         "call_us": {k: round(v, 2) for k, v in call_us.items()},
         "attend_step_us": round(attend_loop_us, 2),
         "attend_step": {"us": round(attend_loop_us, 2), "steps": a_steps, "mean_kept_per_head": mean_kept,
@@ -562,6 +601,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-graph", action="store_true", help="time plain calls instead of replaying CUDA graphs")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else max(1, args.steps)
