@@ -66,6 +66,7 @@ constexpr int kSelectCluster = 4;
 constexpr int kSelectRegThreads = 512;
 constexpr int kSelectRegWarps = kSelectRegThreads / 32;
 constexpr int kSelectKeysPerThread = 16;
+constexpr int kSelectRankMax = 256;                     // candidate lists up to this length are ranked by counting
 constexpr int kSelectRegKeys = kSelectCluster * kSelectRegThreads * kSelectKeysPerThread;
 
 // Sum over the cluster of 4 consecutive histogram bins owned by this thread.
@@ -217,6 +218,26 @@ select_kernel_reg(Shape sh, const float* __restrict__ scores, const int32_t* __r
         ncand += n_peer;
       }
       (void)own;
+      if (ncand <= kSelectRankMax) {
+        // A short list (the usual case: the threshold bin of an 11-bit digit over 32k keys holds tens of keys): the
+        // threshold is the candidate with fewer than `remaining` candidates above it and at least `remaining` at or
+        // above it - one pass of broadcast reads instead of two more histogram passes.
+        __syncthreads();                                   // the gathered list is complete
+        if (tid < ncand) {
+          const uint32_t mine = cand[tid];
+          uint32_t gt = 0, ge = 0;
+          for (int u = 0; u < ncand; ++u) {
+            const uint32_t c = cand[u];
+            gt += c > mine;
+            ge += c >= mine;
+          }
+          if (gt < remaining && remaining <= ge) { sh_digit = mine; sh_remaining = remaining - gt; }   // equal keys write equal values
+        }
+        __syncthreads();
+        prefix = sh_digit;
+        remaining = sh_remaining;
+        bits_left = 0;
+      }
 #pragma unroll 1
       while (bits_left > 0) {
         const int w2 = bits_left >= 11 ? 11 : bits_left;
