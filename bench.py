@@ -170,8 +170,8 @@ def run_layer(ctx, buf, x, live, k_l, alpha, events=None):
 
 
 # DRAM bytes (read + write) of one maskkv_score call at this workload, from the ncu capture summarised in
-# profiles/score_tc_llada32k_ncu.md: sweep 1 284.9 MB + sweep 2 284.5 MB (the key tensor is read once per sweep).
-SCORE_DRAM_TRAFFIC_BYTES = 569.4e6
+# profiles/score_tc_llada32k_ncu.md: sweep 1 279.6 MB + sweep 2 290.7 MB (the key tensor is read once per sweep).
+SCORE_DRAM_TRAFFIC_BYTES = 570.3e6
 
 
 def algorithmic_work(wl, mean_kept_per_head):
