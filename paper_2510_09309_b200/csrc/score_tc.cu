@@ -156,6 +156,18 @@ __device__ __forceinline__ void walker_init(Walker& w, const Shape& sh, int mode
   }
 }
 
+// rel = group * T + tile; the quotient almost always fits 32 bits, where the division is an order of magnitude cheaper
+__device__ __forceinline__ void split_group_tile(long long rel, int T, int& g, int& t) {
+  if (rel < 0x7fffffffLL) {
+    const unsigned r32 = (unsigned)rel, T32 = (unsigned)T;
+    g = (int)(r32 / T32);
+    t = (int)(r32 - (unsigned)g * T32);
+  } else {
+    g = (int)(rel / T);
+    t = (int)(rel % T);
+  }
+}
+
 __device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, Seg& s) {
   if (!w.reverse) {
     if (w.f >= w.f_end) return false;
@@ -170,8 +182,7 @@ __device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, Seg& s) 
     }
     const long long rel = w.f - w.base;
     s.r = w.r;
-    s.g = (int)(rel / s.T);
-    s.t = (int)(rel % s.T);
+    split_group_tile(rel, s.T, s.g, s.t);
     s.dir = 1;
     const long long room = w.f_end - w.f;
     s.len = (int)min((long long)(s.T - s.t), room);
@@ -193,8 +204,7 @@ __device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, Seg& s) 
   }
   const long long rel = last - w.base;
   s.r = w.r;
-  s.g = (int)(rel / s.T);
-  s.t = (int)(rel % s.T);
+  split_group_tile(rel, s.T, s.g, s.t);
   s.dir = -1;
   const long long room = w.f - w.f_end;
   s.len = (int)min((long long)(s.t + 1), room);
@@ -223,6 +233,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + S::kMiscOff);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base + S::kMiscOff + 4);
   pdl_launch_dependents();
+  if (threadIdx.x == 0) { prefetch_tmap(&map_q); prefetch_tmap(&map_kp); prefetch_tmap(&map_km); }   // kernel parameters
   block_setup(bars, 4, tmem_slot, abort_flag);
   pdl_wait();
   // sweep 2 counts finished mass partials per segment in seg_cnt; it reads them after this grid has ended
@@ -236,7 +247,6 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
   if (warp == 0) {
     if (lane == 0) {
-      prefetch_tmap(&map_q); prefetch_tmap(&map_kp); prefetch_tmap(&map_km);
       int kt_it = 0, q_it = 0;
       bool ok = true;
       while (ok && walker_next(wk, sh, s)) {
@@ -459,6 +469,7 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + S::kMiscOff);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base + S::kMiscOff + 4);
   pdl_launch_dependents();
+  if (threadIdx.x == 0) { prefetch_tmap(&map_q); prefetch_tmap(&map_kp); prefetch_tmap(&map_km); }   // kernel parameters
   block_setup(bars, 2, tmem_slot, abort_flag);
   pdl_wait();
   const uint32_t tmem_base = *tmem_slot;
@@ -477,7 +488,6 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
   if (warp == 0) {
     if (lane == 0) {
-      prefetch_tmap(&map_q); prefetch_tmap(&map_kp); prefetch_tmap(&map_km);
       int kt_it = 0, q_it = 0;
       bool ok = true;
       while (ok && walker_next(wk, sh, s)) {
