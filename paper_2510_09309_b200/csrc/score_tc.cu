@@ -6,12 +6,14 @@
 //
 //   sweep 1  score_stats_tc   queries on the TMEM lanes (A = 128-query tile, B = 128-key tile): the thread
 //                             that owns a lane owns a softmax row and keeps its running (max, sum of exp).
-//                             A unit covers 256 queries (two accumulators) x one chunk of key tiles and
-//                             yields one partial per row; a tiny kernel merges the partials into lse_i.
+//                             A unit covers 256 queries (two accumulators) x one run of key tiles and
+//                             yields one partial per row and CTA; sweep 2 merges the partials into lse_i when it
+//                             loads a query block.
 //   sweep 2  score_colsum_tc  keys on the TMEM lanes (A = 128-key tile, B = up to 256 queries): the owning
 //                             thread reads its key's logits against every query, forms
 //                             A_ij = 2^(s_ij*c - lse2_i) and sums over i in a register - the column sum
-//                             needs no cross-thread reduction.
+//                             needs no cross-thread reduction.  It also sums the attention masses; with several
+//                             query blocks per KV head a small kernel adds the blocks' column sums.
 //
 // Both kernels are persistent (one CTA per SM walks an equal, contiguous share of the sweep's tiles, its
 // TMA / MMA / epilogue pipelines running on across segment boundaries) and warp-specialised: warp 0 issues TMA loads (4-stage
