@@ -185,3 +185,24 @@ def test_attend_long_segments_shared_by_two_ctas(ctx, d, n_mask):
     assert np.abs(run.out.float().cpu().numpy() - out).max() <= ATTEND_ATOL["bf16"]
     assert np.abs(run.lse.cpu().numpy() - lse).max() <= 1e-3
     assert ctx.maskkv_check_status() == 0
+
+
+def test_compact_reads_prompt_values_from_pinned_host_memory(ctx):
+    """maskkv_compact is the path's only reader of v_prompt: a caller may leave the prompt values in pinned
+    (device-mapped) host memory and pass that pointer; only the kept rows cross the bus."""
+    wl = synth.scaled(synth.config(2), "host_values", dtype="bf16", prompt_lens=(3000, 700), n_mask=64, n_q_heads=4,
+                      n_kv_heads=4, head_dim=128, mean_budget=200)
+    x = synth.layer_inputs(wl, 0, "cpu")
+    xd = {k: to_dev(v) for k, v in x.items() if torch.is_tensor(v)}
+    run = LayerRun(ctx, wl)
+    run.score(xd); run.budget(); run.select(); run.compact(xd)
+    torch.cuda.synchronize()
+    kc_dev, vc_dev = run.kc.clone(), run.vc.clone()
+    run.kc.zero_(); run.vc.zero_()
+    host = dict(xd)
+    host["v_prompt"] = x["v_prompt"].to(wl.torch_dtype).pin_memory()          # stays on the host
+    host["k_prompt"] = x["k_prompt"].to(wl.torch_dtype).pin_memory()
+    run.compact(host)
+    torch.cuda.synchronize()
+    assert torch.equal(run.kc, kc_dev) and torch.equal(run.vc, vc_dev)
+    assert ctx.maskkv_check_status() == 0
