@@ -284,6 +284,33 @@ def bench_ours(args):
         step(args.warmup + i, ev)
     barrier()
     mean_kept = float(buf.offsets[-1].item()) / wl.n_kv_heads
+    # maskkv_score alone, launched the way the timed steps launch it (graph replays cycling the resident layers): the
+    # duration the roofline objects use
+    score_us = None
+    if graphs is not None:
+        side2 = torch.cuda.Stream(device=device)
+        side2.wait_stream(torch.cuda.current_stream())
+        sgraphs = []
+        with torch.cuda.stream(side2):
+            for j in range(len(resident)):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side2):
+                    ctx.maskkv_score(buf.p, inputs[j]["q_mask"], inputs[j]["k_prompt"], inputs[j]["k_mask"], buf.scores,
+                                     buf.mass_p, buf.mass_m, buf.ws)
+                sgraphs.append(g)
+        torch.cuda.current_stream().wait_stream(side2)
+        for g in sgraphs:
+            g.replay()
+        barrier()
+        s_steps = min(args.steps, 400)
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for i in range(s_steps):
+            sgraphs[i % len(resident)].replay()
+        s1.record()
+        barrier()
+        score_us = 1e3 * max_over_ranks(s0.elapsed_time(s1), device) / s_steps
+        del sgraphs
     call_us = {name: 1e3 * statistics.mean(ev[c].elapsed_time(ev[c + 1]) for ev in per_call) for c, name in enumerate(CALLS)}
     # ---- the later denoising steps: maskkv_attend alone, back to back, as the per-step loop of a layer would issue it.
     # The compacted cache is cloned until the copies exceed twice the L2, and the loop cycles through them.
@@ -441,7 +468,7 @@ def bench_ours(args):
     value = world * N / (ms_per_step * 1e-3)
     peaks = load_peaks()
     work = algorithmic_work(wl, mean_kept)
-    score_s = call_us["score"] * 1e-6
+    score_s = (score_us if score_us is not None else call_us["score"]) * 1e-6
     achieved_tf = work["score_flops"] / score_s / 1e12
     peak_tf = peaks["bf16_tflops_sustained"]
     hbm = peaks["hbm_gbs"]
@@ -474,11 +501,12 @@ def bench_ours(args):
         "gpu_launches": int(launches),
         "clocks": clocks,
         "status_flags": flags,
-        "roofline": {"kernel": "maskkv_score (all its kernels; one Q K^T product counted)", "bound": "tensor",
+        "roofline": {"kernel": "maskkv_score (its two kernels, replayed alone; one Q K^T product counted)", "bound": "tensor",
                      "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
                      "peak_source": peaks["source"] + " (sustained bf16; the kernels run inside a long step)",
                      "traffic": SCORE_DRAM_TRAFFIC_BYTES, "executed_over_algorithmic_flops": 2.0},
-        "roofline_alu": exp_roofline(wl, call_us["score"], clocks.get("sm_max_mhz") or 1965.0),
+        "roofline_alu": exp_roofline(wl, score_s * 1e6, clocks.get("sm_max_mhz") or 1965.0),
+        "score_us": round(score_s * 1e6, 2),
         "roofline_other_calls": other,
         "mean_kept_per_head": mean_kept,
     }
