@@ -237,7 +237,8 @@ int maskkv_create(maskkv_ctx** out, int device) {
   if (const char* e = getenv("MASKKV_FORCE_SIMT")) ctx->force_simt = (unsigned)strtoul(e, nullptr, 0);
   cudaFuncSetAttribute(mkv::select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - mkv::kSelectStaticSmem);
   cudaFuncSetAttribute(mkv::budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-  cudaFuncSetAttribute(mkv::select_kernel_reg, cudaFuncAttributeMaxDynamicSharedMemorySize, mkv::kSelectRegKeys * 4);
+  cudaFuncSetAttribute(mkv::select_kernel_reg<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, mkv::kSelectCandCap * 4);
+  cudaFuncSetAttribute(mkv::select_kernel_reg<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, mkv::kSelectCandCap * 4);
   if (cudaGetLastError() != cudaSuccess) { cudaFree(ctx->status_dev); free(ctx); return MASKKV_E_CUDA; }
   *out = ctx;
   return MASKKV_OK;
@@ -457,9 +458,11 @@ int maskkv_select(maskkv_ctx* ctx, const maskkv_desc_t* desc, const float* score
   if (scores_dev == nullptr || budgets_dev == nullptr || offsets_dev == nullptr || kept_idx_dev == nullptr) return MASKKV_E_INVALID;
   DeviceGuard guard(ctx->device);
   if (sh.maxN <= mkv::kSelectRegKeys) {                  // every segment fits the register-resident kernel
-    mkv::launch_overlapped(mkv::select_kernel_reg, dim3(sh.R * sh.Hkv * mkv::kSelectCluster), dim3(mkv::kSelectRegThreads),
-                           (size_t)mkv::kSelectRegKeys * 4, static_cast<cudaStream_t>(stream), sh, scores_dev, budgets_dev, offsets_dev,
-                           kept_idx_dev, ctx->status_dev);
+    // one wave of clusters (4 CTAs each, one CTA per SM): the leaner-latency variant; more segments: two CTAs per SM
+    const bool one_wave = (long long)sh.R * sh.Hkv * mkv::kSelectCluster <= ctx->sm_count;
+    mkv::launch_overlapped(one_wave ? mkv::select_kernel_reg<1> : mkv::select_kernel_reg<2>, dim3(sh.R * sh.Hkv * mkv::kSelectCluster),
+                           dim3(mkv::kSelectRegThreads), (size_t)mkv::kSelectCandCap * 4, static_cast<cudaStream_t>(stream), sh, scores_dev,
+                           budgets_dev, offsets_dev, kept_idx_dev, ctx->status_dev);
     return launch_status(ctx, 1);
   }
   const int max_cache = (ctx->smem_optin - mkv::kSelectStaticSmem) / 4;

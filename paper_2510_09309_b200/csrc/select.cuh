@@ -66,6 +66,7 @@ constexpr int kSelectCluster = 4;
 constexpr int kSelectRegThreads = 512;
 constexpr int kSelectRegWarps = kSelectRegThreads / 32;
 constexpr int kSelectKeysPerThread = 16;
+constexpr int kSelectCandCap = kSelectRegThreads * kSelectKeysPerThread;   // candidate list a CTA holds: its own keys at most, or all CTAs' when they fit
 constexpr int kSelectRankMax = 256;                     // candidate lists up to this length are ranked by counting
 constexpr int kSelectRegKeys = kSelectCluster * kSelectRegThreads * kSelectKeysPerThread;
 
@@ -102,8 +103,11 @@ __device__ __forceinline__ void find_digit_counts(const uint32_t* c, uint32_t re
   __syncthreads();
 }
 
-// grid = 4 * segments (cluster of 4 per segment); dynamic shared memory: uint32 cand[kSelectRegKeys]
-__global__ void __cluster_dims__(kSelectCluster, 1, 1) __launch_bounds__(kSelectRegThreads, 1)
+// grid = 4 * segments (cluster of 4 per segment); dynamic shared memory: uint32 cand[kSelectCandCap].
+// BLOCKS = CTAs per SM the register budget allows: 1 (94 registers, the fastest single chain: one layer's 32 segments
+// all run at once) or 2 (64 registers, twice the segments in flight: batches).
+template <int BLOCKS>
+__global__ void __cluster_dims__(kSelectCluster, 1, 1) __launch_bounds__(kSelectRegThreads, BLOCKS)
 select_kernel_reg(Shape sh, const float* __restrict__ scores, const int32_t* __restrict__ budgets,
                   const int32_t* __restrict__ offsets, int32_t* __restrict__ kept_idx, uint32_t* __restrict__ status) {
   namespace cg = cooperative_groups;
@@ -209,16 +213,44 @@ select_kernel_reg(Shape sh, const float* __restrict__ scores, const int32_t* __r
       // search on its own: the same list in a different order gives the same histogram, hence the same threshold.
       int ncand = (int)sh_ncand;
       const int own = ncand;
+      int n_peer[kSelectCluster], total = own;
 #pragma unroll
       for (int c = 1; c < kSelectCluster; ++c) {
-        const int peer = (q + c) & (kSelectCluster - 1);
-        const int n_peer = (int)*cluster.map_shared_rank(&sh_ncand, peer);
-        const uint32_t* src = cluster.map_shared_rank(cand, peer);
-        for (int t = tid; t < n_peer; t += kSelectRegThreads) cand[ncand + t] = src[t];
-        ncand += n_peer;
+        n_peer[c] = (int)*cluster.map_shared_rank(&sh_ncand, (q + c) & (kSelectCluster - 1));
+        total += n_peer[c];
       }
-      (void)own;
-      if (ncand <= kSelectRankMax) {
+      if (total > kSelectCandCap) {
+        // Too many keys share the threshold bin (nearly equal scores) for every CTA to hold them all: the lists stay
+        // where they are and the remaining digits are found like the first one, with histograms summed over the cluster.
+#pragma unroll 1
+        while (bits_left > 0) {
+          const int w2 = bits_left >= 11 ? 11 : bits_left;
+          const int sh2 = bits_left - w2;
+          const uint32_t dm2 = (1u << w2) - 1u;
+          for (int b2 = tid; b2 < 2048; b2 += kSelectRegThreads) hist[b2] = 0;
+          __syncthreads();
+          for (int t = tid; t < own; t += kSelectRegThreads) {
+            const uint32_t c = cand[t];
+            if ((c & have_mask) == prefix) atomicAdd(&hist[(c >> sh2) & dm2], 1u);
+          }
+          cluster.sync();
+          cluster_bins(cluster, hist, tid, cnt4);
+          find_digit_counts(cnt4, remaining, warp_tot, &sh_digit, &sh_remaining);
+          prefix |= sh_digit << sh2;
+          remaining = sh_remaining;
+          have_mask |= dm2 << sh2;
+          bits_left = sh2;
+          cluster.sync();                                  // every peer has read this histogram before it is cleared again
+        }
+      } else {
+#pragma unroll
+        for (int c = 1; c < kSelectCluster; ++c) {
+          const uint32_t* src = cluster.map_shared_rank(cand, (q + c) & (kSelectCluster - 1));
+          for (int t = tid; t < n_peer[c]; t += kSelectRegThreads) cand[ncand + t] = src[t];
+          ncand += n_peer[c];
+        }
+      }
+      if (bits_left > 0 && ncand <= kSelectRankMax) {
         // A short list (the usual case: the threshold bin of an 11-bit digit over 32k keys holds tens of keys): the
         // threshold is the candidate with fewer than `remaining` candidates above it and at least `remaining` at or
         // above it - one pass of broadcast reads instead of two more histogram passes.

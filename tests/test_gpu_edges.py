@@ -206,3 +206,31 @@ def test_compact_reads_prompt_values_from_pinned_host_memory(ctx):
     torch.cuda.synchronize()
     assert torch.equal(run.kc, kc_dev) and torch.equal(run.vc, vc_dev)
     assert ctx.maskkv_check_status() == 0
+
+
+def test_select_in_registers_crowded_threshold_bin_and_ties(ctx):
+    """Segments of at most 32768 keys take the register-resident cluster kernel.  Cases: most keys inside one bin of the
+    first radix digit with the cut inside that bin (the candidate lists do not fit one CTA: digits are then found with
+    cluster-summed histograms), the same with exact ties at the cut, a short candidate list (ranked by counting), NaNs,
+    and tiny segments next to full ones."""
+    lens = [32768, 30001, 7, 32768]
+    p, pcu, _ = _problem(ctx, torch.bfloat16, 2, 2, 64, lens, 4)
+    rng = np.random.default_rng(11)
+    sc = rng.random((2, pcu[-1])).astype(np.float32) * 8.0                  # spread over several octaves
+    # request 0, head 0: 24000 keys packed into [1.5, 1.5 + 2^-11) (one bin of the first digit), random low bits
+    crowd = (1.5 + rng.integers(0, 1 << 12, 24000) * 2.0 ** -23).astype(np.float32)
+    pos = rng.permutation(32768)[:24000]
+    sc[0, pos] = crowd
+    # request 0, head 1: the same crowd collapsed onto four values (thousands of exact ties at the cut)
+    sc[1, pos] = (1.5 + rng.integers(0, 4, 24000) * 2.0 ** -23).astype(np.float32)
+    # request 1: ordinary scores with a few NaNs and infinities
+    a = pcu[1]
+    sc[0, a + 5] = np.nan; sc[0, a + 17] = np.inf; sc[1, a + 3] = -np.inf; sc[1, a + 9] = np.nan
+    bud = np.array([[15000, 15000], [300, 29999], [3, 7], [1, 32768]], np.int32)
+    idx, off = O.select(sc, bud, pcu)
+    kept = torch.full((int(off[-1]) + 8,), -1, dtype=torch.int32, device=ctx.device)
+    ctx.maskkv_select(p, to_dev(sc), to_dev(bud), to_dev(off), kept)
+    torch.cuda.synchronize()
+    assert np.array_equal(kept[:int(off[-1])].cpu().numpy(), idx)
+    assert (kept[int(off[-1]):] == -1).all()
+    assert ctx.maskkv_check_status() == 0
