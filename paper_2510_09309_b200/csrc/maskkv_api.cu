@@ -71,7 +71,7 @@ int resolve(const maskkv_desc_t* d, Shape* sh) {
 }
 
 struct ScoreWorkspace {
-  size_t lse_off, part_off, mass_off, cnt_off, base_off, col_off, total;
+  size_t lse_off, part_off, mass_off, cnt_off, col_off, total;
   int C, Tmax;
 };
 
@@ -88,7 +88,6 @@ ScoreWorkspace score_workspace(const maskkv_ctx* ctx, const Shape& sh) {
   w.part_off = off; off = align_up(off + sizeof(float2) * (size_t)sh.H * sh.sumM * w.C, 256);
   w.mass_off = off; off = align_up(off + sizeof(float2) * (size_t)sh.R * sh.Hkv * w.Tmax * 8, 256);
   w.cnt_off = off;  off = align_up(off + sizeof(uint32_t) * (size_t)sh.R * sh.Hkv, 256);
-  w.base_off = off; off = align_up(off + sizeof(long long) * ((size_t)sh.R + 1), 256);
   w.col_off = off;  off = align_up(off + mkv::tc::score_tc_colpart_bytes(sh), 256);   // per-block column sums (grouped heads)
   w.total = off;
   return w;
@@ -112,7 +111,6 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, co
   float2* part = reinterpret_cast<float2*>(ws + w.part_off);
   float2* mass_part = reinterpret_cast<float2*>(ws + w.mass_off);
   uint32_t* seg_cnt = reinterpret_cast<uint32_t*>(ws + w.cnt_off);
-  long long* unit_base = reinterpret_cast<long long*>(ws + w.base_off);
   const int S = sh.R * sh.Hkv;
   const bool tc_ok = mkv::tc::score_tc_supported(ctx, sh);
   const bool want_tc2 = tc_ok && !(ctx->force_simt & 2u);
@@ -120,7 +118,7 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, co
   bool tc1 = false;                                          // sweep 1 ran on the tensor cores: `part` has its layout
   if (sh.sumM > 0) {
     if (tc_ok && !(ctx->force_simt & 1u))
-      tc1 = mkv::tc::launch_score_stats_tc(ctx, sh, desc->prompt_cu, desc->live_cu, q, kp, km, part, w.C, seg_cnt, unit_base, st) == 0;
+      tc1 = mkv::tc::launch_score_stats_tc(ctx, sh, desc->prompt_cu, desc->live_cu, q, kp, km, part, w.C, seg_cnt, st) == 0;
     if (tc1) { ++ctx->tc_launches; ++n; }
     if (!tc1) {
       const int q_tiles = (sh.maxM + mkv::kSimtThreads - 1) / mkv::kSimtThreads;
@@ -137,7 +135,7 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, co
     // after a tensor-core sweep 1 the kernel merges the partials itself; otherwise it reads lse
     int launched = 0;
     float* colpart = reinterpret_cast<float*>(ws + w.col_off);
-    tc2 = mkv::tc::launch_score_colsum_tc(ctx, sh, desc->prompt_cu, desc->live_cu, q, kp, km, lse, tc1 ? part : nullptr, w.C, unit_base, rw,
+    tc2 = mkv::tc::launch_score_colsum_tc(ctx, sh, desc->prompt_cu, desc->live_cu, q, kp, km, lse, tc1 ? part : nullptr, w.C, rw,
                                           scores, colpart, mass_part, w.Tmax, seg_cnt, mass_p, mass_m, any_without_voters, st,
                                           &launched) == 0;
     if (tc2) {
@@ -150,7 +148,7 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, co
     }
   }
   if (!tc2) {
-    if (tc1) { mkv::tc::launch_score_merge_tc(ctx, sh, desc->prompt_cu, desc->live_cu, part, w.C, unit_base, lse, st); ++n; }
+    if (tc1) { mkv::tc::launch_score_merge_tc(ctx, sh, desc->prompt_cu, desc->live_cu, part, w.C, lse, st); ++n; }
     dim3 g2(w.Tmax, sh.Hkv, sh.R);
     mkv::score_colsum_simt<T, D><<<g2, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, lse, rw,
                                                                     scores, mass_part, w.Tmax);

@@ -227,7 +227,7 @@ template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kp,
                const __grid_constant__ CUtensorMap map_km, Shape sh, float2* __restrict__ part, int C, long long F,
-               uint32_t* __restrict__ seg_cnt, long long* __restrict__ unit_base, uint32_t* __restrict__ status) {
+               uint32_t* __restrict__ seg_cnt, uint32_t* __restrict__ status) {
   using S = Smem<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = align_1024(smem_raw);
@@ -241,19 +241,6 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // sweep 2 counts finished mass partials per segment in seg_cnt; it reads them after this grid has ended
   if (blockIdx.x == 0 && seg_cnt != nullptr)
     for (int i = threadIdx.x; i < sh.R * sh.Hkv; i += blockDim.x) seg_cnt[i] = 0u;
-  // unit_base[r] = flat index of request r's first tile in this sweep's walk: sweep 2 needs it to find a row's partials
-  if (blockIdx.x == 0 && unit_base != nullptr) {
-    for (int r = threadIdx.x; r < sh.R; r += blockDim.x) {
-      const int N = sh.prompt_cu[r + 1] - sh.prompt_cu[r], M = sh.live_cu[r + 1] - sh.live_cu[r];
-      unit_base[r + 1] = (long long)walk_groups(sh, kWalkStats, M) * tiles_of(N, M);
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      long long acc = 0;
-      unit_base[0] = 0;
-      for (int r = 0; r < sh.R; ++r) { acc += unit_base[r + 1]; unit_base[r + 1] = acc; }
-    }
-  }
   const uint32_t tmem_base = *tmem_slot;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   Walker wk;
@@ -415,8 +402,12 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 // ln sum_j exp(s_j) of query row `row` (index over all requests) of head h, which lies in 256-query block `qblock` of
 // request r: log-sum-exp merge of the partials the CTAs of sweep 1 left.  F1, G1: flat tile count and grid of sweep 1.
 __device__ __noinline__ float merged_lse(const Shape& sh, const float2* __restrict__ part, int C, long long F1, int G1,
-                                            const long long* __restrict__ unit_base, int r, int h, int qblock, int row) {
-  const long long base = unit_base[r];
+                                            int r, int h, int qblock, int row) {
+  long long base = 0;
+  for (int r2 = 0; r2 < r; ++r2) {
+    const int N2 = sh.prompt_cu[r2 + 1] - sh.prompt_cu[r2], M2 = sh.live_cu[r2 + 1] - sh.live_cu[r2];
+    base += (long long)walk_groups(sh, kWalkStats, M2) * tiles_of(N2, M2);
+  }
   const int N = sh.prompt_cu[r + 1] - sh.prompt_cu[r], M = sh.live_cu[r + 1] - sh.live_cu[r];
   const int T = tiles_of(N, M), qp_n = (M + kQBlock - 1) / kQBlock;
   const long long unit_start = base + ((long long)h * qp_n + qblock) * T;
@@ -443,12 +434,12 @@ __device__ __noinline__ float merged_lse(const Shape& sh, const float2* __restri
 // One thread per (h, row): lse[h*sumM + row].  Only launched when sweep 2 does not run on the tensor-core kernel
 // (which merges the partials itself).
 __global__ void score_merge_stats_tc(Shape sh, const float2* __restrict__ part, int C, long long F, int G,
-                                     const long long* __restrict__ unit_base, float* __restrict__ lse) {
+                                     float* __restrict__ lse) {
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= (long long)sh.H * sh.sumM) return;
   const int h = (int)(t / sh.sumM), row = (int)(t % sh.sumM);
   const int r = find_request(sh.live_cu, sh.R, row);
-  lse[t] = merged_lse(sh, part, C, F, G, unit_base, r, h, (row - sh.live_cu[r]) / kQBlock, row);
+  lse[t] = merged_lse(sh, part, C, F, G, r, h, (row - sh.live_cu[r]) / kQBlock, row);
 }
 
 // =====================================================================================================
@@ -468,7 +459,7 @@ template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kp,
                 const __grid_constant__ CUtensorMap map_km, Shape sh, const float* __restrict__ lse,
-                const float2* __restrict__ part, int C, long long F1, int G1, const long long* __restrict__ unit_base,
+                const float2* __restrict__ part, int C, long long F1, int G1,
                 const float* __restrict__ w, float* __restrict__ scores, float* __restrict__ colpart,
                 float2* __restrict__ mass_part, int Tmax, uint32_t* __restrict__ seg_cnt, float* __restrict__ mass_p,
                 float* __restrict__ mass_m, long long F, uint32_t* __restrict__ status) {
@@ -631,7 +622,7 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         float cst = -INFINITY;                              // 2^(x - inf) = 0: rows that do not exist never vote
         if (row < nq) {
           const int i = s.l0 + qh0 + row;
-          const float ln_z = part != nullptr ? merged_lse(sh, part, C, F1, G1, unit_base, s.r, h, q0 / kQBlock, i)
+          const float ln_z = part != nullptr ? merged_lse(sh, part, C, F1, G1, s.r, h, q0 / kQBlock, i)
                                              : lse[(long long)h * sh.sumM + i];
           cst = (w ? log2f(w[i]) : 0.f) - ln_z * kLog2e;
         }
@@ -786,8 +777,7 @@ bool score_tc_supported(const maskkv_ctx* ctx, const Shape& sh) {
 }
 
 int launch_score_stats_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prompt_cu_host, const int32_t* live_cu_host,
-                          const void* q, const void* kp, const void* km, float2* part, int C, uint32_t* seg_cnt, long long* unit_base,
-                          cudaStream_t st) {
+                          const void* q, const void* kp, const void* km, float2* part, int C, uint32_t* seg_cnt, cudaStream_t st) {
   Maps m;
   if (!build_maps(ctx, sh, q, kp, km, &m)) return 1;
   const long long F = flat_tiles(sh, prompt_cu_host, live_cu_host, kWalkStats);
@@ -796,21 +786,21 @@ int launch_score_stats_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* promp
   if (sh.d == 128) {
     if (set_smem_attr<128>() != cudaSuccess) return 1;
     launch_overlapped(score_stats_tc<128>, dim3(grid), dim3(kThreads), Smem<128>::kDynamic, st, m.q, m.kp, m.km, sh, part, C, F, seg_cnt,
-                      unit_base, ctx->status_dev);
+                      ctx->status_dev);
   } else {
     if (set_smem_attr<64>() != cudaSuccess) return 1;
     launch_overlapped(score_stats_tc<64>, dim3(grid), dim3(kThreads), Smem<64>::kDynamic, st, m.q, m.kp, m.km, sh, part, C, F, seg_cnt,
-                      unit_base, ctx->status_dev);
+                      ctx->status_dev);
   }
   return 0;
 }
 
 void launch_score_merge_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prompt_cu_host, const int32_t* live_cu_host,
-                           const float2* part, int C, const long long* unit_base, float* lse, cudaStream_t st) {
+                           const float2* part, int C, float* lse, cudaStream_t st) {
   const long long F = flat_tiles(sh, prompt_cu_host, live_cu_host, kWalkStats);
   const int grid = (int)(F < ctx->sm_count ? F : ctx->sm_count);
   const long long rows = (long long)sh.H * sh.sumM;
-  score_merge_stats_tc<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(sh, part, C, F, grid, unit_base, lse);
+  score_merge_stats_tc<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(sh, part, C, F, grid, lse);
 }
 
 bool score_tc_split_blocks(const Shape& sh) { return sh.g > 1 || sh.maxM > kQBlock; }
@@ -823,8 +813,8 @@ size_t score_tc_colpart_bytes(const Shape& sh) {
 
 int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prompt_cu_host, const int32_t* live_cu_host,
                            const void* q, const void* kp, const void* km, const float* lse, const float2* part, int C,
-                           const long long* unit_base, const float* w, float* scores, float* colpart, float2* mass_part, int Tmax,
-                           uint32_t* seg_cnt, float* mass_p, float* mass_m, bool any_without_voters, cudaStream_t st, int* launches) {
+                           const float* w, float* scores, float* colpart, float2* mass_part, int Tmax, uint32_t* seg_cnt,
+                           float* mass_p, float* mass_m, bool any_without_voters, cudaStream_t st, int* launches) {
   Maps m;
   if (!build_maps(ctx, sh, q, kp, km, &m)) return 1;
   const bool split = score_tc_split_blocks(sh);
@@ -844,10 +834,10 @@ int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prom
   float* cp = split ? colpart : nullptr;
   if (sh.d == 128)
     launch_overlapped(score_colsum_tc<128>, dim3(grid), dim3(kThreads), Smem<128>::kDynamic, st, m.q, m.kp, m.km, sh, lse, part, C, F1, G1,
-                      unit_base, w, scores, cp, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
+                      w, scores, cp, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
   else
     launch_overlapped(score_colsum_tc<64>, dim3(grid), dim3(kThreads), Smem<64>::kDynamic, st, m.q, m.kp, m.km, sh, lse, part, C, F1, G1,
-                      unit_base, w, scores, cp, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
+                      w, scores, cp, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
   ++*launches;
   if (split) {
     dim3 gr(Tmax, sh.Hkv, sh.R);
