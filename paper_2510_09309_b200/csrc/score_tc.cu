@@ -399,26 +399,19 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   block_teardown(tmem_base);
 }
 
-// ln sum_j exp(s_j) of query row `row` (index over all requests) of head h, which lies in 256-query block `qblock` of
-// request r: log-sum-exp merge of the partials the CTAs of sweep 1 left.  F1, G1: flat tile count and grid of sweep 1.
-__device__ __noinline__ float merged_lse(const Shape& sh, const float2* __restrict__ part, int C, long long F1, int G1,
-                                            int r, int h, int qblock, int row) {
-  long long base = 0;
-  for (int r2 = 0; r2 < r; ++r2) {
-    const int N2 = sh.prompt_cu[r2 + 1] - sh.prompt_cu[r2], M2 = sh.live_cu[r2 + 1] - sh.live_cu[r2];
-    base += (long long)walk_groups(sh, kWalkStats, M2) * tiles_of(N2, M2);
-  }
-  const int N = sh.prompt_cu[r + 1] - sh.prompt_cu[r], M = sh.live_cu[r + 1] - sh.live_cu[r];
-  const int T = tiles_of(N, M), qp_n = (M + kQBlock - 1) / kQBlock;
-  const long long unit_start = base + ((long long)h * qp_n + qblock) * T;
-  const int slots = 2 * (cta_of(unit_start + T - 1, F1, G1) - cta_of(unit_start, F1, G1) + 1);
-  const float2* p = part + (long long)h * C * sh.sumM + row;      // slot c at p[c * sumM]
+// ln sum_j exp(s_j) of query row `row` (index over all requests) of head h: log-sum-exp merge of the partials the CTAs
+// of sweep 1 left for the row's unit, which starts at flat tile `unit_start` of that sweep's walk and has T tiles.
+// F, G: flat tile count and grid of sweep 1.
+__device__ __noinline__ float merged_lse(const float2* __restrict__ part, int C, int sumM, long long F, int G,
+                                            long long unit_start, int T, int h, int row) {
+  const int slots = 2 * (cta_of(unit_start + T - 1, F, G) - cta_of(unit_start, F, G) + 1);
+  const float2* p = part + (long long)h * C * sumM + row;         // slot c at p[c * sumM]
   // the loads of a batch are issued together (a row has 4 to 8 partials on a long prompt)
   float m = -INFINITY, l = 0.f;
   for (int c0 = 0; c0 < slots; c0 += 8) {
     float2 v[8];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) v[k] = c0 + k < slots ? p[(long long)(c0 + k) * sh.sumM] : make_float2(-INFINITY, 0.f);
+    for (int k = 0; k < 8; ++k) v[k] = c0 + k < slots ? p[(long long)(c0 + k) * sumM] : make_float2(-INFINITY, 0.f);
     float bm = m;
 #pragma unroll
     for (int k = 0; k < 8; ++k) bm = fmaxf(bm, v[k].x);
@@ -439,7 +432,14 @@ __global__ void score_merge_stats_tc(Shape sh, const float2* __restrict__ part, 
   if (t >= (long long)sh.H * sh.sumM) return;
   const int h = (int)(t / sh.sumM), row = (int)(t % sh.sumM);
   const int r = find_request(sh.live_cu, sh.R, row);
-  lse[t] = merged_lse(sh, part, C, F, G, r, h, (row - sh.live_cu[r]) / kQBlock, row);
+  long long base = 0;
+  for (int r2 = 0; r2 < r; ++r2) {
+    const int N2 = sh.prompt_cu[r2 + 1] - sh.prompt_cu[r2], M2 = sh.live_cu[r2 + 1] - sh.live_cu[r2];
+    base += (long long)walk_groups(sh, kWalkStats, M2) * tiles_of(N2, M2);
+  }
+  const int N = sh.prompt_cu[r + 1] - sh.prompt_cu[r], l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
+  const int T = tiles_of(N, M), qp_n = (M + kQBlock - 1) / kQBlock;
+  lse[t] = merged_lse(part, C, sh.sumM, F, G, base + ((long long)h * qp_n + (row - l0) / kQBlock) * T, T, h, row);
 }
 
 // =====================================================================================================
@@ -481,6 +481,9 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   walker_init(wk, sh, split ? kWalkColsumSplit : kWalkColsum, true, F);
   Seg s;
   int last_r = -1, last_g = -1;                             // the (request, group) whose queries are resident
+  // Both walks of sweep 2 number their tiles exactly like sweep 1 (KV heads = query heads x blocks when there is one
+  // block per KV head; the same (query head, block) groups otherwise), so a run's unit_start is also the flat index at
+  // which sweep 1 started the rows' unit: that is all the merge of its partials needs.
   // group of a run -> query head, KV head, first query of the block, index of the block among the KV head's blocks
   auto unit_of = [&](const Seg& sg, int& h, int& hk, int& q0, int& blk) {
     if (!split) { h = hk = sg.g; q0 = 0; blk = 0; return; }
@@ -622,7 +625,7 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         float cst = -INFINITY;                              // 2^(x - inf) = 0: rows that do not exist never vote
         if (row < nq) {
           const int i = s.l0 + qh0 + row;
-          const float ln_z = part != nullptr ? merged_lse(sh, part, C, F1, G1, s.r, h, q0 / kQBlock, i)
+          const float ln_z = part != nullptr ? merged_lse(part, C, sh.sumM, F1, G1, s.unit_start, s.T, h, i)
                                              : lse[(long long)h * sh.sumM + i];
           cst = (w ? log2f(w[i]) : 0.f) - ln_z * kLog2e;
         }
