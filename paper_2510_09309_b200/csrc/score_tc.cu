@@ -216,7 +216,11 @@ __device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, Seg& s) 
 }
 
 // CTA whose share contains flat tile f.
-__host__ __device__ __forceinline__ int cta_of(long long f, long long F, int G) { return (int)(((f + 1) * G - 1) / F); }
+__host__ __device__ __forceinline__ int cta_of(long long f, long long F, int G) {
+  const long long num = (f + 1) * G - 1;
+  if (num < 0x7fffffffLL && F < 0x7fffffffLL) return (int)((unsigned)num / (unsigned)F);   // the usual case, a cheap division
+  return (int)(num / F);
+}
 
 // =====================================================================================================
 // sweep 1: per-row (max, sum of exp) over a segment of key tiles.
