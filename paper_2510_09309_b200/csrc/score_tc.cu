@@ -420,12 +420,13 @@ __device__ __noinline__ float merged_lse(const float2* __restrict__ part, int C,
 #pragma unroll
     for (int k = 0; k < 8; ++k) bm = fmaxf(bm, v[k].x);
     if (bm == -INFINITY) continue;
-    l *= expf(m - bm);
+    // special-function exponentials and logarithm (relative error 2^-22): the epilogue waits for this value
+    l *= ex2((m - bm) * kLog2e);
 #pragma unroll
-    for (int k = 0; k < 8; ++k) l += v[k].y * expf(v[k].x - bm);
+    for (int k = 0; k < 8; ++k) l += v[k].y * ex2((v[k].x - bm) * kLog2e);
     m = bm;
   }
-  return m + logf(l);
+  return m + __log2f(l) * 0.6931471805599453f;
 }
 
 // One thread per (h, row): lse[h*sumM + row].  Only launched when sweep 2 does not run on the tensor-core kernel
