@@ -33,6 +33,7 @@ constexpr int kEpiThreadsPerAcc = 256; // two epilogue warpgroups share one accu
 constexpr int kStages = 4;
 constexpr int kTile = 128;             // keys per tile (both sweeps), queries per accumulator (sweep 1)
 constexpr int kQBlock = 256;           // queries resident per CTA
+constexpr int kColsumPad = 3;          // sweep 2: what entering a new unit costs a CTA, in key tiles (see Walker)
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int D>
@@ -121,15 +122,20 @@ __device__ __forceinline__ void block_teardown(uint32_t tmem_base) {
 // contiguous share [c*F/G, (c+1)*F/G) of the F tiles - every CTA gets the same number of tiles to within one -
 // and walks it one segment (a run of tiles of one group) at a time.  Every role of the CTA runs the same walk.
 // =====================================================================================================
-struct Seg { int r, g, t, len, p0, N, l0, M, T, dir; long long unit_start; };   // tiles t, t+dir, ..., len of them
+// tiles t, t+dir, ..., len of them; unit_start = flat index of the unit's first position in this walk (padding included),
+// unit_real = the same without any padding (the index sweep 1's walk gives the unit)
+struct Seg { int r, g, t, len, p0, N, l0, M, T, dir; long long unit_start, unit_real; };
 
 // mode of a walk: sweep 1 (groups = query head x 256-query block), sweep 2 with one query block per KV head (groups =
 // KV heads), sweep 2 with several (groups = query head x block again; the blocks' column sums meet in a later kernel)
 enum { kWalkStats = 0, kWalkColsum = 1, kWalkColsumSplit = 2 };
 
+// `pad`: positions without work put in front of every unit's tiles (sweep 2 only).  Crossing into a new unit costs a CTA
+// about as much as `pad` tiles (new queries, the merge of their normalisers, the hand-over of the attention mass), and
+// the shares are equal in positions, so a share that contains a unit boundary gets that many tiles fewer.
 struct Walker {
-  long long f, f_end, base;   // forward: [f, f_end) still to do; reverse: [f_end, f) still to do, taken from the top
-  int r, mode;
+  long long f, f_end, base, base_real;   // forward: [f, f_end) still to do; reverse: [f_end, f) still to do, taken from the top
+  int r, mode, pad;
   bool reverse;
 };
 
@@ -140,20 +146,24 @@ __device__ __forceinline__ int tiles_of(int N, int M) { return (N + kTile - 1) /
 
 // Sweep 2 walks every share backwards: it then starts on the tiles sweep 1 read last, which are the ones most
 // likely to be still in L2 (the key tensor of a long prompt is larger than L2, so a forward walk would miss all).
-__device__ __forceinline__ void walker_init(Walker& w, const Shape& sh, int mode, bool reverse, long long F) {
+__device__ __forceinline__ void walker_init(Walker& w, const Shape& sh, int mode, bool reverse, long long F, int pad = 0) {
   w.mode = mode;
   w.reverse = reverse;
+  w.pad = pad;
   const long long lo = (long long)blockIdx.x * F / gridDim.x, hi = (long long)(blockIdx.x + 1) * F / gridDim.x;
   w.base = 0;
+  w.base_real = 0;
   w.r = 0;
-  if (!reverse) { w.f = lo; w.f_end = hi; return; }
+  if (!reverse) { w.f = lo; w.f_end = hi; return; }        // forward walks carry no padding
   w.f = hi; w.f_end = lo;
-  // position (r, base) on the request that holds the last tile of the share
+  // position (r, base) on the request that holds the last position of the share
   for (;;) {
     const int N = sh.prompt_cu[w.r + 1] - sh.prompt_cu[w.r], M = sh.live_cu[w.r + 1] - sh.live_cu[w.r];
-    const long long span = (long long)walk_groups(sh, mode, M) * tiles_of(N, M);
+    const long long groups = walk_groups(sh, mode, M);
+    const long long span = groups * (tiles_of(N, M) + pad);
     if (hi <= lo || hi - 1 < w.base + span || w.r + 1 >= sh.R) break;
     w.base += span;
+    w.base_real += groups * tiles_of(N, M);
     ++w.r;
   }
 }
@@ -189,30 +199,42 @@ __device__ __forceinline__ bool walker_next(Walker& w, const Shape& sh, Seg& s) 
     const long long room = w.f_end - w.f;
     s.len = (int)min((long long)(s.T - s.t), room);
     s.unit_start = w.base + (long long)s.g * s.T;
+    s.unit_real = s.unit_start;
     w.f += s.len;
     return true;
   }
-  if (w.f <= w.f_end) return false;
-  const long long last = w.f - 1;                          // highest tile still to do
   for (;;) {
-    s.p0 = sh.prompt_cu[w.r]; s.N = sh.prompt_cu[w.r + 1] - s.p0;
-    s.l0 = sh.live_cu[w.r]; s.M = sh.live_cu[w.r + 1] - s.l0;
-    s.T = tiles_of(s.N, s.M);
-    if (last >= w.base) break;
-    // step back to the previous request
-    --w.r;
-    const int N2 = sh.prompt_cu[w.r + 1] - sh.prompt_cu[w.r], M2 = sh.live_cu[w.r + 1] - sh.live_cu[w.r];
-    w.base -= (long long)walk_groups(sh, w.mode, M2) * tiles_of(N2, M2);
+    if (w.f <= w.f_end) return false;
+    const long long last = w.f - 1;                        // highest position still to do
+    for (;;) {
+      s.p0 = sh.prompt_cu[w.r]; s.N = sh.prompt_cu[w.r + 1] - s.p0;
+      s.l0 = sh.live_cu[w.r]; s.M = sh.live_cu[w.r + 1] - s.l0;
+      s.T = tiles_of(s.N, s.M);
+      if (last >= w.base) break;
+      // step back to the previous request
+      --w.r;
+      const int N2 = sh.prompt_cu[w.r + 1] - sh.prompt_cu[w.r], M2 = sh.live_cu[w.r + 1] - sh.live_cu[w.r];
+      const long long groups2 = walk_groups(sh, w.mode, M2);
+      w.base -= groups2 * (tiles_of(N2, M2) + w.pad);
+      w.base_real -= groups2 * tiles_of(N2, M2);
+    }
+    const long long rel = last - w.base;
+    const int Tv = s.T + w.pad;                            // positions of a unit: padding first, then its tiles
+    int tv;
+    split_group_tile(rel, Tv, s.g, tv);
+    const long long room = w.f - w.f_end;
+    const int lenv = (int)min((long long)(tv + 1), room);
+    w.f -= lenv;
+    const int t_hi = tv - w.pad, t_lo = max(tv - lenv + 1 - w.pad, 0);
+    if (t_hi < 0) continue;                                // this piece of the share is padding only
+    s.r = w.r;
+    s.t = t_hi;
+    s.len = t_hi - t_lo + 1;
+    s.dir = -1;
+    s.unit_start = w.base + (long long)s.g * Tv;
+    s.unit_real = w.base_real + (long long)s.g * s.T;
+    return true;
   }
-  const long long rel = last - w.base;
-  s.r = w.r;
-  split_group_tile(rel, s.T, s.g, s.t);
-  s.dir = -1;
-  const long long room = w.f - w.f_end;
-  s.len = (int)min((long long)(s.t + 1), room);
-  s.unit_start = w.base + (long long)s.g * s.T;
-  w.f -= s.len;
-  return true;
 }
 
 // CTA whose share contains flat tile f.
@@ -483,11 +505,11 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const bool split = colpart != nullptr;
   Walker wk;
-  walker_init(wk, sh, split ? kWalkColsumSplit : kWalkColsum, true, F);
+  walker_init(wk, sh, split ? kWalkColsumSplit : kWalkColsum, true, F, kColsumPad);
   Seg s;
   int last_r = -1, last_g = -1;                             // the (request, group) whose queries are resident
   // Both walks of sweep 2 number their tiles exactly like sweep 1 (KV heads = query heads x blocks when there is one
-  // block per KV head; the same (query head, block) groups otherwise), so a run's unit_start is also the flat index at
+  // block per KV head; the same (query head, block) groups otherwise), so a run's unit_real is also the flat index at
   // which sweep 1 started the rows' unit: that is all the merge of its partials needs.
   // group of a run -> query head, KV head, first query of the block, index of the block among the KV head's blocks
   auto unit_of = [&](const Seg& sg, int& h, int& hk, int& q0, int& blk) {
@@ -587,8 +609,8 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     float run_p = 0.f, run_m = 0.f;
     auto flush = [&]() {
       if (cur_seg < 0 || half != 0) return;
-      const int first = cta_of(cur_start, F, gridDim.x);
-      const unsigned slots = 8u * (unsigned)(cta_of(cur_start + cur_T - 1, F, gridDim.x) - first + 1);
+      const int first = cta_of(cur_start + kColsumPad, F, gridDim.x);          // the CTA with the segment's first tile
+      const unsigned slots = 8u * (unsigned)(cta_of(cur_start + kColsumPad + cur_T - 1, F, gridDim.x) - first + 1);
       float2* mp = mass_part + (long long)cur_seg * Tmax * 8;
       unsigned last = 0;
       if (lane == 0) {
@@ -630,7 +652,7 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         float cst = -INFINITY;                              // 2^(x - inf) = 0: rows that do not exist never vote
         if (row < nq) {
           const int i = s.l0 + qh0 + row;
-          const float ln_z = part != nullptr ? merged_lse(part, C, sh.sumM, F1, G1, s.unit_start, s.T, h, i)
+          const float ln_z = part != nullptr ? merged_lse(part, C, sh.sumM, F1, G1, s.unit_real, s.T, h, i)
                                              : lse[(long long)h * sh.sumM + i];
           cst = (w ? log2f(w[i]) : 0.f) - ln_z * kLog2e;
         }
@@ -748,10 +770,11 @@ bool build_maps(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kp,
 
 // F of the walk: tiles over all (request, group) pairs, from the host's copy of the lengths.
 long long flat_tiles(const Shape& sh, const int32_t* prompt_cu, const int32_t* live_cu, int mode) {
+  const int pad = mode == kWalkStats ? 0 : kColsumPad;
   long long F = 0;
   for (int r = 0; r < sh.R; ++r) {
     const int N = prompt_cu[r + 1] - prompt_cu[r], M = live_cu[r + 1] - live_cu[r];
-    F += (long long)walk_groups(sh, mode, M) * ((N + kTile - 1) / kTile + (M + kTile - 1) / kTile);
+    F += (long long)walk_groups(sh, mode, M) * ((N + kTile - 1) / kTile + (M + kTile - 1) / kTile + pad);
   }
   return F;
 }
