@@ -13,7 +13,8 @@
 // three different threads; key and value tiles come through separate TMA rings (3 and 2 stages) and tiles beyond
 // the rings are requested into L2 ahead of time.  A reference only moves when a logit exceeds it by more than 2^8
 // (then the thread rescales its row of O_w in tensor memory), so nothing per tile waits for a P V product or for the
-// other warpgroup; the two partial softmaxes are merged once, after the last tile.  Columns of a ragged tile's tail
+// other warpgroup; the two partial softmaxes are merged once, after the last tile, straight from tensor memory (a
+// thread can read its row of both accumulators).  Columns of a ragged tile's tail
 // are masked to -inf, and the matching V rows are zeroed in shared memory so that stale cache rows can never leak a
 // NaN into the product.  The output tile leaves through shared memory as whole rows.
 //
@@ -22,7 +23,7 @@
 // first S is ready (tensor maps, Q and K from L2, first MMA group), then about 2.0k per tile - 0.3k reading S and
 // finding the row maximum, 1.4k for the 128 x 128 exponentials (1,024 cycles of the special-function unit by
 // themselves; the two warpgroups stay in phase because the S buffers are shared), packing and the store of P - and
-// 3.5k to merge, normalise and store.  When units are few and their key segments long, a cluster of two CTAs shares a
+// 2.5k to merge, normalise and store.  When units are few and their key segments long, a cluster of two CTAs shares a
 // unit: each walks half of the tiles and CTA 1 hands its (max, sum, output) to CTA 0 through distributed shared
 // memory; that merge costs about three tiles' time, so it is used from eight tiles per unit on.
 #include "attend_tc.h"
@@ -407,10 +408,13 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       mbar_arrive(bars.pready + 2 * b + wg);
       l += rs;
     }
-    // The groups meet: common reference, total sum, and each group's O scaled onto the common reference.  Thread
-    // (wg, row) ends up with output columns [OC wg, OC wg + OC) of its row: it keeps that half of its own O_wg and
-    // passes the other half to its partner through shared memory (the key ring, free by now), 16 bytes per access.
-    if (ok && nt > 0) ok = mbar_wait(bars.odone + 2 * ((nt - 1) & 1) + wg, ((nt - 1) >> 1) & 1, abort_flag, status, 0x30d);
+    // The groups meet: common reference, total sum, and both groups' O scaled onto the common reference.  Thread
+    // (wg, row) ends up with output columns [OC wg, OC wg + OC) of its row; its row of BOTH accumulators sits in
+    // tensor-memory lanes the thread may read, so only the references and sums go through shared memory.
+    if (nt > 0) {                                            // both streams' last P V must have landed
+      if (ok) ok = mbar_wait(bars.odone + 2 * ((nt - 1) & 1), ((nt - 1) >> 1) & 1, abort_flag, status, 0x30d);
+      if (ok) ok = mbar_wait(bars.odone + 2 * ((nt - 1) & 1) + 1, ((nt - 1) >> 1) & 1, abort_flag, status, 0x30e);
+    }
     ok = __all_sync(0xffffffffu, ok);
     if (ok) tc_fence_after();
     mx[wg * kATile + row] = m;
@@ -420,37 +424,25 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     const float m_all = fmaxf(m, m_other);
     const float a_me = m == -INFINITY ? 0.f : ex2((m - m_all) * cs);
     const float a_other = m_other == -INFINITY ? 0.f : ex2((m_other - m_all) * cs);
+    const float a_of[2] = {wg == 0 ? a_me : a_other, wg == 0 ? a_other : a_me};   // scale of stream 0, stream 1
     float o[OC];
-    float4* xg = reinterpret_cast<float4*>(base + S::kKOff);   // [writer group][column group of 4][row] as float4
 #pragma unroll
-    for (int cb = 0; cb < D / 32; ++cb) {
-      float ov[32];
-      if (ok && nt > 0) {                                    // warp-uniform; a group that never saw a valid key holds exact zeros
-        tmem_ld32(o_addr + cb * 32, ov);
-        tmem_ld_wait();
-      } else {
+    for (int c = 0; c < OC; ++c) o[c] = 0.f;
+    if (ok && nt > 0) {                                      // warp-uniform; a stream that never saw a valid key holds exact zeros
 #pragma unroll
-        for (int c = 0; c < 32; ++c) ov[c] = 0.f;
+      for (int w2 = 0; w2 < NW; ++w2) {
+#pragma unroll
+        for (int cb = 0; cb < OC / 32; ++cb) {
+          float ov[32];
+          tmem_ld32(tm_o + lane_addr + w2 * kATile + wg * OC + cb * 32, ov);
+          tmem_ld_wait();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[cb * 32 + c] = fmaf(ov[c], a_of[w2], o[cb * 32 + c]);
+        }
       }
-      if ((cb * 32) / OC == wg) {                            // a chunk of my own half
-#pragma unroll
-        for (int c = 0; c < 32; ++c) o[cb * 32 - wg * OC + c] = ov[c] * a_me;
-      } else {                                               // my partner's half
-        const int c_rel = cb * 32 - (wg ^ 1) * OC;           // column inside the partner's half
-#pragma unroll
-        for (int c = 0; c < 32; c += 4)
-          xg[(wg * (OC / 4) + (c_rel + c) / 4) * kATile + row] = make_float4(ov[c] * a_me, ov[c + 1] * a_me, ov[c + 2] * a_me, ov[c + 3] * a_me);
-      }
-    }
-    named_barrier(1, NW * kATile);
-#pragma unroll
-    for (int c = 0; c < OC; c += 4) {
-      const float4 x4 = xg[((wg ^ 1) * (OC / 4) + c / 4) * kATile + row];
-      o[c] += x4.x; o[c + 1] += x4.y; o[c + 2] += x4.z; o[c + 3] += x4.w;
     }
     l = l * a_me + l_other * a_other;
     m = m_all;
-    named_barrier(1, NW * kATile);                           // the exchange area is reused below
     if (nsplit > 1) {
       // Exchange area in CTA 0: its key ring, free once both CTAs have finished their tiles (first barrier).
       // xo4[column group of 4][row] as float4 (a warp's 32 rows of a group are 512 contiguous bytes, for the remote
