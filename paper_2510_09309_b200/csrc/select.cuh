@@ -135,19 +135,22 @@ select_kernel_reg(Shape sh, const float* __restrict__ scores, const int32_t* __r
     return;
   }
 
-  const int jbase = (q * kSelectRegWarps + warp) * (32 * kSelectKeysPerThread) + lane;
+  // Warp (q, warp) owns a contiguous, ascending run of keys (the emit step relies on that), `n_rows` rows of 32: the runs
+  // are sized to the segment, so a short segment is still spread over all 64 warps of the cluster.
+  const int n_rows = min(kSelectKeysPerThread, (N + 32 * kSelectCluster * kSelectRegWarps - 1) / (32 * kSelectCluster * kSelectRegWarps));
+  const int jbase = (q * kSelectRegWarps + warp) * (32 * n_rows) + lane;
   uint32_t key[kSelectKeysPerThread];
 #pragma unroll
   for (int i = 0; i < kSelectKeysPerThread; ++i) {        // all loads first: the whole segment is in flight at once
     const int j = jbase + i * 32;
-    key[i] = j < N ? __float_as_uint(__ldg(seg + j)) : 0u;
+    key[i] = (i < n_rows && j < N) ? __float_as_uint(__ldg(seg + j)) : 0u;
   }
   uint32_t vmask = 0u;                                   // bit i: key i exists
   uint32_t k_and = 0xffffffffu, k_or = 0u;
 #pragma unroll
   for (int i = 0; i < kSelectKeysPerThread; ++i) {
     key[i] = order_key(__uint_as_float(key[i]));
-    if (jbase + i * 32 < N) { vmask |= 1u << i; k_and &= key[i]; k_or |= key[i]; }
+    if (i < n_rows && jbase + i * 32 < N) { vmask |= 1u << i; k_and &= key[i]; k_or |= key[i]; }
   }
   k_and = __reduce_and_sync(0xffffffffu, k_and);
   k_or = __reduce_or_sync(0xffffffffu, k_or);
