@@ -260,10 +260,13 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const Bars bars = carve_bars(base, S::kBarOff);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + S::kMiscOff);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base + S::kMiscOff + 4);
-  pdl_launch_dependents();
   if (threadIdx.x == 0) { prefetch_tmap(&map_q); prefetch_tmap(&map_kp); prefetch_tmap(&map_km); }   // kernel parameters
   block_setup(bars, 4, tmem_slot, abort_flag);
   pdl_wait();
+  // Only now may sweep 2 be scheduled: once every CTA of this grid is past its wait, everything that precedes the call in
+  // the stream is complete and visible, so sweep 2's loader and MMA issuer - which read nothing but the call's inputs -
+  // may start before this grid has finished (its epilogue still waits for this grid's partials).
+  pdl_launch_dependents();
   // sweep 2 counts finished mass partials per segment in seg_cnt; it reads them after this grid has ended
   if (blockIdx.x == 0 && seg_cnt != nullptr)
     for (int i = threadIdx.x; i < sh.R * sh.Hkv; i += blockDim.x) seg_cnt[i] = 0u;
@@ -500,7 +503,8 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   pdl_launch_dependents();
   if (threadIdx.x == 0) { prefetch_tmap(&map_q); prefetch_tmap(&map_kp); prefetch_tmap(&map_km); }   // kernel parameters
   block_setup(bars, 2, tmem_slot, abort_flag);
-  pdl_wait();
+  // No wait here: the loader and the MMA issuer read only the call's inputs, which are visible (sweep 1 releases this grid
+  // after its own wait); the epilogue waits for sweep 1's results below.
   const uint32_t tmem_base = *tmem_slot;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const bool split = colpart != nullptr;
@@ -607,6 +611,7 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     int cur_seg = -1, cur_T = 0;
     long long cur_start = 0;
     float run_p = 0.f, run_m = 0.f;
+    pdl_wait();                                             // sweep 1's partials (or lse), the cleared segment counters
     auto flush = [&]() {
       if (cur_seg < 0 || half != 0) return;
       const int first = cta_of(cur_start + kColsumPad, F, gridDim.x);          // the CTA with the segment's first tile
