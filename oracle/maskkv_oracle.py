@@ -25,6 +25,7 @@ Readings taken where the paper is silent (each is also listed in the design note
     * argtopk uses the total order (score descending, index ascending); kept indices are
       reported in ascending index order.  NaN scores rank below every number.
     * Eq. 8 (layer importance): a zero hidden-state row counts as cosine 0.
+    * Mask-only projection: the input is the final (already normalised) hidden state; no bias term.
 
 Pins: tests/test_oracle_*.py (brute force, closed forms, invariants, library special cases,
 hand-derived budget examples under tests/golden/).  No function here is "parity unpinned".
@@ -125,6 +126,20 @@ def refresh_set(v_cur, v_prev, delta: float, step: Optional[int] = None, t_r: Op
     if step is not None and t_r is not None and t_r > 0 and step % t_r == 0:
         refresh = np.ones_like(refresh)
     return cos, refresh, np.nonzero(refresh)[0].astype(np.int32)
+
+
+def mask_project(hidden, positions, w_vocab):
+    """Mask-only projection (appendix, "Mask-only Projection"): the vocabulary projection of the final hidden states,
+    taken at the masked positions only - logits[m, v] = sum_k hidden[positions[m], k] * w_vocab[v, k].
+
+    hidden [n_tokens, width], positions [n_mask] (any order, repeats allowed), w_vocab [vocab, width] (one row per
+    vocabulary entry, as an output embedding is stored).  Returns logits [n_mask, vocab] float64: by definition the rows
+    `positions` of the all-token projection, which is what the paper's change must leave untouched."""
+    h, w = _f64(hidden), _f64(w_vocab)
+    pos = np.asarray(positions, dtype=np.int64)
+    if pos.size and (pos.min() < 0 or pos.max() >= h.shape[0]):
+        raise IndexError("mask position outside the sequence")
+    return h[pos] @ w.T
 
 
 def guarded_floor(x: float) -> int:
