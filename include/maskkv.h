@@ -148,6 +148,24 @@ int maskkv_refresh_set(maskkv_ctx* ctx, int32_t dtype, const void* v_cur_dev, co
                        int32_t width, int64_t cur_row_stride, int64_t prev_row_stride, float delta, int32_t refresh_all,
                        float* cos_out_dev, int32_t* idx_out_dev, int32_t* count_out_dev, void* stream);
 
+/* Mask-only projection (appendix, "Mask-only Projection"): the vocabulary projection of the final hidden states at
+ * the masked positions only,
+ *   logits[m][v] = sum_k hidden[positions[m]][k] * w_vocab[v][k],   m < n_mask, v < vocab,
+ * bf16 operands, fp32 accumulation on the tensor cores.  hidden_dev [n_tokens][width] and w_vocab_dev [vocab][width]
+ * are bf16 (dtype must be MASKKV_BF16; anything else returns MASKKV_E_UNSUPPORTED), row strides in elements
+ * (0 = packed), width and the strides multiples of 8 elements, bases 16-byte aligned.  positions_dev [n_mask] holds
+ * the masked token rows (any order, repeats allowed; a position outside [0, n_tokens) gives a zero row and raises
+ * MASKKV_FLAG_BOUNDS); NULL means rows 0..n_mask-1 of hidden_dev, read in place.  logits_out_dev [n_mask][vocab] is
+ * fp32 (out_dtype MASKKV_F32, out_row_stride a multiple of 4) or bf16 rounded to nearest even (MASKKV_BF16, a
+ * multiple of 8), 16-byte aligned, row stride in elements (0 = vocab).  Needs
+ * maskkv_mask_project_workspace_bytes(n_mask, width) bytes of scratch (256-byte aligned; 0 when positions_dev is
+ * NULL) for the packed rows.  Asynchronous on `stream`; n_mask = 0 launches nothing. */
+size_t maskkv_mask_project_workspace_bytes(int64_t n_mask, int32_t width);
+int maskkv_mask_project(maskkv_ctx* ctx, int32_t dtype, const void* hidden_dev, int64_t n_tokens, int32_t width,
+                        int64_t hidden_row_stride, const int32_t* positions_dev, int32_t n_mask, const void* w_vocab_dev,
+                        int32_t vocab, int64_t w_row_stride, int32_t out_dtype, void* logits_out_dev,
+                        int64_t out_row_stride, void* workspace_dev, size_t workspace_bytes, void* stream);
+
 /* Eq. 6-7 and the sums of Eq. 14.  For every request r and KV head h: softmax (fp32) of
  * scale * q_i . k_j over the request's N_r prompt keys followed by its M_r mask keys, for each of the
  * H/H_kv query heads that share h; scores[h][prompt_cu[r] + j] = sum over those heads and mask rows i of

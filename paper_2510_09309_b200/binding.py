@@ -25,7 +25,7 @@ EXPORTS = (
     "maskkv_create", "maskkv_destroy", "maskkv_status_string", "maskkv_check_status", "maskkv_launch_count", "maskkv_last_cuda_error",
     "maskkv_tensor_core_launch_count",
     "maskkv_workspace_bytes",
-    "maskkv_layer_budgets", "maskkv_layer_importance", "maskkv_layer_importance_workspace_bytes", "maskkv_refresh_set", "maskkv_score", "maskkv_score_noalloc", "maskkv_score_noalloc_max_bytes", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend",
+    "maskkv_layer_budgets", "maskkv_layer_importance", "maskkv_layer_importance_workspace_bytes", "maskkv_refresh_set", "maskkv_mask_project", "maskkv_mask_project_workspace_bytes", "maskkv_score", "maskkv_score_noalloc", "maskkv_score_noalloc_max_bytes", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend",
 )
 
 
@@ -72,6 +72,9 @@ def _load() -> C.CDLL:
     lib.maskkv_layer_importance_workspace_bytes.restype = sz
     lib.maskkv_layer_importance.argtypes = [vp, i32, vp, vp, i64, i32, i64, i64, vp, vp, sz, vp]
     lib.maskkv_refresh_set.argtypes = [vp, i32, vp, vp, i64, i32, i64, i64, C.c_float, i32, vp, vp, vp, vp]
+    lib.maskkv_mask_project_workspace_bytes.argtypes = [i64, i32]
+    lib.maskkv_mask_project_workspace_bytes.restype = sz
+    lib.maskkv_mask_project.argtypes = [vp, i32, vp, i64, i32, i64, vp, i32, vp, i32, i64, i32, vp, i64, vp, sz, vp]
     lib.maskkv_score.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.maskkv_score_noalloc.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.maskkv_score_noalloc_max_bytes.argtypes = []
@@ -83,12 +86,16 @@ def _load() -> C.CDLL:
     for name in EXPORTS:
         if name not in ("maskkv_status_string", "maskkv_workspace_bytes", "maskkv_launch_count", "maskkv_tensor_core_launch_count",
                         "maskkv_score_noalloc_max_bytes", "maskkv_last_cuda_error",
-                        "maskkv_layer_importance_workspace_bytes"):
+                        "maskkv_layer_importance_workspace_bytes", "maskkv_mask_project_workspace_bytes"):
             getattr(lib, name).restype = C.c_int
     return lib
 
 
 lib = _load()
+
+
+def maskkv_mask_project_workspace_bytes(n_mask: int, width: int) -> int:
+    return int(lib.maskkv_mask_project_workspace_bytes(int(n_mask), int(width)))
 
 
 def status_string(code: int) -> str:
@@ -198,6 +205,22 @@ class Context:
         _check(lib.maskkv_refresh_set(self._h, dt, _ptr(v_cur), _ptr(v_prev), n, width, v_cur.stride(0) if n else 0,
                                       v_prev.stride(0) if n else 0, float(delta), 1 if refresh_all else 0, _ptr(cos_out),
                                       _ptr(idx_out), _ptr(count_out), _stream()), "maskkv_refresh_set", self._h)
+
+    def maskkv_mask_project(self, hidden, w_vocab, logits_out, positions=None, workspace=None):
+        """Mask-only projection: logits_out[m] = w_vocab @ hidden[positions[m]] (bf16 operands; logits_out fp32 or bf16
+        [n_mask, vocab]).  positions int32 [n_mask] on the device, or None for the first n_mask rows of hidden; workspace
+        of maskkv_mask_project_workspace_bytes(n_mask, width) bytes when positions is given."""
+        if hidden.dtype != torch.bfloat16 or w_vocab.dtype != torch.bfloat16:
+            dt = MASKKV_F32
+        else:
+            dt = MASKKV_BF16
+        n_mask = logits_out.shape[0]
+        _check(lib.maskkv_mask_project(self._h, dt, _ptr(hidden), hidden.shape[0], hidden.shape[1], hidden.stride(0),
+                                       _ptr(positions), n_mask, _ptr(w_vocab), w_vocab.shape[0], w_vocab.stride(0),
+                                       MASKKV_F32 if logits_out.dtype == torch.float32 else MASKKV_BF16, _ptr(logits_out),
+                                       logits_out.stride(0) if n_mask else 0, _ptr(workspace),
+                                       0 if workspace is None else workspace.numel() * workspace.element_size(), _stream()),
+               "maskkv_mask_project", self._h)
 
     def maskkv_score(self, p: Problem, q_mask, k_prompt, k_mask, scores, mass_p, mass_m, workspace, row_weights=None):
         _check(lib.maskkv_score(self._h, C.byref(p.desc), _ptr(q_mask), _ptr(k_prompt), _ptr(k_mask), _ptr(row_weights),

@@ -10,6 +10,7 @@
 #include "common.cuh"
 #include "compact.cuh"
 #include "importance.cuh"
+#include "project_tc.h"
 #include "refresh.cuh"
 #include "score_simt.cuh"
 #include "score_tc.h"
@@ -380,6 +381,43 @@ int maskkv_refresh_set(maskkv_ctx* ctx, int32_t dtype, const void* v_cur_dev, co
   mkv::launch_overlapped(mkv::refresh_compact_kernel, dim3(1), dim3(mkv::kRefreshScanThreads), 0, st, (long long)n_tokens, idx_out_dev,
                          count_out_dev);
   return launch_status(ctx, n + 1);
+}
+
+size_t maskkv_mask_project_workspace_bytes(int64_t n_mask, int32_t width) {
+  return n_mask > 0 && width > 0 ? align_up((size_t)n_mask * (size_t)width * 2, 256) : 0;
+}
+
+int maskkv_mask_project(maskkv_ctx* ctx, int32_t dtype, const void* hidden_dev, int64_t n_tokens, int32_t width,
+                        int64_t hidden_row_stride, const int32_t* positions_dev, int32_t n_mask, const void* w_vocab_dev,
+                        int32_t vocab, int64_t w_row_stride, int32_t out_dtype, void* logits_out_dev, int64_t out_row_stride,
+                        void* workspace_dev, size_t workspace_bytes, void* stream) {
+  if (ctx == nullptr || n_mask < 0 || n_tokens < 0 || width <= 0 || vocab <= 0) return MASKKV_E_INVALID;
+  if (dtype != MASKKV_BF16 || (out_dtype != MASKKV_F32 && out_dtype != MASKKV_BF16)) return MASKKV_E_UNSUPPORTED;
+  if (!mkv::tc::project_tc_supported(ctx)) return MASKKV_E_UNSUPPORTED;
+  if (n_mask == 0) return MASKKV_OK;
+  if (hidden_dev == nullptr || w_vocab_dev == nullptr || logits_out_dev == nullptr) return MASKKV_E_INVALID;
+  if (positions_dev == nullptr && n_mask > n_tokens) return MASKKV_E_INVALID;
+  if (hidden_row_stride == 0) hidden_row_stride = width;
+  if (w_row_stride == 0) w_row_stride = width;
+  if (out_row_stride == 0) out_row_stride = vocab;
+  if (hidden_row_stride < width || w_row_stride < width || out_row_stride < vocab) return MASKKV_E_INVALID;
+  const int out_vec = out_dtype == MASKKV_F32 ? 4 : 8;
+  if (width % 8 || hidden_row_stride % 8 || w_row_stride % 8 || out_row_stride % out_vec || !aligned16(hidden_dev) ||
+      !aligned16(w_vocab_dev) || !aligned16(logits_out_dev) || (reinterpret_cast<uintptr_t>(positions_dev) & 3u))
+    return MASKKV_E_ALIGN;
+  if (positions_dev != nullptr) {
+    if (workspace_dev == nullptr || workspace_bytes < maskkv_mask_project_workspace_bytes(n_mask, width)) return MASKKV_E_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) return MASKKV_E_ALIGN;
+  }
+  DeviceGuard guard(ctx->device);
+  int n = 0;
+  if (mkv::tc::launch_project_tc(ctx, hidden_dev, n_tokens, width, hidden_row_stride, positions_dev, n_mask, w_vocab_dev, vocab,
+                                 w_row_stride, logits_out_dev, out_row_stride, out_dtype == MASKKV_BF16 ? 1 : 0, workspace_dev,
+                                 static_cast<cudaStream_t>(stream), &n) != 0) {
+    ctx->last_cuda_error = (int)cudaGetLastError();
+    return MASKKV_E_CUDA;
+  }
+  return launch_status(ctx, n);
 }
 
 int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_dev, const void* k_prompt_dev,

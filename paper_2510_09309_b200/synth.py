@@ -216,3 +216,30 @@ def live_inputs(wl: Workload, layer: int = 0, step: int = 0, device="cpu") -> Di
 def scaled(wl: Workload, name: str, **over) -> Workload:
     """A scaled-down variant of a config that keeps its structure (for tests the oracle finishes in seconds)."""
     return replace(wl, name=name, **over)
+
+
+def project_inputs(n_tokens: int, width: int, vocab: int, n_mask: int, device="cpu", seed: int = 0,
+                   w_std: float = 0.02) -> Dict[str, torch.Tensor]:
+    """Inputs of the mask-only projection: final hidden states [n_tokens, width] (unit variance, as after the final
+    normalisation), an output embedding [vocab, width] (normal, std 0.02 as at initialisation) and the masked
+    positions (int32, ascending: the last n_mask * 5 / 4 rows with every fifth already decoded, as late in a
+    generation).  bf16; generated in pieces so that the full-size embedding never exists in fp32."""
+    dev = torch.device(device)
+    g = torch.Generator(device=dev)
+    g.manual_seed(BASE_SEED + 77_003 + seed)
+    hidden = torch.randn((n_tokens, width), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    w = torch.empty((vocab, width), dtype=torch.bfloat16, device=dev)
+    step = 8192
+    for v0 in range(0, vocab, step):
+        rows = min(step, vocab - v0)
+        w[v0:v0 + rows] = (torch.randn((rows, width), generator=g, device=dev, dtype=torch.float32) * w_std).to(torch.bfloat16)
+    span = min(n_tokens, n_mask + n_mask // 4)
+    cand = torch.arange(n_tokens - span, n_tokens, dtype=torch.int64)
+    keep = torch.ones(span, dtype=torch.bool)
+    drop = span - min(span, n_mask)
+    if drop > 0:
+        keep[torch.arange(drop) * 5 % span] = False
+    pos = cand[keep][:n_mask]
+    if pos.numel() < n_mask:                                   # fewer tokens than masks: repeat rows
+        pos = torch.arange(n_mask, dtype=torch.int64) % max(n_tokens, 1)
+    return {"hidden": hidden, "w_vocab": w, "positions": pos.to(torch.int32).to(dev)}
