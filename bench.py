@@ -462,6 +462,36 @@ def bench_ours(args):
                              "refreshed": int(r_cnt.item())}
         importance["refresh_set"] = refresh
         del h_in, h_out
+        # the mask-only vocabulary projection of the per-step loop: 256 masked rows x width 4096 x vocabulary 126,464
+        # (LLaDA-8B's output embedding, 1.04 GB read once per call); a dense contraction on the tensor cores
+        px = synth.project_inputs(n_tok, hidden, 126464, wl.n_mask, device, seed=1)
+        p_ws = torch.empty(B.maskkv_mask_project_workspace_bytes(wl.n_mask, hidden), dtype=torch.uint8, device=device)
+        project = {"workload": f"{wl.n_mask} masked rows of {n_tok} x width {hidden} x vocabulary 126464, bf16 operands"}
+        p_flops = 2.0 * wl.n_mask * hidden * 126464
+        for name, odt, osz in (("bf16_logits", torch.bfloat16, 2), ("fp32_logits", torch.float32, 4)):
+            logits = torch.empty((wl.n_mask, 126464), dtype=odt, device=device)
+            reps = 20
+            for _ in range(3):
+                ctx.maskkv_mask_project(px["hidden"], px["w_vocab"], logits, px["positions"], p_ws)
+            torch.cuda.synchronize()
+            p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            p0.record()
+            for _ in range(reps):
+                ctx.maskkv_mask_project(px["hidden"], px["w_vocab"], logits, px["positions"], p_ws)
+            p1.record()
+            torch.cuda.synchronize()
+            us = 1e3 * p0.elapsed_time(p1) / reps
+            p_bytes = 126464.0 * hidden * 2 + wl.n_mask * 126464.0 * osz + 2.0 * wl.n_mask * hidden * 2
+            tf = p_flops / (us * 1e-6) / 1e12
+            peak_tf = load_peaks()["bf16_tflops_sustained"]
+            project[name] = {"us": round(us, 2),
+                             "roofline": {"bound": "tensor", "achieved": round(tf, 1), "peak": peak_tf, "unit": "TFLOP/s",
+                                          "frac": round(tf / peak_tf, 3), "peak_source": "sustained bf16 (20 back-to-back calls)"},
+                             "hbm_GB/s": round(p_bytes / (us * 1e-6) / 1e9, 1),
+                             "frac_of_hbm_peak": round(p_bytes / (us * 1e-6) / 1e9 / load_peaks()["hbm_gbs"], 3)}
+            del logits
+        importance["mask_project"] = project
+        del px, p_ws
 
     if world > 1:
         dist.destroy_process_group()
@@ -517,6 +547,7 @@ def bench_ours(args):
     if importance is not None:
         gbs = importance["bytes"] / (importance["us"] * 1e-6) / 1e9
         line["refresh_set"] = importance.pop("refresh_set", None)
+        line["mask_project"] = importance.pop("mask_project", None)
         line["layer_importance"] = {"workload": importance["workload"], "us": round(importance["us"], 2),
                                     "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm}}
     line["cpu_baseline"] = oracle_baseline(wl, budget_s=15.0)

@@ -8,8 +8,6 @@ namespace tc {
 
 // True when the context can run the tensor-core GEMM (tensor-map encoder resolved, enough shared memory).
 bool project_tc_supported(const maskkv_ctx* ctx);
-// Vocabulary entries per output tile (128...256, a multiple of 32) that wastes least of the last wave of CTAs.
-int project_tile_width(int sm_count, int n_mask, int vocab);
 // Gather (when positions != nullptr; `packed` then holds n_mask * width bf16) + GEMM.  Strides in elements.
 // Returns 0 after its launches, 1 when nothing was launched (tensor map or attribute set-up failed).
 int launch_project_tc(maskkv_ctx* ctx, const void* hidden, long long n_tokens, int width, long long hidden_row_stride,
