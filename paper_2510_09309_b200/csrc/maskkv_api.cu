@@ -414,6 +414,7 @@ int maskkv_mask_project(maskkv_ctx* ctx, int32_t dtype, const void* hidden_dev, 
   if (mkv::tc::launch_project_tc(ctx, hidden_dev, n_tokens, width, hidden_row_stride, positions_dev, n_mask, w_vocab_dev, vocab,
                                  w_row_stride, logits_out_dev, out_row_stride, out_dtype == MASKKV_BF16 ? 1 : 0, workspace_dev,
                                  static_cast<cudaStream_t>(stream), &n) != 0) {
+    ctx->launches += (unsigned long long)n;
     ctx->last_cuda_error = (int)cudaGetLastError();
     return MASKKV_E_CUDA;
   }

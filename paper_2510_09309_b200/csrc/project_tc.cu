@@ -6,15 +6,13 @@
 //   warp 0     TMA producer: per 64-wide k block one [256 rows x 64] box of the packed rows and one [tile width x 64] box of w_vocab
 //   warp 1     one thread issues tcgen05.mma (M = 128 twice, N = tile width, K = 16 x 4 per block) into two TMEM accumulators
 //   warps 2-9  epilogue: a thread owns an output row, reads it from TMEM 32 columns at a time and stores it
-// The vocabulary is cut into units of 16 entries (the granularity of the MMA's N); CTA c of G owns the contiguous
-// units [c*U/G, (c+1)*U/G) and cuts them into the same number of tiles as every other CTA, so all CTAs carry the same
-// load to within one unit and tile widths take at most three values (one tensor map each).  A CTA runs all row
+// The vocabulary is shared out as project_common.cuh describes; a CTA runs all row
 // blocks (256 masked rows each) of a tile before it moves on, so a vocabulary tile comes from DRAM once.  Both
 // accumulators can take all of tensor memory, so a tile's epilogue is not overlapped with the next tile's products;
 // it is about 2 % of a tile's time at width 4096.
 #include "project_tc.h"
 
-#include "tc_common.cuh"
+#include "project_common.cuh"
 
 namespace mkv {
 namespace tc {
@@ -23,30 +21,8 @@ namespace {
 
 constexpr int kPThreads = 320;        // TMA warp, MMA warp, 8 epilogue warps
 constexpr int kPStages = 3;
-constexpr int kPBM = 256;             // output rows per tile (two accumulators of 128)
-constexpr int kPBK = 64;              // bf16 per k block = one 128-byte swizzled box row
 constexpr int kPABytes = kPBM * 128;  // packed-rows operand per stage
 constexpr int kPBarBytes = 128;       // mbarriers, tensor-memory base, abort flag
-constexpr int kPStageOutBytes = 4096; // per epilogue warp: 32 rows x 128 bytes on their way out
-
-constexpr int kPMaxWidths = 3;
-
-// How the vocabulary is shared out (see the top of the file).  widths[] are the tile widths that occur, in entries.
-struct PPlan {
-  int units;                 // ceil(vocab / 16)
-  int n_t;                   // tiles per CTA
-  int widths[kPMaxWidths];   // ascending; unused entries repeat the last one
-  int wmax;
-};
-// Tile ti of this CTA: first vocabulary entry and width (0 = no such tile).
-__host__ __device__ __forceinline__ void project_tile(const PPlan& pl, int cta, int G, int ti, int* col0, int* w) {
-  const long long u0 = (long long)cta * pl.units / G, u1 = (long long)(cta + 1) * pl.units / G;
-  const long long share = u1 - u0;
-  const long long t0 = u0 + share * ti / pl.n_t, t1 = u0 + share * (ti + 1) / pl.n_t;
-  *col0 = (int)(t0 * 16);
-  *w = (int)((t1 - t0) * 16);
-}
-
 struct PBars {
   uint64_t* full;    // [kPStages] operands landed
   uint64_t* empty;   // [kPStages] operands consumed
@@ -58,17 +34,6 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, u
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
                : "memory");
-}
-
-__device__ __forceinline__ void st_stream4(float* p, float a, float b, float c, float d) {
-  asm volatile("st.global.cs.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
-__device__ __forceinline__ void st_stream4u(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-__device__ __forceinline__ uint32_t bf16x2(float lo, float hi) {
-  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&v);
 }
 
 // One warp per masked position: copies its hidden row (16-byte pieces) into the packed operand; a position outside
@@ -199,54 +164,10 @@ project_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       if (!(ok = mbar_wait(bars.tfull, tile_i & 1, abort_flag, status, 0x303))) break;
       tc_fence_after();
       if (half_used) {
-        // A thread holds 32 consecutive logits of its own row; stored like that a warp's store instruction would touch
-        // 32 different lines.  The chunk goes through a 4 KB staging block instead (16-byte pieces, XOR-swizzled so
-        // that neither side has bank conflicts) and leaves as whole 128-byte (fp32) or 64-byte (bf16) row pieces.
         float va[32], vb[32];
         const int row0 = mb * kPBM + a * 128 + lane_group * 32;
         auto store = [&](const float* v, int cc) {
-          const int col0 = tcol0 + cc * 32;
-          if (col0 >= col_end) return;                          // warp-uniform
-          if (out_bf16) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-              *reinterpret_cast<uint4*>(stg + lane * 64 + 16 * (j ^ ((lane >> 1) & 3))) =
-                  make_uint4(bf16x2(v[8 * j], v[8 * j + 1]), bf16x2(v[8 * j + 2], v[8 * j + 3]), bf16x2(v[8 * j + 4], v[8 * j + 5]),
-                             bf16x2(v[8 * j + 6], v[8 * j + 7]));
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const int rl = 8 * i + (lane >> 2), piece = lane & 3;
-              const uint4 x = *reinterpret_cast<const uint4*>(stg + rl * 64 + 16 * (piece ^ ((rl >> 1) & 3)));
-              const int row = row0 + rl, col = col0 + piece * 8;
-              if (row >= n_mask || col >= col_end) continue;
-              __nv_bfloat16* p = static_cast<__nv_bfloat16*>(out) + row * ld_out + col;
-              if (col + 8 <= col_end) st_stream4u(p, x.x, x.y, x.z, x.w);
-              else {
-                const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&x);
-                for (int k = 0; k < 8 && col + k < col_end; ++k) p[k] = e[k];
-              }
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-              *reinterpret_cast<float4*>(stg + lane * 128 + 16 * (j ^ (lane & 7))) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const int rl = 4 * i + (lane >> 3), piece = lane & 7;
-              const float4 x = *reinterpret_cast<const float4*>(stg + rl * 128 + 16 * (piece ^ (rl & 7)));
-              const int row = row0 + rl, col = col0 + piece * 4;
-              if (row >= n_mask || col >= col_end) continue;
-              float* p = static_cast<float*>(out) + row * ld_out + col;
-              if (col + 4 <= col_end) st_stream4(p, x.x, x.y, x.z, x.w);
-              else {
-                const float e[4] = {x.x, x.y, x.z, x.w};
-                for (int k = 0; k < 4 && col + k < col_end; ++k) p[k] = e[k];
-              }
-            }
-          }
-          __syncwarp();                                       // the block is free for the next chunk
+          project_store_chunk(v, stg, lane, row0, n_mask, tcol0 + cc * 32, col_end, out, ld_out, out_bf16);
         };
         tmem_ld32(lane_addr, va);
         for (int c = 0; c < chunks; c += 2) {
@@ -270,52 +191,7 @@ project_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
 }
 
-// [rows][width] bf16 matrix with a byte row stride, viewed as (width, rows); box = 64 x box_rows, 128-byte swizzle,
-// zeros outside the matrix.
-bool make_tmap_matrix(void* encode_fn, CUtensorMap* map, const void* base_ptr, uint64_t width, uint64_t rows,
-                      uint64_t row_stride_bytes, uint32_t box_rows) {
-  if (encode_fn == nullptr || base_ptr == nullptr || rows == 0 || width == 0) return false;
-  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-  const cuuint64_t dims[2] = {width, rows};
-  const cuuint64_t strides[1] = {row_stride_bytes};
-  const cuuint32_t box[2] = {(cuuint32_t)kPBK, box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  return reinterpret_cast<EncodeFn>(encode_fn)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base_ptr), dims, strides,
-                                               box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 size_t project_smem_bytes(int wmax) { return (size_t)kPStages * (kPABytes + wmax * 128) + 1024 + kPBarBytes + 8 * kPStageOutBytes; }
-
-// Grid and plan for a vocabulary of `vocab` entries on `sm_count` SMs: every CTA gets at least four units (64 entries)
-// when there are that many, and the same number of tiles, each at most 256 entries wide.
-int make_plan(int sm_count, int vocab, PPlan* pl) {
-  pl->units = (vocab + 15) / 16;
-  int G = (pl->units + 3) / 4;
-  if (G > sm_count) G = sm_count;
-  if (G < 1) G = 1;
-  const int max_share = (pl->units + G - 1) / G;
-  pl->n_t = (max_share + 15) / 16;
-  int n = 0;
-  for (int c = 0; c < G; ++c)
-    for (int ti = 0; ti < pl->n_t; ++ti) {
-      int col0, w;
-      project_tile(*pl, c, G, ti, &col0, &w);
-      if (w == 0) continue;
-      bool seen = false;
-      for (int k = 0; k < n; ++k) seen = seen || pl->widths[k] == w;
-      if (seen) continue;
-      if (n == kPMaxWidths) return 0;                        // cannot happen: shares differ by one unit at most
-      pl->widths[n++] = w;
-    }
-  if (n == 0) return 0;
-  for (int k = n; k < kPMaxWidths; ++k) pl->widths[k] = pl->widths[n - 1];
-  pl->wmax = 0;
-  for (int k = 0; k < kPMaxWidths; ++k) pl->wmax = pl->widths[k] > pl->wmax ? pl->widths[k] : pl->wmax;
-  return G;
-}
 
 }  // namespace
 
@@ -330,7 +206,7 @@ int launch_project_tc(maskkv_ctx* ctx, const void* hidden, long long n_tokens, i
   const void* a_base = hidden;
   long long a_stride = hidden_row_stride * 2;
   PPlan pl;
-  const int grid = make_plan(ctx->sm_count, vocab, &pl);
+  const int grid = make_project_plan(ctx->sm_count, vocab, &pl);
   if (grid == 0) return 1;
   CUtensorMap map_a, map_w[kPMaxWidths];
   if (positions != nullptr) { a_base = packed; a_stride = (long long)width * 2; }
@@ -353,6 +229,14 @@ int launch_project_tc(maskkv_ctx* ctx, const void* hidden, long long n_tokens, i
                                                                    n_tokens, positions, n_mask, width * 2,
                                                                    static_cast<unsigned char*>(packed), ctx->status_dev);
     ++*launches;
+  }
+  // More than 128 masked rows: a pair of CTAs per tile (project_tc2.cu); otherwise the second CTA would have no rows.
+  static const int no_pair = [] { const char* e = getenv("MASKKV_PROJECT_SINGLE_CTA"); return e != nullptr && e[0] == '1'; }();
+  if (n_mask > 128 && !no_pair && project_tc2_supported(ctx)) {
+    if (launch_project_gemm_tc2(ctx, a_base, a_stride, width, n_mask, w_vocab, vocab, w_row_stride, out, ld_out, out_bf16, st) != 0)
+      return *launches == 0 ? 1 : 2;
+    ++*launches;
+    return 0;
   }
   launch_overlapped(project_gemm_tc, dim3(grid), dim3(kPThreads), smem, st, map_a, map_w[0], map_w[1], map_w[2], pl, n_mask, vocab,
                     width, out, ld_out, out_bf16, ctx->status_dev);
