@@ -92,6 +92,25 @@ def test_rows_in_place_with_strided_operands(ctx):
     assert torch.equal(out, out2)
 
 
+def test_single_cta_and_pair_kernels_agree_bit_for_bit(monkeypatch):
+    """More than 128 masked rows run on pairs of CTAs; bit 3 of MASKKV_FORCE_SIMT (read when a context is created) keeps
+    them on the one-CTA kernel.  Both add the k blocks in the same order, so the logits must be identical."""
+    from paper_2510_09309_b200 import binding as B
+    x = synth.project_inputs(700, 448, 3000, 300, "cuda", seed=4)
+    outs = []
+    for force in ("0", "8"):
+        monkeypatch.setenv("MASKKV_FORCE_SIMT", force)
+        c = B.Context(0)
+        try:
+            out, _ = _run(c, x)
+            assert c.maskkv_check_status() == 0
+            outs.append(out.cpu())
+        finally:
+            c.close()
+    assert torch.equal(outs[0], outs[1])
+    _check(outs[1], x["hidden"].cpu(), x["positions"].cpu().numpy(), x["w_vocab"].cpu())
+
+
 def test_out_of_range_position_is_flagged_and_gives_a_zero_row(ctx):
     from paper_2510_09309_b200 import binding as B
     x = synth.project_inputs(100, 128, 300, 8, "cuda", seed=2)
