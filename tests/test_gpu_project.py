@@ -111,6 +111,31 @@ def test_single_cta_and_pair_kernels_agree_bit_for_bit(monkeypatch):
     _check(outs[1], x["hidden"].cpu(), x["positions"].cpu().numpy(), x["w_vocab"].cpu())
 
 
+def test_seeded_shape_sweep_pair_kernel_against_one_cta_kernel_and_oracle(monkeypatch):
+    """Twenty seeded shapes (129-700 masked rows, widths that are multiples of 8 but mostly not of 64, vocabularies
+    that are multiples of nothing): the pair kernel must reproduce the one-CTA kernel's bits, and both the oracle."""
+    from paper_2510_09309_b200 import binding as B
+    rng = np.random.default_rng(20251009)
+    shapes = [(int(rng.integers(129, 701)), int(rng.integers(8, 140)) * 8, int(rng.integers(40, 9000))) for _ in range(20)]
+    outs = {}
+    for force in ("0", "8"):
+        monkeypatch.setenv("MASKKV_FORCE_SIMT", force)
+        c = B.Context(0)
+        try:
+            for i, (n_mask, width, vocab) in enumerate(shapes):
+                x = synth.project_inputs(n_mask + 50, width, vocab, n_mask, "cuda", seed=100 + i)
+                dt = torch.bfloat16 if i % 3 == 2 else torch.float32
+                out, _ = _run(c, x, dt)
+                outs[(force, i)] = out.cpu()
+                if force == "8":
+                    assert torch.equal(outs[("0", i)], outs[("8", i)]), f"shape {shapes[i]}: the two kernels differ"
+                    if i % 4 == 0:
+                        _check(out.float().cpu(), x["hidden"].cpu(), x["positions"].cpu().numpy(), x["w_vocab"].cpu(), bf16_out=dt == torch.bfloat16)
+            assert c.maskkv_check_status() == 0
+        finally:
+            c.close()
+
+
 def test_out_of_range_position_is_flagged_and_gives_a_zero_row(ctx):
     from paper_2510_09309_b200 import binding as B
     x = synth.project_inputs(100, 128, 300, 8, "cuda", seed=2)
