@@ -176,6 +176,17 @@ int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_
                  float* scores_dev, float* mass_p_dev, float* mass_m_dev, void* workspace_dev,
                  size_t workspace_bytes, void* stream);
 
+/* maskkv_score with one more output, for the voter sets other than the mask tokens that the paper compares in its
+ * voting ablations (all tokens, the prompt tokens, a trailing window of the prompt): scores_live_dev [H_kv][sum_M]
+ * (may be NULL) receives the column sums over the live keys, scores_live[h][live_cu[r] + j] = sum over the voting rows
+ * of A[i][N_r + j].  The call scores every key of K_full = [k_prompt ; k_mask] from the rows of q_mask, so any voter set
+ * is a matter of which tokens are passed where: the voters' queries as q_mask with their own keys as k_mask, every
+ * other token's keys as k_prompt (possibly none: scores_dev may then be NULL).  The importance of a prompt token is
+ * then read from scores_live if it votes and from scores if it does not.  Everything else as in maskkv_score. */
+int maskkv_score_all_keys(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_dev, const void* k_prompt_dev,
+                          const void* k_mask_dev, const float* row_weights_dev, float* scores_dev, float* scores_live_dev,
+                          float* mass_p_dev, float* mass_m_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
+
 /* maskkv_score for callers that cannot hand over a workspace.  (The paper has no counterpart: this is a
  * packaging variant of the call above, same arithmetic, same outputs.)
  *

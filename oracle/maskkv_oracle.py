@@ -96,6 +96,29 @@ def score(q_mask, k_prompt, k_mask, prompt_cu: Sequence[int], live_cu: Sequence[
     return scores, mass_p, mass_m
 
 
+def vote_scores(q, k, voters, n_prompt: int, scale: Optional[float] = None):
+    """The voting ablation (which tokens' attention ranks the prompt): I_j = sum over i in `voters` of A_ij for the
+    n_prompt prompt tokens j, with A = softmax_row(q k^T * scale) over ALL tokens of the sequence [prompt ; response].
+    Mask-Voting takes the mask rows as voters, Prompt-Voting the prompt rows, All-Voting every row, a window the last
+    few prompt rows.  One request: q [T, H, d], k [T, H_kv, d], voters = row indices.  Returns I [H_kv, n_prompt],
+    summed over the query heads that share a KV head as in `score`."""
+    q, k = _f64(q), _f64(k)
+    H, d = q.shape[1], q.shape[2]
+    Hkv = k.shape[1]
+    g = H // Hkv
+    if scale is None or scale <= 0:
+        scale = 1.0 / math.sqrt(d)
+    rows = np.asarray(voters, dtype=np.int64)
+    out = np.zeros((Hkv, n_prompt), F64)
+    for hk in range(Hkv):
+        for h in range(hk * g, (hk + 1) * g):
+            if rows.size == 0:
+                continue
+            a, _ = attention_weights(q[rows, h], k[:, hk], scale)
+            out[hk] += a[:, :n_prompt].sum(axis=0)
+    return out
+
+
 def layer_importance(h_in, h_out) -> float:
     """Eq. 8: I^(l) = 1 - (1/n) sum_i cos_sim(h_in_i, h_out_i) over the n token rows of one layer.
 

@@ -25,7 +25,7 @@ EXPORTS = (
     "maskkv_create", "maskkv_destroy", "maskkv_status_string", "maskkv_check_status", "maskkv_launch_count", "maskkv_last_cuda_error",
     "maskkv_tensor_core_launch_count",
     "maskkv_workspace_bytes",
-    "maskkv_layer_budgets", "maskkv_layer_importance", "maskkv_layer_importance_workspace_bytes", "maskkv_refresh_set", "maskkv_mask_project", "maskkv_mask_project_workspace_bytes", "maskkv_score", "maskkv_score_noalloc", "maskkv_score_noalloc_max_bytes", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend",
+    "maskkv_layer_budgets", "maskkv_layer_importance", "maskkv_layer_importance_workspace_bytes", "maskkv_refresh_set", "maskkv_mask_project", "maskkv_mask_project_workspace_bytes", "maskkv_score", "maskkv_score_all_keys", "maskkv_score_noalloc", "maskkv_score_noalloc_max_bytes", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend",
 )
 
 
@@ -76,6 +76,7 @@ def _load() -> C.CDLL:
     lib.maskkv_mask_project_workspace_bytes.restype = sz
     lib.maskkv_mask_project.argtypes = [vp, i32, vp, i64, i32, i64, vp, i32, vp, i32, i64, i32, vp, i64, vp, sz, vp]
     lib.maskkv_score.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.maskkv_score_all_keys.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.maskkv_score_noalloc.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.maskkv_score_noalloc_max_bytes.argtypes = []
     lib.maskkv_score_noalloc_max_bytes.restype = sz
@@ -227,6 +228,15 @@ class Context:
                                 _ptr(scores), _ptr(mass_p), _ptr(mass_m), _ptr(workspace),
                                 0 if workspace is None else workspace.numel() * workspace.element_size(), _stream()),
                "maskkv_score", self._h)
+
+    def maskkv_score_all_keys(self, p: Problem, q_mask, k_prompt, k_mask, scores, scores_live, mass_p, mass_m, workspace,
+                              row_weights=None):
+        """maskkv_score that also returns the column sums over the live keys (scores_live fp32 [H_kv, sum_M]); with the
+        voters' queries as q_mask, their keys as k_mask and all other keys as k_prompt this scores any voter set."""
+        _check(lib.maskkv_score_all_keys(self._h, C.byref(p.desc), _ptr(q_mask), _ptr(k_prompt), _ptr(k_mask), _ptr(row_weights),
+                                         _ptr(scores), _ptr(scores_live), _ptr(mass_p), _ptr(mass_m), _ptr(workspace),
+                                         0 if workspace is None else workspace.numel() * workspace.element_size(), _stream()),
+               "maskkv_score_all_keys", self._h)
 
     def maskkv_score_noalloc(self, p: Problem, q_mask, k_prompt, k_mask, scores, mass_p, mass_m, row_weights=None):
         """maskkv_score without a workspace argument, for callers that may not allocate device memory: the

@@ -106,8 +106,8 @@ inline int launch_status(maskkv_ctx* ctx, int n) {
 // sweeps on the tensor cores; fp32 problems (and anything the tensor-core path cannot take) on the FP32 pipes.
 template <typename T, int D>
 int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, const ScoreWorkspace& w, bool any_without_voters,
-                 const void* q, const void* kp, const void* km, const float* rw, float* scores, float* mass_p, float* mass_m,
-                 unsigned char* ws, cudaStream_t st) {
+                 const void* q, const void* kp, const void* km, const float* rw, float* scores, float* scores_live, float* mass_p,
+                 float* mass_m, unsigned char* ws, cudaStream_t st) {
   float* lse = reinterpret_cast<float*>(ws + w.lse_off);
   float2* part = reinterpret_cast<float2*>(ws + w.part_off);
   float2* mass_part = reinterpret_cast<float2*>(ws + w.mass_off);
@@ -137,7 +137,7 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, co
     int launched = 0;
     float* colpart = reinterpret_cast<float*>(ws + w.col_off);
     tc2 = mkv::tc::launch_score_colsum_tc(ctx, sh, desc->prompt_cu, desc->live_cu, q, kp, km, lse, tc1 ? part : nullptr, w.C, rw,
-                                          scores, colpart, mass_part, w.Tmax, seg_cnt, mass_p, mass_m, any_without_voters, st,
+                                          scores, colpart, mass_part, w.Tmax, seg_cnt, mass_p, mass_m, scores_live, any_without_voters, st,
                                           &launched) == 0;
     if (tc2) {
       ++ctx->tc_launches;
@@ -152,7 +152,7 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, co
     if (tc1) { mkv::tc::launch_score_merge_tc(ctx, sh, desc->prompt_cu, desc->live_cu, part, w.C, lse, st); ++n; }
     dim3 g2(w.Tmax, sh.Hkv, sh.R);
     mkv::score_colsum_simt<T, D><<<g2, mkv::kSimtThreads, 0, st>>>(sh, (const T*)q, (const T*)kp, (const T*)km, lse, rw,
-                                                                    scores, mass_part, w.Tmax);
+                                                                    scores, scores_live, mass_part, w.Tmax);
     mkv::score_mass_reduce<<<(S + 3) / 4, 128, 0, st>>>(sh, mass_part, w.Tmax, mass_p, mass_m);
     n += 2;
   }
@@ -424,11 +424,19 @@ int maskkv_mask_project(maskkv_ctx* ctx, int32_t dtype, const void* hidden_dev, 
 int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_dev, const void* k_prompt_dev,
                  const void* k_mask_dev, const float* row_weights_dev, float* scores_dev, float* mass_p_dev,
                  float* mass_m_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
+  return maskkv_score_all_keys(ctx, desc, q_mask_dev, k_prompt_dev, k_mask_dev, row_weights_dev, scores_dev, nullptr, mass_p_dev,
+                               mass_m_dev, workspace_dev, workspace_bytes, stream);
+}
+
+int maskkv_score_all_keys(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_dev, const void* k_prompt_dev,
+                          const void* k_mask_dev, const float* row_weights_dev, float* scores_dev, float* scores_live_dev,
+                          float* mass_p_dev, float* mass_m_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
   if (ctx == nullptr) return MASKKV_E_INVALID;
   Shape sh;
   int rc = resolve(desc, &sh);
   if (rc != MASKKV_OK) return rc;
-  if (scores_dev == nullptr || mass_p_dev == nullptr || mass_m_dev == nullptr) return MASKKV_E_INVALID;
+  if ((scores_dev == nullptr && sh.sumN > 0) || mass_p_dev == nullptr || mass_m_dev == nullptr) return MASKKV_E_INVALID;
+  if (reinterpret_cast<uintptr_t>(scores_live_dev) & 3u) return MASKKV_E_ALIGN;
   if ((sh.sumM > 0 && (q_mask_dev == nullptr || k_mask_dev == nullptr)) || (sh.sumN > 0 && k_prompt_dev == nullptr))
     return MASKKV_E_INVALID;
   if (!aligned16(q_mask_dev) || !aligned16(k_prompt_dev) || !aligned16(k_mask_dev) || !aligned16(scores_dev) ||
@@ -442,7 +450,7 @@ int maskkv_score(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_mask_
   bool any_without_voters = false;
   for (int r = 0; r < sh.R; ++r) any_without_voters |= desc->live_cu[r + 1] == desc->live_cu[r];
 #define MKV_SCORE(T, D) launch_score<T, D>(ctx, sh, desc, w, any_without_voters, q_mask_dev, k_prompt_dev, k_mask_dev, row_weights_dev, scores_dev, \
-                                                mass_p_dev, mass_m_dev, ws, st)
+                                                scores_live_dev, mass_p_dev, mass_m_dev, ws, st)
   if (sh.dtype == MASKKV_F32) return sh.d == 64 ? MKV_SCORE(float, 64) : MKV_SCORE(float, 128);
   return sh.d == 64 ? MKV_SCORE(__nv_bfloat16, 64) : MKV_SCORE(__nv_bfloat16, 128);
 #undef MKV_SCORE

@@ -108,7 +108,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads)
 score_colsum_simt(Shape sh, const T* __restrict__ q, const T* __restrict__ kp, const T* __restrict__ km,
                   const float* __restrict__ lse, const float* __restrict__ w, float* __restrict__ scores,
-                  float2* __restrict__ mass_part, int Tmax) {
+                  float* __restrict__ scores_live, float2* __restrict__ mass_part, int Tmax) {
   __shared__ __align__(16) float qs[kSimtStage][D];
   __shared__ float ls[kSimtStage], ws[kSimtStage];
   __shared__ float red[2][kSimtThreads / 32];
@@ -150,6 +150,7 @@ score_colsum_simt(Shape sh, const T* __restrict__ q, const T* __restrict__ kp, c
     }
   }
   if (valid && j < N) scores[(long long)hk * sh.sumN + p0 + j] = acc;
+  if (valid && j >= N && scores_live != nullptr) scores_live[(long long)hk * sh.sumM + l0 + (j - N)] = acc;
   float sp = (valid && j < N) ? acc : 0.f;
   float sm = (valid && j >= N) ? acc : 0.f;
   sp = warp_sum(sp);

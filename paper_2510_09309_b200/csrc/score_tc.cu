@@ -492,7 +492,7 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const float2* __restrict__ part, int C, long long F1, int G1,
                 const float* __restrict__ w, float* __restrict__ scores, float* __restrict__ colpart,
                 float2* __restrict__ mass_part, int Tmax, uint32_t* __restrict__ seg_cnt, float* __restrict__ mass_p,
-                float* __restrict__ mass_m, long long F, uint32_t* __restrict__ status) {
+                float* __restrict__ mass_m, long long F, float* __restrict__ scores_live, uint32_t* __restrict__ status) {
   using S = Smem<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = align_1024(smem_raw);
@@ -711,6 +711,7 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
         if (row >= kt.valid) acc = 0.f;
         if (kt.prompt && row < kt.valid) out_row[kt.token + row] = acc;
+        if (scores_live != nullptr && !kt.prompt && row < kt.valid) scores_live[(long long)hk * sh.sumM + kt.token + row] = acc;
         acc = warp_sum(acc);
         if (kt.prompt) run_p += acc; else run_m += acc;
       }
@@ -725,7 +726,7 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 // the tile's share of the attention masses as the FP32-pipe sweep leaves it (mass_part[((r*H_kv + hk)*Tmax + t)*4 + warp],
 // summed by score_mass_reduce).  A request without voters has no blocks: zeros.  grid (Tmax, H_kv, R), 128 threads.
 __global__ void score_group_reduce(Shape sh, const float* __restrict__ colpart, float* __restrict__ scores,
-                                   float2* __restrict__ mass_part, int Tmax) {
+                                   float* __restrict__ scores_live, float2* __restrict__ mass_part, int Tmax) {
   const int t = blockIdx.x, hk = blockIdx.y, r = blockIdx.z;
   const int p0 = sh.prompt_cu[r], N = sh.prompt_cu[r + 1] - p0;
   const int l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
@@ -739,6 +740,7 @@ __global__ void score_group_reduce(Shape sh, const float* __restrict__ colpart, 
     const float* src = colpart + (long long)hk * keys_total + (kt.prompt ? 0 : sh.sumN) + kt.token + j;
     for (int b = 0; b < blocks; ++b) acc += src[(long long)b * sh.Hkv * keys_total];
     if (kt.prompt) scores[(long long)hk * sh.sumN + kt.token + j] = acc;
+    else if (scores_live != nullptr) scores_live[(long long)hk * sh.sumM + kt.token + j] = acc;
   }
   acc = warp_sum(acc);
   if ((threadIdx.x & 31) == 0)
@@ -850,7 +852,7 @@ size_t score_tc_colpart_bytes(const Shape& sh) {
 int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prompt_cu_host, const int32_t* live_cu_host,
                            const void* q, const void* kp, const void* km, const float* lse, const float2* part, int C,
                            const float* w, float* scores, float* colpart, float2* mass_part, int Tmax, uint32_t* seg_cnt,
-                           float* mass_p, float* mass_m, bool any_without_voters, cudaStream_t st, int* launches) {
+                           float* mass_p, float* mass_m, float* scores_live, bool any_without_voters, cudaStream_t st, int* launches) {
   Maps m;
   if (!build_maps(ctx, sh, q, kp, km, &m)) return 1;
   const bool split = score_tc_split_blocks(sh);
@@ -870,14 +872,14 @@ int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prom
   float* cp = split ? colpart : nullptr;
   if (sh.d == 128)
     launch_overlapped(score_colsum_tc<128>, dim3(grid), dim3(kThreads), Smem<128>::kDynamic, st, m.q, m.kp, m.km, sh, lse, part, C, F1, G1,
-                      w, scores, cp, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
+                      w, scores, cp, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, scores_live, ctx->status_dev);
   else
     launch_overlapped(score_colsum_tc<64>, dim3(grid), dim3(kThreads), Smem<64>::kDynamic, st, m.q, m.kp, m.km, sh, lse, part, C, F1, G1,
-                      w, scores, cp, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, ctx->status_dev);
+                      w, scores, cp, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, scores_live, ctx->status_dev);
   ++*launches;
   if (split) {
     dim3 gr(Tmax, sh.Hkv, sh.R);
-    score_group_reduce<<<gr, kTile, 0, st>>>(sh, colpart, scores, mass_part, Tmax);
+    score_group_reduce<<<gr, kTile, 0, st>>>(sh, colpart, scores, scores_live, mass_part, Tmax);
     ++*launches;
   }
   return 0;

@@ -25,13 +25,14 @@ void launch_score_merge_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prom
 // the warp that finishes a segment's last tile adds up its partials - mass_p / mass_m; `seg_cnt` (R*H_kv words) must
 // be zero on entry.  With several blocks (score_tc_split_blocks) each block's column sums go to `colpart`
 // (score_tc_colpart_bytes), a second kernel adds them into scores and leaves per-tile mass partials in `mass_part` in
-// the layout score_mass_reduce reads: the caller launches that kernel afterwards.  *launches = kernels launched.
+// the layout score_mass_reduce reads: the caller launches that kernel afterwards.  scores_live (may be null) receives the
+// column sums over the live keys, [H_kv][sum_M].  *launches = kernels launched.
 bool score_tc_split_blocks(const Shape& sh);
 size_t score_tc_colpart_bytes(const Shape& sh);
 int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prompt_cu_host, const int32_t* live_cu_host,
                            const void* q, const void* kp, const void* km, const float* lse, const float2* part, int C,
                            const float* w, float* scores, float* colpart, float2* mass_part, int Tmax, uint32_t* seg_cnt,
-                           float* mass_p, float* mass_m, bool any_without_voters, cudaStream_t st, int* launches);
+                           float* mass_p, float* mass_m, float* scores_live, bool any_without_voters, cudaStream_t st, int* launches);
 
 }  // namespace tc
 }  // namespace mkv
