@@ -250,6 +250,19 @@ int maskkv_attend(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_live
                   const void* k_live_dev, const void* v_live_dev, const void* kc_dev, const void* vc_dev,
                   const int32_t* offsets_dev, int64_t capacity, void* out_dev, float* lse_dev, void* stream);
 
+/* The attention step with partial refresh: the feature cache the method builds on recomputes, at most steps, only the
+ * response rows whose value features drifted (maskkv_refresh_set), so only those rows have queries - while the keys and
+ * values are still the compacted prompt cache followed by ALL live rows of the request.  q_rows_dev [rows][H][d] holds
+ * the queries of the refreshed rows, request after request, rows_cu / rows_cu_dev (host and device copies, int32
+ * [n_requests + 1], rows_cu[0] = 0) their cumulative counts; a request may have none.  out_rows_dev has the layout of
+ * q_rows_dev, lse_rows_dev (may be NULL) is f32 [H][rows].  Which live row a query belongs to does not matter (no
+ * mask).  Both rows_cu pointers NULL: the queries are the live rows themselves, i.e. maskkv_attend.  Everything else
+ * as in maskkv_attend. */
+int maskkv_attend_rows(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_rows_dev, const int32_t* rows_cu,
+                       const int32_t* rows_cu_dev, const void* k_live_dev, const void* v_live_dev, const void* kc_dev,
+                       const void* vc_dev, const int32_t* offsets_dev, int64_t capacity, void* out_rows_dev,
+                       float* lse_rows_dev, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -275,12 +275,16 @@ def compact(k_prompt, v_prompt, kept_idx, offsets, prompt_cu: Sequence[int]):
 
 
 def attend(q_live, k_live, v_live, kc, vc, offsets, live_cu: Sequence[int], n_kv_heads: int,
-           scale: Optional[float] = None):
+           scale: Optional[float] = None, rows_cu: Optional[Sequence[int]] = None):
     """Attention of a later step over [compacted prompt segment ; live keys] (appendix proof, Step 3:
     out_m = sum_j alpha_mj V_j with alpha = softmax(q_m k_j / sqrt(d_k))).
 
     q_live [sumM, H, d]; k_live, v_live [sumM, H_kv, d]; kc, vc [total, d]; offsets [R*H_kv+1].
-    Returns out [sumM, H, d] fp64 and lse [H, sumM] fp64 (log of the softmax denominator)."""
+    Returns out [sumM, H, d] fp64 and lse [H, sumM] fp64 (log of the softmax denominator).
+
+    rows_cu (partial refresh of the feature cache, appendix "Response tokens"): only some response rows are recomputed
+    at a step, so q_live then holds the queries of those rows only, rows_cu[r] .. rows_cu[r+1] for request r, while the
+    keys and values stay the segment followed by ALL live rows; out and lse are then per query row."""
     q, kl, vl, kc, vc = _f64(q_live), _f64(k_live), _f64(v_live), _f64(kc), _f64(vc)
     H, d = q.shape[1], q.shape[2]
     Hkv = n_kv_heads
@@ -290,14 +294,18 @@ def attend(q_live, k_live, v_live, kc, vc, offsets, live_cu: Sequence[int], n_kv
         scale = 1.0 / math.sqrt(d)
     out = np.zeros_like(q)
     lse = np.zeros((H, q.shape[0]), F64)
+    q_cu = live_cu if rows_cu is None else rows_cu
     for r in range(R):
         l0, l1 = live_cu[r], live_cu[r + 1]
+        q0, q1 = q_cu[r], q_cu[r + 1]
+        if q1 == q0:
+            continue
         for h in range(H):
             hk = h // g
             s = r * Hkv + hk
             keys = np.concatenate([kc[int(offsets[s]):int(offsets[s + 1])], kl[l0:l1, hk]], axis=0)
             vals = np.concatenate([vc[int(offsets[s]):int(offsets[s + 1])], vl[l0:l1, hk]], axis=0)
-            a, ls = attention_weights(q[l0:l1, h], keys, scale)
-            out[l0:l1, h] = a @ vals
-            lse[h, l0:l1] = ls
+            a, ls = attention_weights(q[q0:q1, h], keys, scale)
+            out[q0:q1, h] = a @ vals
+            lse[h, q0:q1] = ls
     return out, lse

@@ -25,7 +25,7 @@ EXPORTS = (
     "maskkv_create", "maskkv_destroy", "maskkv_status_string", "maskkv_check_status", "maskkv_launch_count", "maskkv_last_cuda_error",
     "maskkv_tensor_core_launch_count",
     "maskkv_workspace_bytes",
-    "maskkv_layer_budgets", "maskkv_layer_importance", "maskkv_layer_importance_workspace_bytes", "maskkv_refresh_set", "maskkv_mask_project", "maskkv_mask_project_workspace_bytes", "maskkv_score", "maskkv_score_all_keys", "maskkv_score_noalloc", "maskkv_score_noalloc_max_bytes", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend",
+    "maskkv_layer_budgets", "maskkv_layer_importance", "maskkv_layer_importance_workspace_bytes", "maskkv_refresh_set", "maskkv_mask_project", "maskkv_mask_project_workspace_bytes", "maskkv_score", "maskkv_score_all_keys", "maskkv_score_noalloc", "maskkv_score_noalloc_max_bytes", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend", "maskkv_attend_rows",
 )
 
 
@@ -84,6 +84,7 @@ def _load() -> C.CDLL:
     lib.maskkv_select.argtypes = [vp, dp, vp, vp, vp, vp, vp, sz, vp]
     lib.maskkv_compact.argtypes = [vp, dp, vp, vp, vp, vp, i64, vp, vp, vp]
     lib.maskkv_attend.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
+    lib.maskkv_attend_rows.argtypes = [vp, dp, vp, C.POINTER(C.c_int32), vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("maskkv_status_string", "maskkv_workspace_bytes", "maskkv_launch_count", "maskkv_tensor_core_launch_count",
                         "maskkv_score_noalloc_max_bytes", "maskkv_last_cuda_error",
@@ -263,3 +264,15 @@ class Context:
     def maskkv_attend(self, p: Problem, q_live, k_live, v_live, kc, vc, offsets, capacity: int, out, lse=None):
         _check(lib.maskkv_attend(self._h, C.byref(p.desc), _ptr(q_live), _ptr(k_live), _ptr(v_live), _ptr(kc), _ptr(vc),
                                  _ptr(offsets), int(capacity), _ptr(out), _ptr(lse), _stream()), "maskkv_attend", self._h)
+
+    def maskkv_attend_rows(self, p: Problem, q_rows, rows_cu: Sequence[int], k_live, v_live, kc, vc, offsets, capacity: int, out_rows,
+                           lse_rows=None):
+        """maskkv_attend for a subset of query rows (partial refresh): q_rows / out_rows [rows, H, d] hold the refreshed
+        rows of every request one after the other, rows_cu their cumulative counts (host list, length n_requests + 1);
+        keys and values remain the compacted cache followed by all live rows."""
+        host = (C.c_int32 * len(rows_cu))(*[int(x) for x in rows_cu])
+        dev = torch.tensor([int(x) for x in rows_cu], dtype=torch.int32, device=p.device)
+        _check(lib.maskkv_attend_rows(self._h, C.byref(p.desc), _ptr(q_rows), host, _ptr(dev), _ptr(k_live), _ptr(v_live), _ptr(kc),
+                                      _ptr(vc), _ptr(offsets), int(capacity), _ptr(out_rows), _ptr(lse_rows), _stream()),
+               "maskkv_attend_rows", self._h)
+        return dev                                           # keep alive until the stream has passed the call

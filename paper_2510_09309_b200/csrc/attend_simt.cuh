@@ -33,24 +33,25 @@ __device__ __forceinline__ void load_lane<__nv_bfloat16, 4>(const __nv_bfloat16*
   dst[2] = __uint_as_float(w.y << 16); dst[3] = __uint_as_float(w.y & 0xffff0000u);
 }
 
-// grid (ceil(maxM / kAttendWarps), H, R); block kAttendWarps * 32.
+// grid (ceil(largest query count / kAttendWarps), H, R); block kAttendWarps * 32.
 template <typename T, int D>
 __global__ void __launch_bounds__(kAttendWarps * 32)
 attend_simt(Shape sh, const T* __restrict__ q, const T* __restrict__ kl, const T* __restrict__ vl,
             const T* __restrict__ kc, const T* __restrict__ vc, const int32_t* __restrict__ offsets,
-            T* __restrict__ out, float* __restrict__ lse) {
+            const int32_t* __restrict__ q_cu, int sum_q, T* __restrict__ out, float* __restrict__ lse) {
   constexpr int E = D / 32;
   const int lane = threadIdx.x & 31;
   const int h = blockIdx.y, r = blockIdx.z, hk = h / sh.g;
   const int l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
+  const int ql0 = q_cu[r], Mq = q_cu[r + 1] - ql0;          // the query rows: the live rows or a subset of them
   const int i = blockIdx.x * kAttendWarps + (threadIdx.x >> 5);
-  if (i >= M) return;
+  if (i >= Mq) return;
   const int s = r * sh.Hkv + hk;
   const int c0 = offsets[s], nc = offsets[s + 1] - c0;
   const int total = nc + M;
 
   float qv[E], acc[E];
-  load_lane<T, E>(q + (long long)(l0 + i) * sh.q_ts + (long long)h * sh.q_hs + lane * E, qv);
+  load_lane<T, E>(q + (long long)(ql0 + i) * sh.q_ts + (long long)h * sh.q_hs + lane * E, qv);
 #pragma unroll
   for (int e = 0; e < E; ++e) { qv[e] *= sh.scale; acc[e] = 0.f; }
   float m = -INFINITY, l = 0.f;
@@ -103,10 +104,10 @@ attend_simt(Shape sh, const T* __restrict__ q, const T* __restrict__ kl, const T
     m = m_new;
   }
   const float inv = 1.f / l;
-  T* o = out + (long long)(l0 + i) * sh.q_ts + (long long)h * sh.q_hs + lane * E;
+  T* o = out + (long long)(ql0 + i) * sh.q_ts + (long long)h * sh.q_hs + lane * E;
 #pragma unroll
   for (int e = 0; e < E; ++e) o[e] = from_f32<T>(acc[e] * inv);
-  if (lse != nullptr && lane == 0) lse[(long long)h * sh.sumM + l0 + i] = m + logf(l);
+  if (lse != nullptr && lane == 0) lse[(long long)h * sum_q + ql0 + i] = m + logf(l);
 }
 
 }  // namespace mkv

@@ -140,7 +140,8 @@ __global__ void __launch_bounds__(AWgs<D>::kThreads, 1)
 attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kl,
           const __grid_constant__ CUtensorMap map_vl, const __grid_constant__ CUtensorMap map_kc,
           const __grid_constant__ CUtensorMap map_vc, Shape sh, const int32_t* __restrict__ offsets,
-          __nv_bfloat16* __restrict__ out, float* __restrict__ lse, uint32_t* __restrict__ status) {
+          const int32_t* __restrict__ q_cu, int sum_q, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
+          uint32_t* __restrict__ status) {
   using S = ASmem<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -179,10 +180,12 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   const int qt = blockIdx.x / nsplit, h = blockIdx.y, r = blockIdx.z, hk = h / sh.g;
   const int seg = r * sh.Hkv + hk;
   // the four loads go out together (they are independent, and nothing can start before them)
+  // q_cu = the query rows of every request: the live rows themselves (q_cu == live_cu), or the refreshed subset of them
   const int l0 = sh.live_cu[r], l1 = sh.live_cu[r + 1], c0 = offsets[seg], c1 = offsets[seg + 1];
-  const int M = l1 - l0, nc = c1 - c0;
+  const int ql0 = q_cu[r], ql1 = q_cu[r + 1];
+  const int M = l1 - l0, nc = c1 - c0, Mq = ql1 - ql0;
   const int q0 = qt * kATile;
-  if (q0 >= M) {                                           // uniform over the block: nothing to do for this tile
+  if (q0 >= Mq) {                                           // uniform over the block: nothing to do for this tile
     if (warp == 1) tmem_dealloc(tmem_base, 512);
     return;
   }
@@ -196,7 +199,7 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   if (warp == 0) {
     if (lane == 0) {
       mbar_expect_tx(bars.qfull, S::kTileBytes);
-      for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kBoxBytes, &map_q, bars.qfull, b * 64, h, l0 + q0);
+      for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kBoxBytes, &map_q, bars.qfull, b * 64, h, ql0 + q0);
       // two independent rings (keys, values): whichever has a free stage gets its next tile, keys first
       int jk = 0, jv = 0;
       const unsigned long long t_start = global_ns();
@@ -491,13 +494,13 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         w.w = pack_bf16(o[c + 6] * inv, o[c + 7] * inv);
         dst[c / 8] = w;
       }
-      if (wg == 0 && lse != nullptr && i < M && !*abort_flag) lse[(long long)h * sh.sumM + l0 + i] = m * sh.scale + logf(l);
+      if (wg == 0 && lse != nullptr && i < Mq && !*abort_flag) lse[(long long)h * sum_q + ql0 + i] = m * sh.scale + logf(l);
     }
     named_barrier(1, NW * kATile);
     if (part == 0 && !*abort_flag) {
       constexpr int PPR = D * 2 / 16;                        // 16-byte pieces per row
-      const int pieces = min(kATile, M - q0) * PPR;
-      uint8_t* out_tile = reinterpret_cast<uint8_t*>(out + (long long)(l0 + q0) * sh.q_ts + (long long)h * sh.q_hs);
+      const int pieces = min(kATile, Mq - q0) * PPR;
+      uint8_t* out_tile = reinterpret_cast<uint8_t*>(out + (long long)(ql0 + q0) * sh.q_ts + (long long)h * sh.q_hs);
       for (int e = tid_all; e < pieces; e += NW * kATile) {
         const int rr = e / PPR, pc = e % PPR;
         *reinterpret_cast<uint4*>(out_tile + (long long)rr * sh.q_ts * 2 + pc * 16) =
@@ -525,14 +528,15 @@ bool attend_tc_supported(const maskkv_ctx* ctx, const Shape& sh) {
   return sh.dtype == MASKKV_BF16 && ctx->encode_tiled != nullptr && sh.sumM > 0 && ctx->smem_optin >= ASmem<128>::kDynamic;
 }
 
-int launch_attend_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kl, const void* vl, const void* kc,
-                     const void* vc, long long cache_rows, const int32_t* offsets, void* out, float* lse, cudaStream_t st) {
+int launch_attend_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const int32_t* q_cu, int sum_q, int max_q, const void* kl,
+                     const void* vl, const void* kc, const void* vc, long long cache_rows, const int32_t* offsets, void* out,
+                     float* lse, cudaStream_t st) {
   CUtensorMap mq, mkl, mvl, mkc, mvc;
   // an empty cache still needs valid maps: point them at the live tensors (no tile of them is ever requested)
   const void* kc_base = cache_rows > 0 && kc ? kc : kl;
   const void* vc_base = cache_rows > 0 && vc ? vc : vl;
   const uint64_t rows = cache_rows > 0 ? (uint64_t)cache_rows : 1;
-  const bool ok = make_tmap_rows(ctx->encode_tiled, &mq, q, sh.d, sh.H, sh.sumM, sh.q_hs * 2, sh.q_ts * 2, kATile) &&
+  const bool ok = make_tmap_rows(ctx->encode_tiled, &mq, q, sh.d, sh.H, (uint64_t)sum_q, sh.q_hs * 2, sh.q_ts * 2, kATile) &&
                   make_tmap_rows(ctx->encode_tiled, &mkl, kl, sh.d, sh.Hkv, sh.sumM, sh.kv_hs * 2, sh.kv_ts * 2, kATile) &&
                   make_tmap_rows(ctx->encode_tiled, &mvl, vl, sh.d, sh.Hkv, sh.sumM, sh.kv_hs * 2, sh.kv_ts * 2, kATile) &&
                   make_tmap_rows(ctx->encode_tiled, &mkc, kc_base, sh.d, 1, rows, (uint64_t)sh.d * 2, (uint64_t)sh.d * 2, kATile) &&
@@ -542,20 +546,20 @@ int launch_attend_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const void
   // then two CTAs share a unit (cluster of 2 along x).  The merge costs about as much as three tiles (64 KB through
   // distributed shared memory), so the split only pays for long chains - eight tiles or more at the mean segment
   // length the capacity allows; with enough units it only adds set-up cost.
-  const unsigned q_tiles = (unsigned)((sh.maxM + kATile - 1) / kATile);
+  const unsigned q_tiles = (unsigned)((max_q + kATile - 1) / kATile);
   const long long units = (long long)q_tiles * sh.H * sh.R;
   const long long mean_rows = cache_rows / ((long long)sh.R * sh.Hkv);
-  const long long chain = (mean_rows + kATile - 1) / kATile + q_tiles;
+  const long long chain = (mean_rows + kATile - 1) / kATile + (sh.maxM + kATile - 1) / kATile;
   const unsigned nsplit = (2 * units <= ctx->sm_count && chain >= kASplitMinTiles) ? 2u : 1u;
   dim3 grid(q_tiles * nsplit, sh.H, sh.R);
   if (sh.d == 128) {
     if (set_attend_attr<128>() != cudaSuccess) return 1;
     (void)launch_overlapped_cluster(attend_tc<128>, grid, dim3(AWgs<128>::kThreads), ASmem<128>::kDynamic, st, nsplit, mq, mkl, mvl, mkc, mvc,
-                                  sh, offsets, (__nv_bfloat16*)out, lse, ctx->status_dev);
+                                  sh, offsets, q_cu, sum_q, (__nv_bfloat16*)out, lse, ctx->status_dev);
   } else {
     if (set_attend_attr<64>() != cudaSuccess) return 1;
     (void)launch_overlapped_cluster(attend_tc<64>, grid, dim3(AWgs<64>::kThreads), ASmem<64>::kDynamic, st, nsplit, mq, mkl, mvl, mkc, mvc,
-                                  sh, offsets, (__nv_bfloat16*)out, lse, ctx->status_dev);
+                                  sh, offsets, q_cu, sum_q, (__nv_bfloat16*)out, lse, ctx->status_dev);
   }
   // a failed launch is reported by the caller through cudaGetLastError
   return 0;

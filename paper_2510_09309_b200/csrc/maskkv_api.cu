@@ -160,12 +160,12 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, co
 }
 
 template <typename T, int D>
-int launch_attend_simt(maskkv_ctx* ctx, const Shape& sh, const void* q, const void* kl, const void* vl, const void* kc, const void* vc,
-                       const int32_t* offsets, void* out, float* lse, cudaStream_t st) {
-  if (sh.maxM == 0) return MASKKV_OK;
-  dim3 grid((sh.maxM + mkv::kAttendWarps - 1) / mkv::kAttendWarps, sh.H, sh.R);
+int launch_attend_simt(maskkv_ctx* ctx, const Shape& sh, const void* q, const int32_t* q_cu, int sum_q, int max_q, const void* kl,
+                       const void* vl, const void* kc, const void* vc, const int32_t* offsets, void* out, float* lse, cudaStream_t st) {
+  if (max_q == 0) return MASKKV_OK;
+  dim3 grid((max_q + mkv::kAttendWarps - 1) / mkv::kAttendWarps, sh.H, sh.R);
   mkv::attend_simt<T, D><<<grid, mkv::kAttendWarps * 32, 0, st>>>(sh, (const T*)q, (const T*)kl, (const T*)vl, (const T*)kc,
-                                                                   (const T*)vc, offsets, (T*)out, lse);
+                                                                   (const T*)vc, offsets, q_cu, sum_q, (T*)out, lse);
   return launch_status(ctx, 1);
 }
 
@@ -547,25 +547,50 @@ int maskkv_compact(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* k_pro
 int maskkv_attend(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_live_dev, const void* k_live_dev,
                   const void* v_live_dev, const void* kc_dev, const void* vc_dev, const int32_t* offsets_dev,
                   int64_t capacity, void* out_dev, float* lse_dev, void* stream) {
+  return maskkv_attend_rows(ctx, desc, q_live_dev, nullptr, nullptr, k_live_dev, v_live_dev, kc_dev, vc_dev, offsets_dev, capacity,
+                            out_dev, lse_dev, stream);
+}
+
+int maskkv_attend_rows(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_rows_dev, const int32_t* rows_cu,
+                       const int32_t* rows_cu_dev, const void* k_live_dev, const void* v_live_dev, const void* kc_dev,
+                       const void* vc_dev, const int32_t* offsets_dev, int64_t capacity, void* out_rows_dev, float* lse_rows_dev,
+                       void* stream) {
   if (ctx == nullptr) return MASKKV_E_INVALID;
   Shape sh;
   int rc = resolve(desc, &sh);
   if (rc != MASKKV_OK) return rc;
   if (offsets_dev == nullptr || capacity < 0) return MASKKV_E_INVALID;
-  if (sh.sumM == 0) return MASKKV_OK;
-  if (q_live_dev == nullptr || k_live_dev == nullptr || v_live_dev == nullptr || out_dev == nullptr) return MASKKV_E_INVALID;
-  if (!aligned16(q_live_dev) || !aligned16(k_live_dev) || !aligned16(v_live_dev) || !aligned16(kc_dev) ||
-      !aligned16(vc_dev) || !aligned16(out_dev))
+  if ((rows_cu == nullptr) != (rows_cu_dev == nullptr)) return MASKKV_E_INVALID;
+  // the query rows: the live rows themselves, or the caller's subset of them
+  const int32_t* q_cu = sh.live_cu;
+  int sum_q = sh.sumM, max_q = sh.maxM;
+  if (rows_cu != nullptr) {
+    if (rows_cu[0] != 0 || (reinterpret_cast<uintptr_t>(rows_cu_dev) & 3u)) return rows_cu[0] != 0 ? MASKKV_E_INVALID : MASKKV_E_ALIGN;
+    max_q = 0;
+    for (int r = 0; r < sh.R; ++r) {
+      const long long n = (long long)rows_cu[r + 1] - rows_cu[r];
+      if (n < 0) return MASKKV_E_INVALID;
+      if (n > max_q) max_q = (int)n;
+    }
+    q_cu = rows_cu_dev;
+    sum_q = rows_cu[sh.R];
+  }
+  if (sum_q == 0) return MASKKV_OK;
+  if (q_rows_dev == nullptr || out_rows_dev == nullptr) return MASKKV_E_INVALID;
+  if (sh.sumM > 0 && (k_live_dev == nullptr || v_live_dev == nullptr)) return MASKKV_E_INVALID;
+  if (!aligned16(q_rows_dev) || !aligned16(k_live_dev) || !aligned16(v_live_dev) || !aligned16(kc_dev) ||
+      !aligned16(vc_dev) || !aligned16(out_rows_dev))
     return MASKKV_E_ALIGN;
   DeviceGuard guard(ctx->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (mkv::tc::attend_tc_supported(ctx, sh) && !(ctx->force_simt & 4u) &&
-      mkv::tc::launch_attend_tc(ctx, sh, q_live_dev, k_live_dev, v_live_dev, kc_dev, vc_dev, capacity, offsets_dev, out_dev,
-                                lse_dev, st) == 0) {
+      mkv::tc::launch_attend_tc(ctx, sh, q_rows_dev, q_cu, sum_q, max_q, k_live_dev, v_live_dev, kc_dev, vc_dev, capacity, offsets_dev,
+                                out_rows_dev, lse_rows_dev, st) == 0) {
     ++ctx->tc_launches;
     return launch_status(ctx, 1);
   }
-#define MKV_ATTEND(T, D) launch_attend_simt<T, D>(ctx, sh, q_live_dev, k_live_dev, v_live_dev, kc_dev, vc_dev, offsets_dev, out_dev, lse_dev, st)
+#define MKV_ATTEND(T, D) launch_attend_simt<T, D>(ctx, sh, q_rows_dev, q_cu, sum_q, max_q, k_live_dev, v_live_dev, kc_dev, vc_dev, \
+                                                  offsets_dev, out_rows_dev, lse_rows_dev, st)
   if (sh.dtype == MASKKV_F32) return sh.d == 64 ? MKV_ATTEND(float, 64) : MKV_ATTEND(float, 128);
   return sh.d == 64 ? MKV_ATTEND(__nv_bfloat16, 64) : MKV_ATTEND(__nv_bfloat16, 128);
 #undef MKV_ATTEND

@@ -83,3 +83,35 @@ def test_closed_forms_single_key_zero_query_and_order_invariance():
     perm = torch.tensor([2, 0, 1, 4, 3])
     out2, _ = O.attend(t["q"], t["kl"], t["vl"], kc[perm], vc[perm], off, lcu, Hkv)
     np.testing.assert_allclose(out1, out2, rtol=1e-12, atol=1e-14)
+
+
+def test_partial_refresh_rows_are_rows_of_the_full_step_and_match_the_library():
+    """With rows_cu the queries are a subset of the live rows while the keys stay all of them: the outputs must be
+    the corresponding rows of the full step, and each row must match the library's attention over
+    [segment ; all live rows]."""
+    t, pcu, lcu = _case(3)
+    R, H, Hkv, M = 2, 4, 2, 5
+    bud = np.array([[6, 2], [0, 9]])
+    idx, off = O.select(t["sc"], bud, pcu)
+    kc, vc = O.compact(t["kp"], t["vp"], idx, off, pcu)
+    full, full_lse = O.attend(t["q"], t["kl"], t["vl"], kc, vc, off, lcu, Hkv)
+    picks = [[4, 1], [2]]                                              # refreshed rows of each request, in list order
+    rows = [lcu[r] + i for r in range(R) for i in picks[r]]
+    rows_cu = [0, 2, 3]
+    out, lse = O.attend(t["q"][rows], t["kl"], t["vl"], kc, vc, off, lcu, Hkv, rows_cu=rows_cu)
+    assert out.shape == (3, H, 8) and lse.shape == (H, 3)
+    np.testing.assert_allclose(out, full[rows], rtol=1e-12, atol=1e-14)      # the library matmul rounds differently per shape
+    np.testing.assert_allclose(lse, full_lse[:, rows], rtol=1e-13)
+    for n, row in enumerate(rows):
+        r = 0 if n < 2 else 1
+        for h in range(H):
+            hk, s = h // 2, r * Hkv + h // 2
+            keys = torch.cat([kc[off[s]:off[s + 1]], t["kl"][lcu[r]:lcu[r + 1], hk]])
+            vals = torch.cat([vc[off[s]:off[s + 1]], t["vl"][lcu[r]:lcu[r + 1], hk]])
+            ref = F.scaled_dot_product_attention(t["q"][row, h][None, None, None], keys[None, None], vals[None, None])[0, 0, 0]
+            np.testing.assert_allclose(out[n, h], ref.numpy(), rtol=1e-11, atol=1e-13)
+    # a request without refreshed rows contributes nothing; no rows at all gives empty outputs
+    out2, _ = O.attend(t["q"][rows[2:]], t["kl"], t["vl"], kc, vc, off, lcu, Hkv, rows_cu=[0, 0, 1])
+    np.testing.assert_allclose(out2, full[rows[2:]], rtol=1e-12, atol=1e-14)
+    out3, lse3 = O.attend(t["q"][:0], t["kl"], t["vl"], kc, vc, off, lcu, Hkv, rows_cu=[0, 0, 0])
+    assert out3.shape == (0, H, 8) and lse3.shape == (H, 0)
