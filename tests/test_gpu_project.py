@@ -60,6 +60,10 @@ def _run(ctx, x, out_dtype=torch.float32, positions="given", out_stride=None):
     (400, 200, 777, 129),        # width not a multiple of 64: the last k block reads zeros; 129 rows = second half by one
     (64, 64, 33, 5),             # everything smaller than one tile
     (2048, 1024, 40000, 512),    # several waves of tiles per CTA
+    (300, 64, 16, 200),          # pair kernel, a vocabulary of one 16-entry unit
+    (300, 72, 8, 130),           # pair kernel, fewer entries than one unit, width 72
+    (40, 8, 100, 10),            # width smaller than a k block
+    (1000, 128, 2368, 1000),     # four row blocks on 148 one-unit tiles
 ])
 def test_parity_fp32_out(ctx, n_tokens, width, vocab, n_mask):
     x = synth.project_inputs(n_tokens, width, vocab, n_mask, "cuda", seed=n_mask)
