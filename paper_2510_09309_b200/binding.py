@@ -265,14 +265,13 @@ class Context:
         _check(lib.maskkv_attend(self._h, C.byref(p.desc), _ptr(q_live), _ptr(k_live), _ptr(v_live), _ptr(kc), _ptr(vc),
                                  _ptr(offsets), int(capacity), _ptr(out), _ptr(lse), _stream()), "maskkv_attend", self._h)
 
-    def maskkv_attend_rows(self, p: Problem, q_rows, rows_cu: Sequence[int], k_live, v_live, kc, vc, offsets, capacity: int, out_rows,
-                           lse_rows=None):
+    def maskkv_attend_rows(self, p: Problem, q_rows, rows_cu: Sequence[int], rows_cu_dev, k_live, v_live, kc, vc, offsets,
+                           capacity: int, out_rows, lse_rows=None):
         """maskkv_attend for a subset of query rows (partial refresh): q_rows / out_rows [rows, H, d] hold the refreshed
-        rows of every request one after the other, rows_cu their cumulative counts (host list, length n_requests + 1);
-        keys and values remain the compacted cache followed by all live rows."""
+        rows of every request one after the other; rows_cu (host list, length n_requests + 1) and rows_cu_dev (the same
+        numbers as an int32 device tensor, owned by the caller) are their cumulative counts; keys and values remain the
+        compacted cache followed by all live rows."""
         host = (C.c_int32 * len(rows_cu))(*[int(x) for x in rows_cu])
-        dev = torch.tensor([int(x) for x in rows_cu], dtype=torch.int32, device=p.device)
-        _check(lib.maskkv_attend_rows(self._h, C.byref(p.desc), _ptr(q_rows), host, _ptr(dev), _ptr(k_live), _ptr(v_live), _ptr(kc),
-                                      _ptr(vc), _ptr(offsets), int(capacity), _ptr(out_rows), _ptr(lse_rows), _stream()),
+        _check(lib.maskkv_attend_rows(self._h, C.byref(p.desc), _ptr(q_rows), host, _ptr(rows_cu_dev), _ptr(k_live), _ptr(v_live),
+                                      _ptr(kc), _ptr(vc), _ptr(offsets), int(capacity), _ptr(out_rows), _ptr(lse_rows), _stream()),
                "maskkv_attend_rows", self._h)
-        return dev                                           # keep alive until the stream has passed the call

@@ -34,10 +34,10 @@ def _check_rows(ctx, run, wl, live, ld, picks, atol):
     q_rows = ld["q_live"][torch.tensor(rows, dtype=torch.long, device=dev)].contiguous() if n else ld["q_live"][:0]
     out = torch.full((max(n, 1), H, d), float("nan"), dtype=wl.torch_dtype, device=dev)
     lse = torch.full((H, max(n, 1)), float("nan"), dtype=torch.float32, device=dev)
-    keep = ctx.maskkv_attend_rows(run.p, q_rows, rows_cu, ld["k_live"], ld["v_live"], run.kc, run.vc, run.offsets, run.kc.shape[0],
-                                  out, lse)
+    rows_cu_dev = torch.tensor(rows_cu, dtype=torch.int32, device=dev)
+    ctx.maskkv_attend_rows(run.p, q_rows, rows_cu, rows_cu_dev, ld["k_live"], ld["v_live"], run.kc, run.vc, run.offsets,
+                           run.kc.shape[0], out, lse)
     torch.cuda.synchronize()
-    del keep
     assert ctx.maskkv_check_status() == 0
     if n == 0:
         assert torch.isnan(out.float()).all()
@@ -120,7 +120,8 @@ def test_argument_errors(monkeypatch):
         before = ctx.maskkv_launch_count()
         for bad in ([1, 4, 4], [0, 4, 2]):                                                  # not starting at 0; decreasing
             with pytest.raises(B.MaskKVError) as e:
-                ctx.maskkv_attend_rows(run.p, q, bad, ld["k_live"], ld["v_live"], run.kc, run.vc, run.offsets, run.kc.shape[0], out)
+                ctx.maskkv_attend_rows(run.p, q, bad, torch.tensor(bad, dtype=torch.int32, device=ctx.device), ld["k_live"],
+                                       ld["v_live"], run.kc, run.vc, run.offsets, run.kc.shape[0], out)
             assert e.value.code == B.MASKKV_E_INVALID
         assert ctx.maskkv_launch_count() == before
     finally:
