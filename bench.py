@@ -312,6 +312,29 @@ def bench_ours(args):
     a1.record()
     barrier()
     attend_loop_us = 1e3 * max_over_ranks(a0.elapsed_time(a1), device) / a_steps
+    # the same step with partial refresh: a quarter of the live rows have queries (maskkv_attend_rows)
+    n_rows = max(1, wl.n_mask // 4)
+    rows_cu = [r * n_rows for r in range(wl.n_requests + 1)]
+    rows_cu_dev = torch.tensor(rows_cu, dtype=torch.int32, device=device)
+    q_rows = [torch.cat([lv["q_live"][r * wl.n_mask:r * wl.n_mask + n_rows] for r in range(wl.n_requests)]).contiguous() for lv in lives]
+    out_rows = torch.empty_like(q_rows[0])
+
+    def attend_rows_step(i):
+        kc, vc = caches[i % n_copies]
+        live = lives[i % len(lives)]
+        ctx.maskkv_attend_rows(p, q_rows[i % len(lives)], rows_cu, rows_cu_dev, live["k_live"], live["v_live"], kc, vc, buf.offsets,
+                               buf.capacity, out_rows)
+
+    for i in range(5):
+        attend_rows_step(i)
+    barrier()
+    r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    r0.record()
+    for i in range(a_steps):
+        attend_rows_step(i)
+    r1.record()
+    barrier()
+    attend_rows_us = 1e3 * max_over_ranks(r0.elapsed_time(r1), device) / a_steps
     del caches
     # maskkv_score alone, launched the way the timed steps launch it (graph replays cycling the resident layers): the
     # duration the roofline objects use
@@ -527,7 +550,9 @@ def bench_ours(args):
         "call_us": {k: round(v, 2) for k, v in call_us.items()},
         "attend_step_us": round(attend_loop_us, 2),
         "attend_step": {"us": round(attend_loop_us, 2), "steps": a_steps, "mean_kept_per_head": mean_kept,
-                        "l2": f"{n_copies} copies of the compacted cache ({cache_bytes * n_copies / 1e6:.0f} MB) cycled"},
+                        "l2": f"{n_copies} copies of the compacted cache ({cache_bytes * n_copies / 1e6:.0f} MB) cycled",
+                        "partial_refresh_us": round(attend_rows_us, 2),
+                        "partial_refresh": f"{n_rows} of {wl.n_mask} live rows have queries (maskkv_attend_rows)"},
         "compress_tokens_per_s": N / (1e-6 * (call_us["score"] + call_us["budget"] + call_us["select"] + call_us["compact"])),
         "e2e": {"value": world * N / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
