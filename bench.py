@@ -188,6 +188,12 @@ def algorithmic_work(wl, mean_kept_per_head):
     }
 
 
+def kv_cache_bytes(tokens_per_head: float, n_kv_heads: int, head_dim: int, elem_bytes: int = 2) -> float:
+    """The paper's accounting of the KV cache of one layer (appendix, "Evaluation metrics"): 2 * L * H * d_head * s,
+    keys and values of L tokens in each of H heads; for the compacted cache L is the mean number of kept tokens."""
+    return 2.0 * tokens_per_head * n_kv_heads * head_dim * elem_bytes
+
+
 def bench_ours(args):
     rank, world, local_rank = rank_world()
     import torch.distributed as dist
@@ -553,6 +559,9 @@ def bench_ours(args):
                         "l2": f"{n_copies} copies of the compacted cache ({cache_bytes * n_copies / 1e6:.0f} MB) cycled",
                         "partial_refresh_us": round(attend_rows_us, 2),
                         "partial_refresh": f"{n_rows} of {wl.n_mask} live rows have queries (maskkv_attend_rows)"},
+        "kv_cache": {"prompt_bytes_per_layer": kv_cache_bytes(N, wl.n_kv_heads, wl.head_dim),
+                     "compacted_bytes_per_layer": kv_cache_bytes(mean_kept, wl.n_kv_heads, wl.head_dim),
+                     "ratio": N / max(mean_kept, 1e-9), "formula": "2 * tokens * heads * d_head * 2 bytes per layer"},
         "compress_tokens_per_s": N / (1e-6 * (call_us["score"] + call_us["budget"] + call_us["select"] + call_us["compact"])),
         "e2e": {"value": world * N / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},

@@ -61,3 +61,14 @@ def test_single_process_helpers_are_no_ops():
     import bench
     assert bench.shard_layers(5, 0, 1) == [0, 1, 2, 3, 4]
     assert bench.max_over_ranks(3.5) == 3.5 and bench.sum_over_ranks(2.0) == 2.0
+
+
+def test_kv_cache_accounting_of_the_32k_layer():
+    """The paper's KV-size formula on the bench workload: a 32k-token LLaDA-shaped layer holds 536.9 MB of prompt keys
+    and values in bf16, 4.19 MB once compacted to a mean budget of 256 tokens per head (a factor of 128)."""
+    import bench
+    full = bench.kv_cache_bytes(32768, 32, 128)
+    kept = bench.kv_cache_bytes(256, 32, 128)
+    assert full == 2 * 32768 * 32 * 128 * 2 == 536870912
+    assert kept == 4194304 and full / kept == 128
+    assert bench.kv_cache_bytes(100, 4, 64, elem_bytes=4) == 2 * 100 * 4 * 64 * 4
