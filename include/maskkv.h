@@ -87,6 +87,12 @@ const char* maskkv_status_string(int code);
  * MASKKV_E_CUDA if the stream reported an error, else MASKKV_OK. */
 int maskkv_check_status(maskkv_ctx* ctx, void* stream, uint32_t* flags_out);
 
+/* Self-test of the bounded waits (every wait on a barrier inside the tensor-core kernels gives up after about one
+ * second instead of spinning forever): enqueues one thread that waits for a signal nothing sends.  The kernel returns
+ * after the limit with MASKKV_FLAG_TIMEOUT raised, so the next maskkv_check_status returns MASKKV_E_TIMEOUT and the
+ * context stays usable.  For tests of the error path; it touches no caller memory. */
+int maskkv_selftest_wait_expiry(maskkv_ctx* ctx, void* stream);
+
 /* Text of the most recent CUDA runtime error behind a MASKKV_E_CUDA return of this context ("" if none). */
 const char* maskkv_last_cuda_error(const maskkv_ctx* ctx);
 

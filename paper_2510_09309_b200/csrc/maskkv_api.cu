@@ -17,6 +17,7 @@
 #include "score_simt.cuh"
 #include "score_tc.h"
 #include "select.cuh"
+#include "selftest.h"
 
 namespace {
 
@@ -272,6 +273,13 @@ int maskkv_check_status(maskkv_ctx* ctx, void* stream, uint32_t* flags_out) {
   if (cudaStreamSynchronize(st) != cudaSuccess) return MASKKV_E_CUDA;
   if (flags_out) *flags_out = flags;
   return (flags & MASKKV_FLAG_TIMEOUT) ? MASKKV_E_TIMEOUT : MASKKV_OK;
+}
+
+int maskkv_selftest_wait_expiry(maskkv_ctx* ctx, void* stream) {
+  if (ctx == nullptr) return MASKKV_E_INVALID;
+  DeviceGuard guard(ctx->device);
+  mkv::tc::launch_wait_expiry_selftest(ctx, static_cast<cudaStream_t>(stream));
+  return launch_status(ctx, 1);
 }
 
 uint64_t maskkv_launch_count(const maskkv_ctx* ctx) { return ctx ? ctx->launches : 0; }
