@@ -342,6 +342,29 @@ def bench_ours(args):
     barrier()
     attend_rows_us = 1e3 * max_over_ranks(r0.elapsed_time(r1), device) / a_steps
     del caches
+    # The loop above ran on the cache of the layer the last step left behind (a boundary layer, the larger budget at
+    # one rank).  Most layers are middle layers with the smaller budget: compress one and time its step too.
+    attend_mid = None
+    mid = [j for j in range(len(resident)) if k_layers[resident[j]] == min(k_layers[l] for l in resident)]
+    if mid and k_layers[resident[mid[0]]] != k_layers[resident[(args.warmup + len(per_call) - 1) % len(resident)]]:
+        step(mid[0])
+        barrier()
+        mid_kept = float(buf.offsets[-1].item()) / wl.n_kv_heads
+        caches = [(buf.kc.clone(), buf.vc.clone()) for _ in range(n_copies)]
+        for i in range(5):
+            attend_step(i)
+        barrier()
+        m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        m0.record()
+        for i in range(a_steps):
+            attend_step(i)
+        m1.record()
+        barrier()
+        attend_mid = {"us": round(1e3 * max_over_ranks(m0.elapsed_time(m1), device) / a_steps, 2), "mean_kept_per_head": mid_kept,
+                      "layer": resident[mid[0]]}
+        del caches
+        step(args.warmup + len(per_call) - 1)                          # leave the buffers as the later sections expect them
+        barrier()
     # maskkv_score alone, launched the way the timed steps launch it (graph replays cycling the resident layers): the
     # duration the roofline objects use
     score_us = None
@@ -558,7 +581,8 @@ def bench_ours(args):
         "attend_step": {"us": round(attend_loop_us, 2), "steps": a_steps, "mean_kept_per_head": mean_kept,
                         "l2": f"{n_copies} copies of the compacted cache ({cache_bytes * n_copies / 1e6:.0f} MB) cycled",
                         "partial_refresh_us": round(attend_rows_us, 2),
-                        "partial_refresh": f"{n_rows} of {wl.n_mask} live rows have queries (maskkv_attend_rows)"},
+                        "partial_refresh": f"{n_rows} of {wl.n_mask} live rows have queries (maskkv_attend_rows)",
+                        "middle_layer": attend_mid},
         "kv_cache": {"prompt_bytes_per_layer": kv_cache_bytes(N, wl.n_kv_heads, wl.head_dim),
                      "compacted_bytes_per_layer": kv_cache_bytes(mean_kept, wl.n_kv_heads, wl.head_dim),
                      "ratio": N / max(mean_kept, 1e-9), "formula": "2 * tokens * heads * d_head * 2 bytes per layer"},
