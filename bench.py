@@ -194,6 +194,68 @@ def kv_cache_bytes(tokens_per_head: float, n_kv_heads: int, head_dim: int, elem_
     return 2.0 * tokens_per_head * n_kv_heads * head_dim * elem_bytes
 
 
+def batched_calls(ctx, B, device):
+    """maskkv_select / maskkv_compact / maskkv_attend on configs[4] (ragged serving: 8 requests of 1k-32k prompt tokens,
+    256 segments, one layer, mean budget 256): per-call time warm (20 calls back to back) and cold (256 MB written
+    between the calls, outside the timed region), with the algorithmic bytes each call must move."""
+    wl = synth.config(5)
+    x = synth.layer_inputs(wl, 1, device)
+    live = synth.live_inputs(wl, 1, 0, device)
+    buf = LayerBuffers(ctx, B, wl, wl.n_requests * wl.n_kv_heads * 2 * wl.mean_budget, device)
+    run_layer(ctx, buf, x, live, wl.mean_budget, wl.alpha)
+    torch.cuda.synchronize()
+    p, d, M = buf.p, wl.head_dim, wl.n_mask
+    S = wl.n_requests * wl.n_kv_heads
+    kept = int(buf.offsets[-1].item())
+    es = 2
+    work = {
+        "select": {"bytes": 4.0 * p.sumN * wl.n_kv_heads + 4.0 * kept},
+        "compact": {"bytes": (4.0 * d * es + 4.0) * kept},
+        "attend": {"bytes": 2.0 * es * p.sumM * wl.n_q_heads * d + 2.0 * es * d * (kept + p.sumM * wl.n_kv_heads),
+                   "flops": 4.0 * M * d * (kept * wl.group + S * wl.group * M)},
+    }
+    calls = {
+        "select": lambda: ctx.maskkv_select(p, buf.scores, buf.budgets, buf.offsets, buf.kept, buf.ws),
+        "compact": lambda: ctx.maskkv_compact(p, x["k_prompt"], x["v_prompt"], buf.kept, buf.offsets, buf.capacity, buf.kc, buf.vc),
+        "attend": lambda: ctx.maskkv_attend(p, live["q_live"], live["k_live"], live["v_live"], buf.kc, buf.vc, buf.offsets,
+                                            buf.capacity, buf.out),
+    }
+    scratch = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    hbm = load_peaks()["hbm_gbs"]
+    out = {"workload": f"configs[4] ragged_serving, one layer: {wl.n_requests} requests, {p.sumN} prompt tokens, {S} segments, "
+                       f"{kept} kept rows; events around single calls include the launch"}
+    for name, call in calls.items():
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize()
+        w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        w0.record()
+        for _ in range(20):
+            call()
+        w1.record()
+        torch.cuda.synchronize()
+        warm_us = 1e3 * w0.elapsed_time(w1) / 20
+        cold = []
+        for i in range(10):
+            scratch.fill_(i)                                           # evicts the call's inputs from L2
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record()
+            call()
+            c1.record()
+            torch.cuda.synchronize()
+            cold.append(1e3 * c0.elapsed_time(c1))
+        cold_us = statistics.median(cold)
+        row = {"warm_us": round(warm_us, 2), "cold_us": round(cold_us, 2), "bytes": work[name]["bytes"],
+               "cold_GB/s": round(work[name]["bytes"] / (cold_us * 1e-6) / 1e9, 1),
+               "cold_frac_of_hbm_peak": round(work[name]["bytes"] / (cold_us * 1e-6) / 1e9 / hbm, 3),
+               "warm_GB/s": round(work[name]["bytes"] / (warm_us * 1e-6) / 1e9, 1)}
+        if "flops" in work[name]:
+            row["warm_TFLOP/s"] = round(work[name]["flops"] / (warm_us * 1e-6) / 1e12, 1)
+        out[name] = row
+    out["status_flags"] = ctx.maskkv_check_status()
+    return out
+
+
 def bench_ours(args):
     rank, world, local_rank = rank_world()
     import torch.distributed as dist
@@ -469,6 +531,10 @@ def bench_ours(args):
         e2e_lazy = {"unavailable": str(exc)[:120]}
     clocks = sampler.stop() if sampler else {}
 
+    # ---- select / compact / attend on a batch: at one layer they are launch- and latency-bound whatever the kernel does
+    # (4-17 MB per call), so a fraction of the memory roof only shows when many segments go into one launch
+    batched = batched_calls(ctx, B, device) if rank == 0 else None
+
     # ---- calibration step of the budget rule (Eq. 8), outside the timed step: a streaming reduction bound by HBM
     importance = None
     if rank == 0:
@@ -602,6 +668,8 @@ def bench_ours(args):
         "roofline_other_calls": other,
         "mean_kept_per_head": mean_kept,
     }
+    if batched is not None:
+        line["batched_calls"] = batched
     if importance is not None:
         gbs = importance["bytes"] / (importance["us"] * 1e-6) / 1e9
         line["refresh_set"] = importance.pop("refresh_set", None)
