@@ -18,7 +18,7 @@ struct maskkv_ctx {
   unsigned long long launches;  // kernels launched through this context so far
   unsigned long long tc_launches;  // of those, kernels of the tcgen05 (tensor-core) paths
   int last_cuda_error;     // cudaError_t of the most recent failed runtime call (0 = none)
-  unsigned force_simt;     // debugging: bit 0 = scoring sweep 1, bit 1 = scoring sweep 2, bit 2 = attention on the FP32 pipes, bit 3 = projection on single CTAs instead of pairs
+  unsigned force_simt;     // debugging: bit 0 = scoring sweep 1, bit 1 = scoring sweep 2, bit 2 = attention on the FP32 pipes, bit 3 = projection on single CTAs instead of pairs, bit 4 / bit 5 = selection always on one CTA per segment / always on clusters
 };
 
 // The descriptor after validation, passed to kernels by value.

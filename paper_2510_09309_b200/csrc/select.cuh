@@ -355,6 +355,239 @@ select_kernel_reg(Shape sh, const float* __restrict__ scores, const int32_t* __r
   cluster.barrier_wait();                                // no CTA leaves while a peer may still read its shared memory
 }
 
+// One CTA per segment, for batches of segments: the keys are staged in shared memory once and every pass over them
+// runs eight rows of 32 keys at a time per warp with the loads ahead of the uses (the cluster kernel above is built
+// for the latency of one layer's few segments; with hundreds of segments its clusters queue up in waves that each
+// wait on cluster barriers).  Passes over all keys: staging (with the common prefix), the first 11-bit histogram,
+// the copy of the threshold bin's keys to a candidate list, and the two emit sweeps; the remaining digits are found
+// on the candidate list (ranked by counting when short).  Warp w owns the contiguous keys [w*span, (w+1)*span).
+// dynamic shared memory: uint32 keys[n_cache] followed by uint32 cand[kSelectCtaCand]; N <= n_cache.
+constexpr int kSelectCtaCand = 4096;
+
+__global__ void __launch_bounds__(kSelectThreads)
+select_kernel_cta(Shape sh, const float* __restrict__ scores, const int32_t* __restrict__ budgets,
+                  const int32_t* __restrict__ offsets, int32_t* __restrict__ kept_idx, int n_cache,
+                  uint32_t* __restrict__ status) {
+  extern __shared__ __align__(16) uint32_t keys_smem[];
+  uint32_t* cand = keys_smem + n_cache;
+  __shared__ uint32_t hist[2048];
+  __shared__ uint32_t sh_digit, sh_remaining, sh_ncand;
+  __shared__ uint32_t warp_gt[kSelectWarps], warp_eq[kSelectWarps], warp_tot[kSelectWarps];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_launch_dependents();
+  pdl_wait();
+  // Blocks are handed out in index order, so the longest prompts go first: block b takes the request that is
+  // number b / H_kv when the requests are sorted by falling length (ties by index) - a ragged batch then ends with
+  // its short segments instead of with a last wave of long ones.
+  if (tid == 0) sh_digit = 0u;
+  __syncthreads();
+  for (int t = tid; t < sh.R; t += kSelectThreads) {
+    const int nt = sh.prompt_cu[t + 1] - sh.prompt_cu[t];
+    int rank = 0;
+    for (int u = 0; u < sh.R; ++u) {
+      const int nu = sh.prompt_cu[u + 1] - sh.prompt_cu[u];
+      rank += (nu > nt || (nu == nt && u < t)) ? 1 : 0;
+    }
+    if (rank == (int)blockIdx.x / sh.Hkv) sh_digit = (uint32_t)t;
+  }
+  __syncthreads();
+  const int r = (int)sh_digit, hk = (int)blockIdx.x % sh.Hkv;
+  const int s = r * sh.Hkv + hk;
+  const int p0 = sh.prompt_cu[r], N = sh.prompt_cu[r + 1] - p0;
+  const int out0 = offsets[s];
+  int k = budgets[s];
+  if (k > N) { k = N; if (threadIdx.x == 0) atomicOr(status, (uint32_t)MASKKV_FLAG_BOUNDS); }
+  if (k <= 0) return;
+  const float* seg = scores + (long long)hk * sh.sumN + p0;
+  if (k == N) {                                          // nothing to evict
+    for (int j = tid; j < N; j += kSelectThreads) kept_idx[out0 + j] = j;
+    return;
+  }
+  __syncthreads();                                       // sh_digit is reused below
+
+  // --- stage the keys and find the bits they all share ---
+  uint32_t k_and = 0xffffffffu, k_or = 0u;
+  auto stage = [&](int j, float f) {
+    const uint32_t key = order_key(f);
+    keys_smem[j] = key;
+    k_and &= key;
+    k_or |= key;
+  };
+  {
+    const int head = min(N, (int)((4 - (((long long)hk * sh.sumN + p0) & 3)) & 3));   // scalars up to the first aligned score
+    const int n4 = (N - head) >> 2;
+    const float4* seg4 = reinterpret_cast<const float4*>(seg + head);
+    for (int j = tid; j < head; j += kSelectThreads) stage(j, seg[j]);
+    for (int i0 = 0; i0 < n4; i0 += 8 * kSelectThreads) {
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int i = i0 + u * kSelectThreads + tid;
+        if (i < n4) v[u] = __ldg(seg4 + i);
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int i = i0 + u * kSelectThreads + tid;
+        if (i < n4) {
+          const int j = head + 4 * i;
+          stage(j, v[u].x); stage(j + 1, v[u].y); stage(j + 2, v[u].z); stage(j + 3, v[u].w);
+        }
+      }
+    }
+    for (int j = head + 4 * n4 + tid; j < N; j += kSelectThreads) stage(j, seg[j]);
+  }
+  k_and = __reduce_and_sync(0xffffffffu, k_and);
+  k_or = __reduce_or_sync(0xffffffffu, k_or);
+  if (lane == 0) { warp_gt[warp] = k_and; warp_eq[warp] = k_or; }
+  for (int b = tid; b < 2048; b += kSelectThreads) hist[b] = 0;
+  if (tid == 0) sh_ncand = 0;
+  __syncthreads();
+  k_and = __reduce_and_sync(0xffffffffu, warp_gt[lane]);
+  k_or = __reduce_or_sync(0xffffffffu, warp_eq[lane]);
+  const int common = __clz(k_and ^ k_or);                // 32 when all keys are equal
+  int bits_left = 32 - common;
+  uint32_t have_mask = common == 0 ? 0u : (common == 32 ? 0xffffffffu : ~(0xffffffffu >> common));
+  uint32_t prefix = k_and & have_mask;
+  uint32_t remaining = (uint32_t)k;
+
+  // this warp's keys: rows of 32 consecutive keys, eight rows per step
+  const int span = ((N + kSelectWarps - 1) / kSelectWarps + 31) & ~31;
+  const int wb = min(warp * span, N), we = min(wb + span, N);
+
+  int ncand = -1;                                        // -1: the candidate list is not in use (all keys still count)
+  if (bits_left > 0) {
+    // first digit: every key matches the common prefix
+    const int width = bits_left >= 11 ? 11 : bits_left;
+    const int shift = bits_left - width;
+    const uint32_t dmask = (1u << width) - 1u;
+    for (int j0 = wb; j0 < we; j0 += 256) {
+      uint32_t kk[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { const int j = j0 + 32 * u + lane; kk[u] = j < we ? keys_smem[j] : 0u; }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { const int j = j0 + 32 * u + lane; if (j < we) atomicAdd(&hist[(kk[u] >> shift) & dmask], 1u); }
+    }
+    __syncthreads();
+    find_digit<kSelectThreads>(hist, 1 << width, remaining, warp_tot, &sh_digit, &sh_remaining);
+    prefix |= sh_digit << shift;
+    remaining = sh_remaining;
+    have_mask |= dmask << shift;
+    bits_left = shift;
+    if (bits_left > 0) {
+      // the keys of the threshold bin become the candidate list (appended per row with one atomic per warp)
+      for (int j0 = wb; j0 < we; j0 += 256) {
+        uint32_t kk[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { const int j = j0 + 32 * u + lane; kk[u] = j < we ? keys_smem[j] : 0u; }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int j = j0 + 32 * u + lane;
+          const bool m = j < we && (kk[u] & have_mask) == prefix;
+          const uint32_t bal = __ballot_sync(0xffffffffu, m);
+          if (bal) {
+            uint32_t pos = 0;
+            if (lane == 0) pos = atomicAdd(&sh_ncand, (uint32_t)__popc(bal));
+            pos = __shfl_sync(0xffffffffu, pos, 0);
+            const uint32_t at = pos + __popc(bal & ((1u << lane) - 1u));
+            if (m && at < (uint32_t)kSelectCtaCand) cand[at] = kk[u];
+          }
+        }
+      }
+      __syncthreads();
+      ncand = (int)sh_ncand;
+      if (ncand > kSelectCtaCand) ncand = -1;            // too many nearly equal scores: keep working on all keys
+    }
+  }
+  if (bits_left > 0 && ncand >= 0 && ncand <= kSelectRankMax) {
+    // a short list: the threshold is the candidate with fewer than `remaining` candidates above it and at least
+    // `remaining` at or above it
+    if (tid < ncand) {
+      const uint32_t mine = cand[tid];
+      uint32_t gt = 0, ge = 0;
+      for (int u = 0; u < ncand; ++u) {
+        const uint32_t c = cand[u];
+        gt += c > mine;
+        ge += c >= mine;
+      }
+      if (gt < remaining && remaining <= ge) { sh_digit = mine; sh_remaining = remaining - gt; }   // equal keys write equal values
+    }
+    __syncthreads();
+    prefix = sh_digit;
+    remaining = sh_remaining;
+    bits_left = 0;
+  }
+#pragma unroll 1
+  while (bits_left > 0) {                                // further digits: on the list, or on all keys when it overflowed
+    const int width = bits_left >= 11 ? 11 : bits_left;
+    const int shift = bits_left - width, bins = 1 << width;
+    const uint32_t dmask = (uint32_t)(bins - 1);
+    __syncthreads();
+    for (int b = tid; b < bins; b += kSelectThreads) hist[b] = 0;
+    __syncthreads();
+    const uint32_t* src = ncand >= 0 ? cand : keys_smem;
+    const int n_src = ncand >= 0 ? ncand : N;
+    for (int j = tid; j < n_src; j += kSelectThreads) {
+      const uint32_t key = src[j];
+      if ((key & have_mask) == prefix) atomicAdd(&hist[(key >> shift) & dmask], 1u);
+    }
+    __syncthreads();
+    find_digit<kSelectThreads>(hist, bins, remaining, warp_tot, &sh_digit, &sh_remaining);
+    prefix |= sh_digit << shift;
+    remaining = sh_remaining;
+    have_mask |= dmask << shift;
+    bits_left = shift;
+  }
+  const uint32_t thr = prefix;                           // threshold key; `remaining` ties are kept, lowest indices first
+
+  // --- emit in ascending index order ---
+  uint32_t n_gt = 0, n_eq = 0;
+  for (int j0 = wb; j0 < we; j0 += 256) {
+    uint32_t kk[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) { const int j = j0 + 32 * u + lane; kk[u] = j < we ? keys_smem[j] : 0u; }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int j = j0 + 32 * u + lane;
+      n_gt += (j < we && kk[u] > thr) ? 1u : 0u;
+      n_eq += (j < we && kk[u] == thr) ? 1u : 0u;
+    }
+  }
+  n_gt = __reduce_add_sync(0xffffffffu, n_gt);
+  n_eq = __reduce_add_sync(0xffffffffu, n_eq);
+  __syncthreads();                                       // warp_gt / warp_eq are reused
+  if (lane == 0) { warp_gt[warp] = n_gt; warp_eq[warp] = n_eq; }
+  __syncthreads();
+  uint32_t eq_before = 0, out_before = 0;                // ties / outputs in lower-index warps
+  for (int w2 = 0; w2 < warp; ++w2) {
+    const uint32_t e2 = warp_eq[w2];
+    const uint32_t take = eq_before >= remaining ? 0u : min(e2, remaining - eq_before);
+    out_before += warp_gt[w2] + take;
+    eq_before += e2;
+  }
+  if (n_gt + n_eq == 0) return;                          // nothing of this warp's range is kept
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  for (int j0 = wb; j0 < we; j0 += 256) {
+    uint32_t kk[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) { const int j = j0 + 32 * u + lane; kk[u] = j < we ? keys_smem[j] : 0u; }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int j = j0 + 32 * u + lane;
+      const bool gt = j < we && kk[u] > thr;
+      const bool eq = j < we && kk[u] == thr;
+      const uint32_t any_bal = __ballot_sync(0xffffffffu, gt || eq);
+      if (any_bal == 0u) continue;                       // warp-uniform: most rows hold no kept key
+      const uint32_t eq_bal = __ballot_sync(0xffffffffu, eq);
+      const bool take = gt || (eq && eq_before + __popc(eq_bal & lt_mask) < remaining);
+      const uint32_t take_bal = __ballot_sync(0xffffffffu, take);
+      if (take) kept_idx[out0 + out_before + __popc(take_bal & lt_mask)] = j;
+      out_before += __popc(take_bal);
+      eq_before += __popc(eq_bal);
+    }
+  }
+}
+
 // dynamic shared memory: uint32 keys[cache_elems] (cache_elems = 0 -> keys are re-read from global)
 __global__ void __launch_bounds__(kSelectThreads)
 select_kernel(Shape sh, const float* __restrict__ scores, const int32_t* __restrict__ budgets,

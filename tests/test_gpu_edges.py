@@ -234,3 +234,31 @@ def test_select_in_registers_crowded_threshold_bin_and_ties(ctx):
     assert np.array_equal(kept[:int(off[-1])].cpu().numpy(), idx)
     assert (kept[int(off[-1]):] == -1).all()
     assert ctx.maskkv_check_status() == 0
+
+
+@pytest.mark.parametrize("force", ["16", "32"])
+def test_both_select_kernels_on_crowded_bins_ties_and_ragged_batches(force, monkeypatch):
+    """The selection runs on clusters (few segments) or on one CTA per segment (batches); bits 4 / 5 of MASKKV_FORCE_SIMT
+    pin the choice.  Both must reproduce the oracle exactly on the crowded-bin / tie / NaN case above and on a ragged
+    batch of 100 segments with budgets from 0 to everything."""
+    from paper_2510_09309_b200 import binding as B
+    monkeypatch.setenv("MASKKV_FORCE_SIMT", force)
+    c = B.Context(0)
+    try:
+        test_select_in_registers_crowded_threshold_bin_and_ties(c)
+        rng = np.random.default_rng(int(force))
+        lens = [int(x) for x in rng.integers(1, 9000, 25)]
+        p, pcu, _ = _problem(c, torch.bfloat16, 4, 4, 64, lens, 4)
+        sc = np.exp(rng.standard_normal((4, pcu[-1]))).astype(np.float32)
+        sc[:, ::7] = np.float32(0.5)                                                   # ties everywhere
+        bud = np.stack([rng.integers(0, n + 1, 4) for n in lens]).astype(np.int32)
+        bud[3] = 0; bud[5] = lens[5]
+        idx, off = O.select(sc, bud, pcu)
+        kept = torch.full((int(off[-1]) + 8,), -1, dtype=torch.int32, device=c.device)
+        c.maskkv_select(p, to_dev(sc), to_dev(bud), to_dev(off), kept)
+        torch.cuda.synchronize()
+        assert np.array_equal(kept[:int(off[-1])].cpu().numpy(), idx)
+        assert (kept[int(off[-1]):] == -1).all()
+        assert c.maskkv_check_status() == 0
+    finally:
+        c.close()
