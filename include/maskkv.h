@@ -19,7 +19,9 @@
  *     pointers that only need to stay valid until the call returns.
  *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default stream) and the
  *     call returns without synchronising.  The only synchronising call is maskkv_check_status.
- *   - Device pointers must be 16-byte aligned (MASKKV_E_ALIGN otherwise); head_dim is contiguous.
+ *   - Device pointers to tensors (Q/K/V/O, scores, kept_idx, the caches, workspaces) must be 16-byte aligned, the small
+ *     int32 / float arrays (budgets, offsets, masses, cumulative lengths) 4-byte aligned (MASKKV_E_ALIGN otherwise);
+ *     head_dim is contiguous.
  *   - Arguments are validated before anything is launched.  A failed validation launches nothing.
  *   - Outputs are fully written for every valid (request, head) segment and untouched elsewhere.
  *     The same inputs give bit-identical outputs on every call (no order-dependent float atomics).
@@ -68,7 +70,11 @@ enum { MASKKV_F32 = 0, MASKKV_BF16 = 1 };
 enum {
   MASKKV_FLAG_TIMEOUT = 1u,   /* a bounded mbarrier wait gave up; that launch's outputs are invalid */
   MASKKV_FLAG_CAPACITY = 2u,  /* maskkv_budget clipped budgets to fit `capacity` */
-  MASKKV_FLAG_BOUNDS = 4u     /* an index read from device memory was out of range and was skipped */
+  MASKKV_FLAG_BOUNDS = 4u,    /* an index read from device memory was out of range and was skipped */
+  MASKKV_FLAG_FALLBACK = 8u   /* a bf16 call the tensor-core kernels should have served ran on the FP32-pipe kernels
+                                 instead (tensor map not encodable, launch refused): results are valid, the call
+                                 was one to two orders of magnitude slower.  Not raised when MASKKV_FORCE_SIMT asks
+                                 for those kernels. */
 };
 
 typedef struct maskkv_ctx maskkv_ctx;
@@ -250,8 +256,11 @@ int maskkv_compact(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* k_pro
 /* One attention step of the live region.  For request r and query head h (KV head h / (H/H_kv)):
  * softmax of scale * q_i . k over the rows [offsets[s], offsets[s+1]) of kc followed by the request's
  * M_r live keys (no mask, own key included); out = weights x [vc rows ; v_live].  bf16: fp32 accumulation
- * and softmax, weights rounded to bf16 before the second product; f32: fp32 throughout.
- * `capacity` is the number of rows kc/vc hold (nothing beyond it is read).  lse_dev (f32 [H][sum_M]) may be NULL. */
+ * and softmax; the tensor-core kernels round the weights to bf16 before the second product (the FP32-pipe kernels that
+ * serve fp32 problems, and bf16 ones under MASKKV_FORCE_SIMT, keep them in fp32).
+ * `capacity` is the number of rows kc/vc hold: nothing beyond it is read, and offsets that point past it are clipped
+ * with MASKKV_FLAG_BOUNDS raised (FP32-pipe kernels) or read as zero rows (tensor-core kernels, through the tensor
+ * map's bounds).  lse_dev (f32 [H][sum_M]) may be NULL. */
 int maskkv_attend(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q_live_dev,
                   const void* k_live_dev, const void* v_live_dev, const void* kc_dev, const void* vc_dev,
                   const int32_t* offsets_dev, int64_t capacity, void* out_dev, float* lse_dev, void* stream);

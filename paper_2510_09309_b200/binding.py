@@ -19,7 +19,7 @@ MASKKV_OK = 0
 MASKKV_E_INVALID, MASKKV_E_UNSUPPORTED, MASKKV_E_ALIGN, MASKKV_E_WORKSPACE = -1, -2, -3, -4
 MASKKV_E_CAPACITY, MASKKV_E_CUDA, MASKKV_E_TIMEOUT = -5, -6, -7
 MASKKV_F32, MASKKV_BF16 = 0, 1
-MASKKV_FLAG_TIMEOUT, MASKKV_FLAG_CAPACITY, MASKKV_FLAG_BOUNDS = 1, 2, 4
+MASKKV_FLAG_TIMEOUT, MASKKV_FLAG_CAPACITY, MASKKV_FLAG_BOUNDS, MASKKV_FLAG_FALLBACK = 1, 2, 4, 8
 
 EXPORTS = (
     "maskkv_create", "maskkv_destroy", "maskkv_status_string", "maskkv_check_status", "maskkv_selftest_wait_expiry", "maskkv_launch_count", "maskkv_last_cuda_error",

@@ -38,7 +38,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kAttendWarps * 32)
 attend_simt(Shape sh, const T* __restrict__ q, const T* __restrict__ kl, const T* __restrict__ vl,
             const T* __restrict__ kc, const T* __restrict__ vc, const int32_t* __restrict__ offsets,
-            const int32_t* __restrict__ q_cu, int sum_q, T* __restrict__ out, float* __restrict__ lse) {
+            const int32_t* __restrict__ q_cu, int sum_q, long long capacity, T* __restrict__ out, float* __restrict__ lse,
+            uint32_t* __restrict__ status) {
   constexpr int E = D / 32;
   const int lane = threadIdx.x & 31;
   const int h = blockIdx.y, r = blockIdx.z, hk = h / sh.g;
@@ -47,7 +48,15 @@ attend_simt(Shape sh, const T* __restrict__ q, const T* __restrict__ kl, const T
   const int i = blockIdx.x * kAttendWarps + (threadIdx.x >> 5);
   if (i >= Mq) return;
   const int s = r * sh.Hkv + hk;
-  const int c0 = offsets[s], nc = offsets[s + 1] - c0;
+  // rows [c0, c0 + nc) of the cache; offsets that point outside the `capacity` rows the cache holds are clipped and
+  // flagged, never dereferenced
+  long long c0 = offsets[s], c1 = offsets[s + 1];
+  if (c0 < 0 || c1 < c0 || c1 > capacity) {
+    if (lane == 0) atomicOr(status, (uint32_t)MASKKV_FLAG_BOUNDS);
+    c0 = c0 < 0 ? 0 : (c0 > capacity ? capacity : c0);
+    c1 = c1 < c0 ? c0 : (c1 > capacity ? capacity : c1);
+  }
+  const int nc = (int)(c1 - c0);
   const int total = nc + M;
 
   float qv[E], acc[E];

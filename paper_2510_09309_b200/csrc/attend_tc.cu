@@ -514,12 +514,15 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
 }
 
 namespace {
+// The opt-in shared-memory size is an attribute of the kernel on ONE device: remembered per device, set with that device
+// current (the entry points hold a device guard).
 template <int D>
-cudaError_t set_attend_attr() {
-  static bool done = false;
-  if (done) return cudaSuccess;
+cudaError_t set_attend_attr(int device) {
+  static bool done[kMaxAttrDevices] = {};
+  if (device < 0 || device >= kMaxAttrDevices) return cudaErrorInvalidDevice;
+  if (done[device]) return cudaSuccess;
   const cudaError_t e = cudaFuncSetAttribute(attend_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, ASmem<D>::kDynamic);
-  done = e == cudaSuccess;
+  done[device] = e == cudaSuccess;
   return e;
 }
 }  // namespace
@@ -552,16 +555,17 @@ int launch_attend_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const int3
   const long long chain = (mean_rows + kATile - 1) / kATile + (sh.maxM + kATile - 1) / kATile;
   const unsigned nsplit = (2 * units <= ctx->sm_count && chain >= kASplitMinTiles) ? 2u : 1u;
   dim3 grid(q_tiles * nsplit, sh.H, sh.R);
+  cudaError_t le;
   if (sh.d == 128) {
-    if (set_attend_attr<128>() != cudaSuccess) return 1;
-    (void)launch_overlapped_cluster(attend_tc<128>, grid, dim3(AWgs<128>::kThreads), ASmem<128>::kDynamic, st, nsplit, mq, mkl, mvl, mkc, mvc,
+    if (set_attend_attr<128>(ctx->device) != cudaSuccess) return 1;
+    le = launch_overlapped_cluster(attend_tc<128>, grid, dim3(AWgs<128>::kThreads), ASmem<128>::kDynamic, st, nsplit, mq, mkl, mvl, mkc, mvc,
                                   sh, offsets, q_cu, sum_q, (__nv_bfloat16*)out, lse, ctx->status_dev);
   } else {
-    if (set_attend_attr<64>() != cudaSuccess) return 1;
-    (void)launch_overlapped_cluster(attend_tc<64>, grid, dim3(AWgs<64>::kThreads), ASmem<64>::kDynamic, st, nsplit, mq, mkl, mvl, mkc, mvc,
+    if (set_attend_attr<64>(ctx->device) != cudaSuccess) return 1;
+    le = launch_overlapped_cluster(attend_tc<64>, grid, dim3(AWgs<64>::kThreads), ASmem<64>::kDynamic, st, nsplit, mq, mkl, mvl, mkc, mvc,
                                   sh, offsets, q_cu, sum_q, (__nv_bfloat16*)out, lse, ctx->status_dev);
   }
-  // a failed launch is reported by the caller through cudaGetLastError
+  if (le != cudaSuccess) { cudaGetLastError(); return 1; }   // a refused launch: the caller falls back and flags it
   return 0;
 }
 

@@ -18,7 +18,9 @@ struct maskkv_ctx {
   unsigned long long launches;  // kernels launched through this context so far
   unsigned long long tc_launches;  // of those, kernels of the tcgen05 (tensor-core) paths
   int last_cuda_error;     // cudaError_t of the most recent failed runtime call (0 = none)
-  unsigned force_simt;     // debugging: bit 0 = scoring sweep 1, bit 1 = scoring sweep 2, bit 2 = attention on the FP32 pipes, bit 3 = projection on single CTAs instead of pairs, bit 4 / bit 5 = selection always on one CTA per segment / always on clusters
+  uint32_t host_flags;     // status bits raised on the host (MASKKV_FLAG_FALLBACK); reported and cleared by maskkv_check_status
+  unsigned force_simt;     // MASKKV_FORCE_SIMT, debugging: bit 0 = scoring sweep 1, bit 1 = scoring sweep 2, bit 2 = attention on the FP32 pipes
+  unsigned kernel_choice;  // MASKKV_KERNEL_CHOICE, debugging: bit 0 = projection on single CTAs instead of pairs, bit 1 / bit 2 = selection always on one CTA per segment / always on clusters
 };
 
 // The descriptor after validation, passed to kernels by value.
@@ -32,6 +34,8 @@ struct Shape {
 };
 
 namespace mkv {
+
+constexpr int kMaxAttrDevices = 64;   // per-device "attribute set" tables of the kernels that opt into large shared memory
 
 // Programmatic dependent launch.  Every kernel of the layer path is launched with launch_overlapped(): its blocks may
 // be scheduled while the previous kernel of the stream is still running, which hides the launch latency and the

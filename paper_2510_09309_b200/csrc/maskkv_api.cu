@@ -131,6 +131,7 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, co
     if (tc_ok && !(ctx->force_simt & 1u))
       tc1 = mkv::tc::launch_score_stats_tc(ctx, sh, desc->prompt_cu, desc->live_cu, q, kp, km, part, w.C, seg_cnt, st) == 0;
     if (tc1) { ++ctx->tc_launches; ++n; }
+    else if (tc_ok && !(ctx->force_simt & 1u)) ctx->host_flags |= MASKKV_FLAG_FALLBACK;   // nobody asked for the FP32 pipes
     if (!tc1) {
       const int q_tiles = (sh.maxM + mkv::kSimtThreads - 1) / mkv::kSimtThreads;
       dim3 g1((unsigned)((sh.maxN + sh.maxM + mkv::kStatsChunk - 1) / mkv::kStatsChunk), sh.H, sh.R * q_tiles);
@@ -149,6 +150,7 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, co
     tc2 = mkv::tc::launch_score_colsum_tc(ctx, sh, desc->prompt_cu, desc->live_cu, q, kp, km, lse, tc1 ? part : nullptr, w.C, rw,
                                           scores, colpart, mass_part, w.Tmax, seg_cnt, mass_p, mass_m, scores_live, any_without_voters, st,
                                           &launched) == 0;
+    if (!tc2) { ctx->host_flags |= MASKKV_FLAG_FALLBACK; n += launched; }
     if (tc2) {
       ++ctx->tc_launches;
       n += launched;
@@ -171,11 +173,13 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, co
 
 template <typename T, int D>
 int launch_attend_simt(maskkv_ctx* ctx, const Shape& sh, const void* q, const int32_t* q_cu, int sum_q, int max_q, const void* kl,
-                       const void* vl, const void* kc, const void* vc, const int32_t* offsets, void* out, float* lse, cudaStream_t st) {
+                       const void* vl, const void* kc, const void* vc, const int32_t* offsets, long long capacity, void* out, float* lse,
+                       cudaStream_t st) {
   if (max_q == 0) return MASKKV_OK;
   dim3 grid((max_q + mkv::kAttendWarps - 1) / mkv::kAttendWarps, sh.H, sh.R);
   mkv::attend_simt<T, D><<<grid, mkv::kAttendWarps * 32, 0, st>>>(sh, (const T*)q, (const T*)kl, (const T*)vl, (const T*)kc,
-                                                                   (const T*)vc, offsets, q_cu, sum_q, (T*)out, lse);
+                                                                   (const T*)vc, offsets, q_cu, sum_q, capacity, (T*)out, lse,
+                                                                   ctx->status_dev);
   return launch_status(ctx, 1);
 }
 
@@ -246,6 +250,7 @@ int maskkv_create(maskkv_ctx** out, int device) {
       qres != cudaDriverEntryPointSuccess)
     ctx->encode_tiled = nullptr;
   if (const char* e = getenv("MASKKV_FORCE_SIMT")) ctx->force_simt = (unsigned)strtoul(e, nullptr, 0);
+  if (const char* e = getenv("MASKKV_KERNEL_CHOICE")) ctx->kernel_choice = (unsigned)strtoul(e, nullptr, 0);
   cudaFuncSetAttribute(mkv::select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - mkv::kSelectStaticSmem);
   cudaFuncSetAttribute(mkv::select_kernel_cta, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - mkv::kSelectStaticSmem);
   cudaFuncSetAttribute(mkv::budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
@@ -272,6 +277,8 @@ int maskkv_check_status(maskkv_ctx* ctx, void* stream, uint32_t* flags_out) {
   if (cudaMemcpyAsync(&flags, ctx->status_dev, sizeof(flags), cudaMemcpyDeviceToHost, st) != cudaSuccess) return MASKKV_E_CUDA;
   if (cudaMemsetAsync(ctx->status_dev, 0, 8, st) != cudaSuccess) return MASKKV_E_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return MASKKV_E_CUDA;
+  flags |= ctx->host_flags;
+  ctx->host_flags = 0;
   if (flags_out) *flags_out = flags;
   return (flags & MASKKV_FLAG_TIMEOUT) ? MASKKV_E_TIMEOUT : MASKKV_OK;
 }
@@ -527,9 +534,12 @@ int maskkv_select(maskkv_ctx* ctx, const maskkv_desc_t* desc, const float* score
   int rc = resolve(desc, &sh);
   if (rc != MASKKV_OK) return rc;
   if (scores_dev == nullptr || budgets_dev == nullptr || offsets_dev == nullptr || kept_idx_dev == nullptr) return MASKKV_E_INVALID;
+  if (!aligned16(scores_dev) || !aligned16(kept_idx_dev) || (reinterpret_cast<uintptr_t>(budgets_dev) & 3u) ||
+      (reinterpret_cast<uintptr_t>(offsets_dev) & 3u))
+    return MASKKV_E_ALIGN;
   DeviceGuard guard(ctx->device);
   const int cta_cache = (ctx->smem_optin - mkv::kSelectStaticSmem) / 4 - mkv::kSelectCtaCand;
-  const int sel_force = (ctx->force_simt & 16u) ? 2 : (ctx->force_simt & 32u) ? 1 : 0;   // debugging: pin the kernel
+  const int sel_force = (ctx->kernel_choice & 2u) ? 2 : (ctx->kernel_choice & 4u) ? 1 : 0;   // debugging: pin the kernel
   // more segments than one wave of clusters (two CTAs per SM): one CTA per segment with the keys in shared memory gets
   // through faster (measured: 128 / 256 segments of up to 32k keys)
   const bool batch = (long long)sh.R * sh.Hkv * mkv::kSelectCluster > 2LL * ctx->sm_count;
@@ -621,14 +631,16 @@ int maskkv_attend_rows(maskkv_ctx* ctx, const maskkv_desc_t* desc, const void* q
     return MASKKV_E_ALIGN;
   DeviceGuard guard(ctx->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (mkv::tc::attend_tc_supported(ctx, sh) && !(ctx->force_simt & 4u) &&
-      mkv::tc::launch_attend_tc(ctx, sh, q_rows_dev, q_cu, sum_q, max_q, k_live_dev, v_live_dev, kc_dev, vc_dev, capacity, offsets_dev,
-                                out_rows_dev, lse_rows_dev, st) == 0) {
-    ++ctx->tc_launches;
-    return launch_status(ctx, 1);
+  if (mkv::tc::attend_tc_supported(ctx, sh) && !(ctx->force_simt & 4u)) {
+    if (mkv::tc::launch_attend_tc(ctx, sh, q_rows_dev, q_cu, sum_q, max_q, k_live_dev, v_live_dev, kc_dev, vc_dev, capacity, offsets_dev,
+                                  out_rows_dev, lse_rows_dev, st) == 0) {
+      ++ctx->tc_launches;
+      return launch_status(ctx, 1);
+    }
+    ctx->host_flags |= MASKKV_FLAG_FALLBACK;               // the FP32-pipe kernel below takes over; nobody asked for it
   }
 #define MKV_ATTEND(T, D) launch_attend_simt<T, D>(ctx, sh, q_rows_dev, q_cu, sum_q, max_q, k_live_dev, v_live_dev, kc_dev, vc_dev, \
-                                                  offsets_dev, out_rows_dev, lse_rows_dev, st)
+                                                  offsets_dev, (long long)capacity, out_rows_dev, lse_rows_dev, st)
   if (sh.dtype == MASKKV_F32) return sh.d == 64 ? MKV_ATTEND(float, 64) : MKV_ATTEND(float, 128);
   return sh.d == 64 ? MKV_ATTEND(__nv_bfloat16, 64) : MKV_ATTEND(__nv_bfloat16, 128);
 #undef MKV_ATTEND

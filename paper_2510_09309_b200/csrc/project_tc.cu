@@ -231,7 +231,7 @@ int launch_project_tc(maskkv_ctx* ctx, const void* hidden, long long n_tokens, i
     ++*launches;
   }
   // More than 128 masked rows: a pair of CTAs per tile (project_tc2.cu); otherwise the second CTA would have no rows.
-  if (n_mask > 128 && !(ctx->force_simt & 8u) && project_tc2_supported(ctx)) {
+  if (n_mask > 128 && !(ctx->kernel_choice & 1u) && project_tc2_supported(ctx)) {
     if (launch_project_gemm_tc2(ctx, a_base, a_stride, width, n_mask, w_vocab, vocab, w_row_stride, out, ld_out, out_bf16, st) != 0)
       return *launches == 0 ? 1 : 2;
     ++*launches;

@@ -76,11 +76,12 @@ __device__ __forceinline__ void umma_ss_pair(uint32_t d_tmem, uint64_t adesc, ui
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// Arrives on `bar` in both CTAs of the pair once every MMA issued so far by this thread has completed.
-__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-               ::"r"(smem_u32(bar)), "h"((uint16_t)3)
-               : "memory");
+// Arrives on `bar` in both CTAs of the pair once every MMA issued so far by this thread has completed: two plain
+// commits, one on this CTA's barrier and one on the peer's copy of it (address from mapa); both track the same MMAs.
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar, uint32_t peer_rank) {
+  const uint32_t own = smem_u32(bar);
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(own) : "memory");
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(map_to_cta(own, peer_rank)) : "memory");
 }
 
 __global__ void __launch_bounds__(k2Threads, 1)
@@ -169,9 +170,9 @@ project_gemm_tc2(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             for (int kk = 0; kk < kPBK / 16; ++kk)
               umma_ss_pair(tmem_base + acc * 256, make_desc(a_lo + ((kk * 32) >> 4), kDescHiSw128),
                            make_desc(b_lo + ((kk * 32) >> 4), kDescHiSw128), idesc, (kb | kk) != 0);
-            umma_commit_pair(bars.empty + stage);
+            umma_commit_pair(bars.empty + stage, rank ^ 1u);
           }
-          if (ok) umma_commit_pair(bars.tfull + acc);
+          if (ok) umma_commit_pair(bars.tfull + acc, rank ^ 1u);
         }
       }
     }

@@ -786,13 +786,16 @@ long long flat_tiles(const Shape& sh, const int32_t* prompt_cu, const int32_t* l
   return F;
 }
 
+// The opt-in shared-memory size is an attribute of the kernel on ONE device: remembered per device, set with that device
+// current (the entry points hold a device guard).
 template <int D>
-cudaError_t set_smem_attr() {
-  static bool done = false;
-  if (done) return cudaSuccess;
+cudaError_t set_smem_attr(int device) {
+  static bool done[kMaxAttrDevices] = {};
+  if (device < 0 || device >= kMaxAttrDevices) return cudaErrorInvalidDevice;
+  if (done[device]) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(score_stats_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::kDynamic);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(score_colsum_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::kDynamic);
-  done = e == cudaSuccess;
+  done[device] = e == cudaSuccess;
   return e;
 }
 
@@ -821,15 +824,17 @@ int launch_score_stats_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* promp
   const long long F = flat_tiles(sh, prompt_cu_host, live_cu_host, kWalkStats);
   if (F <= 0) return 1;
   const int grid = (int)(F < ctx->sm_count ? F : ctx->sm_count);
+  cudaError_t le;
   if (sh.d == 128) {
-    if (set_smem_attr<128>() != cudaSuccess) return 1;
-    launch_overlapped(score_stats_tc<128>, dim3(grid), dim3(kThreads), Smem<128>::kDynamic, st, m.q, m.kp, m.km, sh, part, C, F, seg_cnt,
+    if (set_smem_attr<128>(ctx->device) != cudaSuccess) return 1;
+    le = launch_overlapped(score_stats_tc<128>, dim3(grid), dim3(kThreads), Smem<128>::kDynamic, st, m.q, m.kp, m.km, sh, part, C, F, seg_cnt,
                       ctx->status_dev);
   } else {
-    if (set_smem_attr<64>() != cudaSuccess) return 1;
-    launch_overlapped(score_stats_tc<64>, dim3(grid), dim3(kThreads), Smem<64>::kDynamic, st, m.q, m.kp, m.km, sh, part, C, F, seg_cnt,
+    if (set_smem_attr<64>(ctx->device) != cudaSuccess) return 1;
+    le = launch_overlapped(score_stats_tc<64>, dim3(grid), dim3(kThreads), Smem<64>::kDynamic, st, m.q, m.kp, m.km, sh, part, C, F, seg_cnt,
                       ctx->status_dev);
   }
+  if (le != cudaSuccess) { cudaGetLastError(); return 1; }   // a refused launch: the caller falls back and flags it
   return 0;
 }
 
@@ -862,7 +867,7 @@ int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prom
   const int grid = (int)(F < ctx->sm_count ? F : ctx->sm_count);
   const long long F1 = flat_tiles(sh, prompt_cu_host, live_cu_host, kWalkStats);   // sweep 1's walk, for its partials
   const int G1 = (int)(F1 < ctx->sm_count ? F1 : ctx->sm_count);
-  if (sh.d == 128 ? set_smem_attr<128>() != cudaSuccess : set_smem_attr<64>() != cudaSuccess) return 1;
+  if (sh.d == 128 ? set_smem_attr<128>(ctx->device) != cudaSuccess : set_smem_attr<64>(ctx->device) != cudaSuccess) return 1;
   *launches = 0;
   if (any_without_voters && !split) {                      // with several query blocks the reduce kernel writes the zeros
     dim3 gz(score_tc_max_tiles(sh), sh.Hkv, sh.R);
@@ -870,12 +875,14 @@ int launch_score_colsum_tc(maskkv_ctx* ctx, const Shape& sh, const int32_t* prom
     ++*launches;
   }
   float* cp = split ? colpart : nullptr;
+  cudaError_t le;
   if (sh.d == 128)
-    launch_overlapped(score_colsum_tc<128>, dim3(grid), dim3(kThreads), Smem<128>::kDynamic, st, m.q, m.kp, m.km, sh, lse, part, C, F1, G1,
+    le = launch_overlapped(score_colsum_tc<128>, dim3(grid), dim3(kThreads), Smem<128>::kDynamic, st, m.q, m.kp, m.km, sh, lse, part, C, F1, G1,
                       w, scores, cp, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, scores_live, ctx->status_dev);
   else
-    launch_overlapped(score_colsum_tc<64>, dim3(grid), dim3(kThreads), Smem<64>::kDynamic, st, m.q, m.kp, m.km, sh, lse, part, C, F1, G1,
+    le = launch_overlapped(score_colsum_tc<64>, dim3(grid), dim3(kThreads), Smem<64>::kDynamic, st, m.q, m.kp, m.km, sh, lse, part, C, F1, G1,
                       w, scores, cp, mass_part, Tmax, seg_cnt, mass_p, mass_m, F, scores_live, ctx->status_dev);
+  if (le != cudaSuccess) { cudaGetLastError(); return 1; }   // a refused launch: the caller falls back and flags it
   ++*launches;
   if (split) {
     dim3 gr(Tmax, sh.Hkv, sh.R);

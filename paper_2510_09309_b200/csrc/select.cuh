@@ -116,7 +116,10 @@ select_kernel_reg(Shape sh, const float* __restrict__ scores, const int32_t* __r
   __shared__ __align__(16) uint32_t hist[2048];
   __shared__ uint32_t sh_digit, sh_remaining, sh_ncand;
   __shared__ uint32_t warp_gt[kSelectRegWarps], warp_eq[kSelectRegWarps], warp_tot[kSelectRegWarps];
-  __shared__ uint32_t and_or[2];
+  __shared__ uint32_t and_or[2];                         // this CTA's (AND, OR) of its keys, read by the peers
+  __shared__ uint32_t gt_eq[2];                          // this CTA's (above, at) threshold counts, read by the peers: a pair of
+                                                         // its own, because with all keys equal no cluster barrier lies between a
+                                                         // peer's read of and_or and this CTA's write of its counts
 
   const int s = blockIdx.x / kSelectCluster;
   const int q = (int)cluster.block_rank();
@@ -311,7 +314,7 @@ select_kernel_reg(Shape sh, const float* __restrict__ scores, const int32_t* __r
   if (warp == 0) {                                       // this CTA's totals, for the CTAs after it
     const uint32_t g = __reduce_add_sync(0xffffffffu, lane < kSelectRegWarps ? warp_gt[lane] : 0u);
     const uint32_t e = __reduce_add_sync(0xffffffffu, lane < kSelectRegWarps ? warp_eq[lane] : 0u);
-    if (lane == 0) { and_or[0] = g; and_or[1] = e; }
+    if (lane == 0) { gt_eq[0] = g; gt_eq[1] = e; }
   }
   cluster.sync();
   // ties / outputs that precede this warp: the lower CTAs as wholes, then the lower warps of this CTA
@@ -320,7 +323,7 @@ select_kernel_reg(Shape sh, const float* __restrict__ scores, const int32_t* __r
     uint32_t pg[kSelectCluster], pe[kSelectCluster];
 #pragma unroll
     for (int c = 0; c < kSelectCluster; ++c) {
-      const uint32_t* peer = cluster.map_shared_rank(and_or, c);
+      const uint32_t* peer = cluster.map_shared_rank(gt_eq, c);
       pg[c] = c < q ? peer[0] : 0u;
       pe[c] = c < q ? peer[1] : 0u;
     }

@@ -236,13 +236,13 @@ def test_select_in_registers_crowded_threshold_bin_and_ties(ctx):
     assert ctx.maskkv_check_status() == 0
 
 
-@pytest.mark.parametrize("force", ["16", "32"])
+@pytest.mark.parametrize("force", ["2", "4"])
 def test_both_select_kernels_on_crowded_bins_ties_and_ragged_batches(force, monkeypatch):
-    """The selection runs on clusters (few segments) or on one CTA per segment (batches); bits 4 / 5 of MASKKV_FORCE_SIMT
+    """The selection runs on clusters (few segments) or on one CTA per segment (batches); bits 1 / 2 of MASKKV_KERNEL_CHOICE
     pin the choice.  Both must reproduce the oracle exactly on the crowded-bin / tie / NaN case above and on a ragged
     batch of 100 segments with budgets from 0 to everything."""
     from paper_2510_09309_b200 import binding as B
-    monkeypatch.setenv("MASKKV_FORCE_SIMT", force)
+    monkeypatch.setenv("MASKKV_KERNEL_CHOICE", force)
     c = B.Context(0)
     try:
         test_select_in_registers_crowded_threshold_bin_and_ties(c)
@@ -262,3 +262,65 @@ def test_both_select_kernels_on_crowded_bins_ties_and_ragged_batches(force, monk
         assert c.maskkv_check_status() == 0
     finally:
         c.close()
+
+
+@pytest.mark.parametrize("segments", [8, 48])
+def test_cluster_select_when_every_key_of_a_segment_is_equal(segments, monkeypatch):
+    """All scores of a segment equal (zeros, or all NaN) with 0 < k < N: the keys share all 32 bits, so the cluster
+    kernel skips every radix pass and goes straight from the exchange of the common prefix to the exchange of the
+    threshold counts.  The kept set is the k lowest indices.  Repeated, on the one-wave variant (8 segments) and the
+    two-CTAs-per-SM variant (48 segments), with the cluster kernel pinned."""
+    from paper_2510_09309_b200 import binding as B
+    monkeypatch.setenv("MASKKV_KERNEL_CHOICE", "4")
+    c = B.Context(0)
+    try:
+        rng = np.random.default_rng(segments)
+        heads = 4
+        lens = [int(x) for x in rng.integers(200, 32769, segments // heads)]
+        lens[0] = 32768
+        p, pcu, _ = _problem(c, torch.bfloat16, heads, heads, 64, lens, 4)
+        sc = np.zeros((heads, pcu[-1]), np.float32)
+        sc[1::2] = np.float32("nan")                                               # odd heads: all NaN
+        bud = np.stack([rng.integers(1, n, heads) for n in lens]).astype(np.int32)
+        idx, off = O.select(sc, bud, pcu)
+        for r in range(len(lens)):
+            for h in range(heads):
+                s0 = r * heads + h
+                assert np.array_equal(idx[off[s0]:off[s0 + 1]], np.arange(bud[r, h]))
+        scd, budd, offd = to_dev(sc), to_dev(bud), to_dev(off)
+        kept = torch.empty((int(off[-1]),), dtype=torch.int32, device=c.device)
+        ref = torch.from_numpy(idx).to(c.device)
+        for it in range(300):
+            kept.fill_(-1)
+            c.maskkv_select(p, scd, budd, offd, kept)
+            assert torch.equal(kept, ref), f"repeat {it}"
+        assert c.maskkv_check_status() == 0
+    finally:
+        c.close()
+
+
+def test_attend_fp32_offsets_beyond_capacity_are_clipped_and_flagged(ctx):
+    """The FP32-pipe attention is told how many rows the cache holds: offsets that point past them (a caller's mistake)
+    must raise MASKKV_FLAG_BOUNDS and must not be followed.  The rows behind the declared capacity hold NaN here, so a
+    read past it would show in the output."""
+    from paper_2510_09309_b200 import binding as B
+    wl = synth.scaled(synth.config(1), "cap_clip", prompt_lens=(64,), n_mask=16, n_q_heads=2, n_kv_heads=2, mean_budget=8)
+    live = {k: to_dev(v) for k, v in synth.live_inputs(wl, 0, 0, "cpu").items()}
+    p = B.Problem(wl.torch_dtype, 2, 2, wl.head_dim, wl.prompt_cu(), wl.live_cu(), ctx.device)
+    capacity = 12
+    store_k = torch.full((40, wl.head_dim), float("nan"), dtype=torch.float32, device=ctx.device)
+    store_v = torch.full((40, wl.head_dim), float("nan"), dtype=torch.float32, device=ctx.device)
+    store_k[:capacity] = torch.randn(capacity, wl.head_dim, device=ctx.device)
+    store_v[:capacity] = torch.randn(capacity, wl.head_dim, device=ctx.device)
+    offsets = to_dev(np.array([0, 8, 30], np.int32))            # the second segment claims rows 8..29 of a 12-row cache
+    out = torch.zeros((16, 2, wl.head_dim), dtype=torch.float32, device=ctx.device)
+    lse = torch.zeros((2, 16), dtype=torch.float32, device=ctx.device)
+    assert ctx.maskkv_check_status() == 0
+    ctx.maskkv_attend(p, live["q_live"], live["k_live"], live["v_live"], store_k, store_v, offsets, capacity, out, lse)
+    torch.cuda.synchronize()
+    assert ctx.maskkv_check_status() & B.MASKKV_FLAG_BOUNDS
+    assert torch.isfinite(out).all() and torch.isfinite(lse).all()
+    # the clipped segment is rows 8..11: the oracle on that cache gives the same numbers
+    ref, _ = O.attend(live["q_live"].cpu(), live["k_live"].cpu(), live["v_live"].cpu(), store_k[:capacity].cpu(),
+                      store_v[:capacity].cpu(), np.array([0, 8, 12], np.int32), wl.live_cu(), 2)
+    assert np.abs(out.cpu().numpy() - ref).max() <= 1e-5

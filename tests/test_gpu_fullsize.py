@@ -1,4 +1,4 @@
-"""GPU parity at the full BASELINE sizes, in the launch configuration bench.py times.
+"""GPU parity at the full sizes of the five workloads, in the launch configuration bench.py times.
 
 Inputs are generated on the device (seeded), the whole path runs on the device, and the oracle
 recomputes sampled (request, head) units one by one from the same bytes copied to the host:
@@ -25,9 +25,10 @@ def ctx():
     c.close()
 
 
-def _run_and_check(ctx, wl, layer, k_l, alpha, sample, attend_steps=1):
-    """sample: list of (request, kv_head)."""
-    x = synth.layer_inputs(wl, layer, "cuda")
+def _run_and_check(ctx, wl, layer, k_l, alpha, sample, attend_steps=1, x=None):
+    """sample: list of (request, kv_head); x: the layer's inputs when the caller already holds them."""
+    if x is None:
+        x = synth.layer_inputs(wl, layer, "cuda")
     run = LayerRun(ctx, wl, k_l=k_l)
     run.score(x)
     run.budget(alpha=alpha)
@@ -93,16 +94,22 @@ def _run_and_check(ctx, wl, layer, k_l, alpha, sample, attend_steps=1):
 
 
 def test_config3_llada_32k_layers(ctx):
-    """configs[2]: N=32768, M=256, 32 heads, adaptive budgets; a boundary and a middle layer."""
+    """configs[2]: N=32768, M=256, 32 heads, adaptive budgets.  Layers 0 and 31 (boundary group, 512 per head on
+    average), 1, 15 and 30 (middle group, 238); on each one information head (even) and one structure head (odd)
+    against the oracle, everything else through the properties."""
     from paper_2510_09309_b200 import binding as B
     wl = synth.config(3)
     k_layers = B.maskkv_layer_budgets(wl.total_budget(), wl.beta, wl.layer_importance())
     assert k_layers == O.layer_budgets(wl.total_budget(), wl.beta, wl.layer_importance())
-    assert k_layers[0] == 512 and k_layers[1] == 238
-    for layer, sample in ((0, [(0, 0), (0, 31)]), (1, [(0, 5), (0, 16)])):
+    assert k_layers[0] == 512 and k_layers[1] == 238 and k_layers[31] == 512 and k_layers[15] == 238
+    samples = {0: [(0, 0), (0, 31)], 1: [(0, 5), (0, 16)], 15: [(0, 14), (0, 9)], 30: [(0, 22), (0, 27)],
+               31: [(0, 30), (0, 1)]}
+    for layer, sample in samples.items():
         run = _run_and_check(ctx, wl, layer, k_layers[layer], wl.alpha, sample)
         bud = run.budgets.cpu().numpy()[0]
         assert bud[0::2].mean() > 2 * bud[1::2].mean()       # information heads get the larger share
+        del run
+        torch.cuda.empty_cache()
 
 
 def test_config4_dream_gqa_16k(ctx):
@@ -113,12 +120,28 @@ def test_config4_dream_gqa_16k(ctx):
 
 
 def test_config5_ragged_serving(ctx):
-    """configs[4]: 8 requests with prompts from 1024 to 32768 tokens, budget sweep incl. the clamp at B=1024."""
+    """configs[4]: 8 requests with prompts from 1024 to 32768 tokens; the whole budget sweep B = 64 ... 1024 (the
+    clamp at B = 1024 included), each followed by 16 consecutive attention steps with fresh live tensors.  Sampled
+    against the oracle: per budget two (request, head) units, chosen so that over the sweep every request and both
+    kinds of head occur; the last layer (boundary group) for the sweep, the first and a middle layer at B = 256."""
     from paper_2510_09309_b200 import binding as B
     wl = synth.config(5)
-    for budget, sample, steps in ((64, [(3, 7)], 1), (1024, [(0, 2), (6, 30)], 2)):
+    sweep = ((64, [(3, 7), (0, 12)]), (128, [(1, 0), (7, 21)]), (256, [(2, 9), (5, 4)]), (512, [(4, 18), (6, 3)]),
+             (1024, [(0, 2), (6, 30)]))
+    x = synth.layer_inputs(wl, 31, "cuda")
+    for budget, sample in sweep:
         w2 = synth.scaled(wl, f"ragged_B{budget}", mean_budget=budget)
         k_layers = B.maskkv_layer_budgets(w2.total_budget(), w2.beta, w2.layer_importance())
-        run = _run_and_check(ctx, w2, 31, k_layers[31], w2.alpha, sample, attend_steps=steps)
+        assert k_layers == O.layer_budgets(w2.total_budget(), w2.beta, w2.layer_importance())
+        run = _run_and_check(ctx, w2, 31, k_layers[31], w2.alpha, sample, attend_steps=16, x=x)
         if budget == 1024:
             assert (run.budgets.cpu().numpy()[0] == 1024).any()   # the 1024-token prompt is clamped
+        del run
+        torch.cuda.empty_cache()
+    del x
+    torch.cuda.empty_cache()
+    w2 = synth.scaled(wl, "ragged_B256", mean_budget=256)
+    k_layers = B.maskkv_layer_budgets(w2.total_budget(), w2.beta, w2.layer_importance())
+    for layer, sample in ((0, [(7, 6)]), (16, [(3, 25)])):
+        _run_and_check(ctx, w2, layer, k_layers[layer], w2.alpha, sample, attend_steps=2)
+        torch.cuda.empty_cache()

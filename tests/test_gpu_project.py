@@ -97,13 +97,13 @@ def test_rows_in_place_with_strided_operands(ctx):
 
 
 def test_single_cta_and_pair_kernels_agree_bit_for_bit(monkeypatch):
-    """More than 128 masked rows run on pairs of CTAs; bit 3 of MASKKV_FORCE_SIMT (read when a context is created) keeps
+    """More than 128 masked rows run on pairs of CTAs; bit 0 of MASKKV_KERNEL_CHOICE (read when a context is created) keeps
     them on the one-CTA kernel.  Both add the k blocks in the same order, so the logits must be identical."""
     from paper_2510_09309_b200 import binding as B
     x = synth.project_inputs(700, 448, 3000, 300, "cuda", seed=4)
     outs = []
-    for force in ("0", "8"):
-        monkeypatch.setenv("MASKKV_FORCE_SIMT", force)
+    for force in ("0", "1"):
+        monkeypatch.setenv("MASKKV_KERNEL_CHOICE", force)
         c = B.Context(0)
         try:
             out, _ = _run(c, x)
@@ -122,8 +122,8 @@ def test_seeded_shape_sweep_pair_kernel_against_one_cta_kernel_and_oracle(monkey
     rng = np.random.default_rng(20251009)
     shapes = [(int(rng.integers(129, 701)), int(rng.integers(8, 140)) * 8, int(rng.integers(40, 9000))) for _ in range(20)]
     outs = {}
-    for force in ("0", "8"):
-        monkeypatch.setenv("MASKKV_FORCE_SIMT", force)
+    for force in ("0", "1"):
+        monkeypatch.setenv("MASKKV_KERNEL_CHOICE", force)
         c = B.Context(0)
         try:
             for i, (n_mask, width, vocab) in enumerate(shapes):

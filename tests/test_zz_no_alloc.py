@@ -2,10 +2,10 @@
 loop with a fixed, fully handed-out memory pool; a plugin that receives tensors but no allocator).
 Its scratch is an 8 MiB array inside the library instead of a caller-provided workspace.
 
-The check: called through the C ABI twice in a row on different inputs, it must give the same scores
-and masses as maskkv_score does with a caller-allocated workspace (same kernels, so the same tolerance
-as the other scoring tests holds with room to spare), and it must refuse problems whose scratch would
-not fit.  This file sorts last so that a run that stops at the first failure has already covered
+The check: called through the C ABI twice in a row on different inputs, it must give the same bits as
+maskkv_score does with a caller-allocated workspace (the two run the same kernels on the same inputs),
+it must agree with the CPU oracle within the scoring tolerance like every other scoring test, and it
+must refuse problems whose scratch would not fit.  This file sorts last so that a run that stops at the first failure has already covered
 everything else; it also passes when run on its own in a fresh process."""
 import ctypes
 
@@ -13,8 +13,9 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import maskkv_oracle as O
 from paper_2510_09309_b200 import synth
-from pipeline import SCORE_RTOL, to_dev
+from pipeline import assert_scores_close, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -36,7 +37,8 @@ def _score_both_ways(ctx, B, wl, layer):
             ctx.maskkv_score(p, xd["q_mask"], xd["k_prompt"], xd["k_mask"], scores, mp, mm, ws)
         torch.cuda.synchronize()
         outs.append((scores.cpu().numpy(), mp.cpu().numpy(), mm.cpu().numpy()))
-    return outs
+    ref = O.score(x["q_mask"], x["k_prompt"], x["k_mask"], wl.prompt_cu(), wl.live_cu())
+    return outs, ref
 
 
 def test_noalloc_matches_workspace_call_twice_in_a_row():
@@ -49,11 +51,14 @@ def test_noalloc_matches_workspace_call_twice_in_a_row():
         (synth.config(1), 0),
     ]
     for wl, layer in cases:
-        (s0, p0, m0), (s1, p1, m1) = _score_both_ways(ctx, B, wl, layer)
+        ((s0, p0, m0), (s1, p1, m1)), (ref_s, ref_p, ref_m) = _score_both_ways(ctx, B, wl, layer)
         assert np.isfinite(s1).all() and np.isfinite(p1).all() and np.isfinite(m1).all()
-        for a, b in ((s0, s1), (p0, p1), (m0, m1)):
-            rel = np.abs(a.astype(np.float64) - b) / np.maximum(np.abs(a), 1e-30)
-            assert rel.max() <= SCORE_RTOL
+        # the same kernels on the same inputs: the same bits, wherever the scratch lives
+        assert np.array_equal(s0, s1) and np.array_equal(p0, p1) and np.array_equal(m0, m1)
+        # and the paper's Eq. 6-7 / Eq. 14 sums, from the oracle
+        assert_scores_close(s1, ref_s, what=f"{wl.name}: scores")
+        assert_scores_close(p1, ref_p, what=f"{wl.name}: mass_p")
+        assert_scores_close(m1, ref_m, what=f"{wl.name}: mass_m")
     assert ctx.maskkv_check_status() == 0
     ctx.close()
 
