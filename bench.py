@@ -17,7 +17,9 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import socket
 import statistics
+import subprocess
 
 import sys
 import threading
@@ -169,9 +171,13 @@ def run_layer(ctx, buf, x, live, k_l, alpha, events=None):
     if events: events[5].record()
 
 
-# DRAM bytes (read + write) of one maskkv_score call at this workload, from the ncu capture summarised in
-# profiles/score_tc_llada32k_ncu.md: sweep 1 279.6 MB + sweep 2 290.7 MB (the key tensor is read once per sweep).
+# DRAM bytes (read + write) of one maskkv_score call at this workload.  bench.py cannot read DRAM counters itself: the
+# figure is dram__bytes_read.sum + dram__bytes_write.sum of the call's two kernels from one ncu capture of this very
+# command (sweep 1 279.6 MB + sweep 2 290.7 MB: the key tensor is read once per sweep); the JSON line names the source.
 SCORE_DRAM_TRAFFIC_BYTES = 570.3e6
+SCORE_DRAM_TRAFFIC_SOURCE = ("ncu --set full --clock-control none -k regex:score_(stats|colsum)_tc -s 3 -c 1 python bench.py --steps 4 "
+                             "--warmup 3 --no-graph: dram__bytes_read.sum + dram__bytes_write.sum, sweep 1 279.6 MB + sweep 2 290.7 MB; "
+                             "a constant of this file, not measured by this run")
 
 
 def algorithmic_work(wl, mean_kept_per_head):
@@ -254,6 +260,165 @@ def batched_calls(ctx, B, device):
         out[name] = row
     out["status_flags"] = ctx.maskkv_check_status()
     return out
+
+
+def timed_loop(call, reps, warm=3):
+    """Average device time of `call(i)` over `reps` back-to-back invocations, in microseconds (CUDA events)."""
+    for i in range(warm):
+        call(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(reps):
+        call(warm + i)
+    e1.record()
+    torch.cuda.synchronize()
+    return 1e3 * e0.elapsed_time(e1) / reps
+
+
+def dream_gqa_block(ctx, B, device, peaks, reps=200):
+    """configs[3], one layer per call: 28 query heads on 4 KV heads, N=16384, M=512, d=128, bf16, uniform budget 512 per KV
+    head.  maskkv_score and maskkv_attend alone, back to back, cycling through enough layers' inputs to exceed the L2;
+    attention at these shapes is bound by the tensor cores (every K/V tile serves the 7 x 512 query rows of its group)."""
+    wl = synth.config(4)
+    N, M, H, Hkv, d, g = wl.prompt_lens[0], wl.n_mask, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.group
+    n_sets = 10                                                     # 10 x (16.8 MB keys + 3.7 MB queries) > 126 MB L2
+    xs, lives, caches = [], [], []
+    buf = LayerBuffers(ctx, B, wl, Hkv * 512, device)
+    for l in range(n_sets):
+        x = synth.layer_inputs(wl, l, device)
+        x.pop("planted", None); x.pop("v_mask", None)
+        live = synth.live_inputs(wl, l, 0, device)
+        run_layer(ctx, buf, x, live, 512, 1.0)
+        caches.append((buf.kc.clone(), buf.vc.clone()))
+        xs.append({"q_mask": x["q_mask"], "k_prompt": x["k_prompt"], "k_mask": x["k_mask"]})
+        lives.append(live)
+    torch.cuda.synchronize()
+    p = buf.p
+    outs = [torch.empty_like(buf.out) for _ in range(4)]            # 4 x 3.7 MB of output cycled as well
+
+    def score(i):
+        x = xs[i % n_sets]
+        ctx.maskkv_score(p, x["q_mask"], x["k_prompt"], x["k_mask"], buf.scores, buf.mass_p, buf.mass_m, buf.ws)
+
+    def attend(i):
+        kc, vc = caches[i % n_sets]
+        live = lives[i % n_sets]
+        ctx.maskkv_attend(p, live["q_live"], live["k_live"], live["v_live"], kc, vc, buf.offsets, buf.capacity, outs[i % 4])
+
+    score_us = timed_loop(score, reps)
+    attend_us = timed_loop(attend, reps)
+    k = 512
+    score_flops = 2.0 * M * (N + M) * d * H
+    attend_flops = 4.0 * M * (k + M) * d * H
+    attend_bytes = 2.0 * (2 * M * H * d) + 2.0 * 2 * d * (k + M) * Hkv
+    out = {"workload": f"configs[3] dream_gqa_16k, one layer per call: N={N} M={M} H={H} H_kv={Hkv} d={d}, budget {k} per KV head; "
+                       f"{n_sets} layers' inputs cycled ({n_sets * (N * Hkv + M * H + M * Hkv) * d * 2 / 1e6:.0f} MB > L2), {reps} calls back to back",
+           "score_us": round(score_us, 2), "attend_us": round(attend_us, 2)}
+    for name, us, flops in (("score", score_us, score_flops), ("attend", attend_us, attend_flops)):
+        tf = flops / (us * 1e-6) / 1e12
+        out[name] = {"bound": "tensor", "achieved": round(tf, 1), "unit": "TFLOP/s", "flops": flops,
+                     "frac_burst": round(tf / peaks["bf16_tflops"], 3), "frac_sustained": round(tf / peaks["bf16_tflops_sustained"], 3)}
+    out["score"]["note"] = "one Q K^T counted; the two sweeps execute twice that"
+    out["attend"]["flop_per_byte"] = round(attend_flops / attend_bytes, 1)
+    out["status_flags"] = ctx.maskkv_check_status()
+    return out
+
+
+def kv_peak_bytes(n_layers, prompt_tokens, kept_per_head, n_kv_heads, head_dim, online, elem_bytes=2):
+    """Peak bytes of prompt KV cache held during the first denoising step (paragraph after Eq. 13), with the paper's
+    accounting 2 * tokens * heads * d_head * bytes per layer.  The model runs its layers in order; a layer's prompt K/V
+    exist from the moment the layer has run.  Offline profile: layer l's budget is known beforehand, so the layer is
+    compacted to kept_per_head[l] tokens per head before layer l + 1 runs - at most one uncompressed layer exists at
+    a time.  Online: the budgets need the importance of every layer, i.e. the whole forward pass, so all layers are
+    still uncompressed when the last one has run, and eviction only starts after that peak."""
+    full = kv_cache_bytes(prompt_tokens, n_kv_heads, head_dim, elem_bytes)
+    if online:
+        return n_layers * full
+    peak, held = 0.0, 0.0
+    for l in range(n_layers):
+        peak = max(peak, held + full)
+        held += kv_cache_bytes(kept_per_head[l], n_kv_heads, head_dim, elem_bytes)
+    return max(peak, held)
+
+
+def stack_batched_block(ctx, B, device, peaks):
+    """maskkv_select and maskkv_compact over ALL (layer, head) segments of configs[2] in one call each, with the layer as
+    the request axis: 32 x 32 = 1024 segments of 32768 scores (134 MB) and about 261,000 kept rows (269 MB moved) - the
+    launch in which the two calls have enough bytes for a bandwidth fraction to mean something.  Every layer's inputs
+    are generated from the seed and scored on the device; its scores, masses, keys and values land in the stacked
+    tensors.  The loop is the offline schedule of the paper (budgets known before the layer runs), so it also yields
+    the kept rows per layer for the peak-memory comparison with the online schedule."""
+    wl = synth.config(3)
+    L, N, M, Hkv, H, d = wl.n_layers, wl.prompt_lens[0], wl.n_mask, wl.n_kv_heads, wl.n_q_heads, wl.head_dim
+    k_layers = B.maskkv_layer_budgets(wl.total_budget(), wl.beta, wl.layer_importance())
+    one = LayerBuffers(ctx, B, wl, Hkv * max(k_layers), device)
+    pcu = [l * N for l in range(L + 1)]
+    lcu = [l * M for l in range(L + 1)]
+    p = B.Problem(wl.torch_dtype, H, Hkv, d, pcu, lcu, device)
+    scores = torch.empty((Hkv, L * N), dtype=torch.float32, device=device)
+    mass_p = torch.empty((L, Hkv), dtype=torch.float32, device=device)
+    mass_m = torch.empty((L, Hkv), dtype=torch.float32, device=device)
+    k_all = torch.empty((L * N, Hkv, d), dtype=wl.torch_dtype, device=device)
+    v_all = torch.empty((L * N, Hkv, d), dtype=wl.torch_dtype, device=device)
+    for l in range(L):
+        x = synth.layer_inputs(wl, l, device)
+        ctx.maskkv_score(one.p, x["q_mask"], x["k_prompt"], x["k_mask"], one.scores, one.mass_p, one.mass_m, one.ws)
+        scores[:, l * N:(l + 1) * N] = one.scores
+        mass_p[l] = one.mass_p[0]
+        mass_m[l] = one.mass_m[0]
+        k_all[l * N:(l + 1) * N] = x["k_prompt"]
+        v_all[l * N:(l + 1) * N] = x["v_prompt"]
+        del x
+    capacity = Hkv * sum(k_layers)
+    k_l_dev = torch.tensor(k_layers, dtype=torch.int32, device=device)
+    budgets = torch.empty((L, Hkv), dtype=torch.int32, device=device)
+    offsets = torch.zeros(L * Hkv + 1, dtype=torch.int32, device=device)
+    kept = torch.empty(capacity, dtype=torch.int32, device=device)
+    kc = torch.empty((capacity, d), dtype=wl.torch_dtype, device=device)
+    vc = torch.empty_like(kc)
+    ctx.maskkv_budget(p, 0, wl.alpha, mass_p, mass_m, capacity, budgets, offsets, k_l_dev)
+    ctx.maskkv_select(p, scores, budgets, offsets, kept)
+    ctx.maskkv_compact(p, k_all, v_all, kept, offsets, capacity, kc, vc)
+    torch.cuda.synchronize()
+    rows = int(offsets[-1].item())
+    kept_per_layer = budgets.sum(1).cpu().tolist()
+    work = {"select": 4.0 * L * N * Hkv + 4.0 * rows, "compact": (4.0 * d * 2 + 4.0) * rows}
+    calls = {"select": lambda: ctx.maskkv_select(p, scores, budgets, offsets, kept),
+             "compact": lambda: ctx.maskkv_compact(p, k_all, v_all, kept, offsets, capacity, kc, vc)}
+    scratch = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    hbm = peaks["hbm_gbs"]
+    out = {"workload": f"configs[2] llada_stack_32k, all {L} layers in one call (layer = request axis): {L * Hkv} segments of {N} scores, "
+                       f"{rows} kept rows; warm = 20 calls back to back (inputs of {work['select'] / 1e6:.0f} / {work['compact'] / 1e6:.0f} MB "
+                       "exceed the L2 anyway), cold = 256 MB written before each call"}
+    for name, call in calls.items():
+        warm_us = timed_loop(lambda i: call(), 20)
+        cold = []
+        for i in range(10):
+            scratch.fill_(i)
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record()
+            call()
+            c1.record()
+            torch.cuda.synchronize()
+            cold.append(1e3 * c0.elapsed_time(c1))
+        cold_us = statistics.median(cold)
+        out[name] = {"bound": "hbm", "bytes": work[name], "warm_us": round(warm_us, 2), "cold_us": round(cold_us, 2),
+                     "warm_GB/s": round(work[name] / (warm_us * 1e-6) / 1e9, 1), "cold_GB/s": round(work[name] / (cold_us * 1e-6) / 1e9, 1),
+                     "peak": hbm, "warm_frac_of_hbm_peak": round(work[name] / (warm_us * 1e-6) / 1e9 / hbm, 3),
+                     "cold_frac_of_hbm_peak": round(work[name] / (cold_us * 1e-6) / 1e9 / hbm, 3)}
+    out["status_flags"] = ctx.maskkv_check_status()
+    # peak prompt-KV bytes of the first step under the two schedules of the paragraph after Eq. 13
+    per_head = [r / Hkv for r in kept_per_layer]
+    off_peak = kv_peak_bytes(L, N, per_head, Hkv, d, online=False)
+    on_peak = kv_peak_bytes(L, N, per_head, Hkv, d, online=True)
+    schedules = {"offline_profile_peak_bytes": off_peak, "online_peak_bytes": on_peak, "ratio": on_peak / off_peak,
+                 "after_eviction_bytes": sum(kv_cache_bytes(k, Hkv, d) for k in per_head),
+                 "kept_rows_per_layer": [int(r) for r in kept_per_layer],
+                 "note": "prompt K/V of the 32-layer stack held during the first denoising step; offline = each layer compacted "
+                         "before the next one runs (budgets from a precomputed importance profile), online = budgets need "
+                         "every layer's importance, so nothing can be evicted before the whole stack is resident"}
+    return out, schedules
 
 
 def bench_ours(args):
@@ -534,6 +699,8 @@ def bench_ours(args):
     # ---- select / compact / attend on a batch: at one layer they are launch- and latency-bound whatever the kernel does
     # (4-17 MB per call), so a fraction of the memory roof only shows when many segments go into one launch
     batched = batched_calls(ctx, B, device) if rank == 0 else None
+    dream = dream_gqa_block(ctx, B, device, load_peaks()) if rank == 0 else None
+    stack, schedules = stack_batched_block(ctx, B, device, load_peaks()) if rank == 0 else (None, None)
 
     # ---- calibration step of the budget rule (Eq. 8), outside the timed step: a streaming reduction bound by HBM
     importance = None
@@ -604,7 +771,9 @@ def bench_ours(args):
             peak_tf = load_peaks()["bf16_tflops_sustained"]
             project[name] = {"us": round(us, 2),
                              "roofline": {"bound": "tensor", "achieved": round(tf, 1), "peak": peak_tf, "unit": "TFLOP/s",
-                                          "frac": round(tf / peak_tf, 3), "peak_source": "sustained bf16 (20 back-to-back calls)"},
+                                          "frac": round(tf / peak_tf, 3), "frac_sustained": round(tf / peak_tf, 3),
+                                          "frac_burst": round(tf / load_peaks()["bf16_tflops"], 3),
+                                          "peak_source": "frac = of the sustained bf16 peak; 20 back-to-back calls (4.5 ms)"},
                              "hbm_GB/s": round(p_bytes / (us * 1e-6) / 1e9, 1),
                              "frac_of_hbm_peak": round(p_bytes / (us * 1e-6) / 1e9 / load_peaks()["hbm_gbs"], 3)}
             del logits
@@ -623,6 +792,9 @@ def bench_ours(args):
     score_s = (score_us if score_us is not None else call_us["score"]) * 1e-6
     achieved_tf = work["score_flops"] / score_s / 1e12
     peak_tf = peaks["bf16_tflops_sustained"]
+    # the score-alone loop is a few hundred back-to-back calls (tens of milliseconds): the burst peak is the fairer
+    # denominator for the default short runs, the sustained one for seconds-long loops; both are reported
+    peak_burst_tf = peaks["bf16_tflops"]
     hbm = peaks["hbm_gbs"]
     other = {
         "score_hbm": {"bound": "hbm", "achieved": work["score_bytes"] / score_s / 1e9, "peak": hbm, "unit": "GB/s"},
@@ -661,8 +833,10 @@ def bench_ours(args):
         "status_flags": flags,
         "roofline": {"kernel": "maskkv_score (its two kernels, replayed alone; one Q K^T product counted)", "bound": "tensor",
                      "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
-                     "peak_source": peaks["source"] + " (sustained bf16; the kernels run inside a long step)",
-                     "traffic": SCORE_DRAM_TRAFFIC_BYTES, "executed_over_algorithmic_flops": 2.0},
+                     "frac_sustained": achieved_tf / peak_tf, "frac_burst": achieved_tf / peak_burst_tf, "peak_burst": peak_burst_tf,
+                     "peak_source": peaks["source"] + " (frac = of the sustained bf16 peak; frac_burst = of the burst peak)",
+                     "traffic": SCORE_DRAM_TRAFFIC_BYTES, "traffic_source": SCORE_DRAM_TRAFFIC_SOURCE,
+                     "algorithmic_bytes": work["score_bytes"], "executed_over_algorithmic_flops": 2.0},
         "roofline_alu": exp_roofline(wl, score_s * 1e6, clocks.get("sm_max_mhz") or 1965.0),
         "score_us": round(score_s * 1e6, 2),
         "roofline_other_calls": other,
@@ -670,6 +844,11 @@ def bench_ours(args):
     }
     if batched is not None:
         line["batched_calls"] = batched
+    if dream is not None:
+        line["dream_gqa_16k"] = dream
+    if stack is not None:
+        line["stack_batched"] = stack
+        line["kv_peak_first_step"] = schedules
     if importance is not None:
         gbs = importance["bytes"] / (importance["us"] * 1e-6) / 1e9
         line["refresh_set"] = importance.pop("refresh_set", None)
@@ -700,6 +879,20 @@ def load_peaks():
         return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
                 "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def oracle_threads() -> int:
+    """Threads the oracle's numpy calls actually use: the size of the BLAS pool numpy is linked against (its matrix
+    products are the only multi-threaded part); the host's core count if that cannot be read."""
+    try:
+        from threadpoolctl import threadpool_info
+        import numpy  # noqa: F401  (the pools are listed once the library is loaded)
+        pools = [int(i["num_threads"]) for i in threadpool_info() if i.get("user_api") == "blas"]
+        if pools:
+            return max(pools)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
 
 
 def oracle_sample(wl, n_heads: int, layer: int = 0):
@@ -735,7 +928,7 @@ def oracle_baseline(wl, budget_s: float):
         t = oracle_pass(sub, x, live, 238)
     else:
         t = t1
-    return {"value": N / (t * H / n_heads), "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+    return {"value": N / (t * H / n_heads), "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
             "sample": f"{n_heads} of {H} heads of one 32k layer through the whole path (fp64 numpy), {t:.2f} s; "
                       f"scaled to a full layer by {H}/{n_heads}", "host_cores": os.cpu_count()}
 
@@ -775,13 +968,61 @@ def bench_reference(args):
               f"(fp64 numpy oracle); scaled by {scale:g}")
     return {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": 1e3 * t * scale, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": 1e3 * t * scale, "ms_per_step_is": f"extrapolated: measured {1e3 * t:.1f} ms per sampled step x {scale:g}",
+        "ms_per_sampled_step": 1e3 * t, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": "configs[2] llada_stack_32k, one layer per step (sampled)", "sample": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
+
+
+def launcher_command(n_ranks: int, argv, port: int):
+    """The command that starts `n_ranks` ranks of this script on one node, one per GPU (what a driver would type)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_ranks}", "--master-addr", "127.0.0.1",
+            "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def self_launch(n_ranks: int, argv) -> int:
+    """`python bench.py --gpus N` with N > 1 outside a launcher: start the N ranks ourselves and hand back their exit
+    code.  NCCL's communicator lines go to stderr (NCCL_DEBUG=INFO unless the caller chose otherwise), so that stdout
+    still carries rank 0's one JSON line."""
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")
+    return subprocess.call(launcher_command(n_ranks, argv, port), env=env)
+
+
+def bench_plumbing(args):
+    """The multi-rank plumbing alone (rendezvous, layer sharding, reductions over ranks), on whatever backend the box
+    has - gloo on a machine without GPUs: what the CPU tests run through the launcher."""
+    import torch.distributed as dist
+    rank, world, local_rank = rank_world()
+    use_cuda = torch.cuda.is_available() and torch.cuda.device_count() >= world
+    device = None
+    if world > 1:
+        if use_cuda:
+            torch.cuda.set_device(local_rank)
+            device = torch.device("cuda", local_rank)
+            dist.init_process_group("nccl", device_id=device)
+        else:
+            dist.init_process_group("gloo")
+    mine = shard_layers(synth.config(3).n_layers, rank, world)
+    slowest = max_over_ranks(10.0 + 5.0 * rank, device)
+    total = sum_over_ranks(float(len(mine)), device)
+    gathered = [mine]
+    if world > 1:
+        gathered = [None] * world
+        dist.all_gather_object(gathered, mine)
+        dist.destroy_process_group()
+    if rank != 0:
+        return None
+    return {"plumbing_only": True, "n_gpus": world, "backend": "nccl" if (use_cuda and world > 1) else ("gloo" if world > 1 else "none"),
+            "layers_per_rank": gathered, "layers_total": total, "slowest_rank_time": slowest}
 
 
 def main():
@@ -791,7 +1032,16 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="time plain calls instead of replaying CUDA graphs")
+    ap.add_argument("--plumbing-only", action="store_true",
+                    help="run the multi-rank plumbing (rendezvous, sharding, reductions) and nothing else; needs no GPU")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and "RANK" not in os.environ:
+        raise SystemExit(self_launch(args.gpus, sys.argv[1:]))       # not under a launcher: start the ranks ourselves
+    if args.plumbing_only:
+        line = bench_plumbing(args)
+        if line is not None:
+            print(json.dumps(line), flush=True)
+        return
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else max(1, args.steps)
         args.warmup = 1 if args.warmup is None else max(0, args.warmup)

@@ -14,7 +14,7 @@ Notation (the paper overloads letters; this file uses one meaning each):
     d   head dimension                             k_l per-head mean budget of layer l (Eq. 13)
     k_{l,h} budget of KV head h in layer l (Eq. 15)
 
-Readings taken where the paper is silent (each is also listed in the design notes):
+Readings taken where the paper is silent:
     * K_full is the request's N prompt keys followed by its M mask keys, no attention mask.
     * No smoothing or pooling of I is specified, so none is applied; `row_weights` (default 1)
       weights each mask row's vote and is the only hook.

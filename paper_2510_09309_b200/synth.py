@@ -35,7 +35,7 @@ _T_Q, _T_KP, _T_VP, _T_KM, _T_VM, _T_PLANT, _T_W, _T_QL, _T_KL, _T_VL = range(10
 
 @dataclass(frozen=True)
 class Workload:
-    """One synthetic workload (a BASELINE config or a scaled-down variant)."""
+    """One synthetic workload (one of the five configurations or a scaled-down variant)."""
     name: str
     config_id: int
     dtype: str                       # "f32" | "bf16"
@@ -103,7 +103,7 @@ RAGGED_PROMPT_LENS = (1024, 24615, 30881, 4417, 25124, 24565, 4504, 32768)
 
 
 def config(i: int, **over) -> Workload:
-    """The five BASELINE configurations (1-based, as in the prose)."""
+    """The five configurations (1-based, as in the prose)."""
     if i == 1:
         w = Workload("tiny_fp32", 1, "f32", 1, 4, 4, 64, (512,), 64, planted_per_head=8,
                      planted_gain=3.0, mean_budget=32, alpha=1.0)

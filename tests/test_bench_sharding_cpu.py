@@ -56,6 +56,48 @@ def test_two_ranks_shard_layers_and_reduce_times():
         assert total == 32.0
 
 
+@pytest.mark.timeout(300)
+def test_bench_starts_its_own_ranks_when_asked_for_several_gpus():
+    """`python bench.py --gpus 2` outside a launcher must run as two ranks (here over gloo, plumbing only): rank 0 prints
+    one JSON line that says n_gpus = 2 and shows every layer on exactly one rank."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    env["CUDA_VISIBLE_DEVICES"] = ""
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--plumbing-only"], env=env,
+                         capture_output=True, text=True, timeout=280)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, res.stdout
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["backend"] == "gloo"
+    assert sorted(l for part in line["layers_per_rank"] for l in part) == list(range(32))
+    assert line["layers_total"] == 32.0 and line["slowest_rank_time"] == 15.0
+
+
+def test_launcher_command_is_the_documented_one():
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.launcher_command(4, ["--gpus", "4", "--steps", "7"], 29511)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=4" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29511"
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "7"] and cmd[-5].endswith("bench.py")
+
+
+def test_peak_kv_bytes_of_the_two_schedules():
+    """Paragraph after Eq. 13: with budgets known beforehand a layer is compacted before the next one runs, so the
+    peak is one full layer plus the compacted earlier ones; an online rule holds every layer uncompressed first."""
+    import bench
+    full = bench.kv_cache_bytes(1000, 2, 64)
+    kept = [10.0, 20.0, 30.0]
+    on = bench.kv_peak_bytes(3, 1000, kept, 2, 64, online=True)
+    off = bench.kv_peak_bytes(3, 1000, kept, 2, 64, online=False)
+    assert on == 3 * full
+    assert off == full + bench.kv_cache_bytes(10, 2, 64) + bench.kv_cache_bytes(20, 2, 64)
+    # nothing evicted: both schedules end up holding everything
+    assert bench.kv_peak_bytes(3, 1000, [1000.0] * 3, 2, 64, online=False) == 3 * full
+
+
 def test_single_process_helpers_are_no_ops():
     sys.path.insert(0, ROOT)
     import bench
