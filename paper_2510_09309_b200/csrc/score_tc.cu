@@ -35,6 +35,31 @@ constexpr int kTile = 128;             // keys per tile (both sweeps), queries p
 constexpr int kQBlock = 256;           // queries resident per CTA
 constexpr int kColsumPad = 3;          // sweep 2: what entering a new unit costs a CTA, in key tiles (see Walker)
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+// Share of the exponentials that runs as a polynomial on the FMA pipes instead of on the special-function unit (16 results
+// per clock per SM): this many pairs out of every eight.  Measured on B200 (32k LLaDA layer / 16k Dream layer, whole call):
+// sweep 2 with 0 / 2 / 3 / 4 pairs 171.7 / 169.3 / 176.0 / 182.2 us and 162.4 / 157.8 / 161.3 / 169.6 us; sweep 1 with
+// 0 / 2 / 3 pairs 171.6 / 176.8 / 176.7 us.  A stand-alone loop of the same epilogue gains 24 % at 3 of 8; inside the
+// kernels the sweeps are held by the hand-over of the accumulators and by the key stream as much as by the exponentials,
+// so only the small share in sweep 2 pays.  Compile-time switches so that the comparison can be repeated.
+#ifndef MASKKV_STATS_POLY
+#define MASKKV_STATS_POLY 0
+#endif
+#ifndef MASKKV_COLSUM_POLY
+#define MASKKV_COLSUM_POLY 2
+#endif
+constexpr int kStatsPolyPairs = MASKKV_STATS_POLY;      // sweep 1, degree 2 (row sums average the error away)
+constexpr int kColsumPolyPairs = MASKKV_COLSUM_POLY;
+// Measurement switches (off in the library): MASKKV_DBG_NOMATH leaves the epilogues with their tensor-memory loads and
+// barrier traffic only, MASKKV_DBG_KSTEPS issues that many of the eight MMA k-steps per tile - together they show what the
+// key stream, the products and the accumulator hand-over cost without the exponentials.
+#ifndef MASKKV_DBG_KSTEPS
+#define MASKKV_DBG_KSTEPS 8
+#endif    // sweep 2, degree 4
+// which pairs of a group of eight go to the polynomial: spread out, so that both units always have work in flight
+__host__ __device__ constexpr bool poly_pair(int pair, int n_of_8) {
+  return ((pair & 7) + 1) * n_of_8 / 8 > (pair & 7) * n_of_8 / 8;
+}
 
 template <int D>
 struct Smem {
@@ -45,8 +70,9 @@ struct Smem {
   static constexpr int kKBytes = kBoxes * kKBoxBytes;
   static constexpr int kQOff = 0;
   static constexpr int kKOff = kQBytes;
-  static constexpr int kC2Off = kKOff + kStages * kKBytes;                 // float [4 warpgroups][2][128]
-  static constexpr int kXchOff = kC2Off + 4 * kQBlock * 4;                 // float [2 accumulators][2][128]
+  static constexpr int kC2Off = kKOff + kStages * kKBytes;                 // float [4 warpgroups][2][128] per-query constants
+  static constexpr int kS2Off = kC2Off + 4 * kQBlock * 4;                  // float [4 warpgroups][2][128] second constants (polynomial columns)
+  static constexpr int kXchOff = kS2Off + 4 * kQBlock * 4;                 // float [2 accumulators][2][128]
   static constexpr int kBarOff = kXchOff + 4 * kTile * 4;                  // mbarriers
   static constexpr int kNumBars = 2 * kStages + 2 + 4 + 4;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;                  // tmem base, abort flag
@@ -246,7 +272,8 @@ __host__ __device__ __forceinline__ int cta_of(long long f, long long F, int G) 
 
 // =====================================================================================================
 // sweep 1: per-row (max, sum of exp) over a segment of key tiles.
-// part[(h*C + slot)*sumM + row] = (max of scaled logits, sum of exp), slot = 2*(cta - first cta of the row's unit) + half:
+// part[(h*C + slot)*sumM + row] = (m2, sum of 2^(scaled logit * log2 e - m2)) with m2 an integer reference in log2 units,
+// slot = 2*(cta - first cta of the row's unit) + half:
 // neighbouring rows are neighbours in memory, so a warp's 32 rows of one slot are one 256-byte access.
 // =====================================================================================================
 template <int D>
@@ -326,7 +353,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             tc_fence_after();
             const uint32_t q_lo = q_lo_base + ((a * kTile * 128) >> 4);
 #pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
+            for (int kk = 0; kk < (D / 16) * MASKKV_DBG_KSTEPS / 8; ++kk) {
               const uint32_t qo = ((kk >> 2) * S::kQBoxBytes + (kk & 3) * 32) >> 4;
               const uint32_t ko = ((kk >> 2) * S::kKBoxBytes + (kk & 3) * 32) >> 4;
               umma_ss(tmem_base + acc * kTile, make_desc(q_lo + qo, kDescHiSw128), make_desc(k_lo + ko, kDescHiSw128), idesc, kk > 0);
@@ -353,8 +380,11 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const int h = s.g / qp_n, q0 = (s.g % qp_n) * kQBlock;
       const int n_qtiles = (s.M - q0 > kTile) ? 2 : 1;
       if (a >= n_qtiles) continue;
-      float m = -INFINITY, l = 0.f;                         // m in raw (unscaled) logits
-      // running maximum m and l = sum 2^((s - m) * cs); a chunk's maximum is a tree of 3-input max
+      // The row's reference m2 is an INTEGER in log2 units, at least the largest scaled logit seen so far, and
+      // l = sum 2^(s * cs - m2).  An integer reference costs nothing (any reference at or above the maximum will do) and
+      // lets the polynomial path fold it into its magic number; merging partials is then exact (powers of two).
+      float m2 = -INFINITY, l = 0.f;
+      // a chunk's maximum is a tree of 3-input max
       auto chunk_max = [&](const float* v) {
         float t[11];
 #pragma unroll
@@ -362,8 +392,8 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         t[10] = fmaxf(v[30], v[31]);
         return fmaxf(max3(max3(t[0], t[1], t[2]), max3(t[3], t[4], t[5]), max3(t[6], t[7], t[8])), fmaxf(t[9], t[10]));
       };
-      auto chunk_sum = [&](const float* v, float ref) {
-        const float neg = -ref * cs;
+      auto chunk_sum = [&](const float* v, float ref2) {   // every exponential on the special-function unit
+        const float neg = -ref2;
         const uint64_t cs2 = pack2(cs, cs), neg2 = pack2(neg, neg);
         uint64_t acc_a = pack2(0.f, 0.f), acc_b = pack2(0.f, 0.f);
 #pragma unroll
@@ -378,14 +408,36 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         unpack2(add2(acc_a, acc_b), l0, l1);
         return l0 + l1;
       };
+      // kStatsPolyPairs of every eight pairs as a polynomial on the FMA pipes, the others on the special-function unit;
+      // the two kinds alternate so that both units have work in flight.  All 32 logits must be finite.
+      auto chunk_sum_mixed = [&](const float* v, float ref2) {
+        const float neg = -ref2, mk = kExpMagic - ref2;     // an integer: exact
+        const uint64_t cs2 = pack2(cs, cs), neg2 = pack2(neg, neg), mk2 = pack2(mk, mk);
+        uint64_t acc_a = pack2(0.f, 0.f), acc_b = pack2(0.f, 0.f);
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          const uint64_t v2 = pack2(v[c], v[c + 1]);
+          if (poly_pair(c >> 1, kStatsPolyPairs)) {
+            acc_b = add2(acc_b, exp2_poly_pair<2>(v2, cs2, mk2));
+          } else {
+            float x0, x1;
+            unpack2(fma2(v2, cs2, neg2), x0, x1);
+            acc_a = add2(acc_a, pack2(ex2(x0), ex2(x1)));
+          }
+        }
+        float l0, l1;
+        unpack2(add2(acc_a, acc_b), l0, l1);
+        return l0 + l1;
+      };
       auto absorb = [&](float* v, int col0, int valid) {
-        if (valid - col0 < 32) {
+        const bool ragged = valid - col0 < 32;               // only the last tile of a request's prompt or mask keys
+        if (ragged) {
 #pragma unroll
           for (int c = 0; c < 32; ++c) if (col0 + c >= valid) v[c] = -INFINITY;
         }
-        const float cmax = chunk_max(v);
-        if (cmax > m) { l *= ex2((m - cmax) * cs); m = cmax; }
-        l += chunk_sum(v, m);
+        const float cm2 = chunk_max(v) * cs;
+        if (cm2 > m2) { const float nm = ceilf(cm2); l *= ex2(m2 - nm); m2 = nm; }
+        l += (ragged || kStatsPolyPairs == 0) ? chunk_sum(v, m2) : chunk_sum_mixed(v, m2);
       };
       // Rolling double buffer over the chunk stream (tile 0: c0, c1; tile 1: c0, c1; ...): while one 32-column chunk
       // is being exponentiated the next one - possibly of the next tile - is already on its way from tensor memory.
@@ -405,7 +457,11 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         // chunk 0 of this tile is in flight (into va); start chunk 1 behind it
         tmem_ld_wait();
         tmem_ld32(lane_addr + acc * kTile + 32, vb);
+#ifdef MASKKV_DBG_NOMATH
+        l += va[5];
+#else
         if (valid > col0) absorb(va, col0, valid);
+#endif
         tmem_ld_wait();
         tc_fence_before();
         mbar_arrive(bars.tempty + acc);                     // both chunks of this thread are in registers
@@ -417,22 +473,27 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           valid = key_tile(s.t + it + 1, s.p0, s.N, s.l0, s.M).valid;
           tmem_ld32(lane_addr + (a * 2 + (c2n & 1)) * kTile, va);
         }
+#ifdef MASKKV_DBG_NOMATH
+        l += vb[7];
+#else
         if (valid_now > col0 + 32) absorb(vb, col0 + 32, valid_now);
+#endif
       }
       if (!ok) continue;
       const int i = q0 + a * kTile + row;
       const int slot = 2 * ((int)blockIdx.x - cta_of(s.unit_start, F, gridDim.x)) + half;
-      if (i < s.M) part[((long long)h * C + slot) * sh.sumM + s.l0 + i] = make_float2(m * sh.scale, l);
+      if (i < s.M) part[((long long)h * C + slot) * sh.sumM + s.l0 + i] = make_float2(m2, l);
     }
   }
   block_teardown(tmem_base);
 }
 
-// ln sum_j exp(s_j) of query row `row` (index over all requests) of head h: log-sum-exp merge of the partials the CTAs
-// of sweep 1 left for the row's unit, which starts at flat tile `unit_start` of that sweep's walk and has T tiles.
+// log2 sum_j exp(s_j) of query row `row` (index over all requests) of head h: merge of the partials the CTAs of sweep 1
+// left for the row's unit, which starts at flat tile `unit_start` of that sweep's walk and has T tiles.  The partials'
+// references are integers in log2 units, so bringing them to a common one multiplies by exact powers of two.
 // F, G: flat tile count and grid of sweep 1.
-__device__ __noinline__ float merged_lse(const float2* __restrict__ part, int C, int sumM, long long F, int G,
-                                            long long unit_start, int T, int h, int row) {
+__device__ __noinline__ float merged_lse2(const float2* __restrict__ part, int C, int sumM, long long F, int G,
+                                             long long unit_start, int T, int h, int row) {
   const int slots = 2 * (cta_of(unit_start + T - 1, F, G) - cta_of(unit_start, F, G) + 1);
   const float2* p = part + (long long)h * C * sumM + row;         // slot c at p[c * sumM]
   // the loads of a batch are issued together (a row has 4 to 8 partials on a long prompt)
@@ -445,13 +506,12 @@ __device__ __noinline__ float merged_lse(const float2* __restrict__ part, int C,
 #pragma unroll
     for (int k = 0; k < 8; ++k) bm = fmaxf(bm, v[k].x);
     if (bm == -INFINITY) continue;
-    // special-function exponentials and logarithm (relative error 2^-22): the epilogue waits for this value
-    l *= ex2((m - bm) * kLog2e);
+    l *= ex2(m - bm);
 #pragma unroll
-    for (int k = 0; k < 8; ++k) l += v[k].y * ex2((v[k].x - bm) * kLog2e);
+    for (int k = 0; k < 8; ++k) l += v[k].y * ex2(v[k].x - bm);
     m = bm;
   }
-  return m + __log2f(l) * 0.6931471805599453f;
+  return m + __log2f(l);                                          // special-function logarithm (relative error 2^-22)
 }
 
 // One thread per (h, row): lse[h*sumM + row].  Only launched when sweep 2 does not run on the tensor-core kernel
@@ -469,7 +529,7 @@ __global__ void score_merge_stats_tc(Shape sh, const float2* __restrict__ part, 
   }
   const int N = sh.prompt_cu[r + 1] - sh.prompt_cu[r], l0 = sh.live_cu[r], M = sh.live_cu[r + 1] - l0;
   const int T = tiles_of(N, M), qp_n = (M + kQBlock - 1) / kQBlock;
-  lse[t] = merged_lse(part, C, sh.sumM, F, G, base + ((long long)h * qp_n + (row - l0) / kQBlock) * T, T, h, row);
+  lse[t] = merged_lse2(part, C, sh.sumM, F, G, base + ((long long)h * qp_n + (row - l0) / kQBlock) * T, T, h, row) * kLn2;
 }
 
 // =====================================================================================================
@@ -498,6 +558,7 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   uint8_t* base = align_1024(smem_raw);
   const Bars bars = carve_bars(base, S::kBarOff);
   float* c2s = reinterpret_cast<float*>(base + S::kC2Off);
+  float* s2s = reinterpret_cast<float*>(base + S::kS2Off);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + S::kMiscOff);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base + S::kMiscOff + 4);
   pdl_launch_dependents();
@@ -574,7 +635,7 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           tc_fence_after();
           const uint32_t k_lo = k_lo_base + stage * (S::kKBytes >> 4);
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
+          for (int kk = 0; kk < (D / 16) * MASKKV_DBG_KSTEPS / 8; ++kk) {
             const uint32_t ko = ((kk >> 2) * S::kKBoxBytes + (kk & 3) * 32) >> 4;
             const uint32_t qo = ((kk >> 2) * S::kQBoxBytes + (kk & 3) * 32) >> 4;
             umma_ss(tmem_base + buf * kQBlock, make_desc(k_lo + ko, kDescHiSw128), make_desc(q_lo_base + qo, kDescHiSw128), idesc, kk > 0);
@@ -604,6 +665,7 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     int base_par = 0;
     bool ok = true;
     const float* c2 = c2s;
+    const float* s2 = s2s;
     // Attention mass of the segment in hand (one query block per KV head only), summed over the tiles this warp
     // finished (half-0 warps).  When the walk leaves the segment the warp stores its pair in slot
     // (CTA - first CTA of the segment) * 8 + warp and counts itself in; the warp that completes the count adds the slots
@@ -653,30 +715,53 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       const int nq = max(0, min(kTile, s.M - qh0));
       if (new_q) {
         float* c2w = c2s + (wg * 2 + (c2_it & 1)) * kTile;
+        float* s2w = s2s + (wg * 2 + (c2_it & 1)) * kTile;
         ++c2_it;
         float cst = -INFINITY;                              // 2^(x - inf) = 0: rows that do not exist never vote
         if (row < nq) {
           const int i = s.l0 + qh0 + row;
-          const float ln_z = part != nullptr ? merged_lse(part, C, sh.sumM, F1, G1, s.unit_real, s.T, h, i)
-                                             : lse[(long long)h * sh.sumM + i];
-          cst = (w ? log2f(w[i]) : 0.f) - ln_z * kLog2e;
+          const float lse2 = part != nullptr ? merged_lse2(part, C, sh.sumM, F1, G1, s.unit_real, s.T, h, i)
+                                             : lse[(long long)h * sh.sumM + i] * kLog2e;
+          cst = (w ? log2f(w[i]) : 0.f) - lse2;
         }
-        c2w[row] = cst;                                     // stored negated: x = s*c + cst
+        // Query column `row` of this half: its weight is 2^(s*cs + cst).  A column whose exponentials go to the
+        // special-function unit keeps cst; one that goes to the polynomial keeps the magic number plus the integer part of
+        // cst, and 2^(fraction of cst) as a factor applied when the weight is added (rows that do not vote: factor 0).
+        if (poly_pair((row & 31) >> 1, kColsumPolyPairs)) {
+          const bool votes = cst > -INFINITY;
+          const float ci = rintf(cst);
+          s2w[row] = votes ? ex2(cst - ci) : 0.f;
+          cst = votes ? kExpMagic + fmaxf(ci, -200.f) : kExpMagic - 200.f;
+        }
+        c2w[row] = cst;
         named_barrier(1 + wg, kTile);
         c2 = c2w;
+        s2 = s2w;
       }
       const int chunks = (nq + 31) >> 5;
       auto absorb = [&](const float* v, int cb, uint64_t& acc2) {
-        const float4* cc = reinterpret_cast<const float4*>(c2 + cb * 32);   // negated constants
+        const float4* cc = reinterpret_cast<const float4*>(c2 + cb * 32);   // per-query constants
+        const float4* ss = reinterpret_cast<const float4*>(s2 + cb * 32);
         const uint64_t cs2 = pack2(cs, cs);
 #pragma unroll
         for (int c4 = 0; c4 < 8; ++c4) {
           const float4 k4 = cc[c4];
-          float x0, x1, x2, x3;
-          unpack2(fma2(pack2(v[4 * c4], v[4 * c4 + 1]), cs2, pack2(k4.x, k4.y)), x0, x1);
-          unpack2(fma2(pack2(v[4 * c4 + 2], v[4 * c4 + 3]), cs2, pack2(k4.z, k4.w)), x2, x3);
-          acc2 = add2(acc2, pack2(ex2(x0), ex2(x1)));
-          acc2 = add2(acc2, pack2(ex2(x2), ex2(x3)));
+          float4 f4 = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (poly_pair(2 * c4, kColsumPolyPairs) || poly_pair(2 * c4 + 1, kColsumPolyPairs)) f4 = ss[c4];
+          if (poly_pair(2 * c4, kColsumPolyPairs)) {
+            acc2 = fma2(exp2_poly_pair<4>(pack2(v[4 * c4], v[4 * c4 + 1]), cs2, pack2(k4.x, k4.y)), pack2(f4.x, f4.y), acc2);
+          } else {
+            float x0, x1;
+            unpack2(fma2(pack2(v[4 * c4], v[4 * c4 + 1]), cs2, pack2(k4.x, k4.y)), x0, x1);
+            acc2 = add2(acc2, pack2(ex2(x0), ex2(x1)));
+          }
+          if (poly_pair(2 * c4 + 1, kColsumPolyPairs)) {
+            acc2 = fma2(exp2_poly_pair<4>(pack2(v[4 * c4 + 2], v[4 * c4 + 3]), cs2, pack2(k4.z, k4.w)), pack2(f4.z, f4.w), acc2);
+          } else {
+            float x2, x3;
+            unpack2(fma2(pack2(v[4 * c4 + 2], v[4 * c4 + 3]), cs2, pack2(k4.z, k4.w)), x2, x3);
+            acc2 = add2(acc2, pack2(ex2(x2), ex2(x3)));
+          }
         }
       };
       float* out_row = split ? colpart + ((long long)blk * sh.Hkv + hk) * keys_total : scores + (long long)hk * sh.sumN;
@@ -692,7 +777,11 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tmem_ld32(taddr + cb * 32, v);
             tmem_ld_wait();
             if (cb + 1 == chunks) { tc_fence_before(); mbar_arrive(bars.tempty + buf); }   // last logits are in registers
+#ifdef MASKKV_DBG_NOMATH
+            acc2 = add2(acc2, pack2(v[3], v[9]));
+#else
             absorb(v, cb, acc2);
+#endif
           }
           if (chunks == 0) { tc_fence_before(); mbar_arrive(bars.tempty + buf); }
         }

@@ -188,6 +188,51 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// 2^x on the FMA pipes, for the share of the exponentials that the special-function unit (16 results per clock per SM)
+// has no time for.  x = v*c + K with K an INTEGER known beforehand (the caller folds every fractional constant into a
+// later multiplication): adding the magic number 1.5 * 2^23 + K inside the multiply-add rounds v*c to the nearest
+// integer n and leaves n + K in the low mantissa bits; f = v*c - n lies in [-0.5, 0.5]; 2^f is a polynomial in f; the
+// integer part goes straight into the exponent field.  n + K below -126 is clamped (the result is then a value below
+// 2^-126 times a polynomial in a large |f|: nothing a sum of exponentials can see).  v must be finite.
+constexpr float kExpMagic = 12582912.f;                  // 1.5 * 2^23: one unit in the last place is 1
+constexpr float kExpMagicLow = kExpMagic - 126.f;
+// Least-maximum-relative-error polynomials of 2^f on [-0.5, 0.5], scaled so that the mean relative error is zero.
+// degree 2: |error| <= 1.8e-3 (row sums over thousands of keys: the errors average out), degree 4: <= 2.7e-6.
+template <int DEG>
+__device__ __forceinline__ uint64_t exp2_frac_poly(uint64_t f2) {
+  if (DEG == 2) {
+    const float c0 = 1.000384331f, c1 = 0.703401566f, c2 = 0.238411725f;
+    return fma2(fma2(pack2(c2, c2), f2, pack2(c1, c1)), f2, pack2(c0, c0));
+  } else if (DEG == 3) {
+    const float c0 = 0.999922991f, c1 = 0.693257451f, c2 = 0.242609292f, c3 = 0.0551710390f;
+    return fma2(fma2(fma2(pack2(c3, c3), f2, pack2(c2, c2)), f2, pack2(c1, c1)), f2, pack2(c0, c0));
+  } else {
+    const float c0 = 0.999999225f, c1 = 0.693121791f, c2 = 0.240247443f, c3 = 0.0559178069f, c4 = 0.00957006868f;
+    return fma2(fma2(fma2(fma2(pack2(c4, c4), f2, pack2(c3, c3)), f2, pack2(c2, c2)), f2, pack2(c1, c1)), f2, pack2(c0, c0));
+  }
+}
+// mk2 = (kExpMagic + K) twice.  Returns the pair 2^(v*c + K).
+template <int DEG>
+__device__ __forceinline__ uint64_t exp2_poly_pair(uint64_t v2, uint64_t c2, uint64_t mk2) {
+  float t0, t1;
+  unpack2(fma2(v2, c2, mk2), t0, t1);                    // magic + K + round(v*c)
+  t0 = fmaxf(t0, kExpMagicLow);
+  t1 = fmaxf(t1, kExpMagicLow);
+  const uint64_t nr2 = sub2(mk2, pack2(t0, t1));         // -round(v*c)
+  float p0, p1;
+  unpack2(exp2_frac_poly<DEG>(fma2(v2, c2, nr2)), p0, p1);
+  // (bits of t) << 23 = (n + K) << 23 modulo 2^32: added to the bits of p in [0.70, 1.42] it lowers the exponent by |n + K|
+  p0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
+  p1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
+  return pack2(p0, p1);
+}
+
 __device__ __forceinline__ void named_barrier(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
