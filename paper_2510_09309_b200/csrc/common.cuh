@@ -20,7 +20,7 @@ struct maskkv_ctx {
   int last_cuda_error;     // cudaError_t of the most recent failed runtime call (0 = none)
   uint32_t host_flags;     // status bits raised on the host (MASKKV_FLAG_FALLBACK); reported and cleared by maskkv_check_status
   unsigned force_simt;     // MASKKV_FORCE_SIMT, debugging: bit 0 = scoring sweep 1, bit 1 = scoring sweep 2, bit 2 = attention on the FP32 pipes
-  unsigned kernel_choice;  // MASKKV_KERNEL_CHOICE, debugging: bit 0 = projection on single CTAs instead of pairs, bit 1 / bit 2 = selection always on one CTA per segment / always on clusters
+  unsigned kernel_choice;  // MASKKV_KERNEL_CHOICE, debugging: bit 0 = projection on single CTAs instead of pairs, bit 1 / bit 2 / bit 3 = selection always on one CTA per segment with the keys in shared memory / always on clusters / always on one CTA per segment with the keys in registers
 };
 
 // The descriptor after validation, passed to kernels by value.

@@ -539,10 +539,15 @@ int maskkv_select(maskkv_ctx* ctx, const maskkv_desc_t* desc, const float* score
     return MASKKV_E_ALIGN;
   DeviceGuard guard(ctx->device);
   const int cta_cache = (ctx->smem_optin - mkv::kSelectStaticSmem) / 4 - mkv::kSelectCtaCand;
-  const int sel_force = (ctx->kernel_choice & 2u) ? 2 : (ctx->kernel_choice & 4u) ? 1 : 0;   // debugging: pin the kernel
-  // more segments than one wave of clusters (two CTAs per SM): one CTA per segment with the keys in shared memory gets
-  // through faster (measured: 128 / 256 segments of up to 32k keys)
+  const int sel_force = (ctx->kernel_choice & 2u) ? 2 : (ctx->kernel_choice & 4u) ? 1 : (ctx->kernel_choice & 8u) ? 3 : 0;   // debugging: pin the kernel
+  // more segments than one wave of clusters (two CTAs per SM): one CTA per segment gets through faster - with the keys in
+  // registers up to 32768 scores per segment, staged in shared memory beyond that
   const bool batch = (long long)sh.R * sh.Hkv * mkv::kSelectCluster > 2LL * ctx->sm_count;
+  if (sh.maxN <= mkv::kSelectBlockKeys && ((batch && sel_force == 0) || sel_force == 3)) {
+    mkv::launch_overlapped(mkv::select_kernel_block, dim3(sh.R * sh.Hkv), dim3(mkv::kSelectBlockThreads), 0,
+                           static_cast<cudaStream_t>(stream), sh, scores_dev, budgets_dev, offsets_dev, kept_idx_dev, ctx->status_dev);
+    return launch_status(ctx, 1);
+  }
   if (sh.maxN <= cta_cache && ((batch && sel_force == 0) || sel_force == 2 || sh.maxN > mkv::kSelectRegKeys)) {
     const int n_cache = (sh.maxN + 3) & ~3;
     mkv::launch_overlapped(mkv::select_kernel_cta, dim3(sh.R * sh.Hkv), dim3(mkv::kSelectThreads),

@@ -358,6 +358,266 @@ select_kernel_reg(Shape sh, const float* __restrict__ scores, const int32_t* __r
   cluster.barrier_wait();                                // no CTA leaves while a peer may still read its shared memory
 }
 
+// One CTA per segment with the keys in REGISTERS, for batches of segments of up to kSelectBlockKeys scores (the launch
+// over all (layer, head) segments of a model, a ragged serving batch): 1024 threads hold 32 keys each, so after the one
+// coalesced read of the segment no pass touches memory again - a pass costs two to four instructions per key instead of
+// an index computation, a bounds test and a shared-memory load on top.  Warp w owns the contiguous keys
+// [w * 32 * n_rows, (w + 1) * 32 * n_rows), row i of a thread is key jbase + 32 * i, so ranks inside a row come from a
+// ballot and the output is ascending.
+// The k-th largest key is found inside a window [lo, lo + range] of key values that starts as [smallest key, largest
+// key] and shrinks by a factor of up to 2048 per pass: digit = (key - lo) >> shift with the smallest shift that maps
+// the window onto 2048 bins.  Unlike a digit of fixed bit positions this spreads the keys over the bins whatever
+// power of two the scores happen to straddle (few populated bins would serialise the shared-memory atomics).  After a
+// pass either the threshold bin's keys are gathered into a short list (ranked by counting, or by further digits on the
+// list) or - when that bin holds more than the list - the next digit is taken on the registers again.  One emit pass.
+// Blocks take the requests in order of falling length, so a ragged batch ends with its short segments.
+constexpr int kSelectBlockThreads = 1024;
+constexpr int kSelectBlockWarps = kSelectBlockThreads / 32;
+constexpr int kSelectBlockRows = 32;                     // keys per thread
+constexpr int kSelectBlockKeys = kSelectBlockThreads * kSelectBlockRows;   // 32768
+constexpr int kSelectBlockCand = 4096;
+
+// order_key in five instructions: x + 0 turns -0 into +0 (and keeps everything else, NaN included)
+__device__ __forceinline__ uint32_t order_key_lean(float f) {
+  const uint32_t u = __float_as_uint(f + 0.f);
+  const uint32_t key = u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);
+  return (u & 0x7fffffffu) > 0x7f800000u ? 0u : key;
+}
+
+struct SelectBlockShared {
+  uint32_t hist[2048];
+  uint32_t cand[kSelectBlockCand];
+  uint32_t digit, remaining, ncand;
+  uint32_t warp_a[kSelectBlockWarps], warp_b[kSelectBlockWarps], warp_tot[kSelectBlockWarps];
+};
+
+// FULL: every thread holds kSelectBlockRows keys (N = kSelectBlockKeys), so no row needs a validity test.
+template <bool FULL>
+__device__ __forceinline__ void select_block_body(SelectBlockShared& sm, const float* __restrict__ seg, int N, int k,
+                                                  int32_t* __restrict__ kept) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n_rows = FULL ? kSelectBlockRows : min(kSelectBlockRows, (N + 32 * kSelectBlockWarps - 1) / (32 * kSelectBlockWarps));
+  const int jbase = warp * (32 * n_rows) + lane;
+  const int nv = FULL ? kSelectBlockRows : max(0, min(n_rows, (N - jbase + 31) >> 5));   // rows 0 .. nv-1 hold a key
+  uint32_t key[kSelectBlockRows];
+#pragma unroll
+  for (int i = 0; i < kSelectBlockRows; ++i) key[i] = (FULL || i < nv) ? __float_as_uint(__ldg(seg + jbase + i * 32)) : 0u;   // all loads first
+  // Scores are sums of softmax weights: +0 or positive and finite unless the inputs were not.  The bit patterns of such
+  // floats already order like the numbers, so they serve as keys as they are; one signed minimum and one unsigned
+  // maximum per key find the window and tell whether every score is of that kind (a negative number, -0 or a NaN
+  // shows as a negative minimum or a maximum above +inf).  Otherwise the keys are transformed and the window taken again.
+  int32_t s_min = 0x7fffffff;
+  uint32_t k_max = 0u;
+#pragma unroll
+  for (int i = 0; i < kSelectBlockRows; ++i)
+    if (FULL || i < nv) { s_min = min(s_min, (int32_t)key[i]); k_max = max(k_max, key[i]); }
+  s_min = __reduce_min_sync(0xffffffffu, s_min);
+  k_max = __reduce_max_sync(0xffffffffu, k_max);
+  if (lane == 0) { sm.warp_a[warp] = (uint32_t)s_min; sm.warp_b[warp] = k_max; }
+  for (int b = tid; b < 2048; b += kSelectBlockThreads) sm.hist[b] = 0;
+  if (tid == 0) sm.ncand = 0;
+  __syncthreads();
+  s_min = __reduce_min_sync(0xffffffffu, (int32_t)sm.warp_a[lane]);
+  k_max = __reduce_max_sync(0xffffffffu, sm.warp_b[lane]);
+  uint32_t lo = (uint32_t)s_min;
+  __syncthreads();                                       // warp_a / warp_b are reused below
+  if (s_min < 0 || k_max > 0x7f800000u) {                // block-uniform: some score is negative, -0 or NaN
+    uint32_t k_min = 0xffffffffu;
+    k_max = 0u;
+#pragma unroll
+    for (int i = 0; i < kSelectBlockRows; ++i) {
+      key[i] = order_key_lean(__uint_as_float(key[i]));
+      if (FULL || i < nv) { k_min = min(k_min, key[i]); k_max = max(k_max, key[i]); }
+    }
+    k_min = __reduce_min_sync(0xffffffffu, k_min);
+    k_max = __reduce_max_sync(0xffffffffu, k_max);
+    if (lane == 0) { sm.warp_a[warp] = k_min; sm.warp_b[warp] = k_max; }
+    __syncthreads();
+    lo = __reduce_min_sync(0xffffffffu, sm.warp_a[lane]);
+    k_max = __reduce_max_sync(0xffffffffu, sm.warp_b[lane]);
+    __syncthreads();
+  }
+  uint32_t range = k_max - lo;                           // 0 when all keys are equal
+  uint32_t remaining = (uint32_t)k;
+
+  int ncand = -1;                                        // >= 0: the search continues on cand[0 .. ncand)
+  bool first = true;                                     // every key lies inside the window
+#pragma unroll 1
+  while (range > 0 && ncand < 0) {                       // digits on the registers
+    const int shift = max(0, 21 - __clz(range));         // (range >> shift) < 2048
+    if (first) {
+#pragma unroll
+      for (int i = 0; i < kSelectBlockRows; ++i)
+        if (FULL || i < nv) atomicAdd(&sm.hist[(key[i] - lo) >> shift], 1u);
+    } else {
+#pragma unroll
+      for (int i = 0; i < kSelectBlockRows; ++i) {
+        const uint32_t d = key[i] - lo;
+        if ((FULL || i < nv) && d <= range) atomicAdd(&sm.hist[d >> shift], 1u);
+      }
+    }
+    first = false;
+    __syncthreads();
+    find_digit<kSelectBlockThreads>(sm.hist, 2048, remaining, sm.warp_tot, &sm.digit, &sm.remaining);
+    const uint32_t in_bin = sm.hist[sm.digit];           // keys that share the threshold digit
+    const uint32_t step = sm.digit << shift;
+    lo += step;
+    range = min(range - step, (uint32_t)((1ull << shift) - 1ull));
+    remaining = sm.remaining;
+    __syncthreads();                                     // everyone has read the histogram and the digit
+    if (range > 0) {
+      if (in_bin <= (uint32_t)kSelectBlockCand) {
+        // few enough: gather them (a thread rarely holds more than one) and finish on the list
+#pragma unroll
+        for (int i = 0; i < kSelectBlockRows; ++i)
+          if ((FULL || i < nv) && key[i] - lo <= range) sm.cand[atomicAdd(&sm.ncand, 1u)] = key[i];
+        __syncthreads();
+        ncand = (int)sm.ncand;
+      } else {
+        for (int b = tid; b < 2048; b += kSelectBlockThreads) sm.hist[b] = 0;
+        __syncthreads();
+      }
+    }
+  }
+  if (range > 0 && ncand <= kSelectRankMax) {
+    // a short list: the threshold is the candidate with fewer than `remaining` candidates above it and at least
+    // `remaining` at or above it
+    if (tid < ncand) {
+      const uint32_t mine = sm.cand[tid];
+      uint32_t gt = 0, ge = 0;
+      for (int u = 0; u < ncand; ++u) {
+        const uint32_t c = sm.cand[u];
+        gt += c > mine;
+        ge += c >= mine;
+      }
+      if (gt < remaining && remaining <= ge) { sm.digit = mine; sm.remaining = remaining - gt; }   // equal keys write equal values
+    }
+    __syncthreads();
+    lo = sm.digit;
+    remaining = sm.remaining;
+    range = 0;
+  }
+#pragma unroll 1
+  while (range > 0) {                                    // further digits on the list
+    const int shift = max(0, 21 - __clz(range));
+    __syncthreads();
+    for (int b = tid; b < 2048; b += kSelectBlockThreads) sm.hist[b] = 0;
+    __syncthreads();
+    for (int j = tid; j < ncand; j += kSelectBlockThreads) {
+      const uint32_t d = sm.cand[j] - lo;
+      if (d <= range) atomicAdd(&sm.hist[d >> shift], 1u);
+    }
+    __syncthreads();
+    find_digit<kSelectBlockThreads>(sm.hist, 2048, remaining, sm.warp_tot, &sm.digit, &sm.remaining);
+    const uint32_t step = sm.digit << shift;
+    lo += step;
+    range = min(range - step, (uint32_t)((1ull << shift) - 1ull));
+    remaining = sm.remaining;
+  }
+  const uint32_t thr = lo;                               // threshold key; `remaining` ties are kept, lowest indices first
+
+  // --- emit in ascending index order ---
+  // Usually the ties at the threshold are all kept (one key there, one wanted): then "at or above the threshold" is the
+  // whole test.  Only when more keys tie than are wanted are the ties told apart from the keys above.
+  uint32_t gt_mask = 0u, eq_mask = 0u;
+#pragma unroll
+  for (int i = 0; i < kSelectBlockRows; ++i)
+    if ((FULL || i < nv) && key[i] >= thr) gt_mask |= 1u << i;
+  {
+    const uint32_t n_ge = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(gt_mask));
+    if (lane == 0) sm.warp_a[warp] = n_ge;
+    __syncthreads();
+    const uint32_t total = __reduce_add_sync(0xffffffffu, sm.warp_a[lane]);
+    if (total != (uint32_t)k) {                          // block-uniform: more ties than wanted
+      gt_mask = 0u;
+#pragma unroll
+      for (int i = 0; i < kSelectBlockRows; ++i) {
+        if (FULL || i < nv) {
+          if (key[i] > thr) gt_mask |= 1u << i;
+          if (key[i] == thr) eq_mask |= 1u << i;
+        }
+      }
+    } else {
+      remaining = 0;                                     // no key counts as a tie
+    }
+    __syncthreads();                                     // warp_a is written again below
+  }
+  const uint32_t n_gt = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(gt_mask));
+  const uint32_t n_eq = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(eq_mask));
+  if (lane == 0) { sm.warp_a[warp] = n_gt; sm.warp_b[warp] = n_eq; }
+  __syncthreads();
+  // ties / outputs in lower-index warps: lane l looks at warp l, a warp scan gives the totals before this warp
+  uint32_t eq_before = 0, out_before = 0;
+  {
+    const uint32_t g = sm.warp_a[lane], e = sm.warp_b[lane];
+    uint32_t e_incl = e;                                 // inclusive prefix of the tie counts
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v = __shfl_up_sync(0xffffffffu, e_incl, o);
+      if (lane >= o) e_incl += v;
+    }
+    const uint32_t e_excl = e_incl - e;
+    const uint32_t take = e_excl >= remaining ? 0u : min(e, remaining - e_excl);
+    uint32_t o_incl = g + take;                          // outputs of warp l
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v = __shfl_up_sync(0xffffffffu, o_incl, o);
+      if (lane >= o) o_incl += v;
+    }
+    eq_before = __shfl_sync(0xffffffffu, e_excl, warp);
+    out_before = __shfl_sync(0xffffffffu, o_incl - (g + take), warp);
+  }
+  uint32_t rows = __reduce_or_sync(0xffffffffu, gt_mask | eq_mask);
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  while (rows) {                                         // rows of this warp that hold a key at or above the threshold
+    const int i = __ffs((int)rows) - 1;
+    rows &= rows - 1;
+    const bool gt = (gt_mask >> i) & 1u, eq = (eq_mask >> i) & 1u;
+    const uint32_t eq_bal = __ballot_sync(0xffffffffu, eq);
+    const bool take = gt || (eq && eq_before + __popc(eq_bal & lt_mask) < remaining);
+    const uint32_t take_bal = __ballot_sync(0xffffffffu, take);
+    if (take) kept[out_before + __popc(take_bal & lt_mask)] = jbase + i * 32;
+    out_before += __popc(take_bal);
+    eq_before += __popc(eq_bal);
+  }
+}
+
+__global__ void __launch_bounds__(kSelectBlockThreads, 1)
+select_kernel_block(Shape sh, const float* __restrict__ scores, const int32_t* __restrict__ budgets,
+                    const int32_t* __restrict__ offsets, int32_t* __restrict__ kept_idx, uint32_t* __restrict__ status) {
+  __shared__ __align__(16) SelectBlockShared sm;
+  const int tid = threadIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
+  if (tid == 0) sm.digit = 0u;
+  __syncthreads();
+  for (int t = tid; t < sh.R; t += kSelectBlockThreads) {  // the request that is number blockIdx / H_kv by falling length
+    const int nt = sh.prompt_cu[t + 1] - sh.prompt_cu[t];
+    int rank = 0;
+    for (int u = 0; u < sh.R; ++u) {
+      const int nu = sh.prompt_cu[u + 1] - sh.prompt_cu[u];
+      rank += (nu > nt || (nu == nt && u < t)) ? 1 : 0;
+    }
+    if (rank == (int)blockIdx.x / sh.Hkv) sm.digit = (uint32_t)t;
+  }
+  __syncthreads();
+  const int r = (int)sm.digit, hk = (int)blockIdx.x % sh.Hkv;
+  const int s = r * sh.Hkv + hk;
+  const int p0 = sh.prompt_cu[r], N = sh.prompt_cu[r + 1] - p0;
+  const int out0 = offsets[s];
+  int k = budgets[s];
+  if (k > N) { k = N; if (tid == 0) atomicOr(status, (uint32_t)MASKKV_FLAG_BOUNDS); }
+  if (k <= 0) return;
+  const float* seg = scores + (long long)hk * sh.sumN + p0;
+  if (k == N) {                                          // nothing to evict
+    for (int j = tid; j < N; j += kSelectBlockThreads) kept_idx[out0 + j] = j;
+    return;
+  }
+  __syncthreads();                                       // sm.digit has been read by everyone
+  if (N == kSelectBlockKeys) select_block_body<true>(sm, seg, N, k, kept_idx + out0);
+  else select_block_body<false>(sm, seg, N, k, kept_idx + out0);
+}
+
 // One CTA per segment, for batches of segments: the keys are staged in shared memory once and every pass over them
 // runs eight rows of 32 keys at a time per warp with the loads ahead of the uses (the cluster kernel above is built
 // for the latency of one layer's few segments; with hundreds of segments its clusters queue up in waves that each

@@ -236,10 +236,10 @@ def test_select_in_registers_crowded_threshold_bin_and_ties(ctx):
     assert ctx.maskkv_check_status() == 0
 
 
-@pytest.mark.parametrize("force", ["2", "4"])
+@pytest.mark.parametrize("force", ["2", "4", "8"])
 def test_both_select_kernels_on_crowded_bins_ties_and_ragged_batches(force, monkeypatch):
-    """The selection runs on clusters (few segments) or on one CTA per segment (batches); bits 1 / 2 of MASKKV_KERNEL_CHOICE
-    pin the choice.  Both must reproduce the oracle exactly on the crowded-bin / tie / NaN case above and on a ragged
+    """The selection runs on clusters (few segments) or on one CTA per segment (batches; keys in registers, or staged in
+    shared memory for segments beyond 32768 scores); bits 1 / 2 / 3 of MASKKV_KERNEL_CHOICE pin the choice.  All must reproduce the oracle exactly on the crowded-bin / tie / NaN case above and on a ragged
     batch of 100 segments with budgets from 0 to everything."""
     from paper_2510_09309_b200 import binding as B
     monkeypatch.setenv("MASKKV_KERNEL_CHOICE", force)
