@@ -20,6 +20,8 @@ struct maskkv_ctx {
   int last_cuda_error;     // cudaError_t of the most recent failed runtime call (0 = none)
   uint32_t host_flags;     // status bits raised on the host (MASKKV_FLAG_FALLBACK); reported and cleared by maskkv_check_status
   unsigned force_simt;     // MASKKV_FORCE_SIMT, debugging: bit 0 = scoring sweep 1, bit 1 = scoring sweep 2, bit 2 = attention on the FP32 pipes
+  int score_head_groups;   // MASKKV_SCORE_HEAD_GROUPS: scoring takes the KV heads in this many groups, both sweeps of a group back to
+                           // back, so that sweep 2 finds the group's keys in L2 (1 = all heads at once)
   unsigned kernel_choice;  // MASKKV_KERNEL_CHOICE, debugging: bit 0 = projection on single CTAs instead of pairs, bit 1 / bit 2 / bit 3 = selection always on one CTA per segment with the keys in shared memory / always on clusters / always on one CTA per segment with the keys in registers
 };
 
@@ -31,6 +33,7 @@ struct Shape {
   const int32_t* prompt_cu;               // device
   const int32_t* live_cu;                 // device
   int sumN, sumM, maxN, maxM;
+  int hk0, hkn;                           // KV heads [hk0, hk0 + hkn) a scoring launch covers (all of them unless the heads are taken in groups)
 };
 
 namespace mkv {

@@ -78,6 +78,8 @@ int resolve(const maskkv_desc_t* d, Shape* sh) {
   if ((reinterpret_cast<uintptr_t>(d->prompt_cu_dev) & 3u) || (reinterpret_cast<uintptr_t>(d->live_cu_dev) & 3u)) return MASKKV_E_ALIGN;
   sh->prompt_cu = d->prompt_cu_dev;
   sh->live_cu = d->live_cu_dev;
+  sh->hk0 = 0;
+  sh->hkn = sh->Hkv;
   return MASKKV_OK;
 }
 
@@ -86,11 +88,25 @@ struct ScoreWorkspace {
   int C, Tmax;
 };
 
+// KV heads per scoring launch: all of them, or Hkv / groups when the context takes the heads in groups (only the plain
+// case - one query head per KV head, at most 256 voters per request - is ever grouped).
+int score_heads_per_launch(const maskkv_ctx* ctx, const Shape& sh) {
+  if (ctx == nullptr || ctx->score_head_groups <= 1 || mkv::tc::score_tc_split_blocks(sh) || !mkv::tc::score_tc_supported(ctx, sh) ||
+      (ctx->force_simt & 3u))
+    return sh.Hkv;
+  const int groups = ctx->score_head_groups < sh.Hkv ? ctx->score_head_groups : sh.Hkv;
+  return (sh.Hkv + groups - 1) / groups;
+}
+
 ScoreWorkspace score_workspace(const maskkv_ctx* ctx, const Shape& sh) {
   ScoreWorkspace w;
   const long long keys = (long long)sh.maxN + sh.maxM;
   w.C = (int)((keys + mkv::kStatsChunk - 1) / mkv::kStatsChunk);
-  if (ctx != nullptr && w.C < mkv::tc::score_tc_max_chunks(ctx, sh)) w.C = mkv::tc::score_tc_max_chunks(ctx, sh);
+  if (ctx != nullptr) {
+    Shape per_launch = sh;
+    per_launch.hkn = score_heads_per_launch(ctx, sh);
+    if (w.C < mkv::tc::score_tc_max_chunks(ctx, per_launch)) w.C = mkv::tc::score_tc_max_chunks(ctx, per_launch);
+  }
   if (w.C < 1) w.C = 1;
   w.Tmax = mkv::tc::score_tc_max_tiles(sh);               // >= ceil(keys / 128), the FP32-pipe kernel's tiling
   if (w.Tmax < 1) w.Tmax = 1;
@@ -126,6 +142,30 @@ int launch_score(maskkv_ctx* ctx, const Shape& sh, const maskkv_desc_t* desc, co
   const bool tc_ok = mkv::tc::score_tc_supported(ctx, sh);
   const bool want_tc2 = tc_ok && !(ctx->force_simt & 2u);
   int n = 0;
+  const int per_launch = score_heads_per_launch(ctx, sh);
+  if (per_launch < sh.Hkv && sh.sumM > 0) {
+    // The KV heads in groups, both sweeps of a group back to back: the group's keys (per_launch x N x 2d bytes) are
+    // still in L2 when sweep 2 asks for them, so the key tensor crosses the memory bus once instead of twice.
+    for (int hk0 = 0; hk0 < sh.Hkv; hk0 += per_launch) {
+      Shape g = sh;
+      g.hk0 = hk0;
+      g.hkn = sh.Hkv - hk0 < per_launch ? sh.Hkv - hk0 : per_launch;
+      int launched = 0;
+      if (mkv::tc::launch_score_stats_tc(ctx, g, desc->prompt_cu, desc->live_cu, q, kp, km, part, w.C, seg_cnt, st) != 0) {
+        launch_status(ctx, n);
+        return MASKKV_E_CUDA;
+      }
+      ++n; ++ctx->tc_launches;
+      if (mkv::tc::launch_score_colsum_tc(ctx, g, desc->prompt_cu, desc->live_cu, q, kp, km, lse, part, w.C, rw, scores,
+                                          reinterpret_cast<float*>(ws + w.col_off), mass_part, w.Tmax, seg_cnt, mass_p, mass_m, scores_live,
+                                          any_without_voters, st, &launched) != 0) {
+        launch_status(ctx, n + launched);
+        return MASKKV_E_CUDA;
+      }
+      n += launched; ++ctx->tc_launches;
+    }
+    return launch_status(ctx, n);
+  }
   bool tc1 = false;                                          // sweep 1 ran on the tensor cores: `part` has its layout
   if (sh.sumM > 0) {
     if (tc_ok && !(ctx->force_simt & 1u))
@@ -251,6 +291,8 @@ int maskkv_create(maskkv_ctx** out, int device) {
     ctx->encode_tiled = nullptr;
   if (const char* e = getenv("MASKKV_FORCE_SIMT")) ctx->force_simt = (unsigned)strtoul(e, nullptr, 0);
   if (const char* e = getenv("MASKKV_KERNEL_CHOICE")) ctx->kernel_choice = (unsigned)strtoul(e, nullptr, 0);
+  ctx->score_head_groups = 1;
+  if (const char* e = getenv("MASKKV_SCORE_HEAD_GROUPS")) ctx->score_head_groups = (int)strtol(e, nullptr, 0);
   cudaFuncSetAttribute(mkv::select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - mkv::kSelectStaticSmem);
   cudaFuncSetAttribute(mkv::select_kernel_cta, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - mkv::kSelectStaticSmem);
   cudaFuncSetAttribute(mkv::budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);

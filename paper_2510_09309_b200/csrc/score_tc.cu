@@ -166,7 +166,7 @@ struct Walker {
 };
 
 __host__ __device__ __forceinline__ int walk_groups(const Shape& sh, int mode, int M) {
-  return M <= 0 ? 0 : (mode == kWalkColsum ? sh.Hkv : sh.H * ((M + kQBlock - 1) / kQBlock));
+  return M <= 0 ? 0 : (mode == kWalkColsum ? sh.hkn : sh.hkn * sh.g * ((M + kQBlock - 1) / kQBlock));
 }
 __device__ __forceinline__ int tiles_of(int N, int M) { return (N + kTile - 1) / kTile + (M + kTile - 1) / kTile; }
 
@@ -296,7 +296,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   pdl_launch_dependents();
   // sweep 2 counts finished mass partials per segment in seg_cnt; it reads them after this grid has ended
   if (blockIdx.x == 0 && seg_cnt != nullptr)
-    for (int i = threadIdx.x; i < sh.R * sh.Hkv; i += blockDim.x) seg_cnt[i] = 0u;
+    for (int i = threadIdx.x; i < sh.R * sh.hkn; i += blockDim.x) seg_cnt[(i / sh.hkn) * sh.Hkv + sh.hk0 + i % sh.hkn] = 0u;
   const uint32_t tmem_base = *tmem_slot;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   Walker wk;
@@ -309,7 +309,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       bool ok = true;
       while (ok && walker_next(wk, sh, s)) {
         const int qp_n = (s.M + kQBlock - 1) / kQBlock;
-        const int h = s.g / qp_n, q0 = (s.g % qp_n) * kQBlock, hk = h / sh.g;
+        const int h = sh.hk0 * sh.g + s.g / qp_n, q0 = (s.g % qp_n) * kQBlock, hk = h / sh.g;
         if (!(ok = mbar_wait(bars.qempty, q_it & 1, abort_flag, status, 0x100))) break;   // the MMA warp released the old block
         mbar_expect_tx(bars.qfull, S::kQBytes);
         for (int b = 0; b < S::kBoxes; ++b) tma_load_3d(base + S::kQOff + b * S::kQBoxBytes, &map_q, bars.qfull, b * 64, h, s.l0 + q0);
@@ -377,7 +377,7 @@ score_stats_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     bool ok = true;
     while (ok && walker_next(wk, sh, s)) {
       const int qp_n = (s.M + kQBlock - 1) / kQBlock;
-      const int h = s.g / qp_n, q0 = (s.g % qp_n) * kQBlock;
+      const int h = sh.hk0 * sh.g + s.g / qp_n, q0 = (s.g % qp_n) * kQBlock;
       const int n_qtiles = (s.M - q0 > kTile) ? 2 : 1;
       if (a >= n_qtiles) continue;
       // The row's reference m2 is an INTEGER in log2 units, at least the largest scaled logit seen so far, and
@@ -520,7 +520,7 @@ __global__ void score_merge_stats_tc(Shape sh, const float2* __restrict__ part, 
                                      float* __restrict__ lse) {
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= (long long)sh.H * sh.sumM) return;
-  const int h = (int)(t / sh.sumM), row = (int)(t % sh.sumM);
+  const int h = (int)(t / sh.sumM), row = (int)(t % sh.sumM);      // launched over all heads (hk0 = 0, hkn = H_kv)
   const int r = find_request(sh.live_cu, sh.R, row);
   long long base = 0;
   for (int r2 = 0; r2 < r; ++r2) {
@@ -578,9 +578,9 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   // which sweep 1 started the rows' unit: that is all the merge of its partials needs.
   // group of a run -> query head, KV head, first query of the block, index of the block among the KV head's blocks
   auto unit_of = [&](const Seg& sg, int& h, int& hk, int& q0, int& blk) {
-    if (!split) { h = hk = sg.g; q0 = 0; blk = 0; return; }
+    if (!split) { h = hk = sh.hk0 + sg.g; q0 = 0; blk = 0; return; }
     const int qp_n = (sg.M + kQBlock - 1) / kQBlock;
-    h = sg.g / qp_n; hk = h / sh.g; q0 = (sg.g % qp_n) * kQBlock; blk = (h % sh.g) * qp_n + sg.g % qp_n;
+    h = sh.hk0 * sh.g + sg.g / qp_n; hk = h / sh.g; q0 = (sg.g % qp_n) * kQBlock; blk = (h % sh.g) * qp_n + sg.g % qp_n;
   };
 
   if (warp == 0) {
@@ -895,7 +895,8 @@ int score_tc_max_chunks(const maskkv_ctx* ctx, const Shape& sh) {
   // that contributes at least H*T tiles to the walk, so a CTA's share is at least floor(H*T/G) >= H*T/(2G) tiles (or
   // one tile) and the unit spans at most 2*ceil(G/H) + 1 shares - and never more than T.
   const int T = (sh.maxN + kTile - 1) / kTile + (sh.maxM + kTile - 1) / kTile;
-  const int span = 2 * ((ctx->sm_count + sh.H - 1) / sh.H) + 2;
+  const int heads = sh.hkn * sh.g;                         // query heads one launch walks
+  const int span = 2 * ((ctx->sm_count + heads - 1) / heads) + 2;
   return 2 * (span < T ? span : T);
 }
 
