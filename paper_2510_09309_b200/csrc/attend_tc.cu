@@ -513,6 +513,364 @@ attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
 }
 
+// =====================================================================================================
+// Two query tiles per CTA, for launches with (many) more units than SMs - batches of requests or layers.
+//
+// A unit is a (128-query tile, query head) of one request; two units that share a KV head - the two query tiles of a
+// head, or tiles of different query heads of one group - walk the same key / value tiles, so one CTA takes both: the
+// tiles are fetched once, and while the softmax warpgroup of one unit exponentiates, the tensor cores work on the
+// other unit's products.  Stream w (0 / 1): its logits S_w and, over them, its P in tensor-memory columns
+// [128 w, 128 w + 128), its output O_w in [256 + 128 w, 384 + 128 w); softmax warpgroup w owns the stream (thread =
+// query row, all 128 key columns of a tile in two halves of 64, reference moved lazily as above); P V of stream w is
+// issued by warp 10 + w, both Q K^T by warp 1.  S_w is single-buffered: Q K^T of tile j + 1 of a stream follows its
+// P V of tile j, and the other stream's work fills the tensor pipe meanwhile.  No merge at the end: a warpgroup
+// normalises and stores its own tile.  grid (pairs of units per KV head, H_kv, R).
+// =====================================================================================================
+constexpr int kPKStages = 2;
+constexpr int kPVStages = 2;
+
+template <int D>
+struct PSmem {
+  static constexpr int kBoxes = D / 64;
+  static constexpr int kBoxBytes = kATile * 128;
+  static constexpr int kTileBytes = kBoxes * kBoxBytes;
+  static constexpr int kQOff = 0;                                          // two query tiles
+  static constexpr int kKOff = 2 * kTileBytes;
+  static constexpr int kVOff = kKOff + kPKStages * kTileBytes;
+  static constexpr int kBarOff = kVOff + kPVStages * kTileBytes;
+  static constexpr int kNumBars = 1 + 2 * kPKStages + 2 * kPVStages + 6;
+  static constexpr int kMiscOff = kBarOff + kNumBars * 8;
+  static constexpr int kBytes = kMiscOff + 16;
+  static constexpr int kDynamic = kBytes + 1024;
+};
+
+struct PBars {
+  uint64_t* qfull;
+  uint64_t *kfull, *kempty;                    // [kPKStages]
+  uint64_t *vfull, *vempty;                    // [kPVStages]
+  uint64_t *sfull, *pready, *odone;            // [2 streams]
+};
+__device__ __forceinline__ PBars carve_pbars(uint8_t* base, int off) {
+  uint64_t* b = reinterpret_cast<uint64_t*>(base + off);
+  PBars r;
+  r.qfull = b; r.kfull = b + 1; r.kempty = r.kfull + kPKStages; r.vfull = r.kempty + kPKStages; r.vempty = r.vfull + kPVStages;
+  r.sfull = r.vempty + kPVStages; r.pready = r.sfull + 2; r.odone = r.pready + 2;
+  return r;
+}
+
+template <int D>
+__global__ void __launch_bounds__(AWgs<D>::kThreads, 1)
+attend_pair_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kl,
+               const __grid_constant__ CUtensorMap map_vl, const __grid_constant__ CUtensorMap map_kc,
+               const __grid_constant__ CUtensorMap map_vc, Shape sh, const int32_t* __restrict__ offsets,
+               const int32_t* __restrict__ q_cu, int sum_q, int q_tiles, __nv_bfloat16* __restrict__ out,
+               float* __restrict__ lse, uint32_t* __restrict__ status) {
+  using S = PSmem<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const PBars bars = carve_pbars(base, S::kBarOff);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base + S::kMiscOff);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(base + S::kMiscOff + 4);
+
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    mbar_init(bars.qfull, 1);
+    for (int st = 0; st < kPKStages; ++st) { mbar_init(bars.kfull + st, 1); mbar_init(bars.kempty + st, 1); }
+    for (int st = 0; st < kPVStages; ++st) { mbar_init(bars.vfull + st, 1); mbar_init(bars.vempty + st, 2); }   // both P V issuers release a stage
+    for (int w = 0; w < 2; ++w) { mbar_init(bars.sfull + w, 1); mbar_init(bars.pready + w, kATile); mbar_init(bars.odone + w, 1); }
+    *abort_flag = 0u;
+    fence_barrier_init();
+  }
+  if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) {
+    prefetch_tmap(&map_q); prefetch_tmap(&map_kl); prefetch_tmap(&map_vl); prefetch_tmap(&map_kc); prefetch_tmap(&map_vc);
+  }
+  pdl_wait();
+
+  const int hk = blockIdx.y, r = blockIdx.z;
+  const int seg = r * sh.Hkv + hk;
+  const int l0 = sh.live_cu[r], l1 = sh.live_cu[r + 1], c0 = offsets[seg], c1 = offsets[seg + 1];
+  const int ql0 = q_cu[r], ql1 = q_cu[r + 1];
+  const int M = l1 - l0, nc = c1 - c0, Mq = ql1 - ql0;
+  // the two units of this CTA: unit u of the KV head = (query head hk*g + u / q_tiles, query tile u % q_tiles)
+  int uh[2], uq0[2];
+  bool active[2];
+#pragma unroll
+  for (int w = 0; w < 2; ++w) {
+    const int u = 2 * (int)blockIdx.x + w;
+    uh[w] = hk * sh.g + u / q_tiles;
+    uq0[w] = (u % q_tiles) * kATile;
+    active[w] = u < sh.g * q_tiles && uq0[w] < Mq;
+  }
+  if (!active[0] && !active[1]) {                           // uniform over the block
+    if (warp == 1) tmem_dealloc(tmem_base, 512);
+    return;
+  }
+  const int nt = (nc + kATile - 1) / kATile + (M + kATile - 1) / kATile;
+  const uint32_t tm_s = tmem_base, tm_o = tmem_base + 256;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const int n_act = (active[0] ? 1 : 0) + (active[1] ? 1 : 0);
+      mbar_expect_tx(bars.qfull, n_act * S::kTileBytes);
+      for (int w = 0; w < 2; ++w)
+        if (active[w])
+          for (int b = 0; b < S::kBoxes; ++b)
+            tma_load_3d(base + S::kQOff + w * S::kTileBytes + b * S::kBoxBytes, &map_q, bars.qfull, b * 64, uh[w], ql0 + uq0[w]);
+      int jk = 0, jv = 0;
+      const unsigned long long t_start = global_ns();
+      uint32_t spins = 0;
+      bool ok = true;
+      while (jk < nt || jv < nt) {
+        bool issued = false;
+        if (jk < nt) {
+          const int stage = jk % kPKStages, use = jk / kPKStages;
+          if (mbar_try_wait(bars.kempty + stage, (use & 1) ^ 1)) {
+            const ATile t = a_tile(jk, c0, nc, l0, M);
+            mbar_expect_tx(bars.kfull + stage, S::kTileBytes);
+            for (int b = 0; b < S::kBoxes; ++b)
+              tma_load_3d(base + S::kKOff + stage * S::kTileBytes + b * S::kBoxBytes, t.cache ? &map_kc : &map_kl,
+                          bars.kfull + stage, b * 64, t.cache ? 0 : hk, t.row);
+            ++jk;
+            issued = true;
+          }
+        }
+        if (jv < nt) {
+          const int stage = jv % kPVStages, use = jv / kPVStages;
+          if (mbar_try_wait(bars.vempty + stage, (use & 1) ^ 1)) {
+            const ATile t = a_tile(jv, c0, nc, l0, M);
+            mbar_expect_tx(bars.vfull + stage, S::kTileBytes);
+            for (int b = 0; b < S::kBoxes; ++b)
+              tma_load_3d(base + S::kVOff + stage * S::kTileBytes + b * S::kBoxBytes, t.cache ? &map_vc : &map_vl,
+                          bars.vfull + stage, b * 64, t.cache ? 0 : hk, t.row);
+            ++jv;
+            issued = true;
+          }
+        }
+        if (!issued && (++spins & 255u) == 0u) {             // bounded like every other wait
+          if (*abort_flag) { ok = false; break; }
+          if (global_ns() - t_start > kWaitLimitNs) {
+            *abort_flag = 1u; atomicOr(status, (uint32_t)MASKKV_FLAG_TIMEOUT); atomicExch(status + 1, 0x321u);
+            ok = false; break;
+          }
+        }
+      }
+      if (!ok) {   // wait (bounded) for the copies already issued
+        for (int i = max(0, jk - kPKStages); i < jk; ++i)
+          for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(bars.kfull + i % kPKStages, (i / kPKStages) & 1); ++it) __nanosleep(64);
+        for (int i = max(0, jv - kPVStages); i < jv; ++i)
+          for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(bars.vfull + i % kPVStages, (i / kPVStages) & 1); ++it) __nanosleep(64);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc_qk = idesc_bf16_f32(kATile, kATile);
+      bool ok = mbar_wait(bars.qfull, 0, abort_flag, status, 0x323);
+      tc_fence_after();
+      for (int j = 0; ok && j < nt; ++j) {
+        const int stage = j % kPKStages, use = j / kPKStages;
+        if (!(ok = mbar_wait(bars.kfull + stage, use & 1, abort_flag, status, 0x324))) break;
+        const uint32_t k_lo = smem_desc_lo(smem_u32(base + S::kKOff + stage * S::kTileBytes));
+        for (int w = 0; w < 2 && ok; ++w) {
+          if (!active[w]) continue;
+          // S_w is free once P V of tile j - 1 of this stream has read P from it
+          if (j >= 1 && !(ok = mbar_wait(bars.odone + w, (j - 1) & 1, abort_flag, status, 0x32b))) break;
+          tc_fence_after();
+          const uint32_t q_lo = smem_desc_lo(smem_u32(base + S::kQOff + w * S::kTileBytes));
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t o = ((kk >> 2) * S::kBoxBytes + (kk & 3) * 32) >> 4;
+            umma_ss(tm_s + w * kATile, make_desc(q_lo + o, kDescHiSw128), make_desc(k_lo + o, kDescHiSw128), idesc_qk, kk > 0);
+          }
+          umma_commit(bars.sfull + w);
+        }
+        umma_commit(bars.kempty + stage);
+      }
+    }
+  } else if (warp >= AWgs<D>::kPvWarp) {
+    // P V of stream w: O_w += P_w V over the tile's 128 keys, eight k-steps, accumulated in tensor memory over all tiles
+    const int w = warp - AWgs<D>::kPvWarp;
+    if (lane == 0) {
+      const uint32_t idesc_pv = idesc_bf16_f32_bn(kATile, D);
+      bool ok = true;
+      for (int j = 0; ok && j < nt; ++j) {
+        const int stage = j % kPVStages, use = j / kPVStages;
+        if (!(ok = mbar_wait(bars.vfull + stage, use & 1, abort_flag, status, 0x325))) break;
+        if (active[w]) {
+          if (!(ok = mbar_wait(bars.pready + w, j & 1, abort_flag, status, 0x327))) break;
+          tc_fence_after();
+          const uint32_t v_lo = ((smem_u32(base + S::kVOff + stage * S::kTileBytes) & 0x3ffffu) >> 4) | ((uint32_t)(S::kBoxBytes >> 4) << 16);
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            // P of keys [16 kk, 16 kk + 16) sits in packed columns [8 kk, 8 kk + 8) of S_w
+            umma_ts(tm_o + w * kATile, tm_s + w * kATile + 8 * kk, make_desc(v_lo + ((kk * 16 * 128) >> 4), kDescHiSw128), idesc_pv,
+                    (j > 0 || kk > 0) ? 1u : 0u);
+          umma_commit(bars.odone + w);
+        }
+        umma_commit(bars.vempty + stage);                    // an idle stream releases the stage at once
+      }
+    }
+  } else {
+    constexpr int SC = 64;                                  // key columns per half
+    constexpr float kSlack = 8.f;
+    const int w = (warp - 2) >> 2;                          // this warpgroup's stream
+    const int lane_group = warp & 3;
+    const int row = lane_group * 32 + lane;                 // query inside the tile
+    const int tid_wg = ((warp - 2) & 3) * 32 + lane;        // 0 .. 127 inside the warpgroup
+    const uint32_t lane_addr = (uint32_t)(lane_group * 32) << 16;
+    const uint32_t s_addr = tm_s + lane_addr + w * kATile;
+    const uint32_t o_addr = tm_o + lane_addr + w * kATile;
+    const float cs = sh.scale * kALog2e;
+    float m = -INFINITY, l = 0.f;
+    bool ok = true;
+    const bool mine = active[w];
+    for (int j = 0; j < nt && mine; ++j) {
+      const ATile t = a_tile(j, c0, nc, l0, M);
+      if (ok && t.valid < kATile) {
+        // ragged tail: zero the value rows that do not belong to this tile (each warpgroup clears all of them: its own
+        // P V is released by its own threads only)
+        const int stage = j % kPVStages, su = j / kPVStages;
+        if ((ok = mbar_wait(bars.vfull + stage, su & 1, abort_flag, status, 0x329))) {
+          uint8_t* v_tile = base + S::kVOff + stage * S::kTileBytes;
+          const int n16 = (kATile - t.valid) * 8;
+          for (int bx = 0; bx < S::kBoxes; ++bx) {
+            uint4* dst = reinterpret_cast<uint4*>(v_tile + bx * S::kBoxBytes + t.valid * 128);
+            for (int e = tid_wg; e < n16; e += kATile) dst[e] = make_uint4(0u, 0u, 0u, 0u);
+          }
+          fence_async_smem();
+        }
+      }
+      if (ok) ok = mbar_wait(bars.sfull + w, j & 1, abort_flag, status, 0x32a);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) continue;
+      tc_fence_after();
+      // Both halves of the tile feed one P V product, so they share one reference: a first pass over the logits finds the
+      // row maximum, a second one (the logits are read from tensor memory again, which costs little) forms P.
+      float tmax = -INFINITY;
+#pragma unroll 1
+      for (int hf = 0; hf < 2; ++hf) {
+        const int my_valid = min(SC, max(0, t.valid - hf * SC));
+        if (my_valid == 0) continue;                         // warp-uniform
+        float v[SC];
+#pragma unroll
+        for (int cb = 0; cb < SC / 32; ++cb) tmem_ld32(s_addr + hf * SC + cb * 32, v + cb * 32);
+        tmem_ld_wait();
+        if (my_valid < SC) {
+#pragma unroll
+          for (int c = 0; c < SC; ++c) if (c >= my_valid) v[c] = -INFINITY;
+        }
+#pragma unroll
+        for (int c = 0; c < SC; c += 2) tmax = max3(tmax, v[c], v[c + 1]);
+      }
+      // lazily moved reference: this stream's P V of tile j - 1 landed before Q K^T of tile j was issued, so O_w is at rest
+      const bool grow = m != -INFINITY && (tmax - m) * cs > kSlack;
+      const float f = grow ? ex2((m - tmax) * cs) : 1.f;
+      if (j > 0 && __any_sync(0xffffffffu, grow)) {
+#pragma unroll
+        for (int cb = 0; cb < D / 32; ++cb) {
+          float ov[32];
+          tmem_ld32(o_addr + cb * 32, ov);
+          tmem_ld_wait();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) ov[c] *= f;
+          tmem_st32(o_addr + cb * 32, reinterpret_cast<const uint32_t*>(ov));
+        }
+        tmem_st_wait();
+      }
+      if (grow) { l *= f; m = tmax; }
+      else if (m == -INFINITY) m = tmax;
+      float rs = 0.f;
+      const float neg = -m * cs;
+#pragma unroll 1
+      for (int hf = 0; hf < 2; ++hf) {
+        const int my_valid = min(SC, max(0, t.valid - hf * SC));
+        uint32_t packed[SC / 2];
+        if (my_valid == 0) {                                 // warp-uniform: a half without keys
+#pragma unroll
+          for (int c = 0; c < SC / 2; ++c) packed[c] = 0u;
+        } else {
+          float v[SC];
+#pragma unroll
+          for (int cb = 0; cb < SC / 32; ++cb) tmem_ld32(s_addr + hf * SC + cb * 32, v + cb * 32);
+          tmem_ld_wait();
+          if (my_valid < SC) {
+#pragma unroll
+            for (int c = 0; c < SC; ++c) if (c >= my_valid) v[c] = -INFINITY;
+          }
+#pragma unroll
+          for (int c = 0; c < SC; c += 2) {
+            const float p0 = ex2(fmaf(v[c], cs, neg)), p1 = ex2(fmaf(v[c + 1], cs, neg));
+            rs += p0 + p1;
+            packed[c / 2] = pack_bf16(p0, p1);
+          }
+        }
+        // P of this half over logits that have been read: packed columns [32 hf, 32 hf + 32) of S_w.  (Half 1's logits
+        // sit in columns 64 .. 127 and are read before anything is stored there.)
+        tmem_st32(s_addr + hf * (SC / 2), packed);
+      }
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(bars.pready + w);
+      l += rs;
+    }
+    // the stream's last P V must have landed
+    if (mine && nt > 0 && ok) ok = mbar_wait(bars.odone + w, (nt - 1) & 1, abort_flag, status, 0x32d);
+    ok = __all_sync(0xffffffffu, ok);
+    named_barrier(3, 2 * kATile);                            // ... and the other stream's: nothing reads the rings any more
+    if (mine) {
+      // every other role has finished with shared memory by now (this stream's last P V read the last value tile, and the
+      // key tiles were consumed before it): the tile leaves through the key ring (stream 0) / value ring (stream 1) as
+      // whole 2*D-byte rows, 16 bytes per lane
+      uint8_t* stage_o = base + (w == 0 ? S::kKOff : S::kVOff);
+      constexpr int RS = D * 2 + 16;
+      const int i = uq0[w] + row;
+      if (ok) {
+        tc_fence_after();
+        const float inv = nt > 0 ? 1.f / l : 0.f;
+#pragma unroll
+        for (int cb = 0; cb < D / 32; ++cb) {
+          float ov[32];
+          if (nt > 0) { tmem_ld32(o_addr + cb * 32, ov); tmem_ld_wait(); }
+          else {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) ov[c] = 0.f;
+          }
+          uint4* dst = reinterpret_cast<uint4*>(stage_o + row * RS + cb * 64);
+#pragma unroll
+          for (int c = 0; c < 32; c += 8) {
+            uint4 o4;
+            o4.x = pack_bf16(ov[c] * inv, ov[c + 1] * inv);
+            o4.y = pack_bf16(ov[c + 2] * inv, ov[c + 3] * inv);
+            o4.z = pack_bf16(ov[c + 4] * inv, ov[c + 5] * inv);
+            o4.w = pack_bf16(ov[c + 6] * inv, ov[c + 7] * inv);
+            dst[c / 8] = o4;
+          }
+        }
+        if (lse != nullptr && i < Mq && !*abort_flag) lse[(long long)uh[w] * sum_q + ql0 + i] = m * sh.scale + logf(l);
+      }
+      named_barrier(1 + w, kATile);
+      if (!*abort_flag) {
+        constexpr int PPR = D * 2 / 16;
+        const int pieces = min(kATile, Mq - uq0[w]) * PPR;
+        uint8_t* out_tile = reinterpret_cast<uint8_t*>(out + (long long)(ql0 + uq0[w]) * sh.q_ts + (long long)uh[w] * sh.q_hs);
+        for (int e = tid_wg; e < pieces; e += kATile) {
+          const int rr = e / PPR, pc = e % PPR;
+          *reinterpret_cast<uint4*>(out_tile + (long long)rr * sh.q_ts * 2 + pc * 16) =
+              *reinterpret_cast<const uint4*>(stage_o + rr * RS + pc * 16);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
+}
+
 namespace {
 // The opt-in shared-memory size is an attribute of the kernel on ONE device: remembered per device, set with that device
 // current (the entry points hold a device guard).
@@ -522,6 +880,15 @@ cudaError_t set_attend_attr(int device) {
   if (device < 0 || device >= kMaxAttrDevices) return cudaErrorInvalidDevice;
   if (done[device]) return cudaSuccess;
   const cudaError_t e = cudaFuncSetAttribute(attend_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, ASmem<D>::kDynamic);
+  done[device] = e == cudaSuccess;
+  return e;
+}
+template <int D>
+cudaError_t set_attend_pair_attr(int device) {
+  static bool done[kMaxAttrDevices] = {};
+  if (device < 0 || device >= kMaxAttrDevices) return cudaErrorInvalidDevice;
+  if (done[device]) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(attend_pair_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, PSmem<D>::kDynamic);
   done[device] = e == cudaSuccess;
   return e;
 }
@@ -551,6 +918,26 @@ int launch_attend_tc(maskkv_ctx* ctx, const Shape& sh, const void* q, const int3
   // length the capacity allows; with enough units it only adds set-up cost.
   const unsigned q_tiles = (unsigned)((max_q + kATile - 1) / kATile);
   const long long units = (long long)q_tiles * sh.H * sh.R;
+  // Many more units than SMs (a batch of requests or layers): two units that share a KV head per CTA - their key / value
+  // tiles are fetched once and the two softmax streams keep the tensor cores and the special-function unit busy in
+  // turn.  Few units: one per CTA, so that all of them run at once (the per-layer latency case).
+  const bool pairs_possible = sh.g * q_tiles >= 2;
+  const bool want_pairs = (ctx->kernel_choice & 32u) ? true : (ctx->kernel_choice & 64u) ? false : units >= 2LL * ctx->sm_count;
+  if (pairs_possible && want_pairs) {
+    dim3 grid_p((sh.g * q_tiles + 1) / 2, sh.Hkv, sh.R);
+    cudaError_t le;
+    if (sh.d == 128) {
+      if (set_attend_pair_attr<128>(ctx->device) != cudaSuccess) return 1;
+      le = launch_overlapped(attend_pair_tc<128>, grid_p, dim3(AWgs<128>::kThreads), PSmem<128>::kDynamic, st, mq, mkl, mvl, mkc, mvc, sh,
+                             offsets, q_cu, sum_q, (int)q_tiles, (__nv_bfloat16*)out, lse, ctx->status_dev);
+    } else {
+      if (set_attend_pair_attr<64>(ctx->device) != cudaSuccess) return 1;
+      le = launch_overlapped(attend_pair_tc<64>, grid_p, dim3(AWgs<64>::kThreads), PSmem<64>::kDynamic, st, mq, mkl, mvl, mkc, mvc, sh,
+                             offsets, q_cu, sum_q, (int)q_tiles, (__nv_bfloat16*)out, lse, ctx->status_dev);
+    }
+    if (le != cudaSuccess) { cudaGetLastError(); return 1; }
+    return 0;
+  }
   const long long mean_rows = cache_rows / ((long long)sh.R * sh.Hkv);
   const long long chain = (mean_rows + kATile - 1) / kATile + (sh.maxM + kATile - 1) / kATile;
   const unsigned nsplit = (2 * units <= ctx->sm_count && chain >= kASplitMinTiles) ? 2u : 1u;
