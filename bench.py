@@ -698,13 +698,14 @@ def bench_ours(args):
 
     # ---- select / compact / attend on a batch: at one layer they are launch- and latency-bound whatever the kernel does
     # (4-17 MB per call), so a fraction of the memory roof only shows when many segments go into one launch
-    batched = batched_calls(ctx, B, device) if rank == 0 else None
-    dream = dream_gqa_block(ctx, B, device, load_peaks()) if rank == 0 else None
-    stack, schedules = stack_batched_block(ctx, B, device, load_peaks()) if rank == 0 else (None, None)
+    blocks = set(args.blocks.split(",")) if args.blocks else set()
+    batched = batched_calls(ctx, B, device) if rank == 0 and "batched" in blocks else None
+    dream = dream_gqa_block(ctx, B, device, load_peaks()) if rank == 0 and "dream" in blocks else None
+    stack, schedules = stack_batched_block(ctx, B, device, load_peaks()) if rank == 0 and "stack" in blocks else (None, None)
 
     # ---- calibration step of the budget rule (Eq. 8), outside the timed step: a streaming reduction bound by HBM
     importance = None
-    if rank == 0:
+    if rank == 0 and "extras" in blocks:
         n_tok, hidden = N + wl.n_mask, 4096                       # one LLaDA-8B-shaped layer: 541 MB read per call
         g = torch.Generator(device=device); g.manual_seed(synth.BASE_SEED + 8)
         h_in = torch.randn(n_tok, hidden, generator=g, device=device).bfloat16()
@@ -1032,6 +1033,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="time plain calls instead of replaying CUDA graphs")
+    ap.add_argument("--blocks", default="batched,dream,stack,extras",
+                    help="side measurements to run after the timed steps (comma list; empty = none): batched = select / compact / "
+                         "attend on the ragged serving batch, dream = the Dream-shaped layer, stack = select / compact over all "
+                         "1024 segments of the 32-layer stack, extras = layer importance, refresh test, mask-only projection")
     ap.add_argument("--plumbing-only", action="store_true",
                     help="run the multi-rank plumbing (rendezvous, sharding, reductions) and nothing else; needs no GPU")
     args = ap.parse_args()
