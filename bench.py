@@ -173,10 +173,10 @@ def run_layer(ctx, buf, x, live, k_l, alpha, events=None):
 
 # DRAM bytes (read + write) of one maskkv_score call at this workload.  bench.py cannot read DRAM counters itself: the
 # figure is dram__bytes_read.sum + dram__bytes_write.sum of the call's two kernels from one ncu capture of this very
-# command (sweep 1 279.6 MB + sweep 2 290.7 MB: the key tensor is read once per sweep); the JSON line names the source.
-SCORE_DRAM_TRAFFIC_BYTES = 570.3e6
+# command (sweep 1 279.5 MB + sweep 2 281.6 MB: the key tensor is read once per sweep); the JSON line names the source.
+SCORE_DRAM_TRAFFIC_BYTES = 561.1e6
 SCORE_DRAM_TRAFFIC_SOURCE = ("ncu --set full --clock-control none -k regex:score_(stats|colsum)_tc -s 3 -c 1 python bench.py --steps 4 "
-                             "--warmup 3 --no-graph: dram__bytes_read.sum + dram__bytes_write.sum, sweep 1 279.6 MB + sweep 2 290.7 MB; "
+                             "--warmup 3 --no-graph: dram__bytes_read.sum + dram__bytes_write.sum, sweep 1 279.5 MB + sweep 2 281.6 MB; "
                              "a constant of this file, not measured by this run")
 
 
