@@ -55,7 +55,14 @@ constexpr int kColsumPolyPairs = MASKKV_COLSUM_POLY;
 // key stream, the products and the accumulator hand-over cost without the exponentials.
 #ifndef MASKKV_DBG_KSTEPS
 #define MASKKV_DBG_KSTEPS 8
-#endif    // sweep 2, degree 4
+#endif
+// Two more timing probes for sweep 2 (both give wrong scores): MASKKV_DBG_RELEASE_AT=c hands the accumulator back to the MMA
+// issuer as soon as chunk c of its columns is in registers (0 = three chunks early), MASKKV_DBG_NOTAIL drops everything a
+// warp does per tile after its exponentials (exchange of the halves, score stores, mass sums).  Measured on B200 at the 32k
+// layer, whole call: 175.0 us as shipped; release at chunk 0 / 1 / 2: 174.8 / 174.8 / 175.4; no tail: 173.2; one MMA k-step
+// of eight with all the arithmetic: 164.4.  Neither the hand-over of the accumulators, nor the per-tile tail, nor the
+// products hold the sweeps: the epilogue's own instruction stream does (96 registers per thread where the compiler would
+// take 150 for sweep 2 and 204 for sweep 1 if it could).
 // which pairs of a group of eight go to the polynomial: spread out, so that both units always have work in flight
 __host__ __device__ constexpr bool poly_pair(int pair, int n_of_8) {
   return ((pair & 7) + 1) * n_of_8 / 8 > (pair & 7) * n_of_8 / 8;
@@ -776,7 +783,11 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             float v[32];
             tmem_ld32(taddr + cb * 32, v);
             tmem_ld_wait();
+#ifdef MASKKV_DBG_RELEASE_AT
+            if (cb == MASKKV_DBG_RELEASE_AT) { tc_fence_before(); mbar_arrive(bars.tempty + buf); }
+#else
             if (cb + 1 == chunks) { tc_fence_before(); mbar_arrive(bars.tempty + buf); }   // last logits are in registers
+#endif
 #ifdef MASKKV_DBG_NOMATH
             acc2 = add2(acc2, pack2(v[3], v[9]));
 #else
@@ -789,6 +800,10 @@ score_colsum_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         unpack2(acc2, a0, a1);
         float* slot = xch + (uses & 1) * kTile;
         ++uses;
+#ifdef MASKKV_DBG_NOTAIL
+        slot[row] = a0 + a1;
+        continue;
+#endif
         if (half == 1) slot[row] = a0 + a1;
         named_barrier(5 + buf, 2 * kTile);                  // the pair's two halves of this tile are done
         if (half == 1 || !ok) continue;
