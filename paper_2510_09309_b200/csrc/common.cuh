@@ -22,7 +22,7 @@ struct maskkv_ctx {
   unsigned force_simt;     // MASKKV_FORCE_SIMT, debugging: bit 0 = scoring sweep 1, bit 1 = scoring sweep 2, bit 2 = attention on the FP32 pipes
   int score_head_groups;   // MASKKV_SCORE_HEAD_GROUPS: scoring takes the KV heads in this many groups, both sweeps of a group back to
                            // back, so that sweep 2 finds the group's keys in L2 (1 = all heads at once)
-  unsigned kernel_choice;  // MASKKV_KERNEL_CHOICE, debugging: bit 0 = projection on single CTAs instead of pairs, bit 1 / bit 2 / bit 3 = selection always on one CTA per segment with the keys in shared memory / always on clusters / always on one CTA per segment with the keys in registers, bit 5 / bit 6 = attention always / never with two units per CTA
+  unsigned kernel_choice;  // MASKKV_KERNEL_CHOICE, debugging: bit 0 = projection on single CTAs instead of pairs, bit 1 / bit 2 / bit 3 = selection always on one CTA per segment with the keys in shared memory / always on clusters / always on one CTA per segment with the keys in registers, bit 5 / bit 6 = attention always / never with two units per CTA, bit 7 = selection always on the persistent kernel, bit 8 = that kernel on at most 3 CTAs
 };
 
 // The descriptor after validation, passed to kernels by value.

@@ -295,6 +295,7 @@ int maskkv_create(maskkv_ctx** out, int device) {
   if (const char* e = getenv("MASKKV_SCORE_HEAD_GROUPS")) ctx->score_head_groups = (int)strtol(e, nullptr, 0);
   cudaFuncSetAttribute(mkv::select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - mkv::kSelectStaticSmem);
   cudaFuncSetAttribute(mkv::select_kernel_cta, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - mkv::kSelectStaticSmem);
+  cudaFuncSetAttribute(mkv::select_kernel_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, mkv::kSelectStreamSmem);
   cudaFuncSetAttribute(mkv::budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
   cudaFuncSetAttribute(mkv::select_kernel_reg<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, mkv::kSelectCandCap * 4);
   cudaFuncSetAttribute(mkv::select_kernel_reg<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, mkv::kSelectCandCap * 4);
@@ -585,6 +586,15 @@ int maskkv_select(maskkv_ctx* ctx, const maskkv_desc_t* desc, const float* score
   // more segments than one wave of clusters (two CTAs per SM): one CTA per segment gets through faster - with the keys in
   // registers up to 32768 scores per segment, staged in shared memory beyond that
   const bool batch = (long long)sh.R * sh.Hkv * mkv::kSelectCluster > 2LL * ctx->sm_count;
+  // more segments than SMs: persistent CTAs, the next segment's scores copied to shared memory under the current one's work
+  const bool stream_forced = (ctx->kernel_choice & 128u) != 0;
+  if (sh.maxN <= mkv::kSelectBlockKeys && ((batch && sel_force == 0 && sh.R * sh.Hkv > ctx->sm_count) || stream_forced)) {
+    int grid = sh.R * sh.Hkv < ctx->sm_count ? sh.R * sh.Hkv : ctx->sm_count;
+    if ((ctx->kernel_choice & 256u) && grid > 3) grid = 3;                     // debugging: several segments per CTA on small cases
+    mkv::launch_overlapped(mkv::select_kernel_stream, dim3(grid), dim3(mkv::kSelectBlockThreads), mkv::kSelectStreamSmem,
+                           static_cast<cudaStream_t>(stream), sh, scores_dev, budgets_dev, offsets_dev, kept_idx_dev, ctx->status_dev);
+    return launch_status(ctx, 1);
+  }
   if (sh.maxN <= mkv::kSelectBlockKeys && ((batch && sel_force == 0) || sel_force == 3)) {
     mkv::launch_overlapped(mkv::select_kernel_block, dim3(sh.R * sh.Hkv), dim3(mkv::kSelectBlockThreads), 0,
                            static_cast<cudaStream_t>(stream), sh, scores_dev, budgets_dev, offsets_dev, kept_idx_dev, ctx->status_dev);

@@ -46,7 +46,11 @@ __device__ __forceinline__ void find_digit(const uint32_t* hist, int bins, uint3
   if (lane == 0) warp_tot[warp] = suf;
   __syncthreads();
   uint32_t above = suf - mine;                           // keys with a higher digit
-  for (int w2 = warp + 1; w2 < THREADS / 32; ++w2) above += warp_tot[w2];
+  if (THREADS == 1024) {                                 // 32 warps: lane l looks at warp l
+    above += __reduce_add_sync(0xffffffffu, lane > warp ? warp_tot[lane] : 0u);
+  } else {
+    for (int w2 = warp + 1; w2 < THREADS / 32; ++w2) above += warp_tot[w2];
+  }
 #pragma unroll
   for (int t = BPT - 1; t >= 0; --t) {                   // highest digit first
     if (above < remaining && above + c[t] >= remaining) { *out_digit = BPT * tid + t; *out_remaining = remaining - above; }
@@ -384,24 +388,250 @@ __device__ __forceinline__ uint32_t order_key_lean(float f) {
   return (u & 0x7fffffffu) > 0x7f800000u ? 0u : key;
 }
 
+#ifdef MASKKV_DBG_SELECT_CLOCK
+__device__ unsigned int g_sel_prints = 0;
+#define SEL_STAMP(n) do { if (blockIdx.x == 5 && threadIdx.x == 0) st_[n] = clock64(); } while (0)
+#else
+#define SEL_STAMP(n) do { } while (0)
+#endif
 struct SelectBlockShared {
   uint32_t hist[2048];
   uint32_t cand[kSelectBlockCand];
+  int32_t cand_idx[kSelectBlockCand];                     // indices of the listed keys (sampled short cut)
   uint32_t digit, remaining, ncand;
   uint32_t warp_a[kSelectBlockWarps], warp_b[kSelectBlockWarps], warp_tot[kSelectBlockWarps];
 };
 
 // FULL: every thread holds kSelectBlockRows keys (N = kSelectBlockKeys), so no row needs a validity test.
-template <bool FULL>
-__device__ __forceinline__ void select_block_body(SelectBlockShared& sm, const float* __restrict__ seg, int N, int k,
+// Short cut for the usual case (few keys wanted out of many): one key per thread serves as a sample; a histogram of the
+// samples gives a bound `lo` that - unless the samples mislead - lies below the k-th largest key with few keys above it.
+// One pass over the registers collects the keys at or above `lo` (key and index, in ascending index order) in shared
+// memory; the k-th largest is then found on that list and the kept set is a compaction of the list.  Two passes over
+// the registers less than the full search, and none of its 32 histogram updates per thread.  Returns false, having
+// written nothing, when the short cut does not apply (a sample that is negative, -0 or NaN; too many keys wanted; fewer
+// than k or more than the list holds at or above `lo`): the caller then runs the full search on the same registers.
+template <bool FULL, class Load, class Release>
+__device__ __forceinline__ bool select_block_sampled(SelectBlockShared& sm, const uint32_t (&key)[kSelectBlockRows], int nv, int jbase,
+                                                     int N, int k, int32_t* __restrict__ kept, Load load, Release release) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  const bool has = FULL || nv > 0;
+#ifdef MASKKV_DBG_SELECT_CLOCK
+  long long st_[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#endif
+  SEL_STAMP(0);
+  const uint32_t smp = key[0];
+  {
+    const uint32_t mn = __reduce_min_sync(0xffffffffu, has ? smp : 0xffffffffu);
+    const uint32_t mx = __reduce_max_sync(0xffffffffu, has ? smp : 0u);
+    const uint32_t ns = (uint32_t)__popc(__ballot_sync(0xffffffffu, has));
+    if (lane == 0) { sm.warp_a[warp] = mn; sm.warp_b[warp] = mx; sm.warp_tot[warp] = ns; }
+  }
+  for (int b = tid; b < 2048; b += kSelectBlockThreads) sm.hist[b] = 0;
+  __syncthreads();
+  uint32_t lo = __reduce_min_sync(0xffffffffu, sm.warp_a[lane]);
+  const uint32_t s_max = __reduce_max_sync(0xffffffffu, sm.warp_b[lane]);
+  const uint32_t n_s = __reduce_add_sync(0xffffffffu, sm.warp_tot[lane]);
+  __syncthreads();                                       // the per-warp slots are written again below
+  if (s_max > 0x7f800000u) return false;                 // raw bits do not order like the numbers
+  const float mu = (float)k * (float)n_s / (float)N;     // samples expected above the k-th largest key
+  const uint32_t r_lo = (uint32_t)(mu + 5.f * sqrtf(mu) + 4.f);
+  if (r_lo >= n_s || (long long)r_lo * N > 3072LL * n_s) return false;
+  if (s_max > lo) {
+    const int shift = max(0, 21 - __clz(s_max - lo));
+    if (has) atomicAdd(&sm.hist[(smp - lo) >> shift], 1u);
+    __syncthreads();
+    find_digit<kSelectBlockThreads>(sm.hist, 2048, r_lo, sm.warp_tot, &sm.digit, &sm.remaining);
+    lo += sm.digit << shift;
+  }
+  SEL_STAMP(1);
+  // keys at or above lo: bit i of `mask` = row i of this thread
+  uint32_t mask = 0u;
+#pragma unroll
+  for (int i = 0; i < kSelectBlockRows; ++i)
+    if ((FULL || i < nv) && key[i] >= lo) mask |= 1u << i;
+  // Transpose the warp's 32 x 32 bits: lane i then holds the ballot of row i, so the list positions (ascending index:
+  // warps own consecutive index ranges, rows ascend, lanes ascend) come from one scan over the rows instead of a ballot
+  // per row.  The histogram is free by now: warp w keeps its 32 ballots and 32 row offsets in hist[64 w ...].
+  uint32_t bal = mask;
+#pragma unroll
+  for (int sft = 16; sft >= 1; sft >>= 1) {
+    const uint32_t keep = sft == 16 ? 0x0000ffffu : sft == 8 ? 0x00ff00ffu : sft == 4 ? 0x0f0f0f0fu : sft == 2 ? 0x33333333u : 0x55555555u;
+    const uint32_t other = __shfl_xor_sync(0xffffffffu, bal, sft);
+    bal = (lane & sft) ? (((other >> sft) & keep) | (bal & ~keep)) : ((bal & keep) | ((other & keep) << sft));
+  }
+  __syncthreads();                                       // every thread is done with the histogram of the samples
+  uint32_t C, pos;
+  {
+    const uint32_t cnt = (uint32_t)__popc(bal);
+    uint32_t incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t u = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += u;
+    }
+    sm.hist[warp * 64 + lane] = bal;
+    sm.hist[warp * 64 + 32 + lane] = incl - cnt;
+    if (lane == 31) sm.warp_a[warp] = incl;
+    __syncthreads();
+    const uint32_t v = sm.warp_a[lane];
+    uint32_t w_incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t u = __shfl_up_sync(0xffffffffu, w_incl, o);
+      if (lane >= o) w_incl += u;
+    }
+    C = __shfl_sync(0xffffffffu, w_incl, 31);
+    pos = __shfl_sync(0xffffffffu, w_incl - v, warp);
+  }
+  SEL_STAMP(2);
+  if (C < (uint32_t)k || C > (uint32_t)kSelectBlockCand) { __syncthreads(); return false; }
+  // a thread rarely holds more than one listed key: it lists the indices, and the keys are read back by list position
+  // (the segment is still in the staging buffer or in the caches) - indexing the registers by a run-time row would not do
+  for (uint32_t m = mask; m != 0u; m &= m - 1u) {
+    const int i = __ffs((int)m) - 1;
+    sm.cand_idx[pos + sm.hist[warp * 64 + 32 + i] + __popc(sm.hist[warp * 64 + i] & lt_mask)] = jbase + i * 32;
+  }
+  __syncthreads();
+  {
+    uint32_t l_max = 0u;
+    for (int j = tid; j < (int)C; j += kSelectBlockThreads) {
+      const uint32_t c = load(sm.cand_idx[j]);
+      sm.cand[j] = c;
+      l_max = max(l_max, c);
+    }
+    l_max = __reduce_max_sync(0xffffffffu, l_max);
+    if (lane == 0) sm.warp_b[warp] = l_max;
+  }
+  __syncthreads();
+  release();                                             // the segment's copy is no longer needed
+  const uint32_t k_max = __reduce_max_sync(0xffffffffu, sm.warp_b[lane]);
+  __syncthreads();
+  if (k_max > 0x7f800000u) return false;                 // a negative score, -0 or a NaN somewhere in the segment
+  const int ncand = (int)C;
+  SEL_STAMP(3);
+  uint32_t range = k_max - lo, remaining = (uint32_t)k;
+  // rank by counting on a short list of keys: the wanted key has fewer than `remaining` keys above it and at least
+  // `remaining` at or above it
+  auto rank_short = [&](const uint32_t* list, int n) {
+    if (tid < n) {
+      const uint32_t mine_k = list[tid];
+      uint32_t gt = 0, ge = 0;
+      for (int u = 0; u < n; ++u) {
+        const uint32_t c = list[u];
+        gt += c > mine_k;
+        ge += c >= mine_k;
+      }
+      if (gt < remaining && remaining <= ge) { sm.digit = mine_k; sm.remaining = remaining - gt; }   // equal keys write equal values
+    }
+    __syncthreads();
+    lo = sm.digit;
+    remaining = sm.remaining;
+    range = 0;
+  };
+  if (range > 0 && ncand <= kSelectRankMax) rank_short(sm.cand, ncand);
+#pragma unroll 1
+  while (range > 0) {                                    // digits on the list, within the window [lo, lo + range]
+    const int shift = max(0, 21 - __clz(range));
+    __syncthreads();
+    for (int b = tid; b < 2048; b += kSelectBlockThreads) sm.hist[b] = 0;
+    if (tid == 0) sm.ncand = 0;
+    __syncthreads();
+    for (int j = tid; j < ncand; j += kSelectBlockThreads) {
+      const uint32_t d = sm.cand[j] - lo;
+      if (d <= range) atomicAdd(&sm.hist[d >> shift], 1u);
+    }
+    __syncthreads();
+    find_digit<kSelectBlockThreads>(sm.hist, 2048, remaining, sm.warp_tot, &sm.digit, &sm.remaining);
+    const uint32_t in_bin = sm.hist[sm.digit];
+    const uint32_t step = sm.digit << shift;
+    lo += step;
+    range = min(range - step, (uint32_t)((1ull << shift) - 1ull));
+    remaining = sm.remaining;
+    __syncthreads();                                     // everyone has read the histogram and the digit
+    if (range > 0 && in_bin <= (uint32_t)kSelectRankMax) {
+      // the few keys of the threshold bin, copied over the histogram and ranked by counting
+      for (int j = tid; j < ncand; j += kSelectBlockThreads) {
+        const uint32_t c = sm.cand[j];
+        if (c - lo <= range) sm.hist[atomicAdd(&sm.ncand, 1u)] = c;
+      }
+      __syncthreads();
+      rank_short(sm.hist, (int)sm.ncand);
+    }
+  }
+  const uint32_t thr = lo;                               // the k-th largest key; `remaining` keys equal to it are kept, lowest indices first
+  SEL_STAMP(4);
+  // the kept set: a compaction of the list
+  uint32_t carry_out = 0, carry_eq = 0;
+#pragma unroll 1
+  for (int base = 0; base < ncand; base += kSelectBlockThreads) {
+    const int j = base + tid;
+    const uint32_t kj = j < ncand ? sm.cand[j] : 0u;
+    const bool gt = j < ncand && kj > thr, eq = j < ncand && kj == thr;
+    const uint32_t gt_bal = __ballot_sync(0xffffffffu, gt), eq_bal = __ballot_sync(0xffffffffu, eq);
+    __syncthreads();                                     // the per-warp slots may still be read (previous round, searches above)
+    if (lane == 0) { sm.warp_a[warp] = __popc(gt_bal); sm.warp_b[warp] = __popc(eq_bal); }
+    __syncthreads();
+    const uint32_t g = sm.warp_a[lane], e = sm.warp_b[lane];
+    uint32_t e_incl = e;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v = __shfl_up_sync(0xffffffffu, e_incl, o);
+      if (lane >= o) e_incl += v;
+    }
+    const uint32_t e_excl = carry_eq + e_incl - e;
+    const uint32_t take_w = e_excl >= remaining ? 0u : min(e, remaining - e_excl);
+    uint32_t o_incl = g + take_w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v = __shfl_up_sync(0xffffffffu, o_incl, o);
+      if (lane >= o) o_incl += v;
+    }
+    const uint32_t eq_before = __shfl_sync(0xffffffffu, e_excl, warp);
+    const uint32_t out_before = carry_out + __shfl_sync(0xffffffffu, o_incl - (g + take_w), warp);
+    const bool take = gt || (eq && eq_before + __popc(eq_bal & lt_mask) < remaining);
+    const uint32_t take_bal = __ballot_sync(0xffffffffu, take);
+    if (take) kept[out_before + __popc(take_bal & lt_mask)] = sm.cand_idx[j];
+    carry_eq += __shfl_sync(0xffffffffu, e_incl, 31);
+    carry_out += __shfl_sync(0xffffffffu, o_incl, 31);
+  }
+#ifdef MASKKV_DBG_SELECT_CLOCK
+  SEL_STAMP(5);
+  if (blockIdx.x == 5 && threadIdx.x == 0 && g_sel_prints < 6u)
+    printf("sampled: sample %lld count %lld gather %lld threshold %lld emit %lld ncand %d k %d\n", st_[1] - st_[0], st_[2] - st_[1], st_[3] - st_[2], st_[4] - st_[3], st_[5] - st_[4], ncand, k);
+#endif
+  return true;
+}
+
+// `load(j)` returns the bits of score j of the segment; `loaded()` runs (all threads) once every key is in registers.
+template <bool FULL, class Load, class Loaded>
+__device__ __forceinline__ void select_block_body(SelectBlockShared& sm, Load load, Loaded loaded, int N, int k,
                                                   int32_t* __restrict__ kept) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_rows = FULL ? kSelectBlockRows : min(kSelectBlockRows, (N + 32 * kSelectBlockWarps - 1) / (32 * kSelectBlockWarps));
   const int jbase = warp * (32 * n_rows) + lane;
   const int nv = FULL ? kSelectBlockRows : max(0, min(n_rows, (N - jbase + 31) >> 5));   // rows 0 .. nv-1 hold a key
   uint32_t key[kSelectBlockRows];
+#ifdef MASKKV_DBG_SELECT_CLOCK
+  long long st_[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#endif
+  SEL_STAMP(0);
 #pragma unroll
-  for (int i = 0; i < kSelectBlockRows; ++i) key[i] = (FULL || i < nv) ? __float_as_uint(__ldg(seg + jbase + i * 32)) : 0u;   // all loads first
+  for (int i = 0; i < kSelectBlockRows; ++i) key[i] = (FULL || i < nv) ? load(jbase + i * 32) : 0u;   // all loads first
+  bool released = false;
+  auto release = [&] { if (!released) { loaded(); released = true; } };   // block-uniform
+  SEL_STAMP(1);
+#ifndef MASKKV_SELECT_NO_SAMPLING
+  if (select_block_sampled<FULL>(sm, key, nv, jbase, N, k, kept, load, release)) {
+#ifdef MASKKV_DBG_SELECT_CLOCK
+    SEL_STAMP(6);
+    if (blockIdx.x == 5 && threadIdx.x == 0 && atomicAdd(&g_sel_prints, 1u) < 6u) printf("select sampled path: %lld cycles after the load\n", st_[6] - st_[1]);
+#endif
+    return;
+  }
+  __syncthreads();                                       // the short cut's shared state is reused by the full search
+#endif
+  release();
   // Scores are sums of softmax weights: +0 or positive and finite unless the inputs were not.  The bit patterns of such
   // floats already order like the numbers, so they serve as keys as they are; one signed minimum and one unsigned
   // maximum per key find the window and tell whether every score is of that kind (a negative number, -0 or a NaN
@@ -439,6 +669,7 @@ __device__ __forceinline__ void select_block_body(SelectBlockShared& sm, const f
   }
   uint32_t range = k_max - lo;                           // 0 when all keys are equal
   uint32_t remaining = (uint32_t)k;
+  SEL_STAMP(2);
 
   int ncand = -1;                                        // >= 0: the search continues on cand[0 .. ncand)
   bool first = true;                                     // every key lies inside the window
@@ -458,6 +689,7 @@ __device__ __forceinline__ void select_block_body(SelectBlockShared& sm, const f
     }
     first = false;
     __syncthreads();
+    SEL_STAMP(3);
     find_digit<kSelectBlockThreads>(sm.hist, 2048, remaining, sm.warp_tot, &sm.digit, &sm.remaining);
     const uint32_t in_bin = sm.hist[sm.digit];           // keys that share the threshold digit
     const uint32_t step = sm.digit << shift;
@@ -479,6 +711,7 @@ __device__ __forceinline__ void select_block_body(SelectBlockShared& sm, const f
       }
     }
   }
+  SEL_STAMP(4);
   if (range > 0 && ncand <= kSelectRankMax) {
     // a short list: the threshold is the candidate with fewer than `remaining` candidates above it and at least
     // `remaining` at or above it
@@ -515,6 +748,7 @@ __device__ __forceinline__ void select_block_body(SelectBlockShared& sm, const f
     remaining = sm.remaining;
   }
   const uint32_t thr = lo;                               // threshold key; `remaining` ties are kept, lowest indices first
+  SEL_STAMP(5);
 
   // --- emit in ascending index order ---
   // Usually the ties at the threshold are all kept (one key there, one wanted): then "at or above the threshold" is the
@@ -580,6 +814,12 @@ __device__ __forceinline__ void select_block_body(SelectBlockShared& sm, const f
     out_before += __popc(take_bal);
     eq_before += __popc(eq_bal);
   }
+#ifdef MASKKV_DBG_SELECT_CLOCK
+  SEL_STAMP(6);
+  if (blockIdx.x == 5 && threadIdx.x == 0 && atomicAdd(&g_sel_prints, 1u) < 6u)
+    printf("select phases (cycles): load %lld window %lld hist %lld digit+gather %lld rank %lld emit %lld ncand %d\n", st_[1] - st_[0],
+           st_[2] - st_[1], st_[3] - st_[2], st_[4] - st_[3], st_[5] - st_[4], st_[6] - st_[5], ncand);
+#endif
 }
 
 __global__ void __launch_bounds__(kSelectBlockThreads, 1)
@@ -614,8 +854,149 @@ select_kernel_block(Shape sh, const float* __restrict__ scores, const int32_t* _
     return;
   }
   __syncthreads();                                       // sm.digit has been read by everyone
-  if (N == kSelectBlockKeys) select_block_body<true>(sm, seg, N, k, kept_idx + out0);
-  else select_block_body<false>(sm, seg, N, k, kept_idx + out0);
+  auto load = [&](int j) { return __float_as_uint(__ldg(seg + j)); };
+  auto loaded = [] {};
+  if (N == kSelectBlockKeys) select_block_body<true>(sm, load, loaded, N, k, kept_idx + out0);
+  else select_block_body<false>(sm, load, loaded, N, k, kept_idx + out0);
+}
+
+// ---------------------------------------------------------------------------------------------------------------------
+// The same selection for launches with more segments than SMs: one persistent CTA per SM takes segments b, b + G, ... of
+// the falling-length order, and while it works on one segment the next one's scores arrive in shared memory through ONE
+// bulk copy issued by one thread (no per-thread copy instructions: what a per-thread staging of the next segment cost in
+// instructions used up what it hid).  The buffer is free again as soon as the keys are in registers, so a single buffer
+// gives a whole segment's arithmetic of lead.  The copy moves the 16-byte-aligned middle of the segment; up to three
+// scores at either end are fetched with plain loads.  Waits on the copy are bounded (about a second), then the block
+// raises MASKKV_FLAG_TIMEOUT and leaves.
+__device__ __forceinline__ uint32_t sel_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool sel_mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(sel_smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool sel_mbar_wait(uint64_t* bar, uint32_t parity) {
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (sel_mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 255u) {
+      unsigned long long now;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > 1000000000ull) return false;
+    }
+  }
+}
+
+struct SelectItem { int N, k, out0; const float* seg; };
+constexpr int kSelectStreamSmem = (kSelectBlockKeys + 4) * 4;   // dynamic shared memory: the staged scores
+
+__global__ void __launch_bounds__(kSelectBlockThreads, 1)
+select_kernel_stream(Shape sh, const float* __restrict__ scores, const int32_t* __restrict__ budgets,
+                     const int32_t* __restrict__ offsets, int32_t* __restrict__ kept_idx, uint32_t* __restrict__ status) {
+  extern __shared__ __align__(16) float stage[];           // kSelectBlockKeys + 4 scores
+  __shared__ __align__(16) SelectBlockShared sm;
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int item_r;
+  const int tid = threadIdx.x, n_items = sh.R * sh.Hkv;
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sel_smem_u32(&bar)) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  __syncthreads();
+
+  // segment number `item` of the falling-length order (block-uniform; two barriers)
+  auto locate = [&](int item) {
+    for (int t = tid; t < sh.R; t += kSelectBlockThreads) {
+      const int nt = sh.prompt_cu[t + 1] - sh.prompt_cu[t];
+      int rank = 0;
+      for (int u = 0; u < sh.R; ++u) {
+        const int nu = sh.prompt_cu[u + 1] - sh.prompt_cu[u];
+        rank += (nu > nt || (nu == nt && u < t)) ? 1 : 0;
+      }
+      if (rank == item / sh.Hkv) item_r = t;
+    }
+    __syncthreads();
+    const int r = item_r, hk = item % sh.Hkv, s = r * sh.Hkv + hk;
+    __syncthreads();
+    SelectItem it;
+    const int p0 = sh.prompt_cu[r];
+    it.N = sh.prompt_cu[r + 1] - p0;
+    it.out0 = offsets[s];
+    it.k = budgets[s];
+    if (it.k > it.N) { it.k = it.N; if (tid == 0) atomicOr(status, (uint32_t)MASKKV_FLAG_BOUNDS); }
+    it.seg = scores + (long long)hk * sh.sumN + p0;
+    return it;
+  };
+  auto staged = [](const SelectItem& it) { return it.k > 0 && it.k < it.N; };
+  // score j of the segment lands in stage[mis + j], mis = the segment's offset from a 16-byte boundary in floats
+  auto issue = [&](const SelectItem& it) {
+    if (!staged(it)) return;
+    const int mis = (int)((reinterpret_cast<uintptr_t>(it.seg) & 15u) >> 2);
+    const int e0 = min((4 - mis) & 3, it.N);               // scores in front of the first 16-byte boundary
+    const int n_mid = (it.N - e0) & ~3;
+    float* dst = stage + mis;
+    if (tid == 0) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the buffer was last read with ordinary loads
+      if (n_mid > 0) {
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sel_smem_u32(&bar)), "r"(n_mid * 4) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(sel_smem_u32(dst + e0)), "l"(it.seg + e0), "r"(n_mid * 4), "r"(sel_smem_u32(&bar)) : "memory");
+      } else {
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(sel_smem_u32(&bar)) : "memory");
+      }
+    } else if (tid >= 32 && tid < 40) {
+      const int e = tid - 32;
+      const int j = e < 4 ? e : e0 + n_mid + (e - 4);
+      if (e < 4 ? e < e0 : j < it.N) dst[j] = __ldg(it.seg + j);
+    }
+  };
+
+  int item = blockIdx.x;
+  if (item >= n_items) return;
+  SelectItem cur = locate(item);
+  issue(cur);
+  uint32_t parity = 0;
+  for (;;) {
+    const int next = item + (int)gridDim.x;
+    const bool have_next = next < n_items;
+    SelectItem nxt = cur;
+    if (have_next) nxt = locate(next);
+    bool next_issued = false;
+    if (cur.k >= cur.N && cur.k > 0) {                     // nothing to evict
+      for (int j = tid; j < cur.N; j += kSelectBlockThreads) kept_idx[cur.out0 + j] = j;
+    } else if (cur.k > 0) {
+      const bool ok = sel_mbar_wait(&bar, parity);
+      parity ^= 1u;
+      if (!__syncthreads_and(ok)) {                        // also orders the edge scores written by other threads
+        if (tid == 0) atomicOr(status, (uint32_t)MASKKV_FLAG_TIMEOUT);
+        return;
+      }
+      const float* src = stage + (int)((reinterpret_cast<uintptr_t>(cur.seg) & 15u) >> 2);
+      auto load = [&](int j) { return __float_as_uint(src[j]); };
+      auto loaded = [&] {
+        __syncthreads();                                   // every key is in registers: the buffer is free
+        if (have_next) issue(nxt);
+        next_issued = true;
+      };
+      if (cur.N == kSelectBlockKeys) select_block_body<true>(sm, load, loaded, cur.N, cur.k, kept_idx + cur.out0);
+      else select_block_body<false>(sm, load, loaded, cur.N, cur.k, kept_idx + cur.out0);
+    }
+    if (!have_next) break;
+    __syncthreads();                                       // the body's shared state is reused by the next segment
+    if (!next_issued) issue(nxt);
+    item = next;
+    cur = nxt;
+  }
 }
 
 // One CTA per segment, for batches of segments: the keys are staged in shared memory once and every pass over them

@@ -236,11 +236,14 @@ def test_select_in_registers_crowded_threshold_bin_and_ties(ctx):
     assert ctx.maskkv_check_status() == 0
 
 
-@pytest.mark.parametrize("force", ["2", "4", "8"])
+@pytest.mark.parametrize("force", ["2", "4", "8", "128", "384"])
 def test_both_select_kernels_on_crowded_bins_ties_and_ragged_batches(force, monkeypatch):
-    """The selection runs on clusters (few segments) or on one CTA per segment (batches; keys in registers, or staged in
-    shared memory for segments beyond 32768 scores); bits 1 / 2 / 3 of MASKKV_KERNEL_CHOICE pin the choice.  All must reproduce the oracle exactly on the crowded-bin / tie / NaN case above and on a ragged
-    batch of 100 segments with budgets from 0 to everything."""
+    """The selection runs on clusters (few segments), on one CTA per segment (batches; keys in registers, or staged in
+    shared memory for segments beyond 32768 scores) or on persistent CTAs that copy the next segment's scores to shared
+    memory while they work (more segments than SMs); bits 1 / 2 / 3 / 7 of MASKKV_KERNEL_CHOICE pin the choice, bit 8
+    puts the persistent kernel on three CTAs so that each walks many segments.  All must reproduce the oracle exactly on
+    the crowded-bin / tie / NaN case above and on a ragged batch of 100 segments (starts at every offset from a 16-byte
+    boundary) with budgets from 0 to everything."""
     from paper_2510_09309_b200 import binding as B
     monkeypatch.setenv("MASKKV_KERNEL_CHOICE", force)
     c = B.Context(0)
@@ -324,3 +327,26 @@ def test_attend_fp32_offsets_beyond_capacity_are_clipped_and_flagged(ctx):
     ref, _ = O.attend(live["q_live"].cpu(), live["k_live"].cpu(), live["v_live"].cpu(), store_k[:capacity].cpu(),
                       store_v[:capacity].cpu(), np.array([0, 8, 12], np.int32), wl.live_cu(), 2)
     assert np.abs(out.cpu().numpy() - ref).max() <= 1e-5
+
+
+def test_select_more_segments_than_sms(ctx):
+    """160 full segments of 32768 scores plus a ragged tail of requests: more segments than SMs, so the launch takes the
+    persistent kernel by itself and every CTA walks at least two segments.  Bit-exact against the oracle, twice."""
+    rng = np.random.default_rng(160)
+    heads = 4
+    lens = [32768] * 40 + [int(x) for x in rng.integers(1, 32769, 6)]
+    p, pcu, _ = _problem(ctx, torch.bfloat16, heads, heads, 64, lens, 4)
+    sc = (rng.random((heads, pcu[-1]), dtype=np.float32) * np.float32(1e-3)).astype(np.float32)
+    sc[:, ::11] = np.float32(2.5e-4)                                                    # ties at a common value
+    bud = np.stack([rng.integers(0, min(n, 1024) + 1, heads) for n in lens]).astype(np.int32)
+    bud[1, 0] = lens[1]; bud[2, 1] = 0
+    idx, off = O.select(sc, bud, pcu)
+    scd, budd, offd = to_dev(sc), to_dev(bud), to_dev(off)
+    kept = torch.empty((int(off[-1]) + 8,), dtype=torch.int32, device=ctx.device)
+    for _ in range(2):
+        kept.fill_(-1)
+        ctx.maskkv_select(p, scd, budd, offd, kept)
+        torch.cuda.synchronize()
+        assert np.array_equal(kept[:int(off[-1])].cpu().numpy(), idx)
+        assert (kept[int(off[-1]):] == -1).all()
+    assert ctx.maskkv_check_status() == 0
