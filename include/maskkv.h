@@ -99,6 +99,14 @@ int maskkv_check_status(maskkv_ctx* ctx, void* stream, uint32_t* flags_out);
  * context stays usable.  For tests of the error path; it touches no caller memory. */
 int maskkv_selftest_wait_expiry(maskkv_ctx* ctx, void* stream);
 
+/* Measurement aid (the paper has no counterpart): enqueues a kernel that does nothing but evaluate base-2 exponentials
+ * on the special-function unit - the instruction that bounds maskkv_score, which exponentiates every logit once per
+ * sweep (Eq. 6) - on every SM, `iters` rounds per thread (1 .. 2^20).  *n_exp_out (host) receives the number of
+ * exponentials the launch evaluates; the caller times the launch with events on `stream` and divides, which gives the
+ * measured peak that maskkv_score's exponential throughput is compared with.  `scratch_dev`: one float of device memory
+ * (never written in practice).  Returns MASKKV_E_INVALID on a NULL pointer or an `iters` out of range. */
+int maskkv_selftest_exp_rate(maskkv_ctx* ctx, int iters, float* scratch_dev, int64_t* n_exp_out, void* stream);
+
 /* Text of the most recent CUDA runtime error behind a MASKKV_E_CUDA return of this context ("" if none). */
 const char* maskkv_last_cuda_error(const maskkv_ctx* ctx);
 

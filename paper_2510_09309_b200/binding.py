@@ -22,7 +22,7 @@ MASKKV_F32, MASKKV_BF16 = 0, 1
 MASKKV_FLAG_TIMEOUT, MASKKV_FLAG_CAPACITY, MASKKV_FLAG_BOUNDS, MASKKV_FLAG_FALLBACK = 1, 2, 4, 8
 
 EXPORTS = (
-    "maskkv_create", "maskkv_destroy", "maskkv_status_string", "maskkv_check_status", "maskkv_selftest_wait_expiry", "maskkv_launch_count", "maskkv_last_cuda_error",
+    "maskkv_create", "maskkv_destroy", "maskkv_status_string", "maskkv_check_status", "maskkv_selftest_wait_expiry", "maskkv_selftest_exp_rate", "maskkv_launch_count", "maskkv_last_cuda_error",
     "maskkv_tensor_core_launch_count",
     "maskkv_workspace_bytes",
     "maskkv_layer_budgets", "maskkv_layer_importance", "maskkv_layer_importance_workspace_bytes", "maskkv_refresh_set", "maskkv_mask_project", "maskkv_mask_project_workspace_bytes", "maskkv_score", "maskkv_score_all_keys", "maskkv_score_noalloc", "maskkv_score_noalloc_max_bytes", "maskkv_budget", "maskkv_select", "maskkv_compact", "maskkv_attend", "maskkv_attend_rows",
@@ -62,6 +62,7 @@ def _load() -> C.CDLL:
     lib.maskkv_last_cuda_error.argtypes = [vp]
     lib.maskkv_last_cuda_error.restype = C.c_char_p
     lib.maskkv_selftest_wait_expiry.argtypes = [vp, vp]
+    lib.maskkv_selftest_exp_rate.argtypes = [vp, i32, vp, C.POINTER(C.c_int64), vp]
     lib.maskkv_launch_count.argtypes = [vp]
     lib.maskkv_launch_count.restype = C.c_uint64
     lib.maskkv_tensor_core_launch_count.argtypes = [vp]
@@ -185,6 +186,13 @@ class Context:
     def maskkv_selftest_wait_expiry(self):
         """Enqueues a wait that nothing satisfies: it gives up after about a second and raises MASKKV_FLAG_TIMEOUT."""
         _check(lib.maskkv_selftest_wait_expiry(self._h, _stream()), "maskkv_selftest_wait_expiry", self._h)
+
+    def maskkv_selftest_exp_rate(self, iters: int, scratch: torch.Tensor) -> int:
+        """Enqueues the exponential-rate measurement kernel; returns the number of exponentials it evaluates."""
+        n = C.c_int64(0)
+        _check(lib.maskkv_selftest_exp_rate(self._h, int(iters), scratch.data_ptr(), C.byref(n), _stream()),
+               "maskkv_selftest_exp_rate", self._h)
+        return int(n.value)
 
     def maskkv_check_status(self) -> int:
         flags = C.c_uint32(0)

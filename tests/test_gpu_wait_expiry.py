@@ -42,3 +42,36 @@ def test_a_lost_signal_ends_in_a_status_word_and_the_context_stays_usable():
         assert torch.isfinite(run.out.float()).all() and int(run.offsets[-1].item()) > 0
     finally:
         ctx.close()
+
+
+def test_exp_rate_measurement_counts_its_work_and_rejects_bad_arguments():
+    """maskkv_selftest_exp_rate: the count it returns is grid x threads x 32 x iters, a launch of a few thousand rounds
+    gives a rate between a half and slightly more than the nominal 16 results per clock per SM, and bad arguments launch
+    nothing."""
+    from paper_2510_09309_b200 import binding as B
+    ctx = B.Context(0)
+    try:
+        scratch = torch.zeros(4, dtype=torch.float32, device=ctx.device)
+        sms = torch.cuda.get_device_properties(0).multi_processor_count
+        n0 = ctx.maskkv_launch_count()
+        assert ctx.maskkv_selftest_exp_rate(10, scratch) == sms * 2 * 1024 * 32 * 10
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        best = 0.0
+        for _ in range(4):
+            e0.record()
+            n = ctx.maskkv_selftest_exp_rate(2000, scratch)
+            e1.record()
+            torch.cuda.synchronize()
+            best = max(best, n / (e0.elapsed_time(e1) * 1e-3))
+        per_clock_per_sm = best / sms / 1.965e9                    # at the maximum clock: a lower bound of the per-clock rate
+        assert 8.0 < per_clock_per_sm < 17.0, per_clock_per_sm
+        assert float(scratch.abs().sum()) == 0.0
+        n1 = ctx.maskkv_launch_count()
+        cnt = ctypes.c_int64(0)
+        for iters, ptr in ((0, scratch.data_ptr()), (-3, scratch.data_ptr()), (1 << 21, scratch.data_ptr()), (10, None)):
+            assert B.lib.maskkv_selftest_exp_rate(ctx._h, iters, ptr, ctypes.byref(cnt), None) == B.MASKKV_E_INVALID
+        assert B.lib.maskkv_selftest_exp_rate(ctx._h, 10, scratch.data_ptr(), None, None) == B.MASKKV_E_INVALID
+        assert ctx.maskkv_launch_count() == n1 and n1 == n0 + 5
+        assert ctx.maskkv_check_status() == 0
+    finally:
+        ctx.close()
