@@ -350,3 +350,57 @@ def test_select_more_segments_than_sms(ctx):
         assert np.array_equal(kept[:int(off[-1])].cpu().numpy(), idx)
         assert (kept[int(off[-1]):] == -1).all()
     assert ctx.maskkv_check_status() == 0
+
+
+@pytest.mark.parametrize("force", ["0", "128"])
+def test_select_short_cut_and_its_fallbacks_on_awkward_score_distributions(force, monkeypatch):
+    """The register-resident selection takes a sampled short cut when it can and the full search when it cannot; either
+    way the kept set is the oracle's, bit for bit.  Distributions chosen to hit every exit: sorted ascending and
+    descending scores (the one-key-per-thread sample is then as unrepresentative as it gets), a plateau of equal scores
+    straddling the cut, all but a handful of scores equal, two far-apart clusters, one negative score, one -0, one NaN
+    and one +inf hidden among positive scores, budgets from 1 to most of the segment, full and ragged lengths.  With
+    MASKKV_KERNEL_CHOICE=128 the same runs through the persistent kernel (bulk-copied scores, segment starts at every
+    offset from a 16-byte boundary)."""
+    from paper_2510_09309_b200 import binding as B
+    monkeypatch.setenv("MASKKV_KERNEL_CHOICE", force)
+    c = B.Context(0)
+    try:
+        rng = np.random.default_rng(77)
+        lens = [32768, 32768, 32767, 20001, 9000, 32768, 4097, 32768, 12345, 32768, 32768, 31000]
+        heads = 2
+        p, pcu, _ = _problem(c, torch.bfloat16, heads, heads, 64, lens, 4)
+        sc = np.empty((heads, pcu[-1]), np.float32)
+        bud = np.empty((len(lens), heads), np.int32)
+        for r, n in enumerate(lens):
+            seg = slice(pcu[r], pcu[r + 1])
+            base = (rng.random(n) ** 6).astype(np.float32) * np.float32(1e-2)
+            variants = [
+                np.sort(base), np.sort(base)[::-1].copy(),                                  # 0, 1: sorted both ways
+                np.where(np.arange(n) % 3 == 0, np.float32(5e-3), base),                      # 2: plateau of ties
+                np.where(rng.random(n) < 2e-3, base + 1, np.float32(1e-4)).astype(np.float32),  # 3: nearly all equal
+                np.where(rng.random(n) < 0.5, base, base + np.float32(100)).astype(np.float32),  # 4: two clusters
+                base.copy(), base.copy(), base.copy(), base.copy(),                           # 5-8: one special value each
+                base.copy(), np.full(n, np.float32(0.25)), base.copy(),                       # 9: plain, 10: all equal, 11: plain
+            ]
+            variants[5][n // 2] = np.float32(-1e-3)
+            variants[6][n // 3] = np.float32(-0.0)
+            variants[7][n - 5] = np.float32("nan")
+            variants[8][7] = np.float32("inf")
+            for h in range(heads):
+                sc[h, seg] = variants[r] if h == 0 else variants[(r + 5) % len(variants)]
+            bud[r] = [[1, 300], [256, 2900], [700, 64], [5, 1500], [n // 2, 17], [256, 256], [4000, 9], [512, 33],
+                      [100, n - 1], [3100, 129], [777, 1], [n - 3, 450]][r]
+        idx, off = O.select(sc, bud, pcu)
+        scd, budd, offd = to_dev(sc), to_dev(bud), to_dev(off)
+        kept = torch.empty((int(off[-1]) + 8,), dtype=torch.int32, device=c.device)
+        for _ in range(2):
+            kept.fill_(-1)
+            c.maskkv_select(p, scd, budd, offd, kept)
+            torch.cuda.synchronize()
+            got = kept[:int(off[-1])].cpu().numpy()
+            for s0 in range(len(lens) * heads):
+                assert np.array_equal(got[off[s0]:off[s0 + 1]], idx[off[s0]:off[s0 + 1]]), f"segment {s0}"
+            assert (kept[int(off[-1]):] == -1).all()
+        assert c.maskkv_check_status() == 0
+    finally:
+        c.close()
