@@ -16,6 +16,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import socket
 import statistics
@@ -260,6 +261,34 @@ def batched_calls(ctx, B, device):
         out[name] = row
     out["status_flags"] = ctx.maskkv_check_status()
     return out
+
+
+def replayed_loop_us(call, n_graphs, reps, device):
+    """Microseconds per call of `call(i)`, i = 0 .. n_graphs-1 (each i has its own pointers), when the whole sequence is
+    captured into ONE CUDA graph (the overlapped launches between consecutive calls are kept inside a graph, not between
+    graphs) and the graph is replayed, about `reps` calls in all timed with events.  None if capture is refused."""
+    try:
+        side = torch.cuda.Stream(device=device)
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for j in range(n_graphs):
+                    call(j)
+        torch.cuda.current_stream().wait_stream(side)
+        g.replay()
+        torch.cuda.synchronize()
+        rounds = max(1, reps // n_graphs)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(rounds):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return 1e3 * e0.elapsed_time(e1) / (rounds * n_graphs)
+    except Exception:
+        torch.cuda.synchronize()
+        return None
 
 
 def timed_loop(call, reps, warm=3):
@@ -545,6 +574,12 @@ def bench_ours(args):
     a1.record()
     barrier()
     attend_loop_us = 1e3 * max_over_ranks(a0.elapsed_time(a1), device) / a_steps
+    attend_plain_us = attend_loop_us
+    n_attend_graphs = n_copies                               # graph j: cache copy j, live set j % len(lives)
+    if not args.no_graph and n_attend_graphs <= 64:
+        replayed = replayed_loop_us(attend_step, n_attend_graphs, a_steps, device)
+        if replayed is not None:
+            attend_loop_us = max_over_ranks(replayed, device)
     # the same step with partial refresh: a quarter of the live rows have queries (maskkv_attend_rows)
     n_rows = max(1, wl.n_mask // 4)
     rows_cu = [r * n_rows for r in range(wl.n_requests + 1)]
@@ -568,6 +603,10 @@ def bench_ours(args):
     r1.record()
     barrier()
     attend_rows_us = 1e3 * max_over_ranks(r0.elapsed_time(r1), device) / a_steps
+    if not args.no_graph and n_attend_graphs <= 64:
+        replayed = replayed_loop_us(attend_rows_step, n_attend_graphs, a_steps, device)
+        if replayed is not None:
+            attend_rows_us = max_over_ranks(replayed, device)
     del caches
     # The loop above ran on the cache of the layer the last step left behind (a boundary layer, the larger budget at
     # one rank).  Most layers are middle layers with the smaller budget: compress one and time its step too.
@@ -587,7 +626,13 @@ def bench_ours(args):
             attend_step(i)
         m1.record()
         barrier()
-        attend_mid = {"us": round(1e3 * max_over_ranks(m0.elapsed_time(m1), device) / a_steps, 2), "mean_kept_per_head": mid_kept,
+        mid_plain = 1e3 * max_over_ranks(m0.elapsed_time(m1), device) / a_steps
+        mid_us = mid_plain
+        if not args.no_graph and n_attend_graphs <= 64:
+            replayed = replayed_loop_us(attend_step, n_attend_graphs, a_steps, device)
+            if replayed is not None:
+                mid_us = max_over_ranks(replayed, device)
+        attend_mid = {"us": round(mid_us, 2), "plain_calls_us": round(mid_plain, 2), "mean_kept_per_head": mid_kept,
                       "layer": resident[mid[0]]}
         del caches
         step(args.warmup + len(per_call) - 1)                          # leave the buffers as the later sections expect them
@@ -817,7 +862,10 @@ def bench_ours(args):
         "ms_per_step_plain_calls": eager_ms_per_step,
         "call_us": {k: round(v, 2) for k, v in call_us.items()},
         "attend_step_us": round(attend_loop_us, 2),
-        "attend_step": {"us": round(attend_loop_us, 2), "steps": a_steps, "mean_kept_per_head": mean_kept,
+        "attend_step": {"us": round(attend_loop_us, 2), "plain_calls_us": round(attend_plain_us, 2),
+                        "launch": ("the steps over all cache copies captured in one CUDA graph, replayed" if attend_loop_us != attend_plain_us
+                                   else "plain calls"),
+                        "steps": a_steps, "mean_kept_per_head": mean_kept,
                         "l2": f"{n_copies} copies of the compacted cache ({cache_bytes * n_copies / 1e6:.0f} MB) cycled",
                         "partial_refresh_us": round(attend_rows_us, 2),
                         "partial_refresh": f"{n_rows} of {wl.n_mask} live rows have queries (maskkv_attend_rows)",
